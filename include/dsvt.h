@@ -1,0 +1,192 @@
+/*
+ * dsvt.h -- C ABI of the DSVT dynamic sparse window attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the hot path of the DSVT 3D backbone (arXiv 2301.06051):
+ * rotated set partitioning (Sec. 3.2, Eq. 1-3), batched set attention (Eq. 4-5), the DSVT
+ * layer and block (Eq. 5, Appendix B.1.1) and the attention-style 3D pooling (Eq. 6-7).
+ *
+ * Conventions that hold for every call unless a comment says otherwise:
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  The library reads / writes it
+ *     only during the call's kernels and keeps no reference afterwards.
+ *   - `grid`, `window`, `pool` (3 x int32) and the parameter structs are HOST pointers, read
+ *     before the call returns.
+ *   - Calls are asynchronous: kernels are enqueued on the CUDA stream given to dsvt_create and
+ *     the call returns without synchronising.  Counts produced on the device (`num_sets`,
+ *     `num_out`) stay on the device.
+ *   - Return value: DSVT_OK or a negative DSVT_ERR_* code for errors the host can see (bad
+ *     arguments, unsupported shapes, workspace too small, CUDA launch errors).  Errors only the
+ *     device can see (a coordinate outside the grid, a table index outside [0, n), a table
+ *     larger than its capacity, two voxels in one cell) never trap: the offending item is
+ *     clamped or skipped, a bit is set in the context's device status word, and
+ *     dsvt_status_sync reports it.
+ *   - No call throws, aborts, or frees caller memory.
+ *   - Matrices are row-major; a linear map is y = W x + b with W stored [out][in].
+ *   - precision = DSVT_FP32: weights are float, arithmetic is fp32 throughout.
+ *     precision = DSVT_BF16_FP32ACC: weights are bfloat16 (16-bit storage); products
+ *     accumulate in fp32; residual stream, LayerNorm, softmax and GELU are fp32.
+ *     Features (x, y, feats, out) and biases / LayerNorm parameters are always float.
+ */
+#ifndef DSVT_H_
+#define DSVT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DSVT_OK 0
+#define DSVT_ERR_INVALID_ARG (-1) /* NULL where data is required, negative size, axis not 0/1, ... */
+#define DSVT_ERR_CAPACITY (-2)    /* n, window count or channel count beyond what dsvt_create reserved */
+#define DSVT_ERR_UNSUPPORTED (-3) /* shape the kernels do not cover (see each call) */
+#define DSVT_ERR_CUDA (-4)        /* a CUDA runtime call failed; dsvt_last_cuda_error gives the code */
+#define DSVT_ERR_TIMEOUT (-5)     /* a bounded device-side wait expired (reported by dsvt_status_sync) */
+#define DSVT_ERR_BAD_INPUT (-6)   /* device-detected bad data (reported by dsvt_status_sync) */
+
+#define DSVT_FP32 0
+#define DSVT_BF16_FP32ACC 1
+
+/* Bits of the device status word returned through dsvt_status_sync's `bits`. */
+#define DSVT_STATUS_BAD_COORD 1      /* coordinate or batch index outside the grid (clamped) */
+#define DSVT_STATUS_TABLE_OVERFLOW 2 /* more sets / outputs than the caller's capacity (excess dropped) */
+#define DSVT_STATUS_BAD_INDEX 4      /* set table entry outside [0, n) (slot skipped) */
+#define DSVT_STATUS_DUPLICATE_CELL 8 /* two voxels in the same cell (pooling keeps one of them) */
+#define DSVT_STATUS_TIMEOUT 16       /* a bounded wait inside a kernel expired */
+
+typedef struct dsvt_ctx dsvt_ctx; /* opaque: device workspace, stream, device status word */
+
+/*
+ * Creates a context on CUDA device `device` whose kernels run on `cuda_stream` (a cudaStream_t;
+ * NULL = the legacy default stream).  Reserves all workspace up front for calls with at most
+ * `max_voxels` voxels, `max_windows` windows (or pooling regions) per call and `max_channels`
+ * feature channels; later calls allocate nothing, except dsvt_pool, which grows its dense cell
+ * map once if a call's grid has more cells than any earlier call.
+ * The context must be used by one host thread at a time.
+ */
+int dsvt_create(dsvt_ctx** out, int device, void* cuda_stream, int64_t max_voxels, int64_t max_windows,
+                int32_t max_channels);
+int dsvt_destroy(dsvt_ctx* ctx);
+
+/* Synchronises the context's stream, copies the device status word to *bits (may be NULL), clears
+ * it, and returns DSVT_OK, DSVT_ERR_TIMEOUT, DSVT_ERR_BAD_INPUT or DSVT_ERR_CUDA. */
+int dsvt_status_sync(dsvt_ctx* ctx, int32_t* bits);
+/* The cudaError_t of the most recent failed runtime call on this context (0 if none). */
+int dsvt_last_cuda_error(const dsvt_ctx* ctx);
+/* Static, NUL-terminated description of a DSVT_* return code. */
+const char* dsvt_error_string(int code);
+/* Number of kernels this context has launched since it was created. */
+int64_t dsvt_launch_count(const dsvt_ctx* ctx);
+
+/*
+ * Rotated set partition: Sec. 3.2 "Dynamic set partition" (window partition, Eq. 1 inner-window
+ * id from a sorting strategy, Eq. 2 number of sets, Eq. 3 set index rule) for one sort axis.
+ *
+ *   coords      int32 [n][4] = (b, x, y, z), 16-byte aligned; 0 <= b < batch, 0 <= x < grid[0], ...
+ *   grid        cells per axis (x, y, z); window = (L, W, H); windows start at cell 0 and do not
+ *               cross frames.  Window id = ((b*nWx + x/L)*nWy + y/W)*nWz + z/H, nW* = ceil(grid/window).
+ *   axis        0: X main order, voxels of a window ordered by (x, y, z) of their in-window
+ *               offsets; 1: Y main order, ordered by (y, x, z).  Equal keys keep index order.
+ *   set_table   out, int32 [cap_sets][set_size]: row s = the voxel indices of one set, slot k holding
+ *               the voxel of inner-window rank floor((j*set_size + k) * N / (S*set_size)) (exact
+ *               integer floor), j = the set's number inside its window.  Rows are ordered by
+ *               ascending window id, then j.  Rows [0, *num_sets) are written.
+ *   num_sets    out, device int32: total number of sets.
+ *   set_rowoff  out, optional (NULL to skip), int32 [cap_sets + 1]: set_rowoff[s] = number of
+ *               distinct voxels in the sets before s; entry [*num_sets] = n.  Passing it on to
+ *               dsvt_set_attention / dsvt_layer / dsvt_block saves them a pass over the table.
+ *   perm        out, optional, int32 [n]: voxel indices in (window, inner-window) sorted order.
+ *   win_start, win_setoff   out, optional, int32 [num_windows + 1]: exclusive prefix sums of the
+ *               per-window voxel counts / set counts over ALL windows (empty ones included).
+ *   win_count   out, optional, int32 [num_windows].
+ *
+ * Needs n <= max_voxels, num_windows <= max_windows and num_windows * L*W*H < 2^32
+ * (else DSVT_ERR_CAPACITY / DSVT_ERR_UNSUPPORTED).  cap_sets = n is always enough; if *num_sets
+ * would exceed cap_sets the excess rows are dropped and DSVT_STATUS_TABLE_OVERFLOW is raised.
+ * n = 0 is valid and yields *num_sets = 0.
+ */
+int dsvt_partition(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch, const int32_t grid[3],
+                   const int32_t window[3], int32_t set_size, int32_t axis, int32_t* set_table, int32_t cap_sets,
+                   int32_t* num_sets, int32_t* set_rowoff, int32_t* perm, int32_t* win_start, int32_t* win_count,
+                   int32_t* win_setoff);
+
+/*
+ * Batched set attention: Eq. 4 (INDEX gather of each set's members) followed by the multi-head
+ * self attention of Eq. 5 inside every set, output projection, and scatter back to voxels.
+ * Slot k of a table row is a duplicate, and is masked as a key and not written back, iff k > 0 and
+ * row[k] == row[k-1] (Sec. 3.2: duplicated voxels are masked).
+ *
+ *   feats, out  float [n][C], 16-byte aligned; out may not alias feats.  Rows of voxels that occur in
+ *               no table row are left untouched.  A voxel should occur in at most one set.
+ *   set_table   int32 [cap_sets][set_size]; num_sets: device int32, *num_sets <= cap_sets <= max_voxels.
+ *   set_rowoff  as produced by dsvt_partition, or NULL (then it is derived from the table).
+ *   W_qkv       [3C][C]: rows [0,C) = query map, [C,2C) = key map, [2C,3C) = value map.
+ *   W_o         [C][C].  b_qkv float [3C] or NULL, b_o float [C] or NULL.
+ *   heads       head h owns channels [h*d, (h+1)*d), d = C / heads; logits are scaled by 1/sqrt(d).
+ *   pe          optional float [n][C] positional term, added to the input of the query and key maps only.
+ *
+ * Needs C % 8 == 0, (C/heads) % 4 == 0, set_size <= 128 (else DSVT_ERR_UNSUPPORTED).
+ */
+int dsvt_set_attention(dsvt_ctx* ctx, const float* feats, int32_t n, int32_t C, const int32_t* set_table,
+                       int32_t cap_sets, const int32_t* num_sets, const int32_t* set_rowoff, int32_t set_size,
+                       const void* W_qkv, const float* b_qkv, const void* W_o, const float* b_o, int32_t heads,
+                       const float* pe, int precision, float* out);
+
+/* Parameters of one DSVT layer (Appendix B.1.1).  hidden == 0 drops the MLP; ln1_g == NULL /
+ * ln2_g == NULL drops the corresponding LayerNorm.  hidden <= 2C. */
+typedef struct dsvt_layer_params {
+  int32_t C, heads, hidden, set_size, precision;
+  float ln_eps;
+  const void* W_qkv; /* [3C][C] */
+  const void* W_o;   /* [C][C] */
+  const void* W_1;   /* [hidden][C] */
+  const void* W_2;   /* [C][hidden] */
+  const float *b_qkv, *b_o, *b_1, *b_2;       /* each may be NULL (= 0) */
+  const float *ln1_g, *ln1_b, *ln2_g, *ln2_b; /* float [C]; *_b may be NULL */
+  const float* pe;                            /* float [n][C] or NULL */
+} dsvt_layer_params;
+
+/*
+ * One DSVT layer (Eq. 5 with Appendix B.1.1): x1 = LN1(x + MHSA_sets(x));
+ * y = LN2(x1 + W_2 gelu(W_1 x1 + b_1) + b_2), gelu(t) = t/2 (1 + erf(t/sqrt 2)); LayerNorm over the
+ * C channels with biased variance.  y may alias x (each voxel belongs to one set, and a set is
+ * processed by one thread block).  Rows of voxels in no set are left untouched in y.
+ */
+int dsvt_layer(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* set_table, int32_t cap_sets,
+               const int32_t* num_sets, const int32_t* set_rowoff, const dsvt_layer_params* params, float* y);
+
+/*
+ * One DSVT block (Eq. 5): the layer with the X-axis table, then the layer with the Y-axis table.
+ * layers: HOST array of two parameter structs.  y may alias x.  Every voxel must be covered by
+ * both tables (true for tables made by dsvt_partition).
+ */
+int dsvt_block(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* table_axis0, int32_t cap_sets0,
+               const int32_t* num_sets0, const int32_t* set_rowoff0, const int32_t* table_axis1, int32_t cap_sets1,
+               const int32_t* num_sets1, const int32_t* set_rowoff1, const dsvt_layer_params layers[2], float* y);
+
+/*
+ * Attention-style 3D pooling (Eq. 6, Eq. 7).  Region of voxel (b,x,y,z): (b, x/l, y/w, z/h) with
+ * pool = (l, w, h); slot inside the region: ((x%l)*w + y%w)*h + z%h.  Every non-empty region yields
+ * one output voxel; outputs are ordered by ascending ((b*GX + X)*GY + Y)*GZ + Z, G* = ceil(grid/pool).
+ * The region is padded to l*w*h slots with zero rows; P = channel-wise max over the slots (Eq. 6);
+ * output = W_o MHA(q = W_q P + b_q; k_s = W_k (p_s + e_s) + b_k; v_s = W_v (p_s + e_s) + b_v) + b_o
+ * (Eq. 7), e_s = slot_pe[s] or 0.  mask_empty = 0: max and keys/values run over all l*w*h padded
+ * slots; mask_empty = 1: over the non-empty slots only.
+ *
+ *   out_coords  int32 [cap_m][4] = (b, X, Y, Z); out_feats float [cap_m][C]; num_out device int32.
+ *   region_of   optional int32 [n]: output row of each input voxel; slot_of optional int32 [n].
+ *   cap_m = n is always enough; excess outputs are dropped with DSVT_STATUS_TABLE_OVERFLOW.
+ *
+ * Needs l*w*h <= 32, the number of regions <= max_windows, and the channel limits of
+ * dsvt_set_attention.
+ */
+int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feats, int32_t n, int32_t C, int32_t batch,
+              const int32_t grid[3], const int32_t pool[3], const void* W_q, const void* W_k, const void* W_v,
+              const void* W_o, const float* b_q, const float* b_k, const float* b_v, const float* b_o,
+              const float* slot_pe, int32_t heads, int32_t mask_empty, int precision, int32_t* out_coords,
+              float* out_feats, int32_t cap_m, int32_t* num_out, int32_t* region_of, int32_t* slot_of);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSVT_H_ */

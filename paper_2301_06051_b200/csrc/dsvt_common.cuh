@@ -1,0 +1,77 @@
+// Shared declarations of the CUDA library: context layout, error helpers, launch bookkeeping.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dsvt.h"
+
+struct dsvt_ctx {
+  int device;
+  cudaStream_t stream;
+  int64_t max_voxels, max_windows;
+  int32_t max_channels;
+  int sm_count;
+  int last_cuda_error;
+  int64_t launches;
+  // one device allocation carved into the arrays below
+  void* arena;
+  size_t arena_bytes;
+  int32_t* status;      // device status word
+  uint32_t* keys[2];    // radix sort ping-pong keys        [max_voxels]
+  int32_t* vals[2];     // radix sort ping-pong voxel ids   [max_voxels]
+  int32_t* hist;        // per-tile digit histograms        [256 * sort tiles + 1]
+  int32_t* scan_tmp;    // block sums of the generic scan
+  int32_t* win_count;   // [max_windows + 1]  (pooling: region occupancy flags)
+  int32_t* win_start;   // [max_windows + 1]  (pooling: region rank)
+  int32_t* win_setoff;  // [max_windows + 1]
+  int32_t* rowoff_a;    // [max_voxels + 1] set_rowoff derived from a caller table
+  int32_t* rowoff_b;    // [max_voxels + 1]
+  int32_t* region_key;  // [max_voxels] pooling: dense region id of each output row
+  float* feat_tmp;      // [max_voxels][max_channels] block intermediate
+  // pooling: dense cell -> voxel map, grown on demand
+  int32_t* cell_map;
+  size_t cell_map_entries;
+};
+
+#define DSVT_CUDA_TRY(ctx, expr)          \
+  do {                                    \
+    cudaError_t e_ = (expr);              \
+    if (e_ != cudaSuccess) {              \
+      (ctx)->last_cuda_error = (int)e_;   \
+      return DSVT_ERR_CUDA;               \
+    }                                     \
+  } while (0)
+
+// Call after every kernel launch: counts it and turns a launch error into DSVT_ERR_CUDA.
+#define DSVT_LAUNCHED(ctx)                \
+  do {                                    \
+    (ctx)->launches += 1;                 \
+    cudaError_t e_ = cudaGetLastError();  \
+    if (e_ != cudaSuccess) {              \
+      (ctx)->last_cuda_error = (int)e_;   \
+      return DSVT_ERR_CUDA;               \
+    }                                     \
+  } while (0)
+
+static inline int64_t dsvt_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---- launchers implemented in the .cu files (all enqueue on ctx->stream) ----
+// Exclusive scan; out has count + 1 entries (out[count] = total).  in == out is allowed.
+int dsvt_launch_scan_i32(dsvt_ctx* ctx, const int32_t* in, int32_t* out, int64_t count, int32_t* total_out);
+int dsvt_launch_sort_pairs(dsvt_ctx* ctx, int32_t n, int key_bits, int* final_buf);
+int dsvt_launch_rowoff_from_table(dsvt_ctx* ctx, const int32_t* table, int32_t cap_sets, const int32_t* num_sets,
+                                  int32_t set_size, int32_t* rowoff);
+
+struct dsvt_fused_args {
+  const float* x;
+  float* y;
+  int32_t n;
+  const int32_t* table;
+  const int32_t* num_sets;
+  const int32_t* rowoff;
+  int32_t cap_sets;
+  dsvt_layer_params p;
+  int32_t attention_only;  // 1: y = attention output (no residual, LN, MLP)
+};
+int dsvt_launch_layer_fma(dsvt_ctx* ctx, const dsvt_fused_args& a);

@@ -1,0 +1,430 @@
+// Integer side of the path: window keys, stable LSD radix sort of (key, voxel id) pairs,
+// per-window scans, set table fill (Sec. 3.2, Eq. 1-3).  Everything here is exact int32/uint32/uint64
+// arithmetic, so results are bit-reproducible.
+#include "dsvt_common.cuh"
+
+namespace {
+
+constexpr int kScanThreads = 1024;
+constexpr int kScanItems = 8;                         // per thread
+constexpr int kScanTile = kScanThreads * kScanItems;  // per block iteration
+constexpr int kSortThreads = 256;
+constexpr int kSortRounds = 8;
+constexpr int kSortTile = kSortThreads * kSortRounds;  // keys per block per pass
+constexpr int kRadixBits = 8;
+constexpr int kRadix = 1 << kRadixBits;
+
+__device__ __forceinline__ int warp_incl_scan(int v) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += t;
+  }
+  return v;
+}
+
+// Exclusive scan of one value per thread over the whole block (blockDim.x <= 1024, multiple of 32).
+// warp_tot: shared int[33].  Returns the exclusive prefix; *total = block sum.
+__device__ __forceinline__ int block_excl_scan(int v, int* warp_tot, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  const int incl = warp_incl_scan(v);
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int t = lane < nwarp ? warp_tot[lane] : 0;
+    int ti = warp_incl_scan(t);
+    warp_tot[lane] = ti - t;
+    if (lane == 31) warp_tot[32] = ti;
+  }
+  __syncthreads();
+  const int r = warp_tot[warp] + incl - v;
+  *total = warp_tot[32];
+  __syncthreads();
+  return r;
+}
+
+// ---- generic exclusive scan ------------------------------------------------------------------
+// Single block, loops over the array carrying the running total.  out has count + 1 entries.
+__global__ void __launch_bounds__(kScanThreads) scan_loop_kernel(const int32_t* in, int32_t* out, int64_t count,
+                                                                 int32_t* total_out) {
+  __shared__ int warp_tot[33];
+  int carry = 0;
+  for (int64_t base = 0; base < count; base += kScanTile) {
+    int v[kScanItems];
+    int s = 0;
+    const int64_t i0 = base + (int64_t)threadIdx.x * kScanItems;
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+      v[k] = (i0 + k < count) ? in[i0 + k] : 0;
+      s += v[k];
+    }
+    int tot;
+    int p = carry + block_excl_scan(s, warp_tot, &tot);  // ends with a barrier: all loads precede all stores
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+      if (i0 + k < count) out[i0 + k] = p;
+      p += v[k];
+    }
+    carry += tot;
+  }
+  if (threadIdx.x == 0) {
+    out[count] = carry;
+    if (total_out) *total_out = carry;
+  }
+}
+
+// Multi-block variant: (1) per-block local scan + block sums, (2) scan of block sums, (3) add.
+__global__ void __launch_bounds__(kScanThreads) scan_local_kernel(const int32_t* in, int32_t* out, int64_t count,
+                                                                  int32_t* block_sums) {
+  __shared__ int warp_tot[33];
+  int v[kScanItems];
+  int s = 0;
+  const int64_t i0 = (int64_t)blockIdx.x * kScanTile + (int64_t)threadIdx.x * kScanItems;
+#pragma unroll
+  for (int k = 0; k < kScanItems; ++k) {
+    v[k] = (i0 + k < count) ? in[i0 + k] : 0;
+    s += v[k];
+  }
+  int tot;
+  int p = block_excl_scan(s, warp_tot, &tot);
+#pragma unroll
+  for (int k = 0; k < kScanItems; ++k) {
+    if (i0 + k < count) out[i0 + k] = p;
+    p += v[k];
+  }
+  if (threadIdx.x == 0) block_sums[blockIdx.x] = tot;
+}
+
+__global__ void __launch_bounds__(kScanThreads) scan_add_kernel(int32_t* out, int64_t count,
+                                                                const int32_t* __restrict__ block_offs,
+                                                                int64_t nblocks, int32_t* total_out) {
+  const int add = block_offs[blockIdx.x];
+  const int64_t i0 = (int64_t)blockIdx.x * kScanTile + (int64_t)threadIdx.x * kScanItems;
+#pragma unroll
+  for (int k = 0; k < kScanItems; ++k)
+    if (i0 + k < count) out[i0 + k] += add;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    out[count] = block_offs[nblocks];
+    if (total_out) *total_out = block_offs[nblocks];
+  }
+}
+
+// ---- window keys -----------------------------------------------------------------------------
+struct PartGeom {
+  int32_t batch, gx, gy, gz, L, W, H, nWx, nWy, nWz, axis;
+  uint32_t V;
+};
+
+__global__ void window_key_kernel(const int4* __restrict__ coords, int32_t n, PartGeom g, uint32_t* __restrict__ keys,
+                                  int32_t* __restrict__ vals, int32_t* __restrict__ win_count,
+                                  int32_t* __restrict__ status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  int4 c = coords[i];  // (b, x, y, z)
+  const bool bad =
+      c.x < 0 || c.x >= g.batch || c.y < 0 || c.y >= g.gx || c.z < 0 || c.z >= g.gy || c.w < 0 || c.w >= g.gz;
+  if (bad) {
+    atomicOr(status, DSVT_STATUS_BAD_COORD);
+    c.x = min(max(c.x, 0), g.batch - 1);
+    c.y = min(max(c.y, 0), g.gx - 1);
+    c.z = min(max(c.z, 0), g.gy - 1);
+    c.w = min(max(c.w, 0), g.gz - 1);
+  }
+  const int wx = c.y / g.L, wy = c.z / g.W, wz = c.w / g.H;
+  const int xi = c.y - wx * g.L, yi = c.z - wy * g.W, zi = c.w - wz * g.H;
+  const uint32_t win = (uint32_t)(((c.x * g.nWx + wx) * g.nWy + wy) * g.nWz + wz);
+  const uint32_t inner =
+      g.axis == 0 ? (uint32_t)((xi * g.W + yi) * g.H + zi) : (uint32_t)((yi * g.L + xi) * g.H + zi);
+  keys[i] = win * g.V + inner;
+  vals[i] = i;
+  atomicAdd(&win_count[win], 1);
+}
+
+// ---- stable LSD radix sort, 8 bits per pass ----------------------------------------------------
+__global__ void __launch_bounds__(kSortThreads) radix_hist_kernel(const uint32_t* __restrict__ keys, int32_t n,
+                                                                  int shift, int32_t* __restrict__ hist,
+                                                                  int32_t ntiles) {
+  __shared__ int h[kRadix];
+  h[threadIdx.x] = 0;
+  __syncthreads();
+  const int base = blockIdx.x * kSortTile;
+#pragma unroll
+  for (int r = 0; r < kSortRounds; ++r) {
+    const int i = base + r * kSortThreads + threadIdx.x;
+    if (i < n) atomicAdd(&h[(keys[i] >> shift) & (kRadix - 1)], 1);
+  }
+  __syncthreads();
+  hist[threadIdx.x * ntiles + blockIdx.x] = h[threadIdx.x];  // digit-major: scan order = (digit, tile)
+}
+
+__global__ void __launch_bounds__(kSortThreads) radix_scatter_kernel(const uint32_t* __restrict__ keys_in,
+                                                                     const int32_t* __restrict__ vals_in,
+                                                                     uint32_t* __restrict__ keys_out,
+                                                                     int32_t* __restrict__ vals_out, int32_t n,
+                                                                     int shift, const int32_t* __restrict__ offs,
+                                                                     int32_t ntiles) {
+  constexpr int kWarps = kSortThreads / 32;
+  __shared__ int wcnt[kWarps][kRadix];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int run = offs[threadIdx.x * ntiles + blockIdx.x];  // thread d owns digit d's running output position
+  const int base = blockIdx.x * kSortTile;
+  for (int r = 0; r < kSortRounds; ++r) {
+    if (base + r * kSortThreads >= n) break;  // uniform over the block
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) wcnt[w][threadIdx.x] = 0;
+    __syncthreads();
+    const int i = base + r * kSortThreads + threadIdx.x;
+    const bool live = i < n;
+    uint32_t key = 0;
+    int val = 0, digit = 0, rank = 0;
+    if (live) {
+      key = keys_in[i];
+      val = vals_in[i];
+      digit = (key >> shift) & (kRadix - 1);
+    }
+    const unsigned act = __ballot_sync(0xffffffffu, live);
+    if (live) {
+      const unsigned peers = __match_any_sync(act, digit);
+      rank = __popc(peers & ((1u << lane) - 1u));
+      if (rank == 0) wcnt[warp][digit] = __popc(peers);
+    }
+    __syncthreads();
+    {  // thread d: exclusive prefix over the warps for digit d, starting at its running position
+      int acc = run;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        const int t = wcnt[w][threadIdx.x];
+        wcnt[w][threadIdx.x] = acc;
+        acc += t;
+      }
+      run = acc;
+    }
+    __syncthreads();
+    if (live) {
+      const int dst = wcnt[warp][digit] + rank;
+      keys_out[dst] = key;
+      vals_out[dst] = val;
+    }
+    __syncthreads();
+  }
+}
+
+// ---- per-window scans (Eq. 2) ------------------------------------------------------------------
+// Single block.  win_start = exclusive scan of N_w; win_setoff = exclusive scan of S_w = ceil(N_w / tau).
+__global__ void __launch_bounds__(kScanThreads) window_scan_kernel(const int32_t* __restrict__ win_count,
+                                                                   int32_t num_windows, int32_t tau,
+                                                                   int32_t* win_start, int32_t* win_setoff,
+                                                                   int32_t cap_sets, int32_t* num_sets,
+                                                                   int32_t* status) {
+  __shared__ int warp_tot[33];
+  int carry_n = 0, carry_s = 0;
+  for (int base = 0; base < num_windows; base += kScanTile) {
+    int cn[kScanItems], cs[kScanItems];
+    int sn = 0, ss = 0;
+    const int i0 = base + threadIdx.x * kScanItems;
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+      const int N = (i0 + k < num_windows) ? win_count[i0 + k] : 0;
+      cn[k] = N;
+      cs[k] = N / tau + ((N % tau) > 0 ? 1 : 0);  // Eq. 2
+      sn += cn[k];
+      ss += cs[k];
+    }
+    int tn, ts;
+    int pn = carry_n + block_excl_scan(sn, warp_tot, &tn);
+    int ps = carry_s + block_excl_scan(ss, warp_tot, &ts);
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+      if (i0 + k < num_windows) {
+        win_start[i0 + k] = pn;
+        win_setoff[i0 + k] = ps;
+      }
+      pn += cn[k];
+      ps += cs[k];
+    }
+    carry_n += tn;
+    carry_s += ts;
+  }
+  if (threadIdx.x == 0) {
+    win_start[num_windows] = carry_n;
+    win_setoff[num_windows] = carry_s;
+    if (carry_s > cap_sets) {
+      atomicOr(status, DSVT_STATUS_TABLE_OVERFLOW);
+      carry_s = cap_sets;
+    }
+    *num_sets = carry_s;
+  }
+}
+
+// ---- set table fill (Eq. 3, Eq. 4's rank -> voxel id) -------------------------------------------
+// One warp per set.
+__global__ void table_fill_kernel(const int32_t* __restrict__ sorted_vox, const int32_t* __restrict__ win_count,
+                                  const int32_t* __restrict__ win_start, const int32_t* __restrict__ win_setoff,
+                                  int32_t num_windows, int32_t tau, const int32_t* __restrict__ num_sets,
+                                  int32_t* __restrict__ table, int32_t* __restrict__ rowoff) {
+  const int lane = threadIdx.x & 31;
+  const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int S_all = *num_sets;
+  if (s >= S_all) return;
+  // last window w with win_setoff[w] <= s; it is non-empty because win_setoff[w + 1] > s
+  int lo = 0, hi = num_windows;  // invariant: win_setoff[lo] <= s < win_setoff[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (win_setoff[mid] <= s) lo = mid; else hi = mid;
+  }
+  const int w = lo;
+  const uint64_t N = (uint64_t)win_count[w];
+  const uint64_t Sw = (uint64_t)(win_setoff[w + 1] - win_setoff[w]);
+  const uint64_t j = (uint64_t)(s - win_setoff[w]);
+  const int start = win_start[w];
+  const uint64_t den = Sw * (uint64_t)tau;
+  for (int k = lane; k < tau; k += 32) {
+    const uint64_t q = ((j * (uint64_t)tau + (uint64_t)k) * N) / den;  // Eq. 3, exact integer floor
+    table[(size_t)s * tau + k] = sorted_vox[start + (int)q];
+  }
+  if (rowoff && lane == 0) {
+    rowoff[s] = start + (int)((j * N) / Sw);  // first rank of set j (proof of Theorem A.2)
+    if (s == S_all - 1) rowoff[S_all] = start + (int)(((j + 1) * N) / Sw);
+  }
+}
+
+// ---- distinct-member counts of a caller-supplied table ------------------------------------------
+// cnt[s] = number of slots k with k == 0 or row[k] != row[k-1]; 0 for s >= *num_sets.  One warp per set.
+__global__ void table_unique_count_kernel(const int32_t* __restrict__ table, int32_t cap_sets,
+                                          const int32_t* __restrict__ num_sets, int32_t tau,
+                                          int32_t* __restrict__ cnt) {
+  const int lane = threadIdx.x & 31;
+  const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (s >= cap_sets) return;
+  int c = 0;
+  if (s < *num_sets) {
+    const int32_t* row = table + (size_t)s * tau;
+    for (int k0 = 0; k0 < tau; k0 += 32) {
+      const int k = k0 + lane;
+      const bool uniq = k < tau && (k == 0 || row[k] != row[k - 1]);
+      c += __popc(__ballot_sync(0xffffffffu, uniq));
+    }
+  }
+  if (lane == 0) cnt[s] = c;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------------
+int dsvt_launch_scan_i32(dsvt_ctx* ctx, const int32_t* in, int32_t* out, int64_t count, int32_t* total_out) {
+  if (count <= 8 * (int64_t)kScanTile) {
+    scan_loop_kernel<<<1, kScanThreads, 0, ctx->stream>>>(in, out, count, total_out);
+    DSVT_LAUNCHED(ctx);
+    return DSVT_OK;
+  }
+  const int64_t nblocks = dsvt_ceil_div(count, kScanTile);
+  scan_local_kernel<<<(unsigned)nblocks, kScanThreads, 0, ctx->stream>>>(in, out, count, ctx->scan_tmp);
+  DSVT_LAUNCHED(ctx);
+  scan_loop_kernel<<<1, kScanThreads, 0, ctx->stream>>>(ctx->scan_tmp, ctx->scan_tmp, nblocks, nullptr);
+  DSVT_LAUNCHED(ctx);
+  scan_add_kernel<<<(unsigned)nblocks, kScanThreads, 0, ctx->stream>>>(out, count, ctx->scan_tmp, nblocks, total_out);
+  DSVT_LAUNCHED(ctx);
+  return DSVT_OK;
+}
+
+// Sorts ctx->keys[0] / ctx->vals[0] (n pairs) by the low key_bits bits; *final_buf = index of the
+// buffer pair that holds the result.
+int dsvt_launch_sort_pairs(dsvt_ctx* ctx, int32_t n, int key_bits, int* final_buf) {
+  const int passes = key_bits <= 0 ? 1 : (key_bits + kRadixBits - 1) / kRadixBits;
+  const int32_t ntiles = (int32_t)dsvt_ceil_div(n, kSortTile);
+  int cur = 0;
+  for (int p = 0; p < passes; ++p) {
+    const int shift = p * kRadixBits;
+    radix_hist_kernel<<<ntiles, kSortThreads, 0, ctx->stream>>>(ctx->keys[cur], n, shift, ctx->hist, ntiles);
+    DSVT_LAUNCHED(ctx);
+    int rc = dsvt_launch_scan_i32(ctx, ctx->hist, ctx->hist, (int64_t)kRadix * ntiles, nullptr);
+    if (rc != DSVT_OK) return rc;
+    radix_scatter_kernel<<<ntiles, kSortThreads, 0, ctx->stream>>>(ctx->keys[cur], ctx->vals[cur], ctx->keys[cur ^ 1],
+                                                                    ctx->vals[cur ^ 1], n, shift, ctx->hist, ntiles);
+    DSVT_LAUNCHED(ctx);
+    cur ^= 1;
+  }
+  *final_buf = cur;
+  return DSVT_OK;
+}
+
+int dsvt_launch_rowoff_from_table(dsvt_ctx* ctx, const int32_t* table, int32_t cap_sets, const int32_t* num_sets,
+                                  int32_t set_size, int32_t* rowoff) {
+  const int warps_per_block = 8;
+  if (cap_sets > 0) {
+    const unsigned blocks = (unsigned)dsvt_ceil_div(cap_sets, warps_per_block);
+    table_unique_count_kernel<<<blocks, warps_per_block * 32, 0, ctx->stream>>>(table, cap_sets, num_sets, set_size,
+                                                                                rowoff);
+    DSVT_LAUNCHED(ctx);
+  }
+  return dsvt_launch_scan_i32(ctx, rowoff, rowoff, cap_sets, nullptr);
+}
+
+static int key_bits_for(uint64_t max_key) {
+  int b = 0;
+  while (b < 32 && (max_key >> b) != 0) ++b;
+  return b;
+}
+
+extern "C" int dsvt_partition(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch, const int32_t grid[3],
+                              const int32_t window[3], int32_t set_size, int32_t axis, int32_t* set_table,
+                              int32_t cap_sets, int32_t* num_sets, int32_t* set_rowoff, int32_t* perm,
+                              int32_t* win_start, int32_t* win_count, int32_t* win_setoff) {
+  if (!ctx || !grid || !window || !num_sets || n < 0 || batch < 1 || set_size < 1 || cap_sets < 0 ||
+      (axis != 0 && axis != 1))
+    return DSVT_ERR_INVALID_ARG;
+  for (int a = 0; a < 3; ++a)
+    if (grid[a] < 1 || window[a] < 1) return DSVT_ERR_INVALID_ARG;
+  if (n > 0 && (!coords || !set_table)) return DSVT_ERR_INVALID_ARG;
+  if (((uintptr_t)coords & 15) != 0) return DSVT_ERR_INVALID_ARG;
+  PartGeom g;
+  g.batch = batch; g.gx = grid[0]; g.gy = grid[1]; g.gz = grid[2];
+  g.L = window[0]; g.W = window[1]; g.H = window[2];
+  g.nWx = (int32_t)dsvt_ceil_div(grid[0], window[0]);
+  g.nWy = (int32_t)dsvt_ceil_div(grid[1], window[1]);
+  g.nWz = (int32_t)dsvt_ceil_div(grid[2], window[2]);
+  g.axis = axis;
+  const uint64_t V = (uint64_t)window[0] * window[1] * window[2];
+  const uint64_t num_windows = (uint64_t)batch * g.nWx * g.nWy * g.nWz;
+  if (V >= (1ull << 31) || num_windows >= (1ull << 31) || num_windows * V > 0xFFFFFFFFull) return DSVT_ERR_UNSUPPORTED;
+  g.V = (uint32_t)V;
+  if (n > ctx->max_voxels || (int64_t)num_windows > ctx->max_windows) return DSVT_ERR_CAPACITY;
+  const int32_t nw = (int32_t)num_windows;
+  cudaStream_t st = ctx->stream;
+
+  DSVT_CUDA_TRY(ctx, cudaMemsetAsync(ctx->win_count, 0, sizeof(int32_t) * (size_t)(nw + 1), st));
+  int fin = 0;
+  if (n > 0) {
+    window_key_kernel<<<(unsigned)dsvt_ceil_div(n, 256), 256, 0, st>>>((const int4*)coords, n, g, ctx->keys[0],
+                                                                       ctx->vals[0], ctx->win_count, ctx->status);
+    DSVT_LAUNCHED(ctx);
+    int rc = dsvt_launch_sort_pairs(ctx, n, key_bits_for(num_windows * V - 1), &fin);
+    if (rc != DSVT_OK) return rc;
+  }
+  window_scan_kernel<<<1, kScanThreads, 0, st>>>(ctx->win_count, nw, set_size, ctx->win_start, ctx->win_setoff,
+                                                 cap_sets, num_sets, ctx->status);
+  DSVT_LAUNCHED(ctx);
+  if (n > 0) {
+    // number of sets <= floor(n / tau) + (non-empty windows) <= min(cap_sets, n)
+    int64_t s_bound = (int64_t)n / set_size + (int64_t)(nw < n ? nw : n);
+    if (s_bound > n) s_bound = n;
+    if (s_bound > cap_sets) s_bound = cap_sets;
+    if (s_bound > 0) {
+      table_fill_kernel<<<(unsigned)dsvt_ceil_div(s_bound, 8), 256, 0, st>>>(ctx->vals[fin], ctx->win_count,
+                                                                             ctx->win_start, ctx->win_setoff, nw,
+                                                                             set_size, num_sets, set_table, set_rowoff);
+      DSVT_LAUNCHED(ctx);
+    }
+    if (perm)
+      DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(perm, ctx->vals[fin], sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToDevice, st));
+  }
+  if (set_rowoff && (n == 0 || cap_sets == 0)) DSVT_CUDA_TRY(ctx, cudaMemsetAsync(set_rowoff, 0, sizeof(int32_t), st));
+  if (win_count)
+    DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(win_count, ctx->win_count, sizeof(int32_t) * (size_t)nw, cudaMemcpyDeviceToDevice, st));
+  if (win_start)
+    DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(win_start, ctx->win_start, sizeof(int32_t) * (size_t)(nw + 1), cudaMemcpyDeviceToDevice, st));
+  if (win_setoff)
+    DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(win_setoff, ctx->win_setoff, sizeof(int32_t) * (size_t)(nw + 1), cudaMemcpyDeviceToDevice, st));
+  return DSVT_OK;
+}
