@@ -1,0 +1,303 @@
+#!/usr/bin/env python
+"""Benchmark of the DSVT hot path on synthetic LiDAR-shaped frames.
+
+A step is one pass of the whole path over one frame: rotated set partition (both sort axes), then
+every DSVT block of the backbone (configuration 2: 32,000 pillars on 468 x 468, C = 192, 8 heads,
+set size 36, four blocks of two layers with MLP and LayerNorm, bfloat16 weights, fp32 accumulate).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
+
+Prints one JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own frame: the path shards
+by frame with no collective, so scaling is weak.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "voxels/sec per DSVT block (partition amortised over the backbone); frames_per_sec = backbone frames/sec"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc, self.idx = None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=10)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def algorithmic_flops_per_layer(rowoff: np.ndarray, C: int, hidden: int) -> float:
+    """Projections 8 C^2 + MLP 4 C hidden per voxel, attention 4 m^2 C per set of m distinct voxels."""
+    m = np.diff(rowoff).astype(np.float64)
+    n = float(rowoff[-1])
+    return n * (8.0 * C * C + 4.0 * C * hidden) + 4.0 * C * float((m * m).sum())
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, on a bounded sample of the same workload (rank 0 only)."""
+    rank, _, world = _dist_env()
+    if rank != 0:
+        return
+    import dsvt_inputs as di
+    from oracle import ref
+
+    cores = ref.max_threads()
+    ref.set_threads(cores)
+    cfg = di.make_config(args.config)
+    n_s = min(cfg["n"], 1200)
+    p = ref.partition(cfg["coords"], cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], 0)
+    # whole windows in window order until about n_s voxels
+    w_end = int(np.searchsorted(p.win_start, n_s))
+    sel = np.sort(p.perm[: p.win_start[w_end]])
+    cs, fs = cfg["coords"][sel], cfg["feats"][sel].astype(np.float64)
+
+    def step():
+        t0 = ref.partition(cs, cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], 0)
+        t1 = ref.partition(cs, cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], 1)
+        x = fs
+        for blk in cfg["blocks"]:
+            x = ref.block(x, t0.set_table, t1.set_table, blk)
+        return x
+
+    for _ in range(args.warmup):
+        step()
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t) / args.steps
+    value = sel.shape[0] * len(cfg["blocks"]) / dt
+    sample = "%d voxels (whole windows) of config %d through partition + %d blocks per step" % (
+        sel.shape[0], args.config, len(cfg["blocks"]))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "voxels/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config %d (%s), CPU oracle on a bounded sample" % (args.config, cfg["name"])},
+        "cpu_baseline": {"value": value, "unit": "voxels/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "voxels/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import torch
+
+    import dsvt_inputs as di
+    from paper_2301_06051_b200 import api, pipeline
+
+    rank, local_rank, world = _dist_env()
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    api.load()  # no fallback: a missing library is an error
+
+    cfg = di.make_config(args.config)
+    if cfg.get("pool_shape"):
+        raise SystemExit("bench.py times single-stage configurations (1-4)")
+    n, C, nb = cfg["n"], cfg["C"], len(cfg["blocks"])
+    bb = pipeline.Backbone(cfg, device=local_rank)
+    ctx, stage = bb.ctx, bb.stage1
+    coords_h = torch.from_numpy(cfg["coords"]).pin_memory()
+    feats_h = torch.from_numpy(cfg["feats"]).pin_memory()
+    out_h = torch.empty((n, C), dtype=torch.float32).pin_memory()
+    coords = coords_h.to(dev)
+    x = feats_h.to(dev)
+    y = torch.empty_like(x)
+    flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def step_device():
+        stage.forward(coords, x, y)
+
+    def step_e2e():
+        c = coords_h.to(dev, non_blocking=True)
+        f = feats_h.to(dev, non_blocking=True)
+        stage.forward(c, f, y)
+        out_h.copy_(y, non_blocking=True)
+        stream.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        flush.zero_()
+        step_device()
+    barrier()
+    if ctx.status_sync() != 0:
+        raise SystemExit("device status word is not clean after warm-up")
+
+    # ---- timed region: K steps, L2 flushed (outside the events) before each ----
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3 + nb)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    barrier()
+    for k in range(args.steps):
+        flush.zero_()
+        e = ev[k]
+        e[0].record(stream)
+        stage.partition(coords)
+        e[1].record(stream)
+        src = x
+        for b, blk in enumerate(stage.blocks):
+            ctx.block(src, stage.tables[0], stage.tables[1], blk, y)
+            src = y
+            e[2 + b].record(stream)
+    barrier()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop()
+    t_step = np.array([e[0].elapsed_time(e[1 + nb]) for e in ev])  # ms
+    t_part = np.array([e[0].elapsed_time(e[1]) for e in ev])
+    t_blocks = np.array([[e[1 + b].elapsed_time(e[2 + b]) for b in range(nb)] for e in ev])
+    total_ms = float(t_step.sum())
+
+    # ---- end to end through the public API with pinned host buffers ----
+    for _ in range(2):
+        step_e2e()
+    barrier()
+    t0 = time.perf_counter()
+    e_steps = max(3, min(args.steps, 10))
+    for _ in range(e_steps):
+        step_e2e()
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / e_steps
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+    if ctx.status_sync() != 0:
+        raise SystemExit("device status word is not clean after the timed region")
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = total_ms / args.steps
+    value = world * n * nb / (ms_per_step * 1e-3)
+    peaks = _peaks()
+    # dominant kernel: the fused layer kernel, two launches per block
+    S = int(stage.tables[0].num_sets.item())
+    fl = [algorithmic_flops_per_layer(stage.tables[a].set_rowoff[: S + 1].cpu().numpy(), C, cfg["hidden"])
+          for a in (0, 1)]
+    flops_per_launch = 0.5 * (fl[0] + fl[1])
+    layer_ms = float(t_blocks.mean()) / 2.0
+    achieved = flops_per_launch / (layer_ms * 1e-3) / 1e12
+    pad = 1.0 - n / (S * cfg["set_size"])
+
+    # ---- CPU oracle on a bounded sample (reported baseline, not a target) ----
+    from oracle import ref
+
+    cores = ref.max_threads()
+    ref.set_threads(cores)
+    t0 = time.perf_counter()
+    p0 = ref.partition(cfg["coords"], cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], 0)
+    p1 = ref.partition(cfg["coords"], cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], 1)
+    ref.block(cfg["feats"], p0.set_table, p1.set_table, cfg["blocks"][0])
+    cpu_s = time.perf_counter() - t0
+    cpu = {"value": n / cpu_s, "unit": "voxels/s", "cores": cores, "kind": "oracle",
+           "sample": "the whole frame (%d voxels): both partitions + the first block, one pass, %.1f s" % (n, cpu_s)}
+
+    print(json.dumps({
+        "metric": METRIC, "value": value, "unit": "voxels/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 weights x fp32 activations, fp32 accumulate (FMA pipes)"
+        if cfg["precision"] == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": "config %d (%s): %d voxels, grid %s, window %s, set size %d, C=%d, %d blocks x 2 layers"
+                   % (args.config, cfg["name"], n, cfg["grid"], cfg["window"], cfg["set_size"], C, nb),
+                   "l2": "L2 flushed by a %d MiB write before every step" % (L2_FLUSH_BYTES >> 20),
+                   "num_sets": S, "pad_ratio": pad, "frames_per_rank": 1},
+        "frames_per_sec": world / (ms_per_step * 1e-3),
+        "t_partition_ms": float(t_part.mean()), "t_block_ms": float(t_blocks.mean()),
+        "clocks": clocks,
+        "e2e": {"value": world * n * nb / (e2e_ms * 1e-3), "unit": "voxels/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(coords_h.numel() * 4 + feats_h.numel() * 4),
+                "d2h_bytes_per_step": int(out_h.numel() * 4)},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "fused DSVT layer", "bound": "tensor", "achieved": achieved,
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                     "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"], "peak_source": peaks["source"],
+                     "flops_per_launch": flops_per_launch, "ms_per_launch": layer_ms, "traffic": None},
+        "cpu_baseline": cpu,
+    }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

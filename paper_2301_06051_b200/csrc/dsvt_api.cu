@@ -1,0 +1,216 @@
+// Context management and the attention / layer / block entry points of the C ABI.
+#include <new>
+
+#include "dsvt_common.cuh"
+
+namespace {
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Carver {
+  unsigned char* base;
+  size_t off;
+  template <typename T>
+  T* take(size_t count) {
+    off = align_up(off, 256);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+void carve(dsvt_ctx* c, unsigned char* base, size_t* total) {
+  Carver k{base, 0};
+  const size_t nv = (size_t)c->max_voxels, nw = (size_t)c->max_windows;
+  const size_t sort_tiles = (nv + 2047) / 2048 + 1;
+  const size_t hist = 256 * sort_tiles + 1;
+  size_t longest_scan = hist;
+  if (nw + 1 > longest_scan) longest_scan = nw + 1;
+  if (nv + 1 > longest_scan) longest_scan = nv + 1;
+  c->status = k.take<int32_t>(64);
+  c->keys[0] = k.take<uint32_t>(nv);
+  c->keys[1] = k.take<uint32_t>(nv);
+  c->vals[0] = k.take<int32_t>(nv);
+  c->vals[1] = k.take<int32_t>(nv);
+  c->hist = k.take<int32_t>(hist);
+  c->scan_tmp = k.take<int32_t>(longest_scan / 8192 + 2);
+  c->win_count = k.take<int32_t>(nw + 1);
+  c->win_start = k.take<int32_t>(nw + 1);
+  c->win_setoff = k.take<int32_t>(nw + 1);
+  c->rowoff_a = k.take<int32_t>(nv + 1);
+  c->rowoff_b = k.take<int32_t>(nv + 1);
+  c->region_key = k.take<int32_t>(nv);
+  *total = align_up(k.off, 256);
+}
+
+int check_layer_shape(const dsvt_ctx* ctx, const dsvt_layer_params& p, bool attention_only) {
+  if (p.C < 1 || p.heads < 1 || p.set_size < 1 || p.hidden < 0) return DSVT_ERR_INVALID_ARG;
+  if (p.precision != DSVT_FP32 && p.precision != DSVT_BF16_FP32ACC) return DSVT_ERR_INVALID_ARG;
+  if (!p.W_qkv || !p.W_o) return DSVT_ERR_INVALID_ARG;
+  if (p.C % p.heads != 0 || p.C % 8 != 0 || (p.C / p.heads) % 4 != 0 || p.set_size > 128) return DSVT_ERR_UNSUPPORTED;
+  if (!attention_only && p.hidden > 0) {
+    if (!p.W_1 || !p.W_2) return DSVT_ERR_INVALID_ARG;
+    if (p.hidden % 8 != 0 || p.hidden > 2 * p.C) return DSVT_ERR_UNSUPPORTED;
+  }
+  if (p.C > ctx->max_channels) return DSVT_ERR_CAPACITY;
+  const void* ptrs[] = {p.W_qkv, p.W_o, p.W_1, p.W_2, p.b_qkv, p.b_o, p.b_1, p.b_2, p.pe};
+  for (const void* q : ptrs)
+    if (((uintptr_t)q & 15) != 0) return DSVT_ERR_INVALID_ARG;
+  return DSVT_OK;
+}
+
+// Runs one fused layer; derives the row offsets from the table when the caller has none.
+int run_layer(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* table, int32_t cap_sets,
+              const int32_t* num_sets, const int32_t* rowoff, const dsvt_layer_params& p, float* y,
+              bool attention_only, int32_t* rowoff_scratch) {
+  if (n == 0 || cap_sets == 0) return DSVT_OK;
+  if (!rowoff) {
+    int rc = dsvt_launch_rowoff_from_table(ctx, table, cap_sets, num_sets, p.set_size, rowoff_scratch);
+    if (rc != DSVT_OK) return rc;
+    rowoff = rowoff_scratch;
+  }
+  dsvt_fused_args a;
+  a.x = x; a.y = y; a.n = n; a.table = table; a.num_sets = num_sets; a.rowoff = rowoff; a.cap_sets = cap_sets;
+  a.p = p;
+  a.attention_only = attention_only ? 1 : 0;
+  return dsvt_launch_layer_fma(ctx, a);
+}
+
+int check_common(const dsvt_ctx* ctx, const float* x, const float* y, int32_t n, const int32_t* table,
+                 int32_t cap_sets, const int32_t* num_sets) {
+  if (!ctx || n < 0 || cap_sets < 0) return DSVT_ERR_INVALID_ARG;
+  if (n > 0 && cap_sets > 0 && (!x || !y || !table || !num_sets)) return DSVT_ERR_INVALID_ARG;
+  if (((uintptr_t)x & 15) || ((uintptr_t)y & 15)) return DSVT_ERR_INVALID_ARG;
+  if (n > ctx->max_voxels || cap_sets > ctx->max_voxels) return DSVT_ERR_CAPACITY;
+  return DSVT_OK;
+}
+
+}  // namespace
+
+extern "C" int dsvt_create(dsvt_ctx** out, int device, void* cuda_stream, int64_t max_voxels, int64_t max_windows,
+                           int32_t max_channels) {
+  if (!out || max_voxels < 1 || max_windows < 1 || max_channels < 1) return DSVT_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+    cudaGetLastError();
+    return DSVT_ERR_CUDA;
+  }
+  if (cudaSetDevice(device) != cudaSuccess) return DSVT_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return DSVT_ERR_CUDA;
+  if (prop.major != 10) return DSVT_ERR_UNSUPPORTED;  // kernels are built for sm_100a only
+  dsvt_ctx* c = new (std::nothrow) dsvt_ctx();
+  if (!c) return DSVT_ERR_INVALID_ARG;
+  c->device = device;
+  c->stream = (cudaStream_t)cuda_stream;
+  c->max_voxels = max_voxels;
+  c->max_windows = max_windows;
+  c->max_channels = max_channels;
+  c->sm_count = prop.multiProcessorCount;
+  c->last_cuda_error = 0;
+  c->launches = 0;
+  c->cell_map = nullptr;
+  c->cell_map_entries = 0;
+  size_t total = 0;
+  carve(c, nullptr, &total);
+  cudaError_t e = cudaMalloc(&c->arena, total);
+  if (e != cudaSuccess) {
+    delete c;
+    return e == cudaErrorMemoryAllocation ? DSVT_ERR_CAPACITY : DSVT_ERR_CUDA;
+  }
+  c->arena_bytes = total;
+  carve(c, (unsigned char*)c->arena, &total);
+  if (cudaMemsetAsync(c->status, 0, 64 * sizeof(int32_t), c->stream) != cudaSuccess) {
+    cudaFree(c->arena);
+    delete c;
+    return DSVT_ERR_CUDA;
+  }
+  *out = c;
+  return DSVT_OK;
+}
+
+extern "C" int dsvt_destroy(dsvt_ctx* ctx) {
+  if (!ctx) return DSVT_OK;
+  cudaSetDevice(ctx->device);
+  cudaStreamSynchronize(ctx->stream);
+  if (ctx->cell_map) cudaFree(ctx->cell_map);
+  cudaFree(ctx->arena);
+  delete ctx;
+  return DSVT_OK;
+}
+
+extern "C" int dsvt_status_sync(dsvt_ctx* ctx, int32_t* bits) {
+  if (!ctx) return DSVT_ERR_INVALID_ARG;
+  int32_t h = 0;
+  DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(&h, ctx->status, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+  DSVT_CUDA_TRY(ctx, cudaMemsetAsync(ctx->status, 0, sizeof(int32_t), ctx->stream));
+  DSVT_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+  if (bits) *bits = h;
+  if (h & DSVT_STATUS_TIMEOUT) return DSVT_ERR_TIMEOUT;
+  if (h != 0) return DSVT_ERR_BAD_INPUT;
+  return DSVT_OK;
+}
+
+extern "C" int dsvt_last_cuda_error(const dsvt_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+extern "C" int64_t dsvt_launch_count(const dsvt_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" const char* dsvt_error_string(int code) {
+  switch (code) {
+    case DSVT_OK: return "ok";
+    case DSVT_ERR_INVALID_ARG: return "invalid argument";
+    case DSVT_ERR_CAPACITY: return "beyond the capacity reserved by dsvt_create";
+    case DSVT_ERR_UNSUPPORTED: return "shape not supported by the kernels";
+    case DSVT_ERR_CUDA: return "CUDA runtime error (see dsvt_last_cuda_error)";
+    case DSVT_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case DSVT_ERR_BAD_INPUT: return "bad input detected on the device (see the status bits)";
+  }
+  return "unknown code";
+}
+
+extern "C" int dsvt_set_attention(dsvt_ctx* ctx, const float* feats, int32_t n, int32_t C, const int32_t* set_table,
+                                  int32_t cap_sets, const int32_t* num_sets, const int32_t* set_rowoff,
+                                  int32_t set_size, const void* W_qkv, const float* b_qkv, const void* W_o,
+                                  const float* b_o, int32_t heads, const float* pe, int precision, float* out) {
+  int rc = check_common(ctx, feats, out, n, set_table, cap_sets, num_sets);
+  if (rc != DSVT_OK) return rc;
+  if (n > 0 && feats == out) return DSVT_ERR_INVALID_ARG;
+  dsvt_layer_params p = {};
+  p.C = C; p.heads = heads; p.hidden = 0; p.set_size = set_size; p.precision = precision; p.ln_eps = 0.f;
+  p.W_qkv = W_qkv; p.W_o = W_o; p.b_qkv = b_qkv; p.b_o = b_o; p.pe = pe;
+  rc = check_layer_shape(ctx, p, true);
+  if (rc != DSVT_OK) return rc;
+  return run_layer(ctx, feats, n, set_table, cap_sets, num_sets, set_rowoff, p, out, true, ctx->rowoff_a);
+}
+
+extern "C" int dsvt_layer(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* set_table, int32_t cap_sets,
+                          const int32_t* num_sets, const int32_t* set_rowoff, const dsvt_layer_params* params,
+                          float* y) {
+  if (!params) return DSVT_ERR_INVALID_ARG;
+  int rc = check_common(ctx, x, y, n, set_table, cap_sets, num_sets);
+  if (rc != DSVT_OK) return rc;
+  rc = check_layer_shape(ctx, *params, false);
+  if (rc != DSVT_OK) return rc;
+  return run_layer(ctx, x, n, set_table, cap_sets, num_sets, set_rowoff, *params, y, false, ctx->rowoff_a);
+}
+
+extern "C" int dsvt_block(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* table_axis0, int32_t cap_sets0,
+                          const int32_t* num_sets0, const int32_t* set_rowoff0, const int32_t* table_axis1,
+                          int32_t cap_sets1, const int32_t* num_sets1, const int32_t* set_rowoff1,
+                          const dsvt_layer_params layers[2], float* y) {
+  if (!layers) return DSVT_ERR_INVALID_ARG;
+  int rc = check_common(ctx, x, y, n, table_axis0, cap_sets0, num_sets0);
+  if (rc != DSVT_OK) return rc;
+  rc = check_common(ctx, x, y, n, table_axis1, cap_sets1, num_sets1);
+  if (rc != DSVT_OK) return rc;
+  for (int i = 0; i < 2; ++i) {
+    rc = check_layer_shape(ctx, layers[i], false);
+    if (rc != DSVT_OK) return rc;
+  }
+  if (layers[0].C != layers[1].C) return DSVT_ERR_INVALID_ARG;
+  // X-axis layer writes y (every voxel is in one set, so every row of y is produced); the Y-axis
+  // layer then runs in place on y.
+  rc = run_layer(ctx, x, n, table_axis0, cap_sets0, num_sets0, set_rowoff0, layers[0], y, false, ctx->rowoff_a);
+  if (rc != DSVT_OK) return rc;
+  return run_layer(ctx, y, n, table_axis1, cap_sets1, num_sets1, set_rowoff1, layers[1], y, false, ctx->rowoff_b);
+}

@@ -28,7 +28,6 @@ struct dsvt_ctx {
   int32_t* rowoff_a;    // [max_voxels + 1] set_rowoff derived from a caller table
   int32_t* rowoff_b;    // [max_voxels + 1]
   int32_t* region_key;  // [max_voxels] pooling: dense region id of each output row
-  float* feat_tmp;      // [max_voxels][max_channels] block intermediate
   // pooling: dense cell -> voxel map, grown on demand
   int32_t* cell_map;
   size_t cell_map_entries;

@@ -1,0 +1,79 @@
+"""Sequencing of the C-ABI calls for a whole backbone pass (no arithmetic here).
+
+A DSVT backbone is a stack of blocks; all blocks of a stage share the two rotated set tables of their
+frame, so a pass is: dsvt_partition (X axis), dsvt_partition (Y axis), then one dsvt_block per block,
+and optionally dsvt_pool followed by a second stage on the pooled grid.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+from . import api
+
+
+class Stage:
+    """Blocks that share one grid / window shape: two set tables + per-block weights."""
+
+    def __init__(self, ctx: api.Context, blocks: Sequence[Sequence[Dict]], batch: int, grid, window, set_size: int,
+                 precision: int, max_voxels: int):
+        self.ctx, self.batch, self.grid, self.window, self.set_size = ctx, batch, tuple(grid), tuple(window), set_size
+        dev = ctx.device
+        self.blocks = [[api.device_weights(l, precision, dev) for l in blk] for blk in blocks]
+        cap = max(int(max_voxels), 1)
+        self.tables = [
+            api.SetTable(torch.empty((cap, set_size), dtype=torch.int32, device=dev),
+                         torch.zeros(1, dtype=torch.int32, device=dev),
+                         torch.empty(cap + 1, dtype=torch.int32, device=dev), cap, set_size)
+            for _ in range(2)
+        ]
+
+    def partition(self, coords: torch.Tensor):
+        for axis in (0, 1):
+            self.ctx.partition(coords, self.batch, self.grid, self.window, self.set_size, axis, out=self.tables[axis])
+
+    def forward(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+        """Partition (both axes) then every block; the result ends up in y."""
+        self.partition(coords)
+        src = x
+        for blk in self.blocks:
+            self.ctx.block(src, self.tables[0], self.tables[1], blk, y)
+            src = y
+        return y
+
+
+class Backbone:
+    """One or two stages with an optional attention-style pooling step between them."""
+
+    def __init__(self, cfg: Dict, device: int = 0, max_voxels: Optional[int] = None):
+        n = int(max_voxels or cfg["n"])
+        self.cfg = cfg
+        self.precision = api.BF16_FP32ACC if cfg["precision"] == "bf16" else api.FP32
+        grid, window = cfg["grid"], cfg["window"]
+        nwin = cfg["batch"] * (-(-grid[0] // window[0])) * (-(-grid[1] // window[1])) * (-(-grid[2] // window[2]))
+        max_windows = nwin
+        self.pool_shape = cfg.get("pool_shape")
+        if self.pool_shape:
+            pg = [-(-grid[a] // self.pool_shape[a]) for a in range(3)]
+            max_windows = max(max_windows, cfg["batch"] * pg[0] * pg[1] * pg[2])
+        self.ctx = api.Context(n, max_windows, cfg["C"], device)
+        self.stage1 = Stage(self.ctx, cfg["blocks"], cfg["batch"], grid, window, cfg["set_size"], self.precision, n)
+        self.stage2 = None
+        if self.pool_shape:
+            self.pool_w = api.device_weights(cfg["pool"], self.precision, self.ctx.device)
+            self.pooled_grid = tuple(pg)
+            self.stage2 = Stage(self.ctx, cfg["blocks_after_pool"], cfg["batch"], self.pooled_grid, window,
+                                cfg["set_size"], self.precision, n)
+
+    def forward(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor):
+        """Returns (coords_out, feats_out, num_out); for a single stage these are (coords, y, None)."""
+        self.stage1.forward(coords, x, y)
+        if not self.stage2:
+            return coords, y, None
+        oc, of, num, _, _ = self.ctx.pool(coords, y, self.cfg["batch"], self.cfg["grid"], self.pool_shape, self.pool_w)
+        # the pooled voxel count lives on the device; the second stage needs it as a tensor extent
+        m = int(num.item())
+        oc, of = oc[:m], of[:m]
+        self.stage2.forward(oc, of, of)
+        return oc, of, num

@@ -1,0 +1,329 @@
+"""CUDA path vs the CPU oracle, through the C ABI (ctypes binding).  All tests need a B200."""
+import numpy as np
+import pytest
+import torch
+
+import dsvt_inputs as di
+from gpu_helpers import check_close, dev, precision_of, rowoff_of, table_np, upload_table
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    from paper_2301_06051_b200 import api
+
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    api.load()  # raises if the CUDA library has not been built: there is no fallback
+    return api
+
+
+def _nwin(batch, grid, window):
+    return batch * int(np.prod([-(-g // w) for g, w in zip(grid, window)]))
+
+
+# ------------------------------------------------------------------------------------------------
+# partition: bit-exact
+# ------------------------------------------------------------------------------------------------
+def _check_partition(gpu, oracle, coords, batch, grid, window, tau, ctx=None):
+    n = coords.shape[0]
+    ctx = ctx or gpu.Context(max(n, 1), _nwin(batch, grid, window), 64)
+    dc = dev(coords)
+    for axis in (0, 1):
+        t = ctx.partition(dc, batch, grid, window, tau, axis, extras=True)
+        assert ctx.status_sync() == 0
+        ref = oracle.partition(coords, batch, grid, window, tau, axis)
+        tbl, ro = table_np(t)
+        assert tbl.shape == ref.set_table.shape, (axis, tbl.shape, ref.set_table.shape)
+        assert np.array_equal(tbl, ref.set_table), axis
+        assert np.array_equal(ro, rowoff_of(ref.set_table)), axis
+        assert np.array_equal(t.perm[:n].cpu().numpy(), ref.perm)
+        assert np.array_equal(t.win_count.cpu().numpy(), ref.win_count)
+        assert np.array_equal(t.win_start.cpu().numpy(), ref.win_start)
+        assert np.array_equal(t.win_setoff.cpu().numpy(), ref.win_setoff)
+    return ctx
+
+
+@pytest.mark.parametrize("cid", [1, 2, 3, 4, 5])
+def test_partition_bit_exact_on_every_config(gpu, oracle, cid):
+    cfg = di.make_config(cid, with_feats=False)
+    _check_partition(gpu, oracle, cfg["coords"], cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"])
+
+
+@pytest.mark.parametrize("grid,window,batch,n,tau", [
+    ((20, 17, 1), (6, 5, 1), 1, 200, 7),       # partial edge windows
+    ((9, 9, 6), (4, 4, 3), 2, 500, 10),        # 3D windows, two frames
+    ((5, 5, 5), (5, 5, 5), 1, 125, 36),        # one completely full window
+    ((12, 12, 1), (12, 12, 1), 1, 36, 36),     # N == tau exactly: no duplicates
+    ((12, 12, 1), (12, 12, 1), 1, 1, 36),      # a single voxel
+    ((300, 300, 1), (7, 9, 1), 1, 5000, 90),   # spans several sort tiles and a ragged tail
+    ((64, 64, 8), (64, 64, 8), 1, 20000, 48),  # one huge window (20000 voxels -> 417 sets)
+])
+def test_partition_bit_exact_small_and_edge_cases(gpu, oracle, grid, window, batch, n, tau):
+    rng = np.random.default_rng(n + tau)
+    _check_partition(gpu, oracle, di.unique_cells(rng, n, grid, batch), batch, grid, window, tau)
+
+
+def test_partition_empty_and_errors(gpu):
+    ctx = gpu.Context(100, 64, 64)
+    empty = torch.zeros((0, 4), dtype=torch.int32, device="cuda")
+    t = ctx.partition(empty, 1, (8, 8, 1), (4, 4, 1), 3, 0, extras=True)
+    assert int(t.num_sets.item()) == 0 and int(t.win_start.sum().item()) == 0 and ctx.status_sync() == 0
+    ok = dev(np.array([[0, 1, 1, 0], [0, 2, 2, 0], [0, 7, 7, 0]], dtype=np.int32))
+    with pytest.raises(gpu.DsvtError):
+        ctx.partition(ok, 1, (8, 8, 1), (4, 4, 1), 3, 2)  # bad axis
+    with pytest.raises(gpu.DsvtError):
+        ctx.partition(ok, 1, (800, 800, 1), (4, 4, 1), 3, 0)  # more windows than reserved
+    # device-detected problems raise status bits instead of faulting
+    bad = dev(np.array([[0, 1, 1, 0], [0, 9, 2, 0]], dtype=np.int32))
+    ctx.partition(bad, 1, (8, 8, 1), (4, 4, 1), 3, 0)
+    assert ctx.status_sync() & gpu.STATUS_BAD_COORD
+    t = ctx.partition(ok, 1, (8, 8, 1), (4, 4, 1), 1, 0, cap_sets=2)  # three sets, room for two
+    assert ctx.status_sync() & gpu.STATUS_TABLE_OVERFLOW
+    assert int(t.num_sets.item()) == 2
+    assert ctx.status_sync() == 0  # cleared by the read
+
+
+# ------------------------------------------------------------------------------------------------
+# set attention / layer / block
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed,n,grid,window,tau,C,heads,bf16", [
+    (1, 150, (16, 16, 1), (6, 6, 1), 5, 16, 4, False),
+    (2, 700, (30, 30, 4), (10, 10, 4), 36, 32, 8, False),
+    (3, 90, (12, 12, 1), (12, 12, 1), 36, 64, 2, False),
+    (4, 2500, (64, 64, 1), (12, 12, 1), 36, 128, 8, False),
+    (5, 3000, (96, 96, 1), (30, 30, 1), 90, 128, 8, False),   # nuScenes-like window and set size
+    (6, 1500, (48, 48, 1), (12, 12, 1), 36, 192, 8, True),
+    (7, 1200, (48, 48, 2), (12, 12, 2), 48, 192, 8, True),
+])
+def test_set_attention_matches_oracle(gpu, oracle, seed, n, grid, window, tau, C, heads, bf16):
+    cfg = di.random_case(seed, n, grid, window, tau, C, heads, bf16=bf16)
+    L = cfg["blocks"][0][0]
+    ctx = gpu.Context(n, _nwin(1, grid, window), C)
+    w = gpu.device_weights(L, precision_of(cfg), ctx.device)
+    x = dev(cfg["feats"])
+    for axis in (0, 1):
+        t = ctx.partition(dev(cfg["coords"]), 1, grid, window, tau, axis)
+        out = torch.full_like(x, 123.0)
+        ctx.set_attention(x, t, w, out)
+        out2 = torch.full_like(x, 321.0)
+        ctx.set_attention(x, t, w, out2, use_rowoff=False)  # row offsets derived from the table
+        assert ctx.status_sync() == 0
+        ref_t = oracle.partition(cfg["coords"], 1, grid, window, tau, axis).set_table
+        want, covered = oracle.set_attention(cfg["feats"], ref_t, L["W_qkv"], L["b_qkv"], L["W_o"], L["b_o"], heads)
+        assert covered.all()
+        check_close(out.cpu().numpy(), want, cfg["precision"], "set_attention axis %d" % axis)
+        assert torch.equal(out, out2)
+
+
+def test_set_attention_arbitrary_table_positional_term_and_untouched_rows(gpu, oracle):
+    """A caller-made table (not from dsvt_partition): partial sets, duplicates in odd places,
+    voxels in no set, table capacity larger than the set count, no biases."""
+    rng = np.random.default_rng(5)
+    n, C, heads, tau = 60, 32, 4, 6
+    L = di.make_layer(rng, C, heads, 0, False, False)
+    x = rng.standard_normal((n, C), dtype=np.float32)
+    pe = rng.standard_normal((n, C), dtype=np.float32)
+    table = np.array([[3, 3, 3, 7, 9, 9], [10, 11, 12, 13, 14, 15], [20, 20, 20, 20, 20, 20], [30, 31, 31, 32, 32, 33],
+                      [59, 58, 57, 56, 55, 54], [40, 41, 41, 41, 42, 42]], dtype=np.int32)
+    ctx = gpu.Context(n, 8, C)
+    w = gpu.device_weights(L, gpu.FP32, ctx.device)
+    w["b_qkv"] = None
+    w["b_o"] = None
+    for with_rowoff in (True, False):
+        t = upload_table(table, with_rowoff=with_rowoff, cap_extra=5)
+        out = torch.full((n, C), 55.0, device="cuda")
+        ctx.set_attention(dev(x), t, w, out, pe=dev(pe))
+        assert ctx.status_sync() == 0
+        want = np.full((n, C), 55.0)
+        want, covered = oracle.set_attention(x, table, L["W_qkv"], None, L["W_o"], None, heads, pe=pe, out=want)
+        assert covered.sum() == 23
+        check_close(out.cpu().numpy(), want, "fp32", "arbitrary table")
+        assert np.all(out.cpu().numpy()[covered == 0] == 55.0)
+    # an index outside [0, n) is skipped and flagged, never dereferenced
+    bad = table.copy()
+    bad[1, 2] = n + 5
+    out = torch.zeros((n, C), device="cuda")
+    ctx.set_attention(dev(x), upload_table(bad), w, out)
+    assert ctx.status_sync() & gpu.STATUS_BAD_INDEX
+
+
+def test_empty_inputs_are_no_ops(gpu):
+    ctx = gpu.Context(16, 4, 32)
+    rng = np.random.default_rng(1)
+    L = di.make_layer(rng, 32, 4, 64, True, False)
+    w = gpu.device_weights(L, gpu.FP32, ctx.device)
+    x = torch.zeros((0, 32), device="cuda")
+    t = upload_table(np.zeros((0, 6), dtype=np.int32))
+    ctx.layer(x, t, w, x)
+    ctx.set_attention(x, t, w, torch.zeros((0, 32), device="cuda"))
+    assert ctx.status_sync() == 0
+
+
+def _run_blocks_gpu(gpu, cfg, blocks, coords, feats, ctx=None):
+    from paper_2301_06051_b200 import pipeline
+
+    n = coords.shape[0]
+    ctx = ctx or gpu.Context(n, _nwin(cfg["batch"], cfg["grid"], cfg["window"]), cfg["C"])
+    st = pipeline.Stage(ctx, blocks, cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], precision_of(cfg), n)
+    x = dev(feats)
+    y = torch.empty_like(x)
+    st.forward(dev(coords), x, y)
+    assert ctx.status_sync() == 0
+    return y.cpu().numpy()
+
+
+def _run_blocks_oracle(oracle, cfg, blocks, coords, feats):
+    p0 = oracle.partition(coords, cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], 0)
+    p1 = oracle.partition(coords, cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], 1)
+    x = feats.astype(np.float64)
+    for blk in blocks:
+        x = oracle.block(x, p0.set_table, p1.set_table, blk)
+    return x
+
+
+def test_config1_block_fp32(gpu, oracle):
+    """Config 1: 2000 pillars on 64x64, C = 128, one block of two attention layers, fp32 throughout."""
+    cfg = di.make_config(1)
+    got = _run_blocks_gpu(gpu, cfg, cfg["blocks"], cfg["coords"], cfg["feats"])
+    want = _run_blocks_oracle(oracle, cfg, cfg["blocks"], cfg["coords"], cfg["feats"])
+    check_close(got, want, "fp32", "config 1 block")
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_config1_shape_with_full_layers(gpu, oracle, bf16):
+    """Config 1's frame with MLP and LayerNorm switched on, two blocks; also layer == block halves."""
+    cfg = di.make_config(1)
+    rng = np.random.default_rng(77)
+    cfg["precision"] = "bf16" if bf16 else "fp32"
+    blocks = [[di.make_layer(rng, 128, 8, 256, True, bf16) for _ in range(2)] for _ in range(2)]
+    got = _run_blocks_gpu(gpu, cfg, blocks, cfg["coords"], cfg["feats"])
+    want = _run_blocks_oracle(oracle, cfg, blocks, cfg["coords"], cfg["feats"])
+    check_close(got, want, cfg["precision"], "config 1 frame, full layers")
+    # dsvt_layer on its own, not in place, equals the oracle layer
+    ctx = gpu.Context(cfg["n"], 36, 128)
+    t0 = ctx.partition(dev(cfg["coords"]), 1, cfg["grid"], cfg["window"], 36, 0)
+    w = gpu.device_weights(blocks[0][0], precision_of(cfg), ctx.device)
+    y = torch.empty((cfg["n"], 128), device="cuda")
+    ctx.layer(dev(cfg["feats"]), t0, w, y)
+    ref_t = oracle.partition(cfg["coords"], 1, cfg["grid"], cfg["window"], 36, 0).set_table
+    check_close(y.cpu().numpy(), oracle.layer(cfg["feats"], ref_t, blocks[0][0]), cfg["precision"], "layer")
+
+
+def _sample_windows(oracle, cfg, coords, n_target, seed, win=None):
+    """Voxel indices of randomly chosen whole windows holding about n_target voxels."""
+    win = win or cfg["window"]
+    p = oracle.partition(coords, cfg["batch"], cfg["grid"], win, cfg["set_size"], 0)
+    rng = np.random.default_rng(seed)
+    order = rng.permutation(np.flatnonzero(p.win_count > 0))
+    # always include the fullest and the emptiest windows
+    order = np.concatenate([[np.argmax(p.win_count)], order])
+    sel, total = [], 0
+    for w in order:
+        sel.append(p.perm[p.win_start[w]:p.win_start[w + 1]])
+        total += sel[-1].shape[0]
+        if total >= n_target:
+            break
+    return np.sort(np.unique(np.concatenate(sel)))
+
+
+@pytest.mark.parametrize("cid,n_sample", [(2, 2500), (3, 2500), (4, 2500)])
+def test_backbone_full_size_bf16_on_sampled_windows(gpu, oracle, cid, n_sample):
+    """Configs 2-4 at full size (four blocks, bf16 weights).  The backbone is window-local (both
+    layers of every block use the same windows), so the oracle recomputes whole sampled windows."""
+    cfg = di.make_config(cid)
+    got = _run_blocks_gpu(gpu, cfg, cfg["blocks"], cfg["coords"], cfg["feats"])
+    assert np.all(np.isfinite(got))
+    sel = _sample_windows(oracle, cfg, cfg["coords"], n_sample, cid)
+    want = _run_blocks_oracle(oracle, cfg, cfg["blocks"], cfg["coords"][sel], cfg["feats"][sel])
+    check_close(got[sel], want, "bf16", "config %d backbone, %d sampled voxels" % (cid, sel.shape[0]))
+    # one block on its own as well (per-block error, not only end to end)
+    got1 = _run_blocks_gpu(gpu, cfg, cfg["blocks"][:1], cfg["coords"], cfg["feats"])
+    want1 = _run_blocks_oracle(oracle, cfg, cfg["blocks"][:1], cfg["coords"][sel], cfg["feats"][sel])
+    check_close(got1[sel], want1, "bf16", "config %d first block" % cid)
+
+
+def test_in_place_and_repeatability(gpu):
+    cfg = di.make_config(2, n_override=6000)
+    a = _run_blocks_gpu(gpu, cfg, cfg["blocks"][:2], cfg["coords"], cfg["feats"])
+    b = _run_blocks_gpu(gpu, cfg, cfg["blocks"][:2], cfg["coords"], cfg["feats"])
+    assert np.array_equal(a, b)  # no atomics on the float path: bitwise repeatable
+
+
+# ------------------------------------------------------------------------------------------------
+# pooling
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("mask_empty", [0, 1])
+@pytest.mark.parametrize("grid,pool,batch,n,C,heads,with_pe,bf16", [
+    ((16, 16, 1), (2, 2, 1), 1, 120, 16, 4, False, False),
+    ((9, 7, 8), (2, 2, 2), 2, 400, 32, 4, True, False),
+    ((6, 6, 8), (1, 1, 4), 1, 150, 32, 8, False, False),
+    ((40, 40, 1), (3, 3, 1), 1, 900, 64, 8, True, False),
+    ((100, 100, 1), (2, 2, 1), 1, 4000, 192, 8, False, True),
+    ((20, 20, 16), (2, 2, 4), 1, 3000, 192, 8, True, True),
+])
+def test_pool_matches_oracle(gpu, oracle, grid, pool, batch, n, C, heads, with_pe, bf16, mask_empty):
+    rng = np.random.default_rng(n + C)
+    coords = di.unique_cells(rng, n, grid, batch)
+    feats = rng.standard_normal((n, C), dtype=np.float32)
+    nslots = pool[0] * pool[1] * pool[2]
+    Wt = di.make_pool_weights(rng, C, heads, bf16, nslots, with_pe)
+    regions = batch * int(np.prod([-(-g // p) for g, p in zip(grid, pool)]))
+    ctx = gpu.Context(n, regions, C)
+    w = gpu.device_weights(Wt, gpu.BF16_FP32ACC if bf16 else gpu.FP32, ctx.device)
+    oc, of, num, reg, slot = ctx.pool(dev(coords), dev(feats), batch, grid, pool, w, mask_empty=mask_empty, extras=True)
+    assert ctx.status_sync() == 0
+    ref = oracle.pool(coords, feats, batch, grid, pool, Wt["W_q"], Wt["W_k"], Wt["W_v"], Wt["W_o"], Wt["b_q"],
+                      Wt["b_k"], Wt["b_v"], Wt["b_o"], heads, slot_pe=Wt["slot_pe"], mask_empty=mask_empty)
+    m = int(num.item())
+    assert m == ref.coords.shape[0]
+    assert np.array_equal(oc[:m].cpu().numpy(), ref.coords)
+    assert np.array_equal(reg.cpu().numpy(), ref.region_of)
+    assert np.array_equal(slot.cpu().numpy(), ref.slot_of)
+    check_close(of[:m].cpu().numpy(), ref.feats, "bf16" if bf16 else "fp32", "pool")
+
+
+def test_pool_flags_duplicate_cells_and_overflow(gpu):
+    rng = np.random.default_rng(3)
+    C = 16
+    Wt = di.make_pool_weights(rng, C, 4, False)
+    ctx = gpu.Context(16, 64, C)
+    w = gpu.device_weights(Wt, gpu.FP32, ctx.device)
+    coords = np.array([[0, 1, 1, 0], [0, 1, 1, 0], [0, 5, 5, 0]], dtype=np.int32)
+    feats = rng.standard_normal((3, C), dtype=np.float32)
+    ctx.pool(dev(coords), dev(feats), 1, (8, 8, 1), (2, 2, 1), w)
+    assert ctx.status_sync() & gpu.STATUS_DUPLICATE_CELL
+    coords = np.array([[0, 1, 1, 0], [0, 3, 1, 0], [0, 5, 5, 0]], dtype=np.int32)
+    oc, of, num, _, _ = ctx.pool(dev(coords), dev(feats), 1, (8, 8, 1), (2, 2, 1), w, cap_m=2)
+    assert ctx.status_sync() & gpu.STATUS_TABLE_OVERFLOW
+    assert int(num.item()) == 2
+
+
+def test_config5_blocks_pool_blocks_on_sampled_windows(gpu, oracle):
+    """Config 5 at full size: two blocks, 2x2x1 attention pooling, two blocks at half resolution.
+    A 12x12 window of the pooled grid covers a 24x24 area of the input grid, i.e. four whole input
+    windows, so the chain is local to such areas and the oracle recomputes sampled areas."""
+    from paper_2301_06051_b200 import pipeline
+
+    cfg = di.make_config(5)
+    bb = pipeline.Backbone(cfg)
+    x = dev(cfg["feats"])
+    oc, of, num = bb.forward(dev(cfg["coords"]), x, torch.empty_like(x))
+    assert bb.ctx.status_sync() == 0
+    oc, of = oc.cpu().numpy(), of.cpu().numpy()
+    assert np.all(np.isfinite(of))
+    coords = cfg["coords"]
+    sel = _sample_windows(oracle, cfg, coords, 3000, 5, win=(24, 24, 1))
+    cs, fs = coords[sel], cfg["feats"][sel]
+    mid = _run_blocks_oracle(oracle, cfg, cfg["blocks"], cs, fs)
+    pw = cfg["pool"]
+    pooled = oracle.pool(cs, mid, 1, cfg["grid"], cfg["pool_shape"], pw["W_q"], pw["W_k"], pw["W_v"], pw["W_o"],
+                         pw["b_q"], pw["b_k"], pw["b_v"], pw["b_o"], cfg["heads"])
+    cfg2 = dict(cfg, grid=(468, 468, 1))
+    want = _run_blocks_oracle(oracle, cfg2, cfg["blocks_after_pool"], pooled.coords, pooled.feats)
+    # match rows by pooled coordinate
+    key = lambda c: (c[:, 1].astype(np.int64) * 468 + c[:, 2])
+    pos = {k: i for i, k in enumerate(key(oc).tolist())}
+    rows = np.array([pos[k] for k in key(pooled.coords).tolist()])
+    assert np.all(np.diff(key(oc)) > 0)  # ascending pooled coordinates
+    check_close(of[rows], want, "bf16", "config 5 chain, %d pooled voxels" % rows.shape[0])
