@@ -254,10 +254,13 @@ def run_ours(args):
     t0 = time.perf_counter()
     p0 = ref.partition(cfg["coords"], cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], 0)
     p1 = ref.partition(cfg["coords"], cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"], 1)
-    ref.block(cfg["feats"], p0.set_table, p1.set_table, cfg["blocks"][0])
+    xr = cfg["feats"]
+    for blk in cfg["blocks"]:
+        xr = ref.block(xr, p0.set_table, p1.set_table, blk)
     cpu_s = time.perf_counter() - t0
-    cpu = {"value": n / cpu_s, "unit": "voxels/s", "cores": cores, "kind": "oracle",
-           "sample": "the whole frame (%d voxels): both partitions + the first block, one pass, %.1f s" % (n, cpu_s)}
+    cpu = {"value": n * nb / cpu_s, "unit": "voxels/s", "cores": cores, "kind": "oracle",
+           "sample": "the whole frame (%d voxels): both partitions + all %d blocks, one pass, %.1f s wall"
+                     % (n, nb, cpu_s)}
 
     print(json.dumps({
         "metric": METRIC, "value": value, "unit": "voxels/s", "n_gpus": world, "steps": args.steps,
