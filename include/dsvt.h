@@ -111,6 +111,39 @@ int dsvt_partition(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batc
                    int32_t* win_setoff);
 
 /*
+ * dsvt_partition without any allocation.  (The paper has no counterpart: this is a deployment
+ * variant of dsvt_partition, computing exactly the same table.)
+ *
+ * For callers that may not allocate device memory: a perception loop whose memory was fixed at
+ * start-up, a host framework whose allocator owns the device, a plug-in that only receives a
+ * stream and buffers.  Such callers cannot use dsvt_create, which reserves its workspace with
+ * cudaMalloc.  Here the workspace (sort buffers, digit histograms, per-window arrays) is a fixed
+ * array inside the library image, about 1.9 MB, which every GPU that loads the library holds until
+ * the process exits.  The call makes no cudaMalloc / cudaFree and uses no allocating library.
+ *
+ *   cuda_stream   cudaStream_t of the CURRENT device (NULL = legacy default stream); kernels are
+ *                 enqueued there and the call does not synchronise.
+ *   coords, n, batch, grid, window, set_size, axis, set_table, cap_sets, num_sets, set_rowoff
+ *                 exactly as for dsvt_partition (device pointers owned by the caller).
+ *   status_bits   optional device int32: receives the DSVT_STATUS_* bits of this call.
+ *   cuda_error    optional HOST int32: the cudaError_t behind a DSVT_ERR_CUDA return.
+ *
+ * Limits: n <= DSVT_NOALLOC_MAX_VOXELS and at most DSVT_NOALLOC_MAX_WINDOWS windows, otherwise
+ * DSVT_ERR_CAPACITY is returned and nothing is launched.
+ * The first call on each device looks up the array's device address (once, with that device
+ * current); make that first call before starting any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's contents (the call
+ * clears what has to start at zero): two calls whose kernels overlap on the GPU -- different
+ * streams, or threads -- race on it.  Serialise them on one stream.
+ */
+#define DSVT_NOALLOC_MAX_VOXELS 65536
+#define DSVT_NOALLOC_MAX_WINDOWS 65536
+int dsvt_partition_noalloc(void* cuda_stream, const int32_t* coords, int32_t n, int32_t batch, const int32_t grid[3],
+                           const int32_t window[3], int32_t set_size, int32_t axis, int32_t* set_table,
+                           int32_t cap_sets, int32_t* num_sets, int32_t* set_rowoff, int32_t* status_bits,
+                           int32_t* cuda_error);
+
+/*
  * Batched set attention: Eq. 4 (INDEX gather of each set's members) followed by the multi-head
  * self attention of Eq. 5 inside every set, output projection, and scatter back to voxels.
  * Slot k of a table row is a duplicate, and is masked as a key and not written back, iff k > 0 and

@@ -23,7 +23,7 @@ STATUS_BAD_COORD, STATUS_TABLE_OVERFLOW, STATUS_BAD_INDEX, STATUS_DUPLICATE_CELL
 
 EXPORTS = [
     "dsvt_create", "dsvt_destroy", "dsvt_status_sync", "dsvt_last_cuda_error", "dsvt_error_string",
-    "dsvt_launch_count", "dsvt_partition", "dsvt_set_attention", "dsvt_layer", "dsvt_block", "dsvt_pool",
+    "dsvt_launch_count", "dsvt_partition", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_layer", "dsvt_block", "dsvt_pool",
 ]
 
 _lib = None
@@ -67,6 +67,7 @@ def load():
     lib.dsvt_launch_count.argtypes = [vp]
     lib.dsvt_launch_count.restype = i64
     lib.dsvt_partition.argtypes = [vp, vp, i32, i32, p3, p3, i32, i32, vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.dsvt_partition_noalloc.argtypes = [vp, vp, i32, i32, p3, p3, i32, i32, vp, i32, vp, vp, vp, C.POINTER(i32)]
     lib.dsvt_set_attention.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, i32, vp, vp, vp, vp, i32, vp, C.c_int, vp]
     lib.dsvt_layer.argtypes = [vp, vp, i32, vp, i32, vp, vp, C.POINTER(LayerParams), vp]
     lib.dsvt_block.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, i32, vp, vp, C.POINTER(LayerParams), vp]
@@ -133,6 +134,31 @@ class SetTable:
     win_start: Optional[torch.Tensor] = None
     win_count: Optional[torch.Tensor] = None
     win_setoff: Optional[torch.Tensor] = None
+
+
+NOALLOC_MAX_VOXELS = 65536
+NOALLOC_MAX_WINDOWS = 65536
+
+
+def partition_noalloc(coords: torch.Tensor, batch: int, grid, window, set_size: int, axis: int, out: SetTable,
+                      status_bits: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> SetTable:
+    """dsvt_partition_noalloc: the set partition for callers that must not allocate device memory.
+
+    Needs no Context.  `out` (and `status_bits`, a device int32) are the caller's own buffers; the
+    library's workspace is a fixed array inside the shared library, so at most NOALLOC_MAX_VOXELS voxels
+    and NOALLOC_MAX_WINDOWS windows fit.  Calls that overlap on the GPU race on that array.
+    """
+    lib = load()
+    st = stream if stream is not None else torch.cuda.current_stream(coords.device)
+    err = C.c_int32(0)
+    with torch.cuda.device(coords.device):
+        rc = lib.dsvt_partition_noalloc(C.c_void_p(st.cuda_stream), _ptr(coords), int(coords.shape[0]), int(batch),
+                                        _i3(grid), _i3(window), int(set_size), int(axis), _ptr(out.set_table),
+                                        out.cap_sets, _ptr(out.num_sets), _ptr(out.set_rowoff), _ptr(status_bits),
+                                        C.byref(err))
+    if rc != OK:
+        raise DsvtError(rc, "dsvt_partition_noalloc", int(err.value))
+    return out
 
 
 class Context:
