@@ -265,8 +265,7 @@ def run_ours(args):
     print(json.dumps({
         "metric": METRIC, "value": value, "unit": "voxels/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16 weights x fp32 activations, fp32 accumulate (FMA pipes)"
-        if cfg["precision"] == "bf16" else "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "bf16" if cfg["precision"] == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": "config %d (%s): %d voxels, grid %s, window %s, set size %d, C=%d, %d blocks x 2 layers"
                    % (args.config, cfg["name"], n, cfg["grid"], cfg["window"], cfg["set_size"], C, nb),
                    "l2": "L2 flushed by a %d MiB write before every step" % (L2_FLUSH_BYTES >> 20),

@@ -73,6 +73,7 @@ int run_layer(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* table, in
   a.x = x; a.y = y; a.n = n; a.table = table; a.num_sets = num_sets; a.rowoff = rowoff; a.cap_sets = cap_sets;
   a.p = p;
   a.attention_only = attention_only ? 1 : 0;
+  if (dsvt_layer_tc_supported(a)) return dsvt_launch_layer_tc(ctx, a);
   return dsvt_launch_layer_fma(ctx, a);
 }
 

@@ -74,3 +74,6 @@ struct dsvt_fused_args {
   int32_t attention_only;  // 1: y = attention output (no residual, LN, MLP)
 };
 int dsvt_launch_layer_fma(dsvt_ctx* ctx, const dsvt_fused_args& a);
+// tcgen05 path: bfloat16 weights, C in {64, 128, 192}, head dim in {16, 24, 32}, set size <= 96.
+bool dsvt_layer_tc_supported(const dsvt_fused_args& a);
+int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a);
