@@ -2,12 +2,20 @@
 // accumulation: gather (Eq. 4) -> QKV projection -> per-set multi-head attention (Eq. 5) -> output
 // projection -> residual + LayerNorm -> MLP with GELU -> residual + LayerNorm -> scatter (App. B.1.1).
 //
-// One persistent CTA per SM walks over tiles of up to 128 distinct voxel rows made of whole sets.
-// Roles: warps 0-7 compute (gather, TMEM epilogues, attention), warp 8 streams the weight matrices
-// through a shared-memory ring with TMA (no cluster multicast), warp 9 allocates TMEM and issues the
-// tcgen05.mma instructions.  The four projections of a layer are seven "chunks" of N = C output
-// columns (K, V, Q, O, MLP-1a, MLP-1b, MLP-2); chunk g accumulates in TMEM buffer g & 1, so the
-// tensor pipe works on one chunk while the compute warps drain the previous one.
+// One persistent CTA per SM.  The distinct voxel rows of the frame are cut into one contiguous
+// segment per CTA (equal row counts, cut at set boundaries); inside its segment a CTA packs whole
+// sets greedily into tiles of at most 128 rows (the UMMA M).
+//
+// Roles: warps 0-7 compute (gather, TMEM epilogues, attention); warp 8 is the scheduler and TMA
+// producer: it finds the next tile (binary searches in the row-offset array), publishes it through a
+// two-entry ring, and streams the layer's weight matrices through a shared-memory ring with TMA (no
+// cluster multicast); warp 9 allocates TMEM and issues the tcgen05.mma instructions.
+//
+// The four projections of a layer are chunks of at most 192 output columns (K, V, Q, O, MLP-1 in
+// pieces of 128 or 64 hidden columns, MLP-2).  Accumulators alternate between two TMEM buffers so the
+// tensor pipe works on one chunk while the compute warps drain the previous one.  The fp32 residual
+// stream never leaves the chip inside a layer: x is staged in shared memory for the first residual,
+// and x1 = LN1(x + attention) is parked in spare TMEM columns until the second residual.
 //
 // Every operand tile in shared memory uses the K-major 128-byte-swizzled layout that tcgen05.mma and
 // TMA share: 64 bf16 columns per 128-byte row, 8-row groups of 1024 bytes, 16-byte chunk index XORed
@@ -16,7 +24,7 @@
 // into the A operand of the output projection.
 //
 // Every wait on an mbarrier is bounded; a wait that gives up raises DSVT_STATUS_TIMEOUT and all roles
-// leave the tile loop together.
+// leave their loops.
 #include <cuda.h>
 
 #include "dsvt_common.cuh"
@@ -25,25 +33,25 @@ namespace {
 
 constexpr int kTM = 128;               // tile rows = UMMA M
 constexpr int kComputeThreads = 256;   // warps 0-7
-constexpr int kThreads = 320;          // + TMA warp + MMA warp
+constexpr int kThreads = 320;          // + scheduler/TMA warp + MMA warp
 constexpr int kStages = 3;             // weight ring depth
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxPolls = 1 << 20;
 
 struct TcGeom {
-  int C, hidden, heads, tau, TMn;
-  int nkb;      // C / 64: K blocks of a C-deep contraction
-  int nkb_h;    // hidden / 64
-  int n_f1;     // hidden / C: MLP-1 chunks
-  uint32_t stage_bytes;  // C * 128
+  int hidden, heads, tau;
+  int nkb_h;    // hidden / 64: K blocks of the MLP-2 contraction
+  int NF;       // MLP-1 chunk width (128 or 64)
+  int n_f1;     // hidden / NF
+  int mode;     // 0: attention only, 1: attention + residual + LN1, 2: full layer
   uint32_t off_a, off_kv, off_stage, off_misc;  // byte offsets from the 1024-aligned base
 };
 
 struct Misc {  // small shared state behind the big regions
-  unsigned long long full[kStages], empty[kStages], acc_full[2], acc_free[2], a_ready;
+  unsigned long long full[kStages], empty[kStages], acc_full[2], acc_free[2], a_ready, sched_full[2], sched_empty[2];
   uint32_t tmem_base;
   int abort_flag;
-  int tile[4];  // s_lo, nsets, base row, rows
+  int tile[2][4];  // ring of tiles: first set, number of sets (< 0: no more tiles), first row, rows
   int rowvox[kTM];
   int set_lo[kTM + 1];
   float red[2][2][kTM];  // [exchange][column half][row]
@@ -125,6 +133,24 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
+        "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])),
+        "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])),
+        "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])),
+        "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])),
+        "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -166,21 +192,17 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTM >> 4) << 24);
 }
 
-__device__ __forceinline__ float gelu_erf(float t) { return 0.5f * t * (1.0f + erff(t * 0.70710678118654752440f)); }
-
-// Sets whose first distinct row lies in [t*TMn, (t+1)*TMn).  Same answer for every role.
-__device__ __forceinline__ bool tile_range(const int32_t* __restrict__ rowoff, int S, int t, int TMn, int* out) {
-  const int lo_row = t * TMn, hi_row = lo_row + TMn;
-  int lo = 0, hi = S;
-  while (lo < hi) { const int m = (lo + hi) >> 1; if (rowoff[m] < lo_row) lo = m + 1; else hi = m; }
-  const int s_lo = lo;
-  hi = S;
-  while (lo < hi) { const int m = (lo + hi) >> 1; if (rowoff[m] < hi_row) lo = m + 1; else hi = m; }
-  out[0] = s_lo;
-  out[1] = lo - s_lo;
-  out[2] = rowoff[s_lo];
-  out[3] = rowoff[lo] - rowoff[s_lo];
-  return out[1] > 0 && out[1] <= kTM && out[3] > 0 && out[3] <= kTM;
+// gelu(t) = t/2 (1 + erf(t / sqrt 2)) with the five-term rational approximation of erf
+// (absolute error below 2e-7, far under the bfloat16 rounding applied to the result).
+__device__ __forceinline__ float gelu_fast(float t) {
+  const float z = fabsf(t) * 0.70710678118654752440f;
+  const float k = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
+  float poly = fmaf(1.061405429f, k, -1.453152027f);
+  poly = fmaf(poly, k, 1.421413741f);
+  poly = fmaf(poly, k, -0.284496736f);
+  poly = fmaf(poly, k, 0.254829592f);
+  const float erf_abs = 1.0f - poly * k * __expf(-z * z);
+  return 0.5f * t * (1.0f + copysignf(erf_abs, t));
 }
 
 struct TcMaps {
@@ -262,12 +284,14 @@ __device__ __forceinline__ void attend_tile(uint32_t a_base, uint32_t k_base, ui
 #pragma unroll
       for (int kk = 0; kk < (NT + 1) / 2; ++kk) {
         if (2 * kk < ntu) {
+          constexpr int kLast = NT - 1;
+          const int j1 = (2 * kk + 1 <= kLast) ? 2 * kk + 1 : kLast;
+          const bool two = (2 * kk + 1 <= kLast);
           uint32_t pa[4];
           pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
           pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-          const bool two = (2 * kk + 1 < NT);
-          pa[2] = two ? pack_bf16(s[(2 * kk + 1 < NT) ? 2 * kk + 1 : 0][0], s[(2 * kk + 1 < NT) ? 2 * kk + 1 : 0][1]) : 0u;
-          pa[3] = two ? pack_bf16(s[(2 * kk + 1 < NT) ? 2 * kk + 1 : 0][2], s[(2 * kk + 1 < NT) ? 2 * kk + 1 : 0][3]) : 0u;
+          pa[2] = two ? pack_bf16(s[j1][0], s[j1][1]) : 0u;
+          pa[3] = two ? pack_bf16(s[j1][2], s[j1][3]) : 0u;
           const int row = min(r0 + 16 * kk + (lane & 15), kTM - 1);
 #pragma unroll
           for (int dn = 0; dn < DC; ++dn) {
@@ -293,12 +317,27 @@ __device__ __forceinline__ void attend_tile(uint32_t a_base, uint32_t k_base, ui
   }
 }
 
+// fp32 row staging in the K/V region: row r, 16-byte chunk c4 of C/4, rotated by the row so that both
+// the warp-per-row pattern (global side) and the thread-per-row pattern (TMEM side) are conflict-free.
+template <int C>
+__device__ __forceinline__ uint32_t stage_off(int r, int c4) {
+  constexpr int NCH = C / 4;
+  int idx = c4 + (r % NCH);
+  if (idx >= NCH) idx -= NCH;
+  return (uint32_t)(r * (C * 4) + (idx << 4));
+}
+
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int D, int NT>
+template <int C, int D, int NT>
 __global__ void __launch_bounds__(kThreads, 1)
 layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps, int32_t* __restrict__ status) {
+  constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
+  constexpr int HALF = C / 2;        // epilogue columns per thread for a C-wide chunk
+  constexpr uint32_t COL_B = C;      // second accumulator buffer
+  constexpr uint32_t COL_PARK = kTmemCols - C;  // parked fp32 x1
+  constexpr uint32_t STAGE_BYTES = C * 128;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -307,19 +346,22 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
   Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
   const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int C = g.C;
   const dsvt_layer_params& p = a.p;
   volatile int* abort_flag = &mi->abort_flag;
 
   const int S = min(*a.num_sets, a.cap_sets);
   const int R = S > 0 ? a.rowoff[S] : 0;
-  const int num_tiles = (R + g.TMn - 1) / g.TMn;
-  const bool mlp = g.hidden > 0 && !a.attention_only;
+  const bool mlp = g.mode == 2;
   const int n_chunks = 4 + (mlp ? g.n_f1 + 1 : 0);
 
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(&mi->full[i], 1); mbar_init(&mi->empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&mi->acc_full[i], 1); mbar_init(&mi->acc_free[i], kComputeThreads); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&mi->acc_full[i], 1);
+      mbar_init(&mi->acc_free[i], kComputeThreads);
+      mbar_init(&mi->sched_full[i], 1);
+      mbar_init(&mi->sched_empty[i], kComputeThreads + 1);
+    }
     mbar_init(&mi->a_ready, kComputeThreads);
     mi->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -335,24 +377,54 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
   const uint32_t tmem = mi->tmem_base;
 
   if (warp == 8) {
-    // ================= TMA producer: the layer's weights, chunk by chunk, K block by K block ==========
+    // ================= scheduler + TMA producer =====================================================
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      for (int t = blockIdx.x; t < num_tiles && !*abort_flag; t += gridDim.x) {
-        int info[4];
-        if (!tile_range(a.rowoff, S, t, g.TMn, info)) continue;
+      // this CTA's segment: the sets whose first row lies in [b R / G, (b + 1) R / G)
+      const int row_lo = (int)(((long long)blockIdx.x * R) / gridDim.x);
+      const int row_hi = (int)(((long long)(blockIdx.x + 1) * R) / gridDim.x);
+      int lo = 0, hi = S;
+      while (lo < hi) { const int m = (lo + hi) >> 1; if (a.rowoff[m] < row_lo) lo = m + 1; else hi = m; }
+      int s = lo;
+      hi = S;
+      while (lo < hi) { const int m = (lo + hi) >> 1; if (a.rowoff[m] < row_hi) lo = m + 1; else hi = m; }
+      const int s_end = lo;
+      int stage = 0, slot = 0;
+      uint32_t phase = 0, sphase = 0;
+      for (;;) {
+        if (!mbar_wait(&mi->sched_empty[slot], sphase ^ 1u, abort_flag)) break;
+        int ns = -1, base = 0, rows = 0;
+        while (s < s_end) {  // next tile: as many whole sets as fit in 128 rows
+          base = a.rowoff[s];
+          const int first = a.rowoff[s + 1] - base;
+          if (first <= 0 || first > kTM) {  // offsets that do not describe a set: skip it
+            atomicOr(status, DSVT_STATUS_BAD_INDEX);
+            ++s;
+            continue;
+          }
+          int l2 = s + 1, h2 = s_end;  // last e in (s, s_end] with rowoff[e] - base <= 128
+          while (l2 < h2) { const int m = (l2 + h2 + 1) >> 1; if (a.rowoff[m] - base <= kTM) l2 = m; else h2 = m - 1; }
+          ns = l2 - s;
+          rows = a.rowoff[l2] - base;
+          break;
+        }
+        mi->tile[slot][0] = s; mi->tile[slot][1] = ns; mi->tile[slot][2] = base; mi->tile[slot][3] = rows;
+        mbar_arrive(&mi->sched_full[slot]);
+        if (++slot == 2) { slot = 0; sphase ^= 1u; }
+        if (ns < 0) break;
+        s += ns;
+        // the layer's weights for this tile, chunk by chunk, K block by K block
         for (int c = 0; c < n_chunks; ++c) {
           const CUtensorMap* map;
           int row0, nkb;
-          if (c < 3) { map = &maps.qkv; row0 = (c == 0 ? 1 : c == 1 ? 2 : 0) * C; nkb = g.nkb; }   // K, V, Q
-          else if (c == 3) { map = &maps.o; row0 = 0; nkb = g.nkb; }
-          else if (c < 4 + g.n_f1) { map = &maps.w1; row0 = (c - 4) * C; nkb = g.nkb; }
+          uint32_t bytes = STAGE_BYTES;
+          if (c < 3) { map = &maps.qkv; row0 = (c == 0 ? 1 : c == 1 ? 2 : 0) * C; nkb = NKB; }   // K, V, Q
+          else if (c == 3) { map = &maps.o; row0 = 0; nkb = NKB; }
+          else if (c < 4 + g.n_f1) { map = &maps.w1; row0 = (c - 4) * g.NF; nkb = NKB; bytes = (uint32_t)g.NF * 128u; }
           else { map = &maps.w2; row0 = 0; nkb = g.nkb_h; }
           for (int kb = 0; kb < nkb; ++kb) {
             if (!mbar_wait(&mi->empty[stage], phase ^ 1u, abort_flag)) goto producer_done;
-            mbar_expect_tx(&mi->full[stage], g.stage_bytes);
-            tma_load_2d(st_base + stage * g.stage_bytes, map, kb * 64, row0, &mi->full[stage]);
+            mbar_expect_tx(&mi->full[stage], bytes);
+            tma_load_2d(st_base + stage * STAGE_BYTES, map, kb * 64, row0, &mi->full[stage]);
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
@@ -363,37 +435,45 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
   } else if (warp == 9) {
     // ================= MMA issuer ====================================================================
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc(C);
-      int stage = 0;
-      uint32_t phase = 0, a_phase = 0;
-      uint32_t chunk_seq = 0;  // running chunk number: TMEM buffer = chunk_seq & 1
-      for (int t = blockIdx.x; t < num_tiles && !*abort_flag; t += gridDim.x) {
-        int info[4];
-        if (!tile_range(a.rowoff, S, t, g.TMn, info)) continue;
-        for (int c = 0; c < n_chunks; ++c, ++chunk_seq) {
+      int stage = 0, slot = 0;
+      uint32_t phase = 0, a_phase = 0, sphase = 0;
+      uint32_t uses[2] = {0u, 0u};  // how often each accumulator barrier pair has been used
+      for (;;) {
+        if (!mbar_wait(&mi->sched_full[slot], sphase, abort_flag)) break;
+        const int ns = mi->tile[slot][1];
+        mbar_arrive(&mi->sched_empty[slot]);
+        if (++slot == 2) { slot = 0; sphase ^= 1u; }
+        if (ns < 0) break;
+        for (int c = 0; c < n_chunks; ++c) {
           // a fresh A operand: X (chunks 0-2), attention output (3), x1 (4..), MLP hidden (last)
           if (c == 0 || c == 3 || c == 4 || c == 4 + g.n_f1) {
             if (!mbar_wait(&mi->a_ready, a_phase, abort_flag)) goto mma_done;
             a_phase ^= 1u;
           }
-          const uint32_t buf = chunk_seq & 1u;
-          if (!mbar_wait(&mi->acc_free[buf], ((chunk_seq >> 1) & 1u) ^ 1u, abort_flag)) goto mma_done;
+          // accumulator placement: K -> A, V -> B, Q -> A, O -> A, MLP-1 piece i -> i & 1, MLP-2 -> A
+          uint32_t bar, col, n;
+          if (c < 4) { bar = (c == 1) ? 1u : 0u; col = (c == 1) ? COL_B : 0u; n = C; }
+          else if (c < 4 + g.n_f1) { bar = (uint32_t)(c - 4) & 1u; col = bar * (uint32_t)g.NF; n = (uint32_t)g.NF; }
+          else { bar = (uint32_t)g.n_f1 & 1u; col = 0u; n = C; }
+          if (!mbar_wait(&mi->acc_free[bar], (uses[bar] & 1u) ^ 1u, abort_flag)) goto mma_done;
+          ++uses[bar];
           tc_fence_after();
           const bool last = mlp && c == 4 + g.n_f1;
           const uint32_t abase = last ? kv_base : a_base;
-          const int nkb = last ? g.nkb_h : g.nkb;
-          const uint32_t d_tmem = tmem + buf * 256u;
+          const int nkb = last ? g.nkb_h : NKB;
+          const uint32_t idesc = umma_idesc((int)n);
+          const uint32_t d_tmem = tmem + col;
           for (int kb = 0; kb < nkb; ++kb) {
             if (!mbar_wait(&mi->full[stage], phase, abort_flag)) goto mma_done;
             tc_fence_after();
-            const uint32_t sa = abase + kb * (kTM * 128), sb = st_base + stage * g.stage_bytes;
+            const uint32_t sa = abase + kb * (kTM * 128), sb = st_base + stage * STAGE_BYTES;
 #pragma unroll
             for (int k4 = 0; k4 < 4; ++k4)
               umma_bf16(d_tmem, umma_desc(sa + k4 * 32), umma_desc(sb + k4 * 32), idesc, (kb | k4) != 0 ? 1u : 0u);
             umma_commit(&mi->empty[stage]);  // frees the weight stage once these MMAs have read it
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
-          umma_commit(&mi->acc_full[buf]);
+          umma_commit(&mi->acc_full[bar]);
         }
       }
     mma_done:;
@@ -403,23 +483,42 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
     // ================= compute warps =================================================================
     const int row = 32 * (warp & 3) + lane;  // TMEM lane owned in the epilogues
     const int hh = warp >> 2;                // column half owned in the epilogues
-    const int half = C >> 1;
     const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
-    uint32_t chunk_seq = 0;
+    constexpr int C4 = C / 4;
+    uint32_t uses[2] = {0u, 0u};
+    int slot = 0;
+    uint32_t sphase = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+    auto acc_wait = [&](uint32_t bar) {
+      ok = mbar_wait(&mi->acc_full[bar], uses[bar] & 1u, abort_flag) && ok;
+      ++uses[bar];
+      tc_fence_after();
+    };
+    auto acc_release = [&](uint32_t bar) {
+      tc_fence_before();
+      mbar_arrive(&mi->acc_free[bar]);
+    };
+    // normalised fp32 rows staged in the K/V region -> coalesced global rows
+    auto store_rows = [&](int rows) {
       compute_sync();
-      if (*abort_flag) break;
-      if (tid == 0) {
-        int info[4];
-        const bool valid = tile_range(a.rowoff, S, t, g.TMn, info);
-        mi->tile[0] = info[0]; mi->tile[1] = valid ? info[1] : 0; mi->tile[2] = info[2]; mi->tile[3] = info[3];
-        if (!valid && info[1] > 0) atomicOr(status, DSVT_STATUS_BAD_INDEX);
+      for (int r = warp; r < rows; r += 8) {
+        const int v = mi->rowvox[r];
+        if (v < 0) continue;
+        for (int c4 = lane; c4 < C4; c4 += 32)
+          reinterpret_cast<float4*>(a.y + (size_t)v * C)[c4] =
+              *reinterpret_cast<const float4*>(sm + g.off_kv + stage_off<C>(r, c4));
       }
+    };
+    for (;;) {
+      ok = mbar_wait(&mi->sched_full[slot], sphase, abort_flag) && ok;
+      compute_sync();  // also orders the previous tile's last shared-memory reads before this tile's writes
+      if (*abort_flag) break;
+      const int s_lo = mi->tile[slot][0], nsets = mi->tile[slot][1], base = mi->tile[slot][2], rows = mi->tile[slot][3];
+      mbar_arrive(&mi->sched_empty[slot]);
+      if (++slot == 2) { slot = 0; sphase ^= 1u; }
+      if (nsets < 0) break;
       if (tid < kTM) mi->rowvox[tid] = -1;
       compute_sync();
-      const int s_lo = mi->tile[0], nsets = mi->tile[1], base = mi->tile[2], rows = mi->tile[3];
-      if (nsets <= 0) continue;
       // ---- distinct slots of each set -> tile rows (Eq. 4) ----
       for (int si = warp; si < nsets; si += 8) {
         const int s = s_lo + si;
@@ -433,14 +532,14 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
           if (k < g.tau) { v = trow[k]; uniq = (k == 0) || (v != trow[k - 1]); }
           const unsigned bal = __ballot_sync(0xffffffffu, uniq);
           const int pos = cnt + __popc(bal & ((1u << lane) - 1u));
-          if (uniq && pos < cap && lb + pos < kTM) {
+          if (uniq && pos < cap && lb >= 0 && lb + pos < kTM) {
             if (v < 0 || v >= a.n) { atomicOr(status, DSVT_STATUS_BAD_INDEX); v = -1; }
             mi->rowvox[lb + pos] = v;
           }
           cnt += __popc(bal);
         }
         if (lane == 0) {
-          mi->set_lo[si] = lb;
+          mi->set_lo[si] = min(max(lb, 0), kTM);
           if (cnt != cap) atomicOr(status, DSVT_STATUS_BAD_INDEX);
         }
       }
@@ -462,18 +561,17 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       fence_proxy_async();
       mbar_arrive(&mi->a_ready);  // X is in place
 
-      const int my_v = row < rows ? mi->rowvox[row] : -1;
       // ---- chunks 0..2: K, V, Q epilogues: + bias, to bf16, into the operand layout ----
-      for (int c = 0; c < 3; ++c, ++chunk_seq) {
-        const uint32_t buf = chunk_seq & 1u;
-        ok = mbar_wait(&mi->acc_full[buf], (chunk_seq >> 1) & 1u, abort_flag) && ok;
-        tc_fence_after();
+      for (int c = 0; c < 3; ++c) {
+        const uint32_t bar = (c == 1) ? 1u : 0u;
+        acc_wait(bar);
         const float* bias = p.b_qkv ? p.b_qkv + (c == 0 ? 1 : c == 1 ? 2 : 0) * C : nullptr;
-        unsigned char* dst = sm + (c == 2 ? g.off_a : g.off_kv + (uint32_t)c * (uint32_t)g.nkb * (kTM * 128));
-        for (int j0 = 0; j0 < half; j0 += 32) {
+        unsigned char* dst = sm + (c == 2 ? g.off_a : g.off_kv + (uint32_t)c * (NKB * kTM * 128));
+#pragma unroll 1
+        for (int j0 = 0; j0 < HALF; j0 += 32) {
           float v[32];
-          tmem_ld32(tmem + lane_addr + buf * 256u + hh * half + j0, v);
-          const int col = hh * half + j0;
+          tmem_ld32(tmem + lane_addr + (c == 1 ? COL_B : 0u) + hh * HALF + j0, v);
+          const int col = hh * HALF + j0;
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             float b[8];
@@ -483,211 +581,154 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
                 make_uint4(pack_bf16(b[0], b[1]), pack_bf16(b[2], b[3]), pack_bf16(b[4], b[5]), pack_bf16(b[6], b[7]));
           }
         }
-        tc_fence_before();
-        mbar_arrive(&mi->acc_free[buf]);
+        acc_release(bar);
       }
       compute_sync();
       // ---- attention inside each set ----
-      attend_tile<D, NT>(a_base, kv_base, kv_base + (uint32_t)g.nkb * (kTM * 128), mi->set_lo, nsets, g.heads, warp, lane);
+      attend_tile<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->set_lo, nsets, g.heads, warp, lane);
       fence_proxy_async();
       mbar_arrive(&mi->a_ready);  // attention output is the A operand of the output projection
-
-      // ---- chunk 3: output projection epilogue ----
+      compute_sync();             // every warp is done with K and V: their region becomes fp32 staging
+      if (g.mode != 0) {
+        // x rows (fp32) for the first residual, coalesced
+        for (int r = warp; r < rows; r += 8) {
+          const int v = mi->rowvox[r];
+          for (int c4 = lane; c4 < C4; c4 += 32) {
+            float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (v >= 0) f = __ldg(reinterpret_cast<const float4*>(a.x + (size_t)v * C) + c4);
+            *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(r, c4)) = f;
+          }
+        }
+        compute_sync();
+      }
+      // ---- chunk 3: output projection epilogue: Z + b_o (+ x, LayerNorm) ----
       {
-        const uint32_t buf = chunk_seq & 1u;
-        ok = mbar_wait(&mi->acc_full[buf], (chunk_seq >> 1) & 1u, abort_flag) && ok;
-        tc_fence_after();
-        ++chunk_seq;
-        const uint32_t tsrc = tmem + lane_addr + buf * 256u + hh * half;
-        if (a.attention_only) {
-          for (int j0 = 0; j0 < half; j0 += 32) {
-            float v[32];
-            tmem_ld32(tsrc + j0, v);
-            const int col = hh * half + j0;
-            if (my_v >= 0) {
-#pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                float4 o4;
-                o4.x = v[4 * q] + (p.b_o ? __ldg(p.b_o + col + 4 * q) : 0.f);
-                o4.y = v[4 * q + 1] + (p.b_o ? __ldg(p.b_o + col + 4 * q + 1) : 0.f);
-                o4.z = v[4 * q + 2] + (p.b_o ? __ldg(p.b_o + col + 4 * q + 2) : 0.f);
-                o4.w = v[4 * q + 3] + (p.b_o ? __ldg(p.b_o + col + 4 * q + 3) : 0.f);
-                *reinterpret_cast<float4*>(a.y + (size_t)my_v * C + col + 4 * q) = o4;
-              }
-            }
-          }
-          tc_fence_before();
-          mbar_arrive(&mi->acc_free[buf]);
-          continue;
-        }
-        // x1 = LN1(x + Z): pass 1 sums, pass 2 centred squares, pass 3 normalise (TMEM is re-read)
+        acc_wait(0u);
+        float t[HALF];
         float sum = 0.f;
-        for (int j0 = 0; j0 < half; j0 += 32) {
+#pragma unroll
+        for (int j = 0; j < HALF / 32; ++j) {
           float v[32];
-          tmem_ld32(tsrc + j0, v);
-          const int col = hh * half + j0;
+          tmem_ld32(tmem + lane_addr + hh * HALF + 32 * j, v);
+          const int col = hh * HALF + 32 * j;
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (my_v >= 0) x4 = __ldg(reinterpret_cast<const float4*>(a.x + (size_t)my_v * C + col + 4 * q));
-            sum += v[4 * q] + x4.x + v[4 * q + 1] + x4.y + v[4 * q + 2] + x4.z + v[4 * q + 3] + x4.w;
-            if (p.b_o) sum += __ldg(p.b_o + col + 4 * q) + __ldg(p.b_o + col + 4 * q + 1) + __ldg(p.b_o + col + 4 * q + 2) +
-                              __ldg(p.b_o + col + 4 * q + 3);
-          }
-        }
-        mi->red[0][hh][row] = sum;
-        compute_sync();
-        const float mean = (mi->red[0][0][row] + mi->red[0][1][row]) / (float)C;
-        float sq = 0.f;
-        if (p.ln1_g) {
-          for (int j0 = 0; j0 < half; j0 += 32) {
-            float v[32];
-            tmem_ld32(tsrc + j0, v);
-            const int col = hh * half + j0;
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (my_v >= 0) x4 = __ldg(reinterpret_cast<const float4*>(a.x + (size_t)my_v * C + col + 4 * q));
-              const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float tt = v[4 * q + e] + xs[e] + (p.b_o ? __ldg(p.b_o + col + 4 * q + e) : 0.f) - mean;
-                sq += tt * tt;
-              }
-            }
-          }
-        }
-        mi->red[1][hh][row] = sq;
-        compute_sync();
-        const float inv = p.ln1_g ? rsqrtf((mi->red[1][0][row] + mi->red[1][1][row]) / (float)C + p.ln_eps) : 1.f;
-        for (int j0 = 0; j0 < half; j0 += 32) {
-          float v[32];
-          tmem_ld32(tsrc + j0, v);
-          const int col = hh * half + j0;
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (my_v >= 0) x4 = __ldg(reinterpret_cast<const float4*>(a.x + (size_t)my_v * C + col + 4 * q));
+            if (g.mode != 0 && row < rows)
+              x4 = *reinterpret_cast<const float4*>(sm + g.off_kv + stage_off<C>(row, (col >> 2) + q));
             const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const int cc = col + 4 * q + e;
-              float tt = v[4 * q + e] + xs[e] + (p.b_o ? __ldg(p.b_o + cc) : 0.f);
-              if (p.ln1_g) tt = (tt - mean) * inv * __ldg(p.ln1_g + cc) + (p.ln1_b ? __ldg(p.ln1_b + cc) : 0.f);
-              v[4 * q + e] = tt;
+              const float tt = v[4 * q + e] + xs[e] + (p.b_o ? __ldg(p.b_o + col + 4 * q + e) : 0.f);
+              t[32 * j + 4 * q + e] = tt;
+              sum += tt;
             }
-            // fp32 x1 parks in the voxel's output row (also the final result when there is no MLP)
-            if (my_v >= 0)
-              *reinterpret_cast<float4*>(a.y + (size_t)my_v * C + col + 4 * q) =
-                  make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-          }
-          if (mlp) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-              *reinterpret_cast<uint4*>(sm + g.off_a + swz(row, (col >> 3) + q)) =
-                  make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
-                             pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
           }
         }
+        acc_release(0u);
+        if (g.mode != 0 && p.ln1_g) {
+          mi->red[0][hh][row] = sum;
+          compute_sync();
+          const float mean = (mi->red[0][0][row] + mi->red[0][1][row]) * (1.0f / (float)C);
+          float sq = 0.f;
+#pragma unroll
+          for (int i = 0; i < HALF; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
+          mi->red[1][hh][row] = sq;
+          compute_sync();
+          const float inv = rsqrtf((mi->red[1][0][row] + mi->red[1][1][row]) * (1.0f / (float)C) + p.ln_eps);
+#pragma unroll
+          for (int i = 0; i < HALF; ++i) {
+            const int cc = hh * HALF + i;
+            t[i] = t[i] * inv * __ldg(p.ln1_g + cc) + (p.ln1_b ? __ldg(p.ln1_b + cc) : 0.f);
+          }
+        }
+        if (!mlp) {
+          // final result of this call: stage it (the x staging is dead once every thread has its t)
+          compute_sync();
+#pragma unroll
+          for (int i4 = 0; i4 < HALF / 4; ++i4)
+            *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(row, hh * (HALF / 4) + i4)) =
+                make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
+          store_rows(rows);
+          continue;
+        }
+        // x1: bf16 A operand of MLP-1 in shared memory, fp32 copy parked in TMEM for the second residual
+#pragma unroll
+        for (int j = 0; j < HALF / 32; ++j) {
+          tmem_st32(tmem + lane_addr + COL_PARK + hh * HALF + 32 * j, &t[32 * j]);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4*>(sm + g.off_a + swz(row, ((hh * HALF + 32 * j) >> 3) + q)) =
+                make_uint4(pack_bf16(t[32 * j + 8 * q], t[32 * j + 8 * q + 1]), pack_bf16(t[32 * j + 8 * q + 2], t[32 * j + 8 * q + 3]),
+                           pack_bf16(t[32 * j + 8 * q + 4], t[32 * j + 8 * q + 5]), pack_bf16(t[32 * j + 8 * q + 6], t[32 * j + 8 * q + 7]));
+        }
         tc_fence_before();
-        mbar_arrive(&mi->acc_free[buf]);
-        if (!mlp) continue;
         fence_proxy_async();
         mbar_arrive(&mi->a_ready);  // x1 (bf16) is the A operand of MLP-1
       }
-      // ---- MLP-1 chunks: H = gelu(x1 W_1^T + b_1) as the A operand of MLP-2 ----
-      for (int c = 0; c < g.n_f1; ++c, ++chunk_seq) {
-        const uint32_t buf = chunk_seq & 1u;
-        ok = mbar_wait(&mi->acc_full[buf], (chunk_seq >> 1) & 1u, abort_flag) && ok;
-        tc_fence_after();
-        for (int j0 = 0; j0 < half; j0 += 32) {
+      // ---- MLP-1 pieces: H = gelu(x1 W_1^T + b_1) as the A operand of MLP-2 ----
+      for (int c = 0; c < g.n_f1; ++c) {
+        const uint32_t bar = (uint32_t)c & 1u;
+        acc_wait(bar);
+        const int hw = g.NF >> 1;  // columns per thread
+#pragma unroll 1
+        for (int j0 = 0; j0 < hw; j0 += 32) {
           float v[32];
-          tmem_ld32(tmem + lane_addr + buf * 256u + hh * half + j0, v);
-          const int col = c * C + hh * half + j0;  // hidden column
+          tmem_ld32(tmem + lane_addr + bar * (uint32_t)g.NF + hh * hw + j0, v);
+          const int col = c * g.NF + hh * hw + j0;  // hidden column
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             float b[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) b[e] = gelu_erf(v[8 * q + e] + (p.b_1 ? __ldg(p.b_1 + col + 8 * q + e) : 0.f));
+            for (int e = 0; e < 8; ++e) b[e] = gelu_fast(v[8 * q + e] + (p.b_1 ? __ldg(p.b_1 + col + 8 * q + e) : 0.f));
             *reinterpret_cast<uint4*>(sm + g.off_kv + swz(row, (col >> 3) + q)) =
                 make_uint4(pack_bf16(b[0], b[1]), pack_bf16(b[2], b[3]), pack_bf16(b[4], b[5]), pack_bf16(b[6], b[7]));
           }
         }
-        tc_fence_before();
-        mbar_arrive(&mi->acc_free[buf]);
+        acc_release(bar);
       }
       fence_proxy_async();
       mbar_arrive(&mi->a_ready);  // H is in place
       // ---- MLP-2 epilogue: y = LN2(x1 + M) ----
       {
-        const uint32_t buf = chunk_seq & 1u;
-        ok = mbar_wait(&mi->acc_full[buf], (chunk_seq >> 1) & 1u, abort_flag) && ok;
-        tc_fence_after();
-        ++chunk_seq;
-        const uint32_t tsrc = tmem + lane_addr + buf * 256u + hh * half;
+        const uint32_t bar = (uint32_t)g.n_f1 & 1u;
+        acc_wait(bar);
+        float t[HALF];
         float sum = 0.f;
-        for (int j0 = 0; j0 < half; j0 += 32) {
-          float v[32];
-          tmem_ld32(tsrc + j0, v);
-          const int col = hh * half + j0;
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (my_v >= 0) x4 = *reinterpret_cast<const float4*>(a.y + (size_t)my_v * C + col + 4 * q);
-            sum += v[4 * q] + x4.x + v[4 * q + 1] + x4.y + v[4 * q + 2] + x4.z + v[4 * q + 3] + x4.w;
-            if (p.b_2) sum += __ldg(p.b_2 + col + 4 * q) + __ldg(p.b_2 + col + 4 * q + 1) + __ldg(p.b_2 + col + 4 * q + 2) +
-                              __ldg(p.b_2 + col + 4 * q + 3);
-          }
+        for (int j = 0; j < HALF / 32; ++j) {
+          float v[32];
+          tmem_ld32(tmem + lane_addr + hh * HALF + 32 * j, v);
+          const int col = hh * HALF + 32 * j;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) t[32 * j + e] = v[e] + (p.b_2 ? __ldg(p.b_2 + col + e) : 0.f);
+          tmem_ld32(tmem + lane_addr + COL_PARK + hh * HALF + 32 * j, v);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) { t[32 * j + e] += v[e]; sum += t[32 * j + e]; }
         }
-        mi->red[0][hh][row] = sum;
-        compute_sync();
-        const float mean = (mi->red[0][0][row] + mi->red[0][1][row]) / (float)C;
-        float sq = 0.f;
+        acc_release(bar);
         if (p.ln2_g) {
-          for (int j0 = 0; j0 < half; j0 += 32) {
-            float v[32];
-            tmem_ld32(tsrc + j0, v);
-            const int col = hh * half + j0;
+          mi->red[0][hh][row] = sum;
+          compute_sync();
+          const float mean = (mi->red[0][0][row] + mi->red[0][1][row]) * (1.0f / (float)C);
+          float sq = 0.f;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (my_v >= 0) x4 = *reinterpret_cast<const float4*>(a.y + (size_t)my_v * C + col + 4 * q);
-              const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
+          for (int i = 0; i < HALF; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
+          mi->red[1][hh][row] = sq;
+          compute_sync();
+          const float inv = rsqrtf((mi->red[1][0][row] + mi->red[1][1][row]) * (1.0f / (float)C) + p.ln_eps);
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float tt = v[4 * q + e] + xs[e] + (p.b_2 ? __ldg(p.b_2 + col + 4 * q + e) : 0.f) - mean;
-                sq += tt * tt;
-              }
-            }
+          for (int i = 0; i < HALF; ++i) {
+            const int cc = hh * HALF + i;
+            t[i] = t[i] * inv * __ldg(p.ln2_g + cc) + (p.ln2_b ? __ldg(p.ln2_b + cc) : 0.f);
           }
         }
-        mi->red[1][hh][row] = sq;
-        compute_sync();
-        const float inv = p.ln2_g ? rsqrtf((mi->red[1][0][row] + mi->red[1][1][row]) / (float)C + p.ln_eps) : 1.f;
-        for (int j0 = 0; j0 < half; j0 += 32) {
-          float v[32];
-          tmem_ld32(tsrc + j0, v);
-          const int col = hh * half + j0;
-          if (my_v >= 0) {
+        // the MLP-2 MMAs have read H: its region takes the fp32 output rows
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              float* yp = a.y + (size_t)my_v * C + col + 4 * q;
-              const float4 x4 = *reinterpret_cast<const float4*>(yp);
-              const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
-              float o4[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int cc = col + 4 * q + e;
-                float tt = v[4 * q + e] + xs[e] + (p.b_2 ? __ldg(p.b_2 + cc) : 0.f);
-                if (p.ln2_g) tt = (tt - mean) * inv * __ldg(p.ln2_g + cc) + (p.ln2_b ? __ldg(p.ln2_b + cc) : 0.f);
-                o4[e] = tt;
-              }
-              *reinterpret_cast<float4*>(yp) = make_float4(o4[0], o4[1], o4[2], o4[3]);
-            }
-          }
-        }
-        tc_fence_before();
-        mbar_arrive(&mi->acc_free[buf]);
+        for (int i4 = 0; i4 < HALF / 4; ++i4)
+          *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(row, hh * (HALF / 4) + i4)) =
+              make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
+        store_rows(rows);
       }
     }
     if (!ok || *abort_flag) {
@@ -737,13 +778,21 @@ bool make_weight_map(CUtensorMap* m, const void* w, int rows, int cols, int box_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, int NT>
+template <int C, int D, int NT>
 int launch_tc(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
-  cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<D, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<C, D, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
-  layer_tc_kernel<D, NT><<<grid, kThreads, smem, ctx->stream>>>(a, g, maps, ctx->status);
+  layer_tc_kernel<C, D, NT><<<grid, kThreads, smem, ctx->stream>>>(a, g, maps, ctx->status);
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
+}
+
+template <int C, int D>
+int launch_tc_nt(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
+  const int nt = (g.tau + 7) / 8;
+  if (nt <= 5) return launch_tc<C, D, 5>(ctx, a, g, maps, grid, smem);
+  if (nt <= 6) return launch_tc<C, D, 6>(ctx, a, g, maps, grid, smem);
+  return launch_tc<C, D, 12>(ctx, a, g, maps, grid, smem);
 }
 
 }  // namespace
@@ -752,10 +801,9 @@ int launch_tc(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const Tc
 bool dsvt_layer_tc_supported(const dsvt_fused_args& a) {
   const dsvt_layer_params& p = a.p;
   if (p.precision != DSVT_BF16_FP32ACC || p.pe) return false;
-  if (p.C != 64 && p.C != 128 && p.C != 192) return false;
   const int d = p.C / p.heads;
-  if (d != 16 && d != 24 && d != 32) return false;
-  if (p.set_size > 96) return false;
+  const bool shape = (p.C == 192 && d == 24) || (p.C == 128 && (d == 16 || d == 32)) || (p.C == 64 && d == 16);
+  if (!shape || p.set_size > 96) return false;
   const int hidden = a.attention_only ? 0 : p.hidden;
   if (hidden != 0 && hidden != p.C && hidden != 2 * p.C) return false;
   return encode_fn() != nullptr;
@@ -763,41 +811,38 @@ bool dsvt_layer_tc_supported(const dsvt_fused_args& a) {
 
 int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a) {
   const dsvt_layer_params& p = a.p;
+  const int C = p.C;
   TcGeom g;
-  g.C = p.C; g.hidden = a.attention_only ? 0 : p.hidden; g.heads = p.heads; g.tau = p.set_size;
-  g.TMn = kTM - g.tau + 1;
-  g.nkb = p.C / 64; g.nkb_h = g.hidden / 64; g.n_f1 = g.hidden / p.C;
-  g.stage_bytes = (uint32_t)p.C * 128u;
-  const uint32_t a_bytes = kTM * p.C * 2;
-  const int kv_cols = 2 * p.C > g.hidden ? 2 * p.C : g.hidden;
+  g.hidden = a.attention_only ? 0 : p.hidden;
+  g.heads = p.heads;
+  g.tau = p.set_size;
+  g.mode = a.attention_only ? 0 : (g.hidden > 0 ? 2 : 1);
+  g.nkb_h = g.hidden / 64;
+  g.NF = (g.hidden % 128 == 0 && C >= 128) ? 128 : 64;
+  g.n_f1 = g.hidden / g.NF;
+  const uint32_t a_bytes = kTM * C * 2;
   g.off_a = 0;
   g.off_kv = a_bytes;
-  g.off_stage = g.off_kv + (uint32_t)kTM * kv_cols * 2;
-  g.off_stage = (g.off_stage + 1023u) & ~1023u;
-  g.off_misc = g.off_stage + kStages * g.stage_bytes;
+  g.off_stage = g.off_kv + (uint32_t)kTM * 2 * C * 2;  // K + V (bf16) = fp32 staging = MLP hidden (<= 2C) bytes
+  g.off_misc = g.off_stage + kStages * (uint32_t)C * 128u;
   const size_t smem = (size_t)g.off_misc + sizeof(Misc) + 1024;
   if (smem > 227 * 1024) return DSVT_ERR_UNSUPPORTED;
   TcMaps maps;
-  bool okm = make_weight_map(&maps.qkv, p.W_qkv, 3 * p.C, p.C, p.C) && make_weight_map(&maps.o, p.W_o, p.C, p.C, p.C);
+  bool okm = make_weight_map(&maps.qkv, p.W_qkv, 3 * C, C, C) && make_weight_map(&maps.o, p.W_o, C, C, C);
   if (g.hidden > 0)
-    okm = okm && make_weight_map(&maps.w1, p.W_1, g.hidden, p.C, p.C) && make_weight_map(&maps.w2, p.W_2, p.C, g.hidden, p.C);
+    okm = okm && make_weight_map(&maps.w1, p.W_1, g.hidden, C, g.NF) && make_weight_map(&maps.w2, p.W_2, C, g.hidden, C);
   else {
     maps.w1 = maps.o;
     maps.w2 = maps.o;
   }
   if (!okm) return DSVT_ERR_CUDA;
-  int64_t rmax = (int64_t)a.cap_sets * g.tau;
-  if (rmax > a.n) rmax = a.n;
-  int64_t grid = dsvt_ceil_div(rmax, g.TMn);
-  if (grid < 1) grid = 1;
+  // one CTA per SM, but no more CTAs than there can be sets
+  int64_t grid = a.cap_sets < a.n ? a.cap_sets : a.n;
   if (grid > ctx->sm_count) grid = ctx->sm_count;
-  const int d = p.C / p.heads;
-  const int nt = (g.tau + 7) / 8;
-#define DSVT_TC_CASE(DD, NN) return launch_tc<DD, NN>(ctx, a, g, maps, (int)grid, smem)
-  if (d == 16) { if (nt <= 5) DSVT_TC_CASE(16, 5); if (nt <= 6) DSVT_TC_CASE(16, 6); DSVT_TC_CASE(16, 12); }
-  if (d == 24) { if (nt <= 5) DSVT_TC_CASE(24, 5); if (nt <= 6) DSVT_TC_CASE(24, 6); DSVT_TC_CASE(24, 12); }
-  if (nt <= 5) DSVT_TC_CASE(32, 5);
-  if (nt <= 6) DSVT_TC_CASE(32, 6);
-  DSVT_TC_CASE(32, 12);
-#undef DSVT_TC_CASE
+  if (grid < 1) grid = 1;
+  const int d = C / p.heads;
+  if (C == 192) return launch_tc_nt<192, 24>(ctx, a, g, maps, (int)grid, smem);
+  if (C == 128 && d == 16) return launch_tc_nt<128, 16>(ctx, a, g, maps, (int)grid, smem);
+  if (C == 128) return launch_tc_nt<128, 32>(ctx, a, g, maps, (int)grid, smem);
+  return launch_tc_nt<64, 16>(ctx, a, g, maps, (int)grid, smem);
 }
