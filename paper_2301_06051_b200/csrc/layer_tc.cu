@@ -32,8 +32,10 @@
 namespace {
 
 constexpr int kTM = 128;               // tile rows = UMMA M
-constexpr int kComputeThreads = 256;   // warps 0-7
-constexpr int kThreads = 320;          // + scheduler/TMA warp + MMA warp
+constexpr int kComputeWarps = 16;
+constexpr int kComputeThreads = 32 * kComputeWarps;
+constexpr int kTmaWarp = kComputeWarps, kMmaWarp = kComputeWarps + 1;
+constexpr int kThreads = kComputeThreads + 64;  // + scheduler/TMA warp + MMA warp
 constexpr int kStages = 3;             // weight ring depth
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxPolls = 1 << 20;
@@ -54,7 +56,8 @@ struct Misc {  // small shared state behind the big regions
   int tile[2][4];  // ring of tiles: first set, number of sets (< 0: no more tiles), first row, rows
   int rowvox[kTM];
   int set_lo[kTM + 1];
-  float red[2][2][kTM];  // [exchange][column half][row]
+  short row_lo[kTM], row_hi[kTM];  // tile-row range of the set each row belongs to
+  float red[2][4][kTM];  // [exchange][column quarter][row]
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -95,7 +98,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory"); }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, unsigned long long* bar) {
   asm volatile(
@@ -133,6 +136,38 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
+        "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -173,6 +208,11 @@ __device__ __forceinline__ void mma_1688(float (&c)[4], uint32_t a0, uint32_t a1
       : "r"(a0), "r"(a1), "r"(b0));
 }
 
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
@@ -224,7 +264,7 @@ __device__ __forceinline__ void attend_tile(uint32_t a_base, uint32_t k_base, ui
     const int r0 = set_lo[si], m = set_lo[si + 1] - r0;
     const int mtiles = (m + 15) >> 4, ntu = (m + 7) >> 3;
     for (int hm = 0; hm < heads * mtiles; ++hm, ++item) {
-      if ((item & 7) != warp) continue;
+      if ((item % kComputeWarps) != warp) continue;
       const int h = hm / mtiles, mt = hm - h * mtiles;
       const int c0 = h * DC;
       const int q0 = r0 + 16 * mt;
@@ -317,6 +357,119 @@ __device__ __forceinline__ void attend_tile(uint32_t a_base, uint32_t k_base, ui
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Attention of one tile, blocked by 16 consecutive tile rows instead of by set: one warp per (row
+// block, head).  The keys of a block are the rows of every set that the block touches; a score is
+// kept only where query and key belong to the same set (row_lo / row_hi give each row's set range).
+// The arithmetic per query row is exactly the per-set softmax attention, but sparse regions with
+// many tiny sets cost one item per 16 rows instead of one per set.
+// NTB = key blocks of 8 a row block can need: ceil((2 tau + 14) / 8).
+// ---------------------------------------------------------------------------------------------
+template <int D, int NTB>
+__device__ __forceinline__ void attend_blocked(uint32_t a_base, uint32_t k_base, uint32_t v_base,
+                                               const short* row_lo, const short* row_hi, int rows, int heads,
+                                               int warp, int lane) {
+  constexpr int DC = D / 8;  // 16-byte chunks per head
+  const int g = lane >> 2, t4 = lane & 3;
+  const float sc = 1.4426950408889634f * rsqrtf((float)D);  // log2(e) / sqrt(d)
+  const int nblk = (rows + 15) >> 4;
+  for (int item = warp; item < nblk * heads; item += kComputeWarps) {
+    const int blk = item / heads, h = item - blk * heads;
+    const int c0 = h * DC;
+    const int q0 = 16 * blk;
+    const int k_lo = row_lo[q0], k_hi = row_hi[min(q0 + 15, rows - 1)];
+    const int ntu = min((k_hi - k_lo + 7) >> 3, NTB);
+    const int ra = q0 + g, rb = q0 + g + 8;
+    // each thread's two query rows: the key range of their sets, relative to k_lo
+    const int loA = ra < rows ? row_lo[ra] - k_lo : 0, hiA = ra < rows ? row_hi[ra] - k_lo : 0;
+    const int loB = rb < rows ? row_lo[rb] - k_lo : 0, hiB = rb < rows ? row_hi[rb] - k_lo : 0;
+    uint32_t qa[4], qb[4];
+    {
+      const int row = min(q0 + (lane & 15), kTM - 1);
+      ldsm_x4(a_base + swz(row, c0 + (lane >> 4)), qa);
+      if (D > 16) ldsm_x4(a_base + swz(row, c0 + 2 + ((D == 32) ? (lane >> 4) : 0)), qb);
+    }
+    float s[NTB][4];
+    float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < NTB; ++j) {
+      if (j < ntu) {
+        s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+        uint32_t kf[4];
+        const int row = min(k_lo + 8 * j + (lane & 7), kTM - 1);
+        const int ch = min(lane >> 3, DC - 1);
+        ldsm_x4(k_base + swz(row, c0 + ch), kf);
+        mma_16816(s[j], qa, kf[0], kf[1]);
+        if (D == 24) mma_1688(s[j], qb[0], qb[1], kf[2]);
+        if (D == 32) mma_16816(s[j], qb, kf[2], kf[3]);
+        const int key = 8 * j + 2 * t4;
+        if (key < loA || key >= hiA) s[j][0] = -INFINITY;
+        if (key + 1 < loA || key + 1 >= hiA) s[j][1] = -INFINITY;
+        if (key < loB || key >= hiB) s[j][2] = -INFINITY;
+        if (key + 1 < loB || key + 1 >= hiB) s[j][3] = -INFINITY;
+        mx0 = fmaxf(mx0, fmaxf(s[j][0], s[j][1]));
+        mx1 = fmaxf(mx1, fmaxf(s[j][2], s[j][3]));
+      }
+    }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    // rows past the tile have no keys: keep their (unused) arithmetic finite
+    const float off0 = (mx0 == -INFINITY) ? 0.f : -mx0 * sc, off1 = (mx1 == -INFINITY) ? 0.f : -mx1 * sc;
+    float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+    for (int j = 0; j < NTB; ++j) {
+      if (j < ntu) {
+        s[j][0] = ex2_approx(fmaf(s[j][0], sc, off0));
+        s[j][1] = ex2_approx(fmaf(s[j][1], sc, off0));
+        s[j][2] = ex2_approx(fmaf(s[j][2], sc, off1));
+        s[j][3] = ex2_approx(fmaf(s[j][3], sc, off1));
+        l0 += s[j][0] + s[j][1];
+        l1 += s[j][2] + s[j][3];
+      }
+    }
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    float o[DC][4];
+#pragma unroll
+    for (int dn = 0; dn < DC; ++dn) o[dn][0] = o[dn][1] = o[dn][2] = o[dn][3] = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < (NTB + 1) / 2; ++kk) {
+      if (2 * kk < ntu) {
+        constexpr int kLast = NTB - 1;
+        const int j1 = (2 * kk + 1 <= kLast) ? 2 * kk + 1 : kLast;
+        const bool two = (2 * kk + 1 <= kLast) && (2 * kk + 1 < ntu);
+        uint32_t pa[4];
+        pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
+        pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
+        pa[2] = two ? pack_bf16(s[j1][0], s[j1][1]) : 0u;
+        pa[3] = two ? pack_bf16(s[j1][2], s[j1][3]) : 0u;
+        const int row = min(k_lo + 16 * kk + (lane & 15), kTM - 1);
+#pragma unroll
+        for (int dn = 0; dn < DC; ++dn) {
+          uint32_t vf[2];
+          ldsm_x2_trans(v_base + swz(row, c0 + dn), vf);
+          mma_16816(o[dn], pa, vf[0], vf[1]);
+        }
+      }
+    }
+    const float i0 = __fdividef(1.0f, l0), i1 = __fdividef(1.0f, l1);
+#pragma unroll
+    for (int dn = 0; dn < DC; ++dn) {
+      // the query rows of this block and head are dead now: their slots take the attention output
+      if (ra < rows)
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(a_base + swz(ra, c0 + dn) + 4 * t4),
+                     "r"(pack_bf16(o[dn][0] * i0, o[dn][1] * i0)) : "memory");
+      if (rb < rows)
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(a_base + swz(rb, c0 + dn) + 4 * t4),
+                     "r"(pack_bf16(o[dn][2] * i1, o[dn][3] * i1)) : "memory");
+    }
+  }
+}
+
 // fp32 row staging in the K/V region: row r, 16-byte chunk c4 of C/4, rotated by the row so that both
 // the warp-per-row pattern (global side) and the thread-per-row pattern (TMEM side) are conflict-free.
 template <int C>
@@ -330,14 +483,15 @@ __device__ __forceinline__ uint32_t stage_off(int r, int c4) {
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int C, int D, int NT>
+template <int C, int D, int NT, bool BLOCKED>
 __global__ void __launch_bounds__(kThreads, 1)
 layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps, int32_t* __restrict__ status) {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
-  constexpr int HALF = C / 2;        // epilogue columns per thread for a C-wide chunk
+  constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
   constexpr uint32_t COL_B = C;      // second accumulator buffer
   constexpr uint32_t COL_PARK = kTmemCols - C;  // parked fp32 x1
   constexpr uint32_t STAGE_BYTES = C * 128;
+  constexpr int C4 = C / 4;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -366,17 +520,21 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
     mi->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 9) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&mi->tmem_base)),
                  "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // rows of K / V past the end of a tile are read (and masked) by the attention: never let them hold
+  // uninitialised bit patterns
+  for (uint32_t i = tid; i < (uint32_t)kTM * 2 * C * 2 / 16; i += kThreads)
+    reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = mi->tmem_base;
 
-  if (warp == 8) {
+  if (warp == kTmaWarp) {
     // ================= scheduler + TMA producer =====================================================
     if (lane == 0) {
       // this CTA's segment: the sets whose first row lies in [b R / G, (b + 1) R / G)
@@ -388,30 +546,36 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       hi = S;
       while (lo < hi) { const int m = (lo + hi) >> 1; if (a.rowoff[m] < row_hi) lo = m + 1; else hi = m; }
       const int s_end = lo;
-      int stage = 0, slot = 0;
-      uint32_t phase = 0, sphase = 0;
-      for (;;) {
-        if (!mbar_wait(&mi->sched_empty[slot], sphase ^ 1u, abort_flag)) break;
-        int ns = -1, base = 0, rows = 0;
-        while (s < s_end) {  // next tile: as many whole sets as fit in 128 rows
-          base = a.rowoff[s];
-          const int first = a.rowoff[s + 1] - base;
+      // next tile from set s on: as many whole sets as fit in 128 rows; ns < 0: none left
+      auto next_tile = [&](int& s0, int& ns, int& base, int& rows) {
+        ns = -1; base = 0; rows = 0;
+        while (s0 < s_end) {
+          base = a.rowoff[s0];
+          const int first = a.rowoff[s0 + 1] - base;
           if (first <= 0 || first > kTM) {  // offsets that do not describe a set: skip it
             atomicOr(status, DSVT_STATUS_BAD_INDEX);
-            ++s;
+            ++s0;
             continue;
           }
-          int l2 = s + 1, h2 = s_end;  // last e in (s, s_end] with rowoff[e] - base <= 128
+          int l2 = s0 + 1, h2 = s_end;  // last e in (s0, s_end] with rowoff[e] - base <= 128
           while (l2 < h2) { const int m = (l2 + h2 + 1) >> 1; if (a.rowoff[m] - base <= kTM) l2 = m; else h2 = m - 1; }
-          ns = l2 - s;
+          ns = l2 - s0;
           rows = a.rowoff[l2] - base;
-          break;
+          return;
         }
+      };
+      int stage = 0, slot = 0;
+      uint32_t phase = 0, sphase = 0;
+      int ns, base, rows;
+      next_tile(s, ns, base, rows);
+      for (;;) {
+        if (!mbar_wait(&mi->sched_empty[slot], sphase ^ 1u, abort_flag)) break;
         mi->tile[slot][0] = s; mi->tile[slot][1] = ns; mi->tile[slot][2] = base; mi->tile[slot][3] = rows;
         mbar_arrive(&mi->sched_full[slot]);
         if (++slot == 2) { slot = 0; sphase ^= 1u; }
         if (ns < 0) break;
         s += ns;
+        next_tile(s, ns, base, rows);  // found now, published as soon as this tile's weights are on their way
         // the layer's weights for this tile, chunk by chunk, K block by K block
         for (int c = 0; c < n_chunks; ++c) {
           const CUtensorMap* map;
@@ -432,7 +596,7 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
     producer_done:;
     }
     __syncwarp();
-  } else if (warp == 9) {
+  } else if (warp == kMmaWarp) {
     // ================= MMA issuer ====================================================================
     if (lane == 0) {
       int stage = 0, slot = 0;
@@ -481,10 +645,10 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
     __syncwarp();
   } else {
     // ================= compute warps =================================================================
-    const int row = 32 * (warp & 3) + lane;  // TMEM lane owned in the epilogues
-    const int hh = warp >> 2;                // column half owned in the epilogues
+    // epilogues: four threads per tile row; warp w owns TMEM lanes 32 (w % 4) .. + 31 and column quarter w / 4
+    const int row = 32 * (warp & 3) + lane;
+    const int hq = warp >> 2;
     const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
-    constexpr int C4 = C / 4;
     uint32_t uses[2] = {0u, 0u};
     int slot = 0;
     uint32_t sphase = 0;
@@ -498,15 +662,38 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       tc_fence_before();
       mbar_arrive(&mi->acc_free[bar]);
     };
-    // normalised fp32 rows staged in the K/V region -> coalesced global rows
+    // fp32 rows staged in the K/V region -> coalesced global rows
     auto store_rows = [&](int rows) {
       compute_sync();
-      for (int r = warp; r < rows; r += 8) {
+      for (int r = warp; r < rows; r += kComputeWarps) {
         const int v = mi->rowvox[r];
         if (v < 0) continue;
         for (int c4 = lane; c4 < C4; c4 += 32)
           reinterpret_cast<float4*>(a.y + (size_t)v * C)[c4] =
               *reinterpret_cast<const float4*>(sm + g.off_kv + stage_off<C>(r, c4));
+      }
+    };
+    // LayerNorm over the row that four threads share: t holds this thread's QC values
+    auto layer_norm = [&](float (&t)[QC], float sum, const float* gain, const float* shift) {
+      mi->red[0][hq][row] = sum;
+      compute_sync();
+      const float mean = (mi->red[0][0][row] + mi->red[0][1][row] + mi->red[0][2][row] + mi->red[0][3][row]) * (1.0f / (float)C);
+      float sq = 0.f;
+#pragma unroll
+      for (int i = 0; i < QC; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
+      mi->red[1][hq][row] = sq;
+      compute_sync();
+      const float var = (mi->red[1][0][row] + mi->red[1][1][row] + mi->red[1][2][row] + mi->red[1][3][row]) * (1.0f / (float)C);
+      const float inv = rsqrtf(var + p.ln_eps);
+#pragma unroll
+      for (int i4 = 0; i4 < QC / 4; ++i4) {
+        const float4 g4 = __ldg(reinterpret_cast<const float4*>(gain + hq * QC) + i4);
+        float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (shift) b4 = __ldg(reinterpret_cast<const float4*>(shift + hq * QC) + i4);
+        t[4 * i4] = t[4 * i4] * inv * g4.x + b4.x;
+        t[4 * i4 + 1] = t[4 * i4 + 1] * inv * g4.y + b4.y;
+        t[4 * i4 + 2] = t[4 * i4 + 2] * inv * g4.z + b4.z;
+        t[4 * i4 + 3] = t[4 * i4 + 3] * inv * g4.w + b4.w;
       }
     };
     for (;;) {
@@ -517,10 +704,13 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       mbar_arrive(&mi->sched_empty[slot]);
       if (++slot == 2) { slot = 0; sphase ^= 1u; }
       if (nsets < 0) break;
-      if (tid < kTM) mi->rowvox[tid] = -1;
+      const bool live = 32 * (warp & 3) < rows;  // this warp's 32 tile rows hold at least one voxel
+      // the attention pads its key blocks up to 15 rows past the tile: those K / V rows must be real bf16
+      const bool live_kv = 32 * (warp & 3) < rows + 16;
+      if (tid < kTM) { mi->rowvox[tid] = -1; mi->row_lo[tid] = (short)tid; mi->row_hi[tid] = (short)(tid + 1); }
       compute_sync();
       // ---- distinct slots of each set -> tile rows (Eq. 4) ----
-      for (int si = warp; si < nsets; si += 8) {
+      for (int si = warp; si < nsets; si += kComputeWarps) {
         const int s = s_lo + si;
         const int32_t* trow = a.table + (size_t)s * g.tau;
         const int lb = a.rowoff[s] - base, cap = a.rowoff[s + 1] - a.rowoff[s];
@@ -538,6 +728,11 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
           }
           cnt += __popc(bal);
         }
+        if (lb >= 0)
+          for (int i = lane; i < cap && lb + i < kTM; i += 32) {
+            mi->row_lo[lb + i] = (short)lb;
+            mi->row_hi[lb + i] = (short)min(lb + cap, kTM);
+          }
         if (lane == 0) {
           mi->set_lo[si] = min(max(lb, 0), kTM);
           if (cnt != cap) atomicOr(status, DSVT_STATUS_BAD_INDEX);
@@ -545,17 +740,26 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       }
       if (tid == 0) mi->set_lo[nsets] = rows;
       compute_sync();
-      // ---- gather: fp32 rows -> bf16 A operand ----
-      for (int r = warp; r < kTM; r += 8) {
-        const int v = r < rows ? mi->rowvox[r] : -1;
-        if (lane < (C >> 3)) {
-          uint4 pk = make_uint4(0u, 0u, 0u, 0u);
-          if (v >= 0) {
+      // ---- gather: fp32 rows -> bf16 A operand (four rows in flight per warp) ----
+      for (int r0 = warp; r0 < kTM; r0 += 4 * kComputeWarps) {
+        float4 f[4][2];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int r = r0 + kComputeWarps * u;
+          const int v = r < rows ? mi->rowvox[r] : -1;
+          f[u][0] = f[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (v >= 0 && lane < (C >> 3)) {
             const float4* src = reinterpret_cast<const float4*>(a.x + (size_t)v * C) + 2 * lane;
-            const float4 f0 = __ldg(src), f1 = __ldg(src + 1);
-            pk = make_uint4(pack_bf16(f0.x, f0.y), pack_bf16(f0.z, f0.w), pack_bf16(f1.x, f1.y), pack_bf16(f1.z, f1.w));
+            f[u][0] = __ldg(src);
+            f[u][1] = __ldg(src + 1);
           }
-          *reinterpret_cast<uint4*>(sm + g.off_a + swz(r, lane)) = pk;
+        }
+        if (lane < (C >> 3)) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            *reinterpret_cast<uint4*>(sm + g.off_a + swz(r0 + kComputeWarps * u, lane)) =
+                make_uint4(pack_bf16(f[u][0].x, f[u][0].y), pack_bf16(f[u][0].z, f[u][0].w),
+                           pack_bf16(f[u][1].x, f[u][1].y), pack_bf16(f[u][1].z, f[u][1].w));
         }
       }
       fence_proxy_async();
@@ -565,38 +769,63 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       for (int c = 0; c < 3; ++c) {
         const uint32_t bar = (c == 1) ? 1u : 0u;
         acc_wait(bar);
-        const float* bias = p.b_qkv ? p.b_qkv + (c == 0 ? 1 : c == 1 ? 2 : 0) * C : nullptr;
-        unsigned char* dst = sm + (c == 2 ? g.off_a : g.off_kv + (uint32_t)c * (NKB * kTM * 128));
-#pragma unroll 1
-        for (int j0 = 0; j0 < HALF; j0 += 32) {
-          float v[32];
-          tmem_ld32(tmem + lane_addr + (c == 1 ? COL_B : 0u) + hh * HALF + j0, v);
-          const int col = hh * HALF + j0;
+        if (c == 2 ? live : live_kv) {
+          uint32_t rr[QC];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            float b[8];
+          for (int j = 0; j < QC / 16; ++j)
+            tmem_ld16_nowait(tmem + lane_addr + (c == 1 ? COL_B : 0u) + hq * QC + 16 * j, &rr[16 * j]);
+          tmem_wait_ld();
+          acc_release(bar);  // the accumulator is in registers now
+          const float* bias = p.b_qkv ? p.b_qkv + (c == 0 ? 1 : c == 1 ? 2 : 0) * C + hq * QC : nullptr;
+          unsigned char* dst = sm + (c == 2 ? g.off_a : g.off_kv + (uint32_t)c * (NKB * kTM * 128));
 #pragma unroll
-            for (int e = 0; e < 8; ++e) b[e] = v[8 * q + e] + (bias ? __ldg(bias + col + 8 * q + e) : 0.f);
-            *reinterpret_cast<uint4*>(dst + swz(row, (col >> 3) + q)) =
-                make_uint4(pack_bf16(b[0], b[1]), pack_bf16(b[2], b[3]), pack_bf16(b[4], b[5]), pack_bf16(b[6], b[7]));
+          for (int q = 0; q < QC / 8; ++q) {
+            float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+            if (bias) { b0 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q); b1 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q + 1); }
+            const uint32_t* r8 = &rr[8 * q];
+            *reinterpret_cast<uint4*>(dst + swz(row, ((hq * QC) >> 3) + q)) =
+                make_uint4(pack_bf16(__uint_as_float(r8[0]) + b0.x, __uint_as_float(r8[1]) + b0.y),
+                           pack_bf16(__uint_as_float(r8[2]) + b0.z, __uint_as_float(r8[3]) + b0.w),
+                           pack_bf16(__uint_as_float(r8[4]) + b1.x, __uint_as_float(r8[5]) + b1.y),
+                           pack_bf16(__uint_as_float(r8[6]) + b1.z, __uint_as_float(r8[7]) + b1.w));
           }
+        } else {
+          acc_release(bar);
         }
-        acc_release(bar);
       }
       compute_sync();
       // ---- attention inside each set ----
-      attend_tile<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->set_lo, nsets, g.heads, warp, lane);
+      if (BLOCKED)
+        attend_blocked<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->row_lo, mi->row_hi, rows, g.heads, warp, lane);
+      else
+        attend_tile<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->set_lo, nsets, g.heads, warp, lane);
       fence_proxy_async();
       mbar_arrive(&mi->a_ready);  // attention output is the A operand of the output projection
       compute_sync();             // every warp is done with K and V: their region becomes fp32 staging
       if (g.mode != 0) {
-        // x rows (fp32) for the first residual, coalesced
-        for (int r = warp; r < rows; r += 8) {
-          const int v = mi->rowvox[r];
-          for (int c4 = lane; c4 < C4; c4 += 32) {
-            float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (v >= 0) f = __ldg(reinterpret_cast<const float4*>(a.x + (size_t)v * C) + c4);
-            *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(r, c4)) = f;
+        // x rows (fp32) for the first residual, coalesced, four rows in flight per warp
+        constexpr int XL = (C4 + 31) / 32;
+        for (int r0 = warp; r0 < rows; r0 += 4 * kComputeWarps) {
+          float4 f[4][XL];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int r = r0 + kComputeWarps * u;
+            const int v = r < rows ? mi->rowvox[r] : -1;
+#pragma unroll
+            for (int i = 0; i < XL; ++i) {
+              const int c4 = lane + 32 * i;
+              f[u][i] = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (v >= 0 && c4 < C4) f[u][i] = __ldg(reinterpret_cast<const float4*>(a.x + (size_t)v * C) + c4);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int r = r0 + kComputeWarps * u;
+#pragma unroll
+            for (int i = 0; i < XL; ++i) {
+              const int c4 = lane + 32 * i;
+              if (r < rows && c4 < C4) *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(r, c4)) = f[u][i];
+            }
           }
         }
         compute_sync();
@@ -604,64 +833,47 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       // ---- chunk 3: output projection epilogue: Z + b_o (+ x, LayerNorm) ----
       {
         acc_wait(0u);
-        float t[HALF];
+        float t[QC];
         float sum = 0.f;
+        {
+          uint32_t rr[QC];
 #pragma unroll
-        for (int j = 0; j < HALF / 32; ++j) {
-          float v[32];
-          tmem_ld32(tmem + lane_addr + hh * HALF + 32 * j, v);
-          const int col = hh * HALF + 32 * j;
+          for (int j = 0; j < QC / 16; ++j) tmem_ld16_nowait(tmem + lane_addr + hq * QC + 16 * j, &rr[16 * j]);
+          tmem_wait_ld();
+          acc_release(0u);
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int q = 0; q < QC / 4; ++q) {
+            float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f), b4 = x4;
             if (g.mode != 0 && row < rows)
-              x4 = *reinterpret_cast<const float4*>(sm + g.off_kv + stage_off<C>(row, (col >> 2) + q));
-            const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float tt = v[4 * q + e] + xs[e] + (p.b_o ? __ldg(p.b_o + col + 4 * q + e) : 0.f);
-              t[32 * j + 4 * q + e] = tt;
-              sum += tt;
-            }
+              x4 = *reinterpret_cast<const float4*>(sm + g.off_kv + stage_off<C>(row, hq * (QC / 4) + q));
+            if (p.b_o) b4 = __ldg(reinterpret_cast<const float4*>(p.b_o + hq * QC) + q);
+            t[4 * q] = __uint_as_float(rr[4 * q]) + x4.x + b4.x;
+            t[4 * q + 1] = __uint_as_float(rr[4 * q + 1]) + x4.y + b4.y;
+            t[4 * q + 2] = __uint_as_float(rr[4 * q + 2]) + x4.z + b4.z;
+            t[4 * q + 3] = __uint_as_float(rr[4 * q + 3]) + x4.w + b4.w;
+            sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
           }
         }
-        acc_release(0u);
-        if (g.mode != 0 && p.ln1_g) {
-          mi->red[0][hh][row] = sum;
-          compute_sync();
-          const float mean = (mi->red[0][0][row] + mi->red[0][1][row]) * (1.0f / (float)C);
-          float sq = 0.f;
-#pragma unroll
-          for (int i = 0; i < HALF; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
-          mi->red[1][hh][row] = sq;
-          compute_sync();
-          const float inv = rsqrtf((mi->red[1][0][row] + mi->red[1][1][row]) * (1.0f / (float)C) + p.ln_eps);
-#pragma unroll
-          for (int i = 0; i < HALF; ++i) {
-            const int cc = hh * HALF + i;
-            t[i] = t[i] * inv * __ldg(p.ln1_g + cc) + (p.ln1_b ? __ldg(p.ln1_b + cc) : 0.f);
-          }
-        }
+        if (g.mode != 0 && p.ln1_g) layer_norm(t, sum, p.ln1_g, p.ln1_b);
         if (!mlp) {
           // final result of this call: stage it (the x staging is dead once every thread has its t)
           compute_sync();
 #pragma unroll
-          for (int i4 = 0; i4 < HALF / 4; ++i4)
-            *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(row, hh * (HALF / 4) + i4)) =
+          for (int i4 = 0; i4 < QC / 4; ++i4)
+            *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(row, hq * (QC / 4) + i4)) =
                 make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
           store_rows(rows);
           continue;
         }
         // x1: bf16 A operand of MLP-1 in shared memory, fp32 copy parked in TMEM for the second residual
 #pragma unroll
-        for (int j = 0; j < HALF / 32; ++j) {
-          tmem_st32(tmem + lane_addr + COL_PARK + hh * HALF + 32 * j, &t[32 * j]);
+        for (int j = 0; j < QC / 16; ++j) tmem_st16(tmem + lane_addr + COL_PARK + hq * QC + 16 * j, &t[16 * j]);
+        tmem_wait_st();
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            *reinterpret_cast<uint4*>(sm + g.off_a + swz(row, ((hh * HALF + 32 * j) >> 3) + q)) =
-                make_uint4(pack_bf16(t[32 * j + 8 * q], t[32 * j + 8 * q + 1]), pack_bf16(t[32 * j + 8 * q + 2], t[32 * j + 8 * q + 3]),
-                           pack_bf16(t[32 * j + 8 * q + 4], t[32 * j + 8 * q + 5]), pack_bf16(t[32 * j + 8 * q + 6], t[32 * j + 8 * q + 7]));
-        }
+        for (int q = 0; q < QC / 8; ++q)
+          *reinterpret_cast<uint4*>(sm + g.off_a + swz(row, ((hq * QC) >> 3) + q)) =
+              make_uint4(pack_bf16(t[8 * q], t[8 * q + 1]), pack_bf16(t[8 * q + 2], t[8 * q + 3]),
+                         pack_bf16(t[8 * q + 4], t[8 * q + 5]), pack_bf16(t[8 * q + 6], t[8 * q + 7]));
         tc_fence_before();
         fence_proxy_async();
         mbar_arrive(&mi->a_ready);  // x1 (bf16) is the A operand of MLP-1
@@ -670,22 +882,30 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       for (int c = 0; c < g.n_f1; ++c) {
         const uint32_t bar = (uint32_t)c & 1u;
         acc_wait(bar);
-        const int hw = g.NF >> 1;  // columns per thread
-#pragma unroll 1
-        for (int j0 = 0; j0 < hw; j0 += 32) {
-          float v[32];
-          tmem_ld32(tmem + lane_addr + bar * (uint32_t)g.NF + hh * hw + j0, v);
-          const int col = c * g.NF + hh * hw + j0;  // hidden column
+        if (live) {
+          const int qw = g.NF >> 2;  // columns per thread: 32 or 16
+          uint32_t rr[32];
+          tmem_ld16_nowait(tmem + lane_addr + bar * (uint32_t)g.NF + hq * qw, &rr[0]);
+          if (qw > 16) tmem_ld16_nowait(tmem + lane_addr + bar * (uint32_t)g.NF + hq * qw + 16, &rr[16]);
+          tmem_wait_ld();
+          acc_release(bar);
+          const int col0 = c * g.NF + hq * qw;  // first hidden column of this thread
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            float b[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) b[e] = gelu_fast(v[8 * q + e] + (p.b_1 ? __ldg(p.b_1 + col + 8 * q + e) : 0.f));
-            *reinterpret_cast<uint4*>(sm + g.off_kv + swz(row, (col >> 3) + q)) =
-                make_uint4(pack_bf16(b[0], b[1]), pack_bf16(b[2], b[3]), pack_bf16(b[4], b[5]), pack_bf16(b[6], b[7]));
+            if (8 * q < qw) {
+              float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+              if (p.b_1) { b0 = __ldg(reinterpret_cast<const float4*>(p.b_1 + col0) + 2 * q); b1 = __ldg(reinterpret_cast<const float4*>(p.b_1 + col0) + 2 * q + 1); }
+              const uint32_t* r8 = &rr[8 * q];
+              *reinterpret_cast<uint4*>(sm + g.off_kv + swz(row, (col0 >> 3) + q)) =
+                  make_uint4(pack_bf16(gelu_fast(__uint_as_float(r8[0]) + b0.x), gelu_fast(__uint_as_float(r8[1]) + b0.y)),
+                             pack_bf16(gelu_fast(__uint_as_float(r8[2]) + b0.z), gelu_fast(__uint_as_float(r8[3]) + b0.w)),
+                             pack_bf16(gelu_fast(__uint_as_float(r8[4]) + b1.x), gelu_fast(__uint_as_float(r8[5]) + b1.y)),
+                             pack_bf16(gelu_fast(__uint_as_float(r8[6]) + b1.z), gelu_fast(__uint_as_float(r8[7]) + b1.w)));
+            }
           }
+        } else {
+          acc_release(bar);
         }
-        acc_release(bar);
       }
       fence_proxy_async();
       mbar_arrive(&mi->a_ready);  // H is in place
@@ -693,40 +913,33 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       {
         const uint32_t bar = (uint32_t)g.n_f1 & 1u;
         acc_wait(bar);
-        float t[HALF];
+        float t[QC];
         float sum = 0.f;
+        {
+          uint32_t rr[QC], rp[QC];
 #pragma unroll
-        for (int j = 0; j < HALF / 32; ++j) {
-          float v[32];
-          tmem_ld32(tmem + lane_addr + hh * HALF + 32 * j, v);
-          const int col = hh * HALF + 32 * j;
+          for (int j = 0; j < QC / 16; ++j) {
+            tmem_ld16_nowait(tmem + lane_addr + hq * QC + 16 * j, &rr[16 * j]);
+            tmem_ld16_nowait(tmem + lane_addr + COL_PARK + hq * QC + 16 * j, &rp[16 * j]);
+          }
+          tmem_wait_ld();
+          acc_release(bar);
 #pragma unroll
-          for (int e = 0; e < 32; ++e) t[32 * j + e] = v[e] + (p.b_2 ? __ldg(p.b_2 + col + e) : 0.f);
-          tmem_ld32(tmem + lane_addr + COL_PARK + hh * HALF + 32 * j, v);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) { t[32 * j + e] += v[e]; sum += t[32 * j + e]; }
-        }
-        acc_release(bar);
-        if (p.ln2_g) {
-          mi->red[0][hh][row] = sum;
-          compute_sync();
-          const float mean = (mi->red[0][0][row] + mi->red[0][1][row]) * (1.0f / (float)C);
-          float sq = 0.f;
-#pragma unroll
-          for (int i = 0; i < HALF; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
-          mi->red[1][hh][row] = sq;
-          compute_sync();
-          const float inv = rsqrtf((mi->red[1][0][row] + mi->red[1][1][row]) * (1.0f / (float)C) + p.ln_eps);
-#pragma unroll
-          for (int i = 0; i < HALF; ++i) {
-            const int cc = hh * HALF + i;
-            t[i] = t[i] * inv * __ldg(p.ln2_g + cc) + (p.ln2_b ? __ldg(p.ln2_b + cc) : 0.f);
+          for (int q = 0; q < QC / 4; ++q) {
+            float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (p.b_2) b4 = __ldg(reinterpret_cast<const float4*>(p.b_2 + hq * QC) + q);
+            t[4 * q] = __uint_as_float(rr[4 * q]) + __uint_as_float(rp[4 * q]) + b4.x;
+            t[4 * q + 1] = __uint_as_float(rr[4 * q + 1]) + __uint_as_float(rp[4 * q + 1]) + b4.y;
+            t[4 * q + 2] = __uint_as_float(rr[4 * q + 2]) + __uint_as_float(rp[4 * q + 2]) + b4.z;
+            t[4 * q + 3] = __uint_as_float(rr[4 * q + 3]) + __uint_as_float(rp[4 * q + 3]) + b4.w;
+            sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
           }
         }
+        if (p.ln2_g) layer_norm(t, sum, p.ln2_g, p.ln2_b);
         // the MLP-2 MMAs have read H: its region takes the fp32 output rows
 #pragma unroll
-        for (int i4 = 0; i4 < HALF / 4; ++i4)
-          *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(row, hh * (HALF / 4) + i4)) =
+        for (int i4 = 0; i4 < QC / 4; ++i4)
+          *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(row, hq * (QC / 4) + i4)) =
               make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
         store_rows(rows);
       }
@@ -738,7 +951,7 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
   // ---- teardown: everyone meets here, then the allocating warp returns the TMEM columns ----
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
@@ -778,21 +991,23 @@ bool make_weight_map(CUtensorMap* m, const void* w, int rows, int cols, int box_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int C, int D, int NT>
+template <int C, int D, int NT, bool BLOCKED>
 int launch_tc(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
-  cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<C, D, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e =
+      cudaFuncSetAttribute(layer_tc_kernel<C, D, NT, BLOCKED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
-  layer_tc_kernel<C, D, NT><<<grid, kThreads, smem, ctx->stream>>>(a, g, maps, ctx->status);
+  layer_tc_kernel<C, D, NT, BLOCKED><<<grid, kThreads, smem, ctx->stream>>>(a, g, maps, ctx->status);
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
 }
 
 template <int C, int D>
 int launch_tc_nt(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
-  const int nt = (g.tau + 7) / 8;
-  if (nt <= 5) return launch_tc<C, D, 5>(ctx, a, g, maps, grid, smem);
-  if (nt <= 6) return launch_tc<C, D, 6>(ctx, a, g, maps, grid, smem);
-  return launch_tc<C, D, 12>(ctx, a, g, maps, grid, smem);
+  // up to set size 48 the attention runs per 16-row block (key blocks: ceil((2 tau + 14) / 8)); larger
+  // sets keep one item per set (key blocks: ceil(tau / 8))
+  if (g.tau <= 36) return launch_tc<C, D, 11, true>(ctx, a, g, maps, grid, smem);
+  if (g.tau <= 48) return launch_tc<C, D, 14, true>(ctx, a, g, maps, grid, smem);
+  return launch_tc<C, D, 12, false>(ctx, a, g, maps, grid, smem);
 }
 
 }  // namespace
