@@ -90,6 +90,24 @@ def algorithmic_flops_per_layer(rowoff: np.ndarray, C: int, hidden: int) -> floa
     return n * (8.0 * C * C + 4.0 * C * hidden) + 4.0 * C * float((m * m).sum())
 
 
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks (identity when not distributed)."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def job_throughput(world: int, units_per_rank: float, ms_per_step: float) -> float:
+    """Whole-job units per second: every rank processes units_per_rank per step (weak scaling), and a
+    step takes as long as the slowest rank."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 def run_reference(args):
     """The CPU oracle as it stands, on a bounded sample of the same workload (rank 0 only)."""
     rank, _, world = _dist_env()
@@ -223,10 +241,7 @@ def run_ours(args):
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e_steps
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], device=dev)
     if ctx.status_sync() != 0:
         raise SystemExit("device status word is not clean after the timed region")
     if rank != 0:
@@ -235,7 +250,7 @@ def run_ours(args):
         return
 
     ms_per_step = total_ms / args.steps
-    value = world * n * nb / (ms_per_step * 1e-3)
+    value = job_throughput(world, n * nb, ms_per_step)
     peaks = _peaks()
     # dominant kernel: the fused layer kernel, two launches per block
     S = int(stage.tables[0].num_sets.item())
@@ -273,7 +288,7 @@ def run_ours(args):
         "frames_per_sec": world / (ms_per_step * 1e-3),
         "t_partition_ms": float(t_part.mean()), "t_block_ms": float(t_blocks.mean()),
         "clocks": clocks,
-        "e2e": {"value": world * n * nb / (e2e_ms * 1e-3), "unit": "voxels/s", "ms_per_step": e2e_ms,
+        "e2e": {"value": job_throughput(world, n * nb, e2e_ms), "unit": "voxels/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(coords_h.numel() * 4 + feats_h.numel() * 4),
                 "d2h_bytes_per_step": int(out_h.numel() * 4)},
         "gpu_launches": int(launches),
