@@ -92,9 +92,13 @@ int64_t dsvt_launch_count(const dsvt_ctx* ctx);
  *               integer floor), j = the set's number inside its window.  Rows are ordered by
  *               ascending window id, then j.  Rows [0, *num_sets) are written.
  *   num_sets    out, device int32: total number of sets.
- *   set_rowoff  out, optional (NULL to skip), int32 [cap_sets + 1]: set_rowoff[s] = number of
- *               distinct voxels in the sets before s; entry [*num_sets] = n.  Passing it on to
- *               dsvt_set_attention / dsvt_layer / dsvt_block saves them a pass over the table.
+ *   set_rowoff  out, optional (NULL to skip), int32 [2 * cap_sets + 3].  Entries [0, cap_sets]:
+ *               set_rowoff[s] = number of distinct voxels in the sets before s; entry [*num_sets] = n.
+ *               Entries from [cap_sets + 1] on: a tile plan for the tensor-core layer kernel (number of
+ *               tiles, then the first set of each tile of at most 128 distinct rows; -1 = no plan).
+ *               Passing the buffer on to dsvt_set_attention / dsvt_layer / dsvt_block saves them two
+ *               passes over the table.  A caller that fills the row offsets by hand sets entry
+ *               [cap_sets + 1] to -1.
  *   perm        out, optional, int32 [n]: voxel indices in (window, inner-window) sorted order.
  *   win_start, win_setoff   out, optional, int32 [num_windows + 1]: exclusive prefix sums of the
  *               per-window voxel counts / set counts over ALL windows (empty ones included).

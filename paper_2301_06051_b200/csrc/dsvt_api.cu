@@ -37,8 +37,8 @@ void carve(dsvt_ctx* c, unsigned char* base, size_t* total) {
   c->win_count = k.take<int32_t>(nw + 1);
   c->win_start = k.take<int32_t>(nw + 1);
   c->win_setoff = k.take<int32_t>(nw + 1);
-  c->rowoff_a = k.take<int32_t>(nv + 1);
-  c->rowoff_b = k.take<int32_t>(nv + 1);
+  c->rowoff_a = k.take<int32_t>(2 * nv + 3);
+  c->rowoff_b = k.take<int32_t>(2 * nv + 3);
   c->region_key = k.take<int32_t>(nv);
   *total = align_up(k.off, 256);
 }
@@ -64,16 +64,21 @@ int run_layer(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* table, in
               const int32_t* num_sets, const int32_t* rowoff, const dsvt_layer_params& p, float* y,
               bool attention_only, int32_t* rowoff_scratch) {
   if (n == 0 || cap_sets == 0) return DSVT_OK;
-  if (!rowoff) {
-    int rc = dsvt_launch_rowoff_from_table(ctx, table, cap_sets, num_sets, p.set_size, rowoff_scratch);
-    if (rc != DSVT_OK) return rc;
-    rowoff = rowoff_scratch;
-  }
   dsvt_fused_args a;
   a.x = x; a.y = y; a.n = n; a.table = table; a.num_sets = num_sets; a.rowoff = rowoff; a.cap_sets = cap_sets;
   a.p = p;
   a.attention_only = attention_only ? 1 : 0;
-  if (dsvt_layer_tc_supported(a)) return dsvt_launch_layer_tc(ctx, a);
+  const bool tc = dsvt_layer_tc_supported(a);
+  if (!rowoff) {
+    int rc = dsvt_launch_rowoff_from_table(ctx, table, cap_sets, num_sets, p.set_size, rowoff_scratch);
+    if (rc != DSVT_OK) return rc;
+    if (tc) {
+      rc = dsvt_launch_tile_plan(ctx, num_sets, cap_sets, rowoff_scratch);
+      if (rc != DSVT_OK) return rc;
+    }
+    a.rowoff = rowoff_scratch;
+  }
+  if (tc) return dsvt_launch_layer_tc(ctx, a);
   return dsvt_launch_layer_fma(ctx, a);
 }
 

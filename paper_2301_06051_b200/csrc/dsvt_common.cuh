@@ -25,8 +25,8 @@ struct dsvt_ctx {
   int32_t* win_count;   // [max_windows + 1]  (pooling: region occupancy flags)
   int32_t* win_start;   // [max_windows + 1]  (pooling: region rank)
   int32_t* win_setoff;  // [max_windows + 1]
-  int32_t* rowoff_a;    // [max_voxels + 1] set_rowoff derived from a caller table
-  int32_t* rowoff_b;    // [max_voxels + 1]
+  int32_t* rowoff_a;    // [2 max_voxels + 3] row offsets + tile plan derived from a caller table
+  int32_t* rowoff_b;    // [2 max_voxels + 3]
   int32_t* region_key;  // [max_voxels] pooling: dense region id of each output row
   // pooling: dense cell -> voxel map, grown on demand
   int32_t* cell_map;
@@ -61,6 +61,8 @@ int dsvt_launch_scan_i32(dsvt_ctx* ctx, const int32_t* in, int32_t* out, int64_t
 int dsvt_launch_sort_pairs(dsvt_ctx* ctx, int32_t n, int key_bits, int* final_buf);
 int dsvt_launch_rowoff_from_table(dsvt_ctx* ctx, const int32_t* table, int32_t cap_sets, const int32_t* num_sets,
                                   int32_t set_size, int32_t* rowoff);
+
+int dsvt_launch_tile_plan(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap_sets, int32_t* set_rowoff);
 
 struct dsvt_fused_args {
   const float* x;

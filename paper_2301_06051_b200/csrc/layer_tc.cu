@@ -537,18 +537,40 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
   if (warp == kTmaWarp) {
     // ================= scheduler + TMA producer =====================================================
     if (lane == 0) {
-      // this CTA's segment: the sets whose first row lies in [b R / G, (b + 1) R / G)
-      const int row_lo = (int)(((long long)blockIdx.x * R) / gridDim.x);
-      const int row_hi = (int)(((long long)(blockIdx.x + 1) * R) / gridDim.x);
-      int lo = 0, hi = S;
-      while (lo < hi) { const int m = (lo + hi) >> 1; if (a.rowoff[m] < row_lo) lo = m + 1; else hi = m; }
-      int s = lo;
-      hi = S;
-      while (lo < hi) { const int m = (lo + hi) >> 1; if (a.rowoff[m] < row_hi) lo = m + 1; else hi = m; }
-      const int s_end = lo;
-      // next tile from set s on: as many whole sets as fit in 128 rows; ns < 0: none left
+      // Tiles come from the plan behind the row offsets (greedy packing of the whole frame, tile t goes to
+      // CTA t mod G); without a plan each CTA packs its own segment, the sets whose first row lies in
+      // [b R / G, (b + 1) R / G).
+      const int32_t* plan = a.rowoff + a.cap_sets + 1;
+      const int n_plan = plan[0];
+      int t_next = blockIdx.x;
+      int s = 0, s_end = 0;
+      if (n_plan < 0) {
+        const int row_lo = (int)(((long long)blockIdx.x * R) / gridDim.x);
+        const int row_hi = (int)(((long long)(blockIdx.x + 1) * R) / gridDim.x);
+        int lo = 0, hi = S;
+        while (lo < hi) { const int m = (lo + hi) >> 1; if (a.rowoff[m] < row_lo) lo = m + 1; else hi = m; }
+        s = lo;
+        hi = S;
+        while (lo < hi) { const int m = (lo + hi) >> 1; if (a.rowoff[m] < row_hi) lo = m + 1; else hi = m; }
+        s_end = lo;
+      }
+      // next tile: first set s0, ns sets (< 0: none left), first row, rows
       auto next_tile = [&](int& s0, int& ns, int& base, int& rows) {
         ns = -1; base = 0; rows = 0;
+        if (n_plan >= 0) {
+          while (t_next < n_plan) {
+            const int f = plan[1 + t_next], l = plan[2 + t_next];
+            t_next += gridDim.x;
+            if (f < 0 || l <= f || l > S) { atomicOr(status, DSVT_STATUS_BAD_INDEX); continue; }
+            base = a.rowoff[f];
+            rows = a.rowoff[l] - base;
+            if (rows <= 0 || rows > kTM || l - f > kTM) { atomicOr(status, DSVT_STATUS_BAD_INDEX); continue; }
+            s0 = f;
+            ns = l - f;
+            return;
+          }
+          return;
+        }
         while (s0 < s_end) {
           base = a.rowoff[s0];
           const int first = a.rowoff[s0 + 1] - base;

@@ -309,6 +309,65 @@ __global__ void table_unique_count_kernel(const int32_t* __restrict__ table, int
   if (lane == 0) cnt[s] = c;
 }
 
+// ---- tile plan for the tensor-core layer kernel -------------------------------------------------
+// Greedy packing of whole sets, in table order, into tiles of at most max_rows distinct rows:
+// plan[0] = number of tiles, plan[1 + t] = first set of tile t, plan[1 + tiles] = number of sets;
+// plan[0] = -1 if there are more sets than this kernel handles (the layer kernel then schedules by
+// row segments).  The greedy chain 0 -> next(0) -> next(next(0)) ... is found by pointer doubling, all
+// sets in parallel: single block, arrays in shared memory.
+constexpr int kPlanMaxSets = 24576;
+__global__ void __launch_bounds__(kScanThreads) tile_plan_kernel(const int32_t* __restrict__ rowoff,
+                                                                 const int32_t* __restrict__ num_sets, int32_t cap_sets,
+                                                                 int32_t smax, int32_t max_rows, int32_t* __restrict__ plan) {
+  extern __shared__ int plan_smem[];
+  __shared__ int warp_tot[33];
+  int* cur = plan_smem;
+  int* nxt = cur + (smax + 1);
+  unsigned char* mark = reinterpret_cast<unsigned char*>(nxt + (smax + 1));
+  const int tid = threadIdx.x;
+  const int S = min(*num_sets, cap_sets);
+  if (S > smax) {
+    if (tid == 0) plan[0] = -1;
+    return;
+  }
+  if (S <= 0) {
+    if (tid == 0) { plan[0] = 0; plan[1] = 0; }
+    return;
+  }
+  for (int s = tid; s < S; s += kScanThreads) {
+    const int base = rowoff[s];
+    int e = s + 1;
+    const int first = rowoff[s + 1] - base;
+    if (first > 0 && first <= max_rows) {  // last e in (s, S] with rowoff[e] - base <= max_rows
+      int lo = s + 1, hi = min(S, s + max_rows);
+      while (lo < hi) { const int m = (lo + hi + 1) >> 1; if (rowoff[m] - base <= max_rows) lo = m; else hi = m - 1; }
+      e = lo;
+    }
+    cur[s] = e;
+    mark[s] = (s == 0);
+  }
+  if (tid == 0) cur[S] = S;
+  __syncthreads();
+  for (int len = 1; len < S; len <<= 1) {
+    // marked sets are tile starts; cur = 'next' applied len times
+    for (int s = tid; s < S; s += kScanThreads)
+      if (mark[s] && cur[s] < S) mark[cur[s]] = 1;
+    for (int s = tid; s <= S; s += kScanThreads) nxt[s] = cur[cur[s]];
+    __syncthreads();
+    int* t = cur; cur = nxt; nxt = t;
+  }
+  // ordered compaction of the marks
+  const int chunk = (S + kScanThreads - 1) / kScanThreads;
+  const int s0 = min(tid * chunk, S), s1 = min(s0 + chunk, S);
+  int cnt = 0;
+  for (int s = s0; s < s1; ++s) cnt += mark[s];
+  int total;
+  int off = block_excl_scan(cnt, warp_tot, &total);
+  for (int s = s0; s < s1; ++s)
+    if (mark[s]) plan[1 + off++] = s;
+  if (tid == 0) { plan[0] = total; plan[1 + total] = S; }
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------------------
@@ -359,6 +418,22 @@ int dsvt_launch_rowoff_from_table(dsvt_ctx* ctx, const int32_t* table, int32_t c
     DSVT_LAUNCHED(ctx);
   }
   return dsvt_launch_scan_i32(ctx, rowoff, rowoff, cap_sets, nullptr);
+}
+
+// Tile plan behind the row offsets: set_rowoff + cap_sets + 1 (see include/dsvt.h).
+int dsvt_launch_tile_plan(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap_sets, int32_t* set_rowoff) {
+  const int32_t smax = cap_sets < kPlanMaxSets ? cap_sets : kPlanMaxSets;
+  const size_t smem = (size_t)(smax + 1) * 8 + (size_t)smax + 16;
+  static bool attr_set = false;
+  if (!attr_set) {
+    DSVT_CUDA_TRY(ctx, cudaFuncSetAttribute(tile_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)((size_t)(kPlanMaxSets + 1) * 8 + kPlanMaxSets + 16)));
+    attr_set = true;
+  }
+  tile_plan_kernel<<<1, kScanThreads, smem, ctx->stream>>>(set_rowoff, num_sets, cap_sets, smax, 128,
+                                                          set_rowoff + cap_sets + 1);
+  DSVT_LAUNCHED(ctx);
+  return DSVT_OK;
 }
 
 static int key_bits_for(uint64_t max_key) {
@@ -416,10 +491,15 @@ extern "C" int dsvt_partition(dsvt_ctx* ctx, const int32_t* coords, int32_t n, i
                                                                              set_size, num_sets, set_table, set_rowoff);
       DSVT_LAUNCHED(ctx);
     }
+    if (set_rowoff && s_bound > 0) {
+      int rc = dsvt_launch_tile_plan(ctx, num_sets, cap_sets, set_rowoff);
+      if (rc != DSVT_OK) return rc;
+    }
     if (perm)
       DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(perm, ctx->vals[fin], sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToDevice, st));
   }
-  if (set_rowoff && (n == 0 || cap_sets == 0)) DSVT_CUDA_TRY(ctx, cudaMemsetAsync(set_rowoff, 0, sizeof(int32_t), st));
+  if (set_rowoff && (n == 0 || cap_sets == 0))  // no sets: row offset 0, empty tile plan
+    DSVT_CUDA_TRY(ctx, cudaMemsetAsync(set_rowoff, 0, sizeof(int32_t) * (size_t)(2 * (size_t)cap_sets + 3), st));
   if (win_count)
     DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(win_count, ctx->win_count, sizeof(int32_t) * (size_t)nw, cudaMemcpyDeviceToDevice, st));
   if (win_start)

@@ -25,7 +25,7 @@ class Stage:
         self.tables = [
             api.SetTable(torch.empty((cap, set_size), dtype=torch.int32, device=dev),
                          torch.zeros(1, dtype=torch.int32, device=dev),
-                         torch.empty(cap + 1, dtype=torch.int32, device=dev), cap, set_size)
+                         torch.empty(2 * cap + 3, dtype=torch.int32, device=dev), cap, set_size)
             for _ in range(2)
         ]
 

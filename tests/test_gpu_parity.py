@@ -37,6 +37,21 @@ def _check_partition(gpu, oracle, coords, batch, grid, window, tau, ctx=None):
         assert tbl.shape == ref.set_table.shape, (axis, tbl.shape, ref.set_table.shape)
         assert np.array_equal(tbl, ref.set_table), axis
         assert np.array_equal(ro, rowoff_of(ref.set_table)), axis
+        # tile plan behind the row offsets: greedy packing of whole sets into tiles of at most 128 rows
+        plan = t.set_rowoff[t.cap_sets + 1:].cpu().numpy()
+        S = tbl.shape[0]
+        starts, s = [], 0
+        while s < S:
+            starts.append(s)
+            e = s + 1
+            while e < S and ro[e + 1] - ro[s] <= 128:
+                e += 1
+            s = e
+        if S <= 24576:
+            assert plan[0] == len(starts), axis
+            assert np.array_equal(plan[1:1 + len(starts)], np.array(starts, dtype=np.int32)) and plan[1 + len(starts)] == S
+        else:
+            assert plan[0] == -1
         assert np.array_equal(t.perm[:n].cpu().numpy(), ref.perm)
         assert np.array_equal(t.win_count.cpu().numpy(), ref.win_count)
         assert np.array_equal(t.win_start.cpu().numpy(), ref.win_start)

@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 def _blank_table(api, cap, tau):
     return api.SetTable(torch.full((cap, tau), -1, dtype=torch.int32, device="cuda"),
                         torch.full((1,), -1, dtype=torch.int32, device="cuda"),
-                        torch.full((cap + 1,), -1, dtype=torch.int32, device="cuda"), cap, tau)
+                        torch.full((2 * cap + 3,), -1, dtype=torch.int32, device="cuda"), cap, tau)
 
 
 def _same(api, ctx, coords, batch, grid, window, tau, axis, check_memory=True):
@@ -38,6 +38,9 @@ def _same(api, ctx, coords, batch, grid, window, tau, axis, check_memory=True):
     assert int(got.num_sets.item()) == S
     assert torch.equal(got.set_table[:S], want.set_table[:S])  # integer outputs: bit-exact
     assert torch.equal(got.set_rowoff[: S + 1], want.set_rowoff[: S + 1])
+    cap = want.cap_sets  # the tile plan behind the row offsets: tile count, tile starts, terminator
+    tiles = int(want.set_rowoff[cap + 1].item())
+    assert torch.equal(got.set_rowoff[cap + 1: cap + 3 + tiles], want.set_rowoff[cap + 1: cap + 3 + tiles])
     assert torch.all(got.set_table[S:] == -1)  # nothing written past the last set
     return S
 
