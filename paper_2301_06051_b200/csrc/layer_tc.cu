@@ -232,17 +232,19 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTM >> 4) << 24);
 }
 
-// gelu(t) = t/2 (1 + erf(t / sqrt 2)) with the five-term rational approximation of erf
-// (absolute error below 2e-7, far under the bfloat16 rounding applied to the result).
+// gelu(t) = t Phi(t), Phi(t) = 1 - erfc(|t| / sqrt 2) / 2 for t >= 0 and erfc(|t| / sqrt 2) / 2 for t < 0.
+// erfc(z) is evaluated as 2^p(|t|) with p a degree-5 polynomial: a weighted least-squares fit of
+// log2 erfc(|t| / sqrt 2) on |t| <= 8.4 (beyond that erfc < 1e-16).  One ex2 and six FMAs; the absolute error of
+// gelu is below 2e-6 for all t, far under the bfloat16 rounding applied to the result.
 __device__ __forceinline__ float gelu_fast(float t) {
-  const float z = fabsf(t) * 0.70710678118654752440f;
-  const float k = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
-  float poly = fmaf(1.061405429f, k, -1.453152027f);
-  poly = fmaf(poly, k, 1.421413741f);
-  poly = fmaf(poly, k, -0.284496736f);
-  poly = fmaf(poly, k, 0.254829592f);
-  const float erf_abs = 1.0f - poly * k * __expf(-z * z);
-  return 0.5f * t * (1.0f + copysignf(erf_abs, t));
+  const float a = fminf(fabsf(t), 8.4f);
+  float q = fmaf(-5.189499352e-04f, a, 7.387642749e-03f);
+  q = fmaf(q, a, -5.253871530e-02f);
+  q = fmaf(q, a, -4.592762589e-01f);
+  q = fmaf(q, a, -1.151083231e+00f);
+  q = fmaf(q, a, -8.382420447e-07f);
+  const float h = 0.5f * ex2_approx(q);  // erfc(|t| / sqrt 2) / 2
+  return t * (t < 0.f ? h : 1.0f - h);
 }
 
 struct TcMaps {
@@ -825,31 +827,20 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       mbar_arrive(&mi->a_ready);  // attention output is the A operand of the output projection
       compute_sync();             // every warp is done with K and V: their region becomes fp32 staging
       if (g.mode != 0) {
-        // x rows (fp32) for the first residual, coalesced, four rows in flight per warp
-        constexpr int XL = (C4 + 31) / 32;
-        for (int r0 = warp; r0 < rows; r0 += 4 * kComputeWarps) {
-          float4 f[4][XL];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int r = r0 + kComputeWarps * u;
-            const int v = r < rows ? mi->rowvox[r] : -1;
-#pragma unroll
-            for (int i = 0; i < XL; ++i) {
-              const int c4 = lane + 32 * i;
-              f[u][i] = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (v >= 0 && c4 < C4) f[u][i] = __ldg(reinterpret_cast<const float4*>(a.x + (size_t)v * C) + c4);
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int r = r0 + kComputeWarps * u;
-#pragma unroll
-            for (int i = 0; i < XL; ++i) {
-              const int c4 = lane + 32 * i;
-              if (r < rows && c4 < C4) *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(r, c4)) = f[u][i];
-            }
+        // x rows (fp32) for the first residual: asynchronous 16-byte copies global -> shared, all of a
+        // warp's rows in flight at once, no registers involved
+        for (int r = warp; r < rows; r += kComputeWarps) {
+          const int v = mi->rowvox[r];
+          for (int c4 = lane; c4 < C4; c4 += 32) {
+            const uint32_t dst = sbase + g.off_kv + stage_off<C>(r, c4);
+            if (v >= 0)
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst),
+                           "l"(reinterpret_cast<const float4*>(a.x + (size_t)v * C) + c4) : "memory");
+            else
+              *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(r, c4)) = make_float4(0.f, 0.f, 0.f, 0.f);
           }
         }
+        asm volatile("cp.async.wait_all;" ::: "memory");
         compute_sync();
       }
       // ---- chunk 3: output projection epilogue: Z + b_o (+ x, LayerNorm) ----
