@@ -27,6 +27,8 @@
 // leave their loops.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "dsvt_common.cuh"
 
 namespace {
@@ -167,6 +169,41 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// 16 fp32 columns of this thread's TMEM lane into / from elements [OFF, OFF + 16) of a register array
+// (compile-time offsets keep the array in registers).
+template <int OFF, int N>
+__device__ __forceinline__ void tmem_ld16_at(uint32_t taddr, float (&r)[N]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=f"(r[OFF + 0]), "=f"(r[OFF + 1]), "=f"(r[OFF + 2]), "=f"(r[OFF + 3]), "=f"(r[OFF + 4]), "=f"(r[OFF + 5]),
+        "=f"(r[OFF + 6]), "=f"(r[OFF + 7]), "=f"(r[OFF + 8]), "=f"(r[OFF + 9]), "=f"(r[OFF + 10]), "=f"(r[OFF + 11]),
+        "=f"(r[OFF + 12]), "=f"(r[OFF + 13]), "=f"(r[OFF + 14]), "=f"(r[OFF + 15])
+      : "r"(taddr));
+}
+template <int OFF, int N>
+__device__ __forceinline__ void tmem_st16_at(uint32_t taddr, const float (&v)[N]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "f"(v[OFF + 0]), "f"(v[OFF + 1]), "f"(v[OFF + 2]), "f"(v[OFF + 3]), "f"(v[OFF + 4]), "f"(v[OFF + 5]),
+        "f"(v[OFF + 6]), "f"(v[OFF + 7]), "f"(v[OFF + 8]), "f"(v[OFF + 9]), "f"(v[OFF + 10]), "f"(v[OFF + 11]),
+        "f"(v[OFF + 12]), "f"(v[OFF + 13]), "f"(v[OFF + 14]), "f"(v[OFF + 15])
+      : "memory");
+}
+template <int N>
+__device__ __forceinline__ void tmem_ld_row(uint32_t taddr, float (&r)[N]) {
+  static_assert(N == 16 || N == 32 || N == 48, "column count per thread");
+  tmem_ld16_at<0>(taddr, r);
+  if constexpr (N > 16) tmem_ld16_at<16>(taddr + 16, r);
+  if constexpr (N > 32) tmem_ld16_at<32>(taddr + 32, r);
+}
+template <int N>
+__device__ __forceinline__ void tmem_st_row(uint32_t taddr, const float (&v)[N]) {
+  tmem_st16_at<0>(taddr, v);
+  if constexpr (N > 16) tmem_st16_at<16>(taddr + 16, v);
+  if constexpr (N > 32) tmem_st16_at<32>(taddr + 32, v);
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
   asm volatile(
@@ -256,7 +293,7 @@ struct TcMaps {
 // D = head dim (16 / 24 / 32), NT = key blocks of 8 a set can have.
 // ---------------------------------------------------------------------------------------------
 template <int D, int NT>
-__device__ __forceinline__ void attend_tile(uint32_t a_base, uint32_t k_base, uint32_t v_base, const int* set_lo,
+__device__ __noinline__ void attend_tile(uint32_t a_base, uint32_t k_base, uint32_t v_base, const int* set_lo,
                                             int nsets, int heads, int warp, int lane) {
   constexpr int DC = D / 8;  // 16-byte chunks per head
   const int g = lane >> 2, t4 = lane & 3;
@@ -368,10 +405,11 @@ __device__ __forceinline__ void attend_tile(uint32_t a_base, uint32_t k_base, ui
 // NTB = key blocks of 8 a row block can need: ceil((2 tau + 14) / 8).
 // ---------------------------------------------------------------------------------------------
 template <int D, int NTB>
-__device__ __forceinline__ void attend_blocked(uint32_t a_base, uint32_t k_base, uint32_t v_base,
+__device__ __noinline__ void attend_blocked(uint32_t a_base, uint32_t k_base, uint32_t v_base,
                                                const short* row_lo, const short* row_hi, int rows, int heads,
                                                int warp, int lane) {
   constexpr int DC = D / 8;  // 16-byte chunks per head
+  constexpr int PW = 4;      // key blocks of 8 per pass (running softmax across passes keeps registers low)
   const int g = lane >> 2, t4 = lane & 3;
   const float sc = 1.4426950408889634f * rsqrtf((float)D);  // log2(e) / sqrt(d)
   const int nblk = (rows + 15) >> 4;
@@ -391,73 +429,84 @@ __device__ __forceinline__ void attend_blocked(uint32_t a_base, uint32_t k_base,
       ldsm_x4(a_base + swz(row, c0 + (lane >> 4)), qa);
       if (D > 16) ldsm_x4(a_base + swz(row, c0 + 2 + ((D == 32) ? (lane >> 4) : 0)), qb);
     }
-    float s[NTB][4];
-    float mx0 = -INFINITY, mx1 = -INFINITY;
+    float o[DC][4];
 #pragma unroll
-    for (int j = 0; j < NTB; ++j) {
-      if (j < ntu) {
-        s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
-        uint32_t kf[4];
-        const int row = min(k_lo + 8 * j + (lane & 7), kTM - 1);
-        const int ch = min(lane >> 3, DC - 1);
-        ldsm_x4(k_base + swz(row, c0 + ch), kf);
-        mma_16816(s[j], qa, kf[0], kf[1]);
-        if (D == 24) mma_1688(s[j], qb[0], qb[1], kf[2]);
-        if (D == 32) mma_16816(s[j], qb, kf[2], kf[3]);
-        const int key = 8 * j + 2 * t4;
-        if (key < loA || key >= hiA) s[j][0] = -INFINITY;
-        if (key + 1 < loA || key + 1 >= hiA) s[j][1] = -INFINITY;
-        if (key < loB || key >= hiB) s[j][2] = -INFINITY;
-        if (key + 1 < loB || key + 1 >= hiB) s[j][3] = -INFINITY;
-        mx0 = fmaxf(mx0, fmaxf(s[j][0], s[j][1]));
-        mx1 = fmaxf(mx1, fmaxf(s[j][2], s[j][3]));
+    for (int dn = 0; dn < DC; ++dn) o[dn][0] = o[dn][1] = o[dn][2] = o[dn][3] = 0.f;
+    float mA = -INFINITY, mB = -INFINITY, l0 = 0.f, l1 = 0.f;  // running row maxima and sums
+    for (int j0 = 0; j0 < ntu; j0 += PW) {
+      float s[PW][4];
+      float mx0 = mA, mx1 = mB;
+#pragma unroll
+      for (int jj = 0; jj < PW; ++jj) {
+        const int j = j0 + jj;
+        if (j < ntu) {
+          s[jj][0] = s[jj][1] = s[jj][2] = s[jj][3] = 0.f;
+          uint32_t kf[4];
+          const int row = min(k_lo + 8 * j + (lane & 7), kTM - 1);
+          const int ch = min(lane >> 3, DC - 1);
+          ldsm_x4(k_base + swz(row, c0 + ch), kf);
+          mma_16816(s[jj], qa, kf[0], kf[1]);
+          if (D == 24) mma_1688(s[jj], qb[0], qb[1], kf[2]);
+          if (D == 32) mma_16816(s[jj], qb, kf[2], kf[3]);
+          const int key = 8 * j + 2 * t4;
+          if (key < loA || key >= hiA) s[jj][0] = -INFINITY;
+          if (key + 1 < loA || key + 1 >= hiA) s[jj][1] = -INFINITY;
+          if (key < loB || key >= hiB) s[jj][2] = -INFINITY;
+          if (key + 1 < loB || key + 1 >= hiB) s[jj][3] = -INFINITY;
+          mx0 = fmaxf(mx0, fmaxf(s[jj][0], s[jj][1]));
+          mx1 = fmaxf(mx1, fmaxf(s[jj][2], s[jj][3]));
+        }
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      // rows without any key so far (rows past the tile) keep finite arithmetic
+      const float off0 = (mx0 == -INFINITY) ? 0.f : -mx0 * sc, off1 = (mx1 == -INFINITY) ? 0.f : -mx1 * sc;
+      // rescale what the earlier passes accumulated to the new maxima
+      const float al0 = (mA == -INFINITY) ? 0.f : ex2_approx(fmaf(mA, sc, off0));
+      const float al1 = (mB == -INFINITY) ? 0.f : ex2_approx(fmaf(mB, sc, off1));
+      mA = mx0;
+      mB = mx1;
+      l0 *= al0;
+      l1 *= al1;
+#pragma unroll
+      for (int dn = 0; dn < DC; ++dn) { o[dn][0] *= al0; o[dn][1] *= al0; o[dn][2] *= al1; o[dn][3] *= al1; }
+#pragma unroll
+      for (int jj = 0; jj < PW; ++jj) {
+        if (j0 + jj < ntu) {
+          s[jj][0] = ex2_approx(fmaf(s[jj][0], sc, off0));
+          s[jj][1] = ex2_approx(fmaf(s[jj][1], sc, off0));
+          s[jj][2] = ex2_approx(fmaf(s[jj][2], sc, off1));
+          s[jj][3] = ex2_approx(fmaf(s[jj][3], sc, off1));
+          l0 += s[jj][0] + s[jj][1];
+          l1 += s[jj][2] + s[jj][3];
+        }
+      }
+#pragma unroll
+      for (int kk = 0; kk < PW / 2; ++kk) {
+        if (j0 + 2 * kk < ntu) {
+          const bool two = j0 + 2 * kk + 1 < ntu;
+          uint32_t pa[4];
+          pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
+          pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
+          pa[2] = two ? pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]) : 0u;
+          pa[3] = two ? pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]) : 0u;
+          const int row = min(k_lo + 8 * j0 + 16 * kk + (lane & 15), kTM - 1);
+#pragma unroll
+          for (int dn = 0; dn < DC; ++dn) {
+            uint32_t vf[2];
+            ldsm_x2_trans(v_base + swz(row, c0 + dn), vf);
+            mma_16816(o[dn], pa, vf[0], vf[1]);
+          }
+        }
       }
     }
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-    // rows past the tile have no keys: keep their (unused) arithmetic finite
-    const float off0 = (mx0 == -INFINITY) ? 0.f : -mx0 * sc, off1 = (mx1 == -INFINITY) ? 0.f : -mx1 * sc;
-    float l0 = 0.f, l1 = 0.f;
-#pragma unroll
-    for (int j = 0; j < NTB; ++j) {
-      if (j < ntu) {
-        s[j][0] = ex2_approx(fmaf(s[j][0], sc, off0));
-        s[j][1] = ex2_approx(fmaf(s[j][1], sc, off0));
-        s[j][2] = ex2_approx(fmaf(s[j][2], sc, off1));
-        s[j][3] = ex2_approx(fmaf(s[j][3], sc, off1));
-        l0 += s[j][0] + s[j][1];
-        l1 += s[j][2] + s[j][3];
-      }
-    }
+    // the per-thread partial sums of a row live in the four threads of its quad
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
     l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-    float o[DC][4];
-#pragma unroll
-    for (int dn = 0; dn < DC; ++dn) o[dn][0] = o[dn][1] = o[dn][2] = o[dn][3] = 0.f;
-#pragma unroll
-    for (int kk = 0; kk < (NTB + 1) / 2; ++kk) {
-      if (2 * kk < ntu) {
-        constexpr int kLast = NTB - 1;
-        const int j1 = (2 * kk + 1 <= kLast) ? 2 * kk + 1 : kLast;
-        const bool two = (2 * kk + 1 <= kLast) && (2 * kk + 1 < ntu);
-        uint32_t pa[4];
-        pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-        pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-        pa[2] = two ? pack_bf16(s[j1][0], s[j1][1]) : 0u;
-        pa[3] = two ? pack_bf16(s[j1][2], s[j1][3]) : 0u;
-        const int row = min(k_lo + 16 * kk + (lane & 15), kTM - 1);
-#pragma unroll
-        for (int dn = 0; dn < DC; ++dn) {
-          uint32_t vf[2];
-          ldsm_x2_trans(v_base + swz(row, c0 + dn), vf);
-          mma_16816(o[dn], pa, vf[0], vf[1]);
-        }
-      }
-    }
     const float i0 = __fdividef(1.0f, l0), i1 = __fdividef(1.0f, l1);
 #pragma unroll
     for (int dn = 0; dn < DC; ++dn) {
@@ -483,61 +532,37 @@ __device__ __forceinline__ uint32_t stage_off(int r, int c4) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// The kernel
+// Roles
 // ---------------------------------------------------------------------------------------------
-template <int C, int D, int NT, bool BLOCKED>
-__global__ void __launch_bounds__(kThreads, 1)
-layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps, int32_t* __restrict__ status) {
+struct RoleCtx {
+  unsigned char* sm;  // 1024-aligned shared-memory base (generic address) and its shared-space address
+  uint32_t sbase;
+  uint32_t tmem;      // TMEM base address of the CTA's allocation
+  int S, R;           // number of sets, number of distinct rows
+};
+
+// The scheduler and the MMA issuer are separate (not inlined) functions so that their polling loops get
+// their own, spill-free register allocation; the compute role is inlined into the kernel, where the
+// kernel parameters are constant-bank operands.
+
+// ================= scheduler + TMA producer (one thread) ===============================================
+template <int C>
+__device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps,
+                                           int32_t* __restrict__ status, const RoleCtx rc) {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
-  constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
   constexpr uint32_t COL_B = C;      // second accumulator buffer
-  constexpr uint32_t COL_PARK = kTmemCols - C;  // parked fp32 x1
   constexpr uint32_t STAGE_BYTES = C * 128;
-  constexpr int C4 = C / 4;
-  extern __shared__ unsigned char smem_raw[];
-  const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
-  unsigned char* sm = smem_raw + pad;
-  const uint32_t sbase = raw + pad;
+  unsigned char* sm = rc.sm;
+  const uint32_t sbase = rc.sbase, tmem = rc.tmem;
   Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
   const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const dsvt_layer_params& p = a.p;
   volatile int* abort_flag = &mi->abort_flag;
-
-  const int S = min(*a.num_sets, a.cap_sets);
-  const int R = S > 0 ? a.rowoff[S] : 0;
+  const int S = rc.S, R = rc.R;
   const bool mlp = g.mode == 2;
   const int n_chunks = 4 + (mlp ? g.n_f1 + 1 : 0);
-
-  if (tid == 0) {
-    for (int i = 0; i < kStages; ++i) { mbar_init(&mi->full[i], 1); mbar_init(&mi->empty[i], 1); }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&mi->acc_full[i], 1);
-      mbar_init(&mi->acc_free[i], kComputeThreads);
-      mbar_init(&mi->sched_full[i], 1);
-      mbar_init(&mi->sched_empty[i], kComputeThreads + 1);
-    }
-    mbar_init(&mi->a_ready, kComputeThreads);
-    mi->abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == kMmaWarp) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&mi->tmem_base)),
-                 "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  // rows of K / V past the end of a tile are read (and masked) by the attention: never let them hold
-  // uninitialised bit patterns
-  for (uint32_t i = tid; i < (uint32_t)kTM * 2 * C * 2 / 16; i += kThreads)
-    reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = mi->tmem_base;
-
-  if (warp == kTmaWarp) {
-    // ================= scheduler + TMA producer =====================================================
+  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp; (void)R;
+  (void)tmem; (void)S; (void)n_chunks; (void)tid;
     if (lane == 0) {
       // Tiles come from the plan behind the row offsets (greedy packing of the whole frame, tile t goes to
       // CTA t mod G); without a plan each CTA packs its own segment, the sets whose first row lies in
@@ -619,9 +644,25 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       }
     producer_done:;
     }
-    __syncwarp();
-  } else if (warp == kMmaWarp) {
-    // ================= MMA issuer ====================================================================
+}
+
+// ================= MMA issuer (one thread) =============================================================
+template <int C>
+__device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g, const RoleCtx rc) {
+  constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
+  constexpr uint32_t COL_B = C;      // second accumulator buffer
+  constexpr uint32_t STAGE_BYTES = C * 128;
+  unsigned char* sm = rc.sm;
+  const uint32_t sbase = rc.sbase, tmem = rc.tmem;
+  Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
+  const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  volatile int* abort_flag = &mi->abort_flag;
+  const int S = rc.S, R = rc.R;
+  const bool mlp = g.mode == 2;
+  const int n_chunks = 4 + (mlp ? g.n_f1 + 1 : 0);
+  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp; (void)R;
+  (void)tmem; (void)S; (void)n_chunks; (void)tid;
     if (lane == 0) {
       int stage = 0, slot = 0;
       uint32_t phase = 0, a_phase = 0, sphase = 0;
@@ -666,9 +707,30 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
       }
     mma_done:;
     }
-    __syncwarp();
-  } else {
-    // ================= compute warps =================================================================
+}
+
+// ================= compute warps ========================================================================
+template <int C, int D, int NT, bool BLOCKED>
+__device__ __forceinline__ void compute_role(const dsvt_fused_args& a, const TcGeom& g, int32_t* __restrict__ status,
+                                          const RoleCtx rc) {
+  constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
+  constexpr uint32_t COL_PARK = kTmemCols - C;  // parked fp32 x1
+  constexpr int C4 = C / 4;
+  const dsvt_layer_params& p = a.p;
+  constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
+  constexpr uint32_t COL_B = C;      // second accumulator buffer
+  constexpr uint32_t STAGE_BYTES = C * 128;
+  unsigned char* sm = rc.sm;
+  const uint32_t sbase = rc.sbase, tmem = rc.tmem;
+  Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
+  const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  volatile int* abort_flag = &mi->abort_flag;
+  const int S = rc.S, R = rc.R;
+  const bool mlp = g.mode == 2;
+  const int n_chunks = 4 + (mlp ? g.n_f1 + 1 : 0);
+  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp; (void)R;
+  (void)tmem; (void)S; (void)n_chunks; (void)tid;
     // epilogues: four threads per tile row; warp w owns TMEM lanes 32 (w % 4) .. + 31 and column quarter w / 4
     const int row = 32 * (warp & 3) + lane;
     const int hq = warp >> 2;
@@ -794,10 +856,8 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
         const uint32_t bar = (c == 1) ? 1u : 0u;
         acc_wait(bar);
         if (c == 2 ? live : live_kv) {
-          uint32_t rr[QC];
-#pragma unroll
-          for (int j = 0; j < QC / 16; ++j)
-            tmem_ld16_nowait(tmem + lane_addr + (c == 1 ? COL_B : 0u) + hq * QC + 16 * j, &rr[16 * j]);
+          float rr[QC];
+          tmem_ld_row(tmem + lane_addr + (c == 1 ? COL_B : 0u) + hq * QC, rr);
           tmem_wait_ld();
           acc_release(bar);  // the accumulator is in registers now
           const float* bias = p.b_qkv ? p.b_qkv + (c == 0 ? 1 : c == 1 ? 2 : 0) * C + hq * QC : nullptr;
@@ -806,12 +866,9 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
           for (int q = 0; q < QC / 8; ++q) {
             float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
             if (bias) { b0 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q); b1 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q + 1); }
-            const uint32_t* r8 = &rr[8 * q];
             *reinterpret_cast<uint4*>(dst + swz(row, ((hq * QC) >> 3) + q)) =
-                make_uint4(pack_bf16(__uint_as_float(r8[0]) + b0.x, __uint_as_float(r8[1]) + b0.y),
-                           pack_bf16(__uint_as_float(r8[2]) + b0.z, __uint_as_float(r8[3]) + b0.w),
-                           pack_bf16(__uint_as_float(r8[4]) + b1.x, __uint_as_float(r8[5]) + b1.y),
-                           pack_bf16(__uint_as_float(r8[6]) + b1.z, __uint_as_float(r8[7]) + b1.w));
+                make_uint4(pack_bf16(rr[8 * q] + b0.x, rr[8 * q + 1] + b0.y), pack_bf16(rr[8 * q + 2] + b0.z, rr[8 * q + 3] + b0.w),
+                           pack_bf16(rr[8 * q + 4] + b1.x, rr[8 * q + 5] + b1.y), pack_bf16(rr[8 * q + 6] + b1.z, rr[8 * q + 7] + b1.w));
           }
         } else {
           acc_release(bar);
@@ -849,9 +906,7 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
         float t[QC];
         float sum = 0.f;
         {
-          uint32_t rr[QC];
-#pragma unroll
-          for (int j = 0; j < QC / 16; ++j) tmem_ld16_nowait(tmem + lane_addr + hq * QC + 16 * j, &rr[16 * j]);
+          tmem_ld_row(tmem + lane_addr + hq * QC, t);
           tmem_wait_ld();
           acc_release(0u);
 #pragma unroll
@@ -860,10 +915,10 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
             if (g.mode != 0 && row < rows)
               x4 = *reinterpret_cast<const float4*>(sm + g.off_kv + stage_off<C>(row, hq * (QC / 4) + q));
             if (p.b_o) b4 = __ldg(reinterpret_cast<const float4*>(p.b_o + hq * QC) + q);
-            t[4 * q] = __uint_as_float(rr[4 * q]) + x4.x + b4.x;
-            t[4 * q + 1] = __uint_as_float(rr[4 * q + 1]) + x4.y + b4.y;
-            t[4 * q + 2] = __uint_as_float(rr[4 * q + 2]) + x4.z + b4.z;
-            t[4 * q + 3] = __uint_as_float(rr[4 * q + 3]) + x4.w + b4.w;
+            t[4 * q] += x4.x + b4.x;
+            t[4 * q + 1] += x4.y + b4.y;
+            t[4 * q + 2] += x4.z + b4.z;
+            t[4 * q + 3] += x4.w + b4.w;
             sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
           }
         }
@@ -879,8 +934,7 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
           continue;
         }
         // x1: bf16 A operand of MLP-1 in shared memory, fp32 copy parked in TMEM for the second residual
-#pragma unroll
-        for (int j = 0; j < QC / 16; ++j) tmem_st16(tmem + lane_addr + COL_PARK + hq * QC + 16 * j, &t[16 * j]);
+        tmem_st_row(tmem + lane_addr + COL_PARK + hq * QC, t);
         tmem_wait_st();
 #pragma unroll
         for (int q = 0; q < QC / 8; ++q)
@@ -897,9 +951,10 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
         acc_wait(bar);
         if (live) {
           const int qw = g.NF >> 2;  // columns per thread: 32 or 16
-          uint32_t rr[32];
-          tmem_ld16_nowait(tmem + lane_addr + bar * (uint32_t)g.NF + hq * qw, &rr[0]);
-          if (qw > 16) tmem_ld16_nowait(tmem + lane_addr + bar * (uint32_t)g.NF + hq * qw + 16, &rr[16]);
+          float rr[32];
+          const uint32_t src = tmem + lane_addr + bar * (uint32_t)g.NF + hq * qw;
+          tmem_ld16_at<0>(src, rr);
+          if (qw > 16) tmem_ld16_at<16>(src + 16, rr);
           tmem_wait_ld();
           acc_release(bar);
           const int col0 = c * g.NF + hq * qw;  // first hidden column of this thread
@@ -908,12 +963,11 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
             if (8 * q < qw) {
               float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
               if (p.b_1) { b0 = __ldg(reinterpret_cast<const float4*>(p.b_1 + col0) + 2 * q); b1 = __ldg(reinterpret_cast<const float4*>(p.b_1 + col0) + 2 * q + 1); }
-              const uint32_t* r8 = &rr[8 * q];
               *reinterpret_cast<uint4*>(sm + g.off_kv + swz(row, (col0 >> 3) + q)) =
-                  make_uint4(pack_bf16(gelu_fast(__uint_as_float(r8[0]) + b0.x), gelu_fast(__uint_as_float(r8[1]) + b0.y)),
-                             pack_bf16(gelu_fast(__uint_as_float(r8[2]) + b0.z), gelu_fast(__uint_as_float(r8[3]) + b0.w)),
-                             pack_bf16(gelu_fast(__uint_as_float(r8[4]) + b1.x), gelu_fast(__uint_as_float(r8[5]) + b1.y)),
-                             pack_bf16(gelu_fast(__uint_as_float(r8[6]) + b1.z), gelu_fast(__uint_as_float(r8[7]) + b1.w)));
+                  make_uint4(pack_bf16(gelu_fast(rr[8 * q] + b0.x), gelu_fast(rr[8 * q + 1] + b0.y)),
+                             pack_bf16(gelu_fast(rr[8 * q + 2] + b0.z), gelu_fast(rr[8 * q + 3] + b0.w)),
+                             pack_bf16(gelu_fast(rr[8 * q + 4] + b1.x), gelu_fast(rr[8 * q + 5] + b1.y)),
+                             pack_bf16(gelu_fast(rr[8 * q + 6] + b1.z), gelu_fast(rr[8 * q + 7] + b1.w)));
             }
           }
         } else {
@@ -929,24 +983,29 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
         float t[QC];
         float sum = 0.f;
         {
-          uint32_t rr[QC], rp[QC];
-#pragma unroll
-          for (int j = 0; j < QC / 16; ++j) {
-            tmem_ld16_nowait(tmem + lane_addr + hq * QC + 16 * j, &rr[16 * j]);
-            tmem_ld16_nowait(tmem + lane_addr + COL_PARK + hq * QC + 16 * j, &rp[16 * j]);
-          }
+          tmem_ld_row(tmem + lane_addr + hq * QC, t);
           tmem_wait_ld();
           acc_release(bar);
+          // + parked x1 and bias, 16 columns at a time (keeps the register footprint at one row quarter)
+          auto add_park = [&](auto off) {
+            constexpr int OFF = decltype(off)::value;
+            float rp[16];
+            tmem_ld16_at<0>(tmem + lane_addr + COL_PARK + hq * QC + OFF, rp);
+            tmem_wait_ld();
 #pragma unroll
-          for (int q = 0; q < QC / 4; ++q) {
-            float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (p.b_2) b4 = __ldg(reinterpret_cast<const float4*>(p.b_2 + hq * QC) + q);
-            t[4 * q] = __uint_as_float(rr[4 * q]) + __uint_as_float(rp[4 * q]) + b4.x;
-            t[4 * q + 1] = __uint_as_float(rr[4 * q + 1]) + __uint_as_float(rp[4 * q + 1]) + b4.y;
-            t[4 * q + 2] = __uint_as_float(rr[4 * q + 2]) + __uint_as_float(rp[4 * q + 2]) + b4.z;
-            t[4 * q + 3] = __uint_as_float(rr[4 * q + 3]) + __uint_as_float(rp[4 * q + 3]) + b4.w;
-            sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
-          }
+            for (int q = 0; q < 4; ++q) {
+              float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (p.b_2) b4 = __ldg(reinterpret_cast<const float4*>(p.b_2 + hq * QC + OFF) + q);
+              t[OFF + 4 * q] += rp[4 * q] + b4.x;
+              t[OFF + 4 * q + 1] += rp[4 * q + 1] + b4.y;
+              t[OFF + 4 * q + 2] += rp[4 * q + 2] + b4.z;
+              t[OFF + 4 * q + 3] += rp[4 * q + 3] + b4.w;
+              sum += (t[OFF + 4 * q] + t[OFF + 4 * q + 1]) + (t[OFF + 4 * q + 2] + t[OFF + 4 * q + 3]);
+            }
+          };
+          add_park(std::integral_constant<int, 0>{});
+          if constexpr (QC > 16) add_park(std::integral_constant<int, 16>{});
+          if constexpr (QC > 32) add_park(std::integral_constant<int, 32>{});
         }
         if (p.ln2_g) layer_norm(t, sum, p.ln2_g, p.ln2_b);
         // the MLP-2 MMAs have read H: its region takes the fp32 output rows
@@ -960,13 +1019,67 @@ layer_tc_kernel(dsvt_fused_args a, TcGeom g, const __grid_constant__ TcMaps maps
     if (!ok || *abort_flag) {
       if (tid == 0) atomicOr(status, DSVT_STATUS_TIMEOUT);
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------------------------
+template <int C, int D, int NT, bool BLOCKED>
+__global__ void __launch_bounds__(kThreads, 1)
+layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant__ TcGeom g,
+                const __grid_constant__ TcMaps maps, int32_t* __restrict__ status) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
+  unsigned char* sm = smem_raw + pad;
+  Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i) { mbar_init(&mi->full[i], 1); mbar_init(&mi->empty[i], 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&mi->acc_full[i], 1);
+      mbar_init(&mi->acc_free[i], kComputeThreads);
+      mbar_init(&mi->sched_full[i], 1);
+      mbar_init(&mi->sched_empty[i], kComputeThreads + 1);
+    }
+    mbar_init(&mi->a_ready, kComputeThreads);
+    mi->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kMmaWarp) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&mi->tmem_base)),
+                 "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // rows of K / V past the end of a tile are read (and masked) by the attention: never let them hold
+  // uninitialised bit patterns
+  for (uint32_t i = tid; i < (uint32_t)kTM * 2 * C * 2 / 16; i += kThreads)
+    reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  RoleCtx rc;
+  rc.sm = sm;
+  rc.sbase = raw + pad;
+  rc.tmem = mi->tmem_base;
+  rc.S = min(*a.num_sets, a.cap_sets);
+  rc.R = rc.S > 0 ? a.rowoff[rc.S] : 0;
+
+  if (warp == kTmaWarp) {
+    if ((tid & 31) == 0) producer_role<C>(a, g, maps, status, rc);
+    __syncwarp();
+  } else if (warp == kMmaWarp) {
+    if ((tid & 31) == 0) mma_role<C>(a, g, rc);
+    __syncwarp();
+  } else {
+    compute_role<C, D, NT, BLOCKED>(a, g, status, rc);
   }
   // ---- teardown: everyone meets here, then the allocating warp returns the TMEM columns ----
   tc_fence_before();
   __syncthreads();
   if (warp == kMmaWarp) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(rc.tmem), "r"(kTmemCols) : "memory");
   }
 }
 
