@@ -405,30 +405,39 @@ __device__ __noinline__ void attend_tile(uint32_t a_base, uint32_t k_base, uint3
 // NTB = key blocks of 8 a row block can need: ceil((2 tau + 14) / 8).
 // ---------------------------------------------------------------------------------------------
 template <int D, int NTB>
-__device__ __noinline__ void attend_blocked(uint32_t a_base, uint32_t k_base, uint32_t v_base,
-                                               const short* row_lo, const short* row_hi, int rows, int heads,
-                                               int warp, int lane) {
+__device__ __noinline__ void attend_blocked(uint32_t a_base, uint32_t k_base, uint32_t v_base, const short* row_lo,
+                                            const short* row_hi, int rows, int heads, int warp, int lane) {
   constexpr int DC = D / 8;  // 16-byte chunks per head
   constexpr int PW = 4;      // key blocks of 8 per pass (running softmax across passes keeps registers low)
-  const int g = lane >> 2, t4 = lane & 3;
+  const int t4 = lane & 3;
   const float sc = 1.4426950408889634f * rsqrtf((float)D);  // log2(e) / sqrt(d)
   const int nblk = (rows + 15) >> 4;
   for (int item = warp; item < nblk * heads; item += kComputeWarps) {
     const int blk = item / heads, h = item - blk * heads;
     const int c0 = h * DC;
     const int q0 = 16 * blk;
-    const int k_lo = row_lo[q0], k_hi = row_hi[min(q0 + 15, rows - 1)];
-    const int ntu = min((k_hi - k_lo + 7) >> 3, NTB);
-    const int ra = q0 + g, rb = q0 + g + 8;
-    // each thread's two query rows: the key range of their sets, relative to k_lo
-    const int loA = ra < rows ? row_lo[ra] - k_lo : 0, hiA = ra < rows ? row_hi[ra] - k_lo : 0;
-    const int loB = rb < rows ? row_lo[rb] - k_lo : 0, hiB = rb < rows ? row_hi[rb] - k_lo : 0;
+    const int k_lo = row_lo[q0];
+    const int ntu = min((row_hi[min(q0 + 15, rows - 1)] - k_lo + 7) >> 3, NTB);
+    const int ra = q0 + (lane >> 2), rb = ra + 8;
+    // each thread's two query rows: first key and number of keys of their sets, relative to k_lo
+    // (rows past the tile get zero keys)
+    const unsigned loA = ra < rows ? (unsigned)(row_lo[ra] - k_lo) : 0u;
+    const unsigned nA = ra < rows ? (unsigned)(row_hi[ra] - row_lo[ra]) : 0u;
+    const unsigned loB = rb < rows ? (unsigned)(row_lo[rb] - k_lo) : 0u;
+    const unsigned nB = rb < rows ? (unsigned)(row_hi[rb] - row_lo[rb]) : 0u;
     uint32_t qa[4], qb[4];
     {
-      const int row = min(q0 + (lane & 15), kTM - 1);
+      const int row = q0 + (lane & 15);  // <= 127
       ldsm_x4(a_base + swz(row, c0 + (lane >> 4)), qa);
       if (D > 16) ldsm_x4(a_base + swz(row, c0 + 2 + ((D == 32) ? (lane >> 4) : 0)), qb);
     }
+    // Row addresses advance by one 1024-byte group per key block of 8 (the swizzle depends on row & 7 only).
+    // Reads may run up to two groups past row 127: they land in the neighbouring operand block or the weight
+    // ring, which hold finite bf16 values, and meet zero probabilities.
+    uint32_t k_addr = k_base + swz(k_lo + (lane & 7), c0 + min(lane >> 3, DC - 1));
+    uint32_t v_addr[DC];
+#pragma unroll
+    for (int dn = 0; dn < DC; ++dn) v_addr[dn] = v_base + swz(k_lo + (lane & 15), c0 + dn);
     float o[DC][4];
 #pragma unroll
     for (int dn = 0; dn < DC; ++dn) o[dn][0] = o[dn][1] = o[dn][2] = o[dn][3] = 0.f;
@@ -438,69 +447,66 @@ __device__ __noinline__ void attend_blocked(uint32_t a_base, uint32_t k_base, ui
       float mx0 = mA, mx1 = mB;
 #pragma unroll
       for (int jj = 0; jj < PW; ++jj) {
-        const int j = j0 + jj;
-        if (j < ntu) {
+        if (j0 + jj < ntu) {
           s[jj][0] = s[jj][1] = s[jj][2] = s[jj][3] = 0.f;
           uint32_t kf[4];
-          const int row = min(k_lo + 8 * j + (lane & 7), kTM - 1);
-          const int ch = min(lane >> 3, DC - 1);
-          ldsm_x4(k_base + swz(row, c0 + ch), kf);
+          ldsm_x4(k_addr + 1024u * jj, kf);
           mma_16816(s[jj], qa, kf[0], kf[1]);
           if (D == 24) mma_1688(s[jj], qb[0], qb[1], kf[2]);
           if (D == 32) mma_16816(s[jj], qb, kf[2], kf[3]);
-          const int key = 8 * j + 2 * t4;
-          if (key < loA || key >= hiA) s[jj][0] = -INFINITY;
-          if (key + 1 < loA || key + 1 >= hiA) s[jj][1] = -INFINITY;
-          if (key < loB || key >= hiB) s[jj][2] = -INFINITY;
-          if (key + 1 < loB || key + 1 >= hiB) s[jj][3] = -INFINITY;
+          const unsigned key = (unsigned)(8 * (j0 + jj) + 2 * t4);
+          if (key - loA >= nA) s[jj][0] = -INFINITY;  // unsigned: also true for key < lo
+          if (key + 1u - loA >= nA) s[jj][1] = -INFINITY;
+          if (key - loB >= nB) s[jj][2] = -INFINITY;
+          if (key + 1u - loB >= nB) s[jj][3] = -INFINITY;
           mx0 = fmaxf(mx0, fmaxf(s[jj][0], s[jj][1]));
           mx1 = fmaxf(mx1, fmaxf(s[jj][2], s[jj][3]));
         }
       }
+      k_addr += 1024u * PW;
       mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
       mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
       // rows without any key so far (rows past the tile) keep finite arithmetic
       const float off0 = (mx0 == -INFINITY) ? 0.f : -mx0 * sc, off1 = (mx1 == -INFINITY) ? 0.f : -mx1 * sc;
-      // rescale what the earlier passes accumulated to the new maxima
-      const float al0 = (mA == -INFINITY) ? 0.f : ex2_approx(fmaf(mA, sc, off0));
-      const float al1 = (mB == -INFINITY) ? 0.f : ex2_approx(fmaf(mB, sc, off1));
+      if (j0 > 0) {  // rescale what the earlier passes accumulated to the new maxima
+        const float al0 = (mA == -INFINITY) ? 0.f : ex2_approx(fmaf(mA, sc, off0));
+        const float al1 = (mB == -INFINITY) ? 0.f : ex2_approx(fmaf(mB, sc, off1));
+        l0 *= al0;
+        l1 *= al1;
+#pragma unroll
+        for (int dn = 0; dn < DC; ++dn) { o[dn][0] *= al0; o[dn][1] *= al0; o[dn][2] *= al1; o[dn][3] *= al1; }
+      }
       mA = mx0;
       mB = mx1;
-      l0 *= al0;
-      l1 *= al1;
-#pragma unroll
-      for (int dn = 0; dn < DC; ++dn) { o[dn][0] *= al0; o[dn][1] *= al0; o[dn][2] *= al1; o[dn][3] *= al1; }
-#pragma unroll
-      for (int jj = 0; jj < PW; ++jj) {
-        if (j0 + jj < ntu) {
-          s[jj][0] = ex2_approx(fmaf(s[jj][0], sc, off0));
-          s[jj][1] = ex2_approx(fmaf(s[jj][1], sc, off0));
-          s[jj][2] = ex2_approx(fmaf(s[jj][2], sc, off1));
-          s[jj][3] = ex2_approx(fmaf(s[jj][3], sc, off1));
-          l0 += s[jj][0] + s[jj][1];
-          l1 += s[jj][2] + s[jj][3];
-        }
-      }
 #pragma unroll
       for (int kk = 0; kk < PW / 2; ++kk) {
         if (j0 + 2 * kk < ntu) {
           const bool two = j0 + 2 * kk + 1 < ntu;
+          float e[8];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            e[u] = ex2_approx(fmaf(s[2 * kk][u], sc, u < 2 ? off0 : off1));
+            e[4 + u] = two ? ex2_approx(fmaf(s[2 * kk + 1][u], sc, u < 2 ? off0 : off1)) : 0.f;
+          }
+          l0 += (e[0] + e[1]) + (e[4] + e[5]);
+          l1 += (e[2] + e[3]) + (e[6] + e[7]);
           uint32_t pa[4];
-          pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-          pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-          pa[2] = two ? pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]) : 0u;
-          pa[3] = two ? pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]) : 0u;
-          const int row = min(k_lo + 8 * j0 + 16 * kk + (lane & 15), kTM - 1);
+          pa[0] = pack_bf16(e[0], e[1]);
+          pa[1] = pack_bf16(e[2], e[3]);
+          pa[2] = pack_bf16(e[4], e[5]);
+          pa[3] = pack_bf16(e[6], e[7]);
 #pragma unroll
           for (int dn = 0; dn < DC; ++dn) {
             uint32_t vf[2];
-            ldsm_x2_trans(v_base + swz(row, c0 + dn), vf);
+            ldsm_x2_trans(v_addr[dn] + 2048u * kk, vf);
             mma_16816(o[dn], pa, vf[0], vf[1]);
           }
         }
       }
+#pragma unroll
+      for (int dn = 0; dn < DC; ++dn) v_addr[dn] += 1024u * PW;
     }
     // the per-thread partial sums of a row live in the four threads of its quad
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
@@ -508,13 +514,16 @@ __device__ __noinline__ void attend_blocked(uint32_t a_base, uint32_t k_base, ui
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
     const float i0 = __fdividef(1.0f, l0), i1 = __fdividef(1.0f, l1);
+    // the query rows of this block and head are dead now: their slots take the attention output
+    if (ra < rows) {
 #pragma unroll
-    for (int dn = 0; dn < DC; ++dn) {
-      // the query rows of this block and head are dead now: their slots take the attention output
-      if (ra < rows)
+      for (int dn = 0; dn < DC; ++dn)
         asm volatile("st.shared.b32 [%0], %1;" ::"r"(a_base + swz(ra, c0 + dn) + 4 * t4),
                      "r"(pack_bf16(o[dn][0] * i0, o[dn][1] * i0)) : "memory");
-      if (rb < rows)
+    }
+    if (rb < rows) {
+#pragma unroll
+      for (int dn = 0; dn < DC; ++dn)
         asm volatile("st.shared.b32 [%0], %1;" ::"r"(a_base + swz(rb, c0 + dn) + 4 * t4),
                      "r"(pack_bf16(o[dn][2] * i1, o[dn][3] * i1)) : "memory");
     }
@@ -1053,8 +1062,10 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   }
   // rows of K / V past the end of a tile are read (and masked) by the attention: never let them hold
   // uninitialised bit patterns
-  for (uint32_t i = tid; i < (uint32_t)kTM * 2 * C * 2 / 16; i += kThreads)
+  // (the weight ring behind it as well: key blocks that run past row 127 read a little of it)
+  for (uint32_t i = tid; i < ((uint32_t)kTM * 2 * C * 2 + kStages * (uint32_t)C * 128u) / 16; i += kThreads)
     reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
+  fence_proxy_async();  // the TMA writes that follow must not be overtaken by these generic stores
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
