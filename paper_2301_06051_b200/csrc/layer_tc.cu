@@ -719,315 +719,368 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
 }
 
 // ================= compute warps ========================================================================
+// Each phase of a tile is a separate (not inlined) function with a handful of scalar arguments, so that each
+// gets a register allocation of its own and the tile loop keeps only a few values alive across them.
+
+// Distinct slots of each set -> tile rows (Eq. 4), per-row set ranges, per-set first rows.
+__device__ __noinline__ void phase_row_list(const int32_t* __restrict__ table, const int32_t* __restrict__ rowoff, int n,
+                                            int tau, int s_lo, int nsets, int base, int rows, Misc* mi,
+                                            int32_t* __restrict__ status) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int si = warp; si < nsets; si += kComputeWarps) {
+    const int s = s_lo + si;
+    const int32_t* trow = table + (size_t)s * tau;
+    const int lb = rowoff[s] - base, cap = rowoff[s + 1] - rowoff[s];
+    int cnt = 0;
+    for (int k0 = 0; k0 < tau; k0 += 32) {
+      const int k = k0 + lane;
+      int v = -1;
+      bool uniq = false;
+      if (k < tau) { v = trow[k]; uniq = (k == 0) || (v != trow[k - 1]); }
+      const unsigned bal = __ballot_sync(0xffffffffu, uniq);
+      const int pos = cnt + __popc(bal & ((1u << lane) - 1u));
+      if (uniq && pos < cap && lb >= 0 && lb + pos < kTM) {
+        if (v < 0 || v >= n) { atomicOr(status, DSVT_STATUS_BAD_INDEX); v = -1; }
+        mi->rowvox[lb + pos] = v;
+      }
+      cnt += __popc(bal);
+    }
+    if (lb >= 0)
+      for (int i = lane; i < cap && lb + i < kTM; i += 32) {
+        mi->row_lo[lb + i] = (short)lb;
+        mi->row_hi[lb + i] = (short)min(lb + cap, kTM);
+      }
+    if (lane == 0) {
+      mi->set_lo[si] = min(max(lb, 0), kTM);
+      if (cnt != cap) atomicOr(status, DSVT_STATUS_BAD_INDEX);
+    }
+  }
+  if (tid == 0) mi->set_lo[nsets] = rows;
+}
+
+// Gather: fp32 rows -> bf16 A operand (four rows in flight per warp); all 128 rows are written.
+template <int C>
+__device__ __noinline__ void phase_gather(const float* __restrict__ x, const int* rowvox, int rows, unsigned char* a_tile) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int r0 = warp; r0 < kTM; r0 += 4 * kComputeWarps) {
+    float4 f[4][2];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = r0 + kComputeWarps * u;
+      const int v = r < rows ? rowvox[r] : -1;
+      f[u][0] = f[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (v >= 0 && lane < (C >> 3)) {
+        const float4* src = reinterpret_cast<const float4*>(x + (size_t)v * C) + 2 * lane;
+        f[u][0] = __ldg(src);
+        f[u][1] = __ldg(src + 1);
+      }
+    }
+    if (lane < (C >> 3)) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        *reinterpret_cast<uint4*>(a_tile + swz(r0 + kComputeWarps * u, lane)) =
+            make_uint4(pack_bf16(f[u][0].x, f[u][0].y), pack_bf16(f[u][0].z, f[u][0].w),
+                       pack_bf16(f[u][1].x, f[u][1].y), pack_bf16(f[u][1].z, f[u][1].w));
+    }
+  }
+}
+
+// Epilogue of a projection chunk: QC accumulator columns + bias -> bf16 into an operand tile.
+// GELU = true applies gelu first (MLP-1).  c8 = first 16-byte chunk of this thread in the destination.
+template <int QC, bool GELU>
+__device__ __noinline__ void phase_epi_bf16(uint32_t taddr, unsigned long long* acc_free, const float* __restrict__ bias,
+                                            unsigned char* dst, int row, int c8) {
+  float rr[QC];
+  tmem_ld_row(taddr, rr);
+  tmem_wait_ld();
+  tc_fence_before();
+  mbar_arrive(acc_free);  // the accumulator is in registers now
+#pragma unroll
+  for (int q = 0; q < QC / 8; ++q) {
+    float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+    if (bias) { b0 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q); b1 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q + 1); }
+    float v[8] = {rr[8 * q] + b0.x, rr[8 * q + 1] + b0.y, rr[8 * q + 2] + b0.z, rr[8 * q + 3] + b0.w,
+                  rr[8 * q + 4] + b1.x, rr[8 * q + 5] + b1.y, rr[8 * q + 6] + b1.z, rr[8 * q + 7] + b1.w};
+    if (GELU) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = gelu_fast(v[e]);
+    }
+    *reinterpret_cast<uint4*>(dst + swz(row, c8 + q)) =
+        make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+  }
+}
+
+// x rows (fp32) for the first residual: asynchronous 16-byte copies global -> shared staging.
+template <int C>
+__device__ __noinline__ void phase_stage_x(const float* __restrict__ x, const int* rowvox, int rows, unsigned char* stage,
+                                           uint32_t stage_saddr) {
+  constexpr int C4 = C / 4;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int r = warp; r < rows; r += kComputeWarps) {
+    const int v = rowvox[r];
+    for (int c4 = lane; c4 < C4; c4 += 32) {
+      const uint32_t off = stage_off<C>(r, c4);
+      if (v >= 0)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_saddr + off),
+                     "l"(reinterpret_cast<const float4*>(x + (size_t)v * C) + c4) : "memory");
+      else
+        *reinterpret_cast<float4*>(stage + off) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+}
+
+// fp32 rows staged in shared memory -> coalesced global rows.
+template <int C>
+__device__ __noinline__ void phase_store_rows(float* __restrict__ y, const int* rowvox, int rows, const unsigned char* stage) {
+  constexpr int C4 = C / 4;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int r = warp; r < rows; r += kComputeWarps) {
+    const int v = rowvox[r];
+    if (v < 0) continue;
+    for (int c4 = lane; c4 < C4; c4 += 32)
+      reinterpret_cast<float4*>(y + (size_t)v * C)[c4] = *reinterpret_cast<const float4*>(stage + stage_off<C>(r, c4));
+  }
+}
+
+struct LnArgs {
+  const float *bias, *gain, *shift;  // projection bias, LayerNorm gain (NULL: no LayerNorm) and shift
+  float eps;
+};
+
+// LayerNorm over the row that four threads share: t holds this thread's QC values.
+template <int C, int QC>
+__device__ __forceinline__ void layer_norm_rows(float (&t)[QC], float sum, const LnArgs& ln, Misc* mi, int row, int hq) {
+  mi->red[0][hq][row] = sum;
+  compute_sync();
+  const float mean = (mi->red[0][0][row] + mi->red[0][1][row] + mi->red[0][2][row] + mi->red[0][3][row]) * (1.0f / (float)C);
+  float sq = 0.f;
+#pragma unroll
+  for (int i = 0; i < QC; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
+  mi->red[1][hq][row] = sq;
+  compute_sync();
+  const float var = (mi->red[1][0][row] + mi->red[1][1][row] + mi->red[1][2][row] + mi->red[1][3][row]) * (1.0f / (float)C);
+  const float inv = rsqrtf(var + ln.eps);
+#pragma unroll
+  for (int i4 = 0; i4 < QC / 4; ++i4) {
+    const float4 g4 = __ldg(reinterpret_cast<const float4*>(ln.gain + hq * QC) + i4);
+    float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (ln.shift) b4 = __ldg(reinterpret_cast<const float4*>(ln.shift + hq * QC) + i4);
+    t[4 * i4] = t[4 * i4] * inv * g4.x + b4.x;
+    t[4 * i4 + 1] = t[4 * i4 + 1] * inv * g4.y + b4.y;
+    t[4 * i4 + 2] = t[4 * i4 + 2] * inv * g4.z + b4.z;
+    t[4 * i4 + 3] = t[4 * i4 + 3] * inv * g4.w + b4.w;
+  }
+}
+
+// Output-projection epilogue: t = Z + b_o (+ staged x); LayerNorm; then either the fp32 rows go to the staging
+// area (final result of the call: to_stage) or x1 goes to TMEM (fp32 park) and to the A operand (bf16).
+template <int C, int QC>
+__device__ __noinline__ void phase_epi_o(uint32_t taddr, unsigned long long* acc_free, LnArgs ln, bool add_x, bool to_stage,
+                                         unsigned char* stage, unsigned char* a_tile, uint32_t park_addr, Misc* mi,
+                                         int rows) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = 32 * (warp & 3) + lane, hq = warp >> 2;
+  float t[QC];
+  float sum = 0.f;
+  tmem_ld_row(taddr, t);
+  tmem_wait_ld();
+  tc_fence_before();
+  mbar_arrive(acc_free);
+#pragma unroll
+  for (int q = 0; q < QC / 4; ++q) {
+    float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f), b4 = x4;
+    if (add_x && row < rows) x4 = *reinterpret_cast<const float4*>(stage + stage_off<C>(row, hq * (QC / 4) + q));
+    if (ln.bias) b4 = __ldg(reinterpret_cast<const float4*>(ln.bias + hq * QC) + q);
+    t[4 * q] += x4.x + b4.x;
+    t[4 * q + 1] += x4.y + b4.y;
+    t[4 * q + 2] += x4.z + b4.z;
+    t[4 * q + 3] += x4.w + b4.w;
+    sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
+  }
+  if (ln.gain) layer_norm_rows<C, QC>(t, sum, ln, mi, row, hq);
+  if (to_stage) {
+    compute_sync();  // the x staging is dead once every thread has its t
+#pragma unroll
+    for (int i4 = 0; i4 < QC / 4; ++i4)
+      *reinterpret_cast<float4*>(stage + stage_off<C>(row, hq * (QC / 4) + i4)) =
+          make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
+    return;
+  }
+  tmem_st_row(park_addr, t);
+  tmem_wait_st();
+#pragma unroll
+  for (int q = 0; q < QC / 8; ++q)
+    *reinterpret_cast<uint4*>(a_tile + swz(row, ((hq * QC) >> 3) + q)) =
+        make_uint4(pack_bf16(t[8 * q], t[8 * q + 1]), pack_bf16(t[8 * q + 2], t[8 * q + 3]),
+                   pack_bf16(t[8 * q + 4], t[8 * q + 5]), pack_bf16(t[8 * q + 6], t[8 * q + 7]));
+  tc_fence_before();
+}
+
+// MLP-2 epilogue: t = M + b_2 + parked x1; LayerNorm; fp32 rows to the staging area.
+template <int C, int QC>
+__device__ __noinline__ void phase_epi_f2(uint32_t taddr, unsigned long long* acc_free, LnArgs ln, unsigned char* stage,
+                                          uint32_t park_addr, Misc* mi) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = 32 * (warp & 3) + lane, hq = warp >> 2;
+  float t[QC];
+  float sum = 0.f;
+  tmem_ld_row(taddr, t);
+  tmem_wait_ld();
+  tc_fence_before();
+  mbar_arrive(acc_free);
+  {
+    float rp[QC];
+    tmem_ld_row(park_addr, rp);
+    tmem_wait_ld();
+#pragma unroll
+    for (int q = 0; q < QC / 4; ++q) {
+      float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (ln.bias) b4 = __ldg(reinterpret_cast<const float4*>(ln.bias + hq * QC) + q);
+      t[4 * q] += rp[4 * q] + b4.x;
+      t[4 * q + 1] += rp[4 * q + 1] + b4.y;
+      t[4 * q + 2] += rp[4 * q + 2] + b4.z;
+      t[4 * q + 3] += rp[4 * q + 3] + b4.w;
+      sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
+    }
+  }
+  if (ln.gain) layer_norm_rows<C, QC>(t, sum, ln, mi, row, hq);
+  // the MLP-2 MMAs have read H: its region takes the fp32 output rows
+#pragma unroll
+  for (int i4 = 0; i4 < QC / 4; ++i4)
+    *reinterpret_cast<float4*>(stage + stage_off<C>(row, hq * (QC / 4) + i4)) =
+        make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
+}
+
 template <int C, int D, int NT, bool BLOCKED>
 __device__ __forceinline__ void compute_role(const dsvt_fused_args& a, const TcGeom& g, int32_t* __restrict__ status,
-                                          const RoleCtx rc) {
-  constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
-  constexpr uint32_t COL_PARK = kTmemCols - C;  // parked fp32 x1
-  constexpr int C4 = C / 4;
-  const dsvt_layer_params& p = a.p;
+                                             const RoleCtx rc) {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
+  constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
   constexpr uint32_t COL_B = C;      // second accumulator buffer
-  constexpr uint32_t STAGE_BYTES = C * 128;
+  constexpr uint32_t COL_PARK = kTmemCols - C;  // parked fp32 x1
+  const dsvt_layer_params& p = a.p;
   unsigned char* sm = rc.sm;
   const uint32_t sbase = rc.sbase, tmem = rc.tmem;
   Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
-  const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
+  const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &mi->abort_flag;
-  const int S = rc.S, R = rc.R;
-  const bool mlp = g.mode == 2;
-  const int n_chunks = 4 + (mlp ? g.n_f1 + 1 : 0);
-  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp; (void)R;
-  (void)tmem; (void)S; (void)n_chunks; (void)tid;
-    // epilogues: four threads per tile row; warp w owns TMEM lanes 32 (w % 4) .. + 31 and column quarter w / 4
-    const int row = 32 * (warp & 3) + lane;
-    const int hq = warp >> 2;
-    const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
-    uint32_t uses[2] = {0u, 0u};
-    int slot = 0;
-    uint32_t sphase = 0;
-    bool ok = true;
-    auto acc_wait = [&](uint32_t bar) {
-      ok = mbar_wait(&mi->acc_full[bar], uses[bar] & 1u, abort_flag) && ok;
-      ++uses[bar];
-      tc_fence_after();
-    };
-    auto acc_release = [&](uint32_t bar) {
-      tc_fence_before();
-      mbar_arrive(&mi->acc_free[bar]);
-    };
-    // fp32 rows staged in the K/V region -> coalesced global rows
-    auto store_rows = [&](int rows) {
-      compute_sync();
-      for (int r = warp; r < rows; r += kComputeWarps) {
-        const int v = mi->rowvox[r];
-        if (v < 0) continue;
-        for (int c4 = lane; c4 < C4; c4 += 32)
-          reinterpret_cast<float4*>(a.y + (size_t)v * C)[c4] =
-              *reinterpret_cast<const float4*>(sm + g.off_kv + stage_off<C>(r, c4));
-      }
-    };
-    // LayerNorm over the row that four threads share: t holds this thread's QC values
-    auto layer_norm = [&](float (&t)[QC], float sum, const float* gain, const float* shift) {
-      mi->red[0][hq][row] = sum;
-      compute_sync();
-      const float mean = (mi->red[0][0][row] + mi->red[0][1][row] + mi->red[0][2][row] + mi->red[0][3][row]) * (1.0f / (float)C);
-      float sq = 0.f;
-#pragma unroll
-      for (int i = 0; i < QC; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
-      mi->red[1][hq][row] = sq;
-      compute_sync();
-      const float var = (mi->red[1][0][row] + mi->red[1][1][row] + mi->red[1][2][row] + mi->red[1][3][row]) * (1.0f / (float)C);
-      const float inv = rsqrtf(var + p.ln_eps);
-#pragma unroll
-      for (int i4 = 0; i4 < QC / 4; ++i4) {
-        const float4 g4 = __ldg(reinterpret_cast<const float4*>(gain + hq * QC) + i4);
-        float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (shift) b4 = __ldg(reinterpret_cast<const float4*>(shift + hq * QC) + i4);
-        t[4 * i4] = t[4 * i4] * inv * g4.x + b4.x;
-        t[4 * i4 + 1] = t[4 * i4 + 1] * inv * g4.y + b4.y;
-        t[4 * i4 + 2] = t[4 * i4 + 2] * inv * g4.z + b4.z;
-        t[4 * i4 + 3] = t[4 * i4 + 3] * inv * g4.w + b4.w;
-      }
-    };
-    for (;;) {
-      ok = mbar_wait(&mi->sched_full[slot], sphase, abort_flag) && ok;
-      compute_sync();  // also orders the previous tile's last shared-memory reads before this tile's writes
-      if (*abort_flag) break;
-      const int s_lo = mi->tile[slot][0], nsets = mi->tile[slot][1], base = mi->tile[slot][2], rows = mi->tile[slot][3];
-      mbar_arrive(&mi->sched_empty[slot]);
-      if (++slot == 2) { slot = 0; sphase ^= 1u; }
-      if (nsets < 0) break;
-      const bool live = 32 * (warp & 3) < rows;  // this warp's 32 tile rows hold at least one voxel
-      // the attention pads its key blocks up to 15 rows past the tile: those K / V rows must be real bf16
-      const bool live_kv = 32 * (warp & 3) < rows + 16;
-      if (tid < kTM) { mi->rowvox[tid] = -1; mi->row_lo[tid] = (short)tid; mi->row_hi[tid] = (short)(tid + 1); }
-      compute_sync();
-      // ---- distinct slots of each set -> tile rows (Eq. 4) ----
-      for (int si = warp; si < nsets; si += kComputeWarps) {
-        const int s = s_lo + si;
-        const int32_t* trow = a.table + (size_t)s * g.tau;
-        const int lb = a.rowoff[s] - base, cap = a.rowoff[s + 1] - a.rowoff[s];
-        int cnt = 0;
-        for (int k0 = 0; k0 < g.tau; k0 += 32) {
-          const int k = k0 + lane;
-          int v = -1;
-          bool uniq = false;
-          if (k < g.tau) { v = trow[k]; uniq = (k == 0) || (v != trow[k - 1]); }
-          const unsigned bal = __ballot_sync(0xffffffffu, uniq);
-          const int pos = cnt + __popc(bal & ((1u << lane) - 1u));
-          if (uniq && pos < cap && lb >= 0 && lb + pos < kTM) {
-            if (v < 0 || v >= a.n) { atomicOr(status, DSVT_STATUS_BAD_INDEX); v = -1; }
-            mi->rowvox[lb + pos] = v;
-          }
-          cnt += __popc(bal);
-        }
-        if (lb >= 0)
-          for (int i = lane; i < cap && lb + i < kTM; i += 32) {
-            mi->row_lo[lb + i] = (short)lb;
-            mi->row_hi[lb + i] = (short)min(lb + cap, kTM);
-          }
-        if (lane == 0) {
-          mi->set_lo[si] = min(max(lb, 0), kTM);
-          if (cnt != cap) atomicOr(status, DSVT_STATUS_BAD_INDEX);
-        }
-      }
-      if (tid == 0) mi->set_lo[nsets] = rows;
-      compute_sync();
-      // ---- gather: fp32 rows -> bf16 A operand (four rows in flight per warp) ----
-      for (int r0 = warp; r0 < kTM; r0 += 4 * kComputeWarps) {
-        float4 f[4][2];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int r = r0 + kComputeWarps * u;
-          const int v = r < rows ? mi->rowvox[r] : -1;
-          f[u][0] = f[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (v >= 0 && lane < (C >> 3)) {
-            const float4* src = reinterpret_cast<const float4*>(a.x + (size_t)v * C) + 2 * lane;
-            f[u][0] = __ldg(src);
-            f[u][1] = __ldg(src + 1);
-          }
-        }
-        if (lane < (C >> 3)) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-            *reinterpret_cast<uint4*>(sm + g.off_a + swz(r0 + kComputeWarps * u, lane)) =
-                make_uint4(pack_bf16(f[u][0].x, f[u][0].y), pack_bf16(f[u][0].z, f[u][0].w),
-                           pack_bf16(f[u][1].x, f[u][1].y), pack_bf16(f[u][1].z, f[u][1].w));
-        }
-      }
-      fence_proxy_async();
-      mbar_arrive(&mi->a_ready);  // X is in place
+  // epilogues: four threads per tile row; warp w owns TMEM lanes 32 (w % 4) .. + 31 and column quarter w / 4
+  const int row = 32 * (warp & 3) + lane;
+  const int hq = warp >> 2;
+  const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+  uint32_t uses[2] = {0u, 0u};
+  int slot = 0;
+  uint32_t sphase = 0;
+  bool ok = true;
+  auto acc_wait = [&](uint32_t bar) {
+    ok = mbar_wait(&mi->acc_full[bar], uses[bar] & 1u, abort_flag) && ok;
+    ++uses[bar];
+    tc_fence_after();
+  };
+  auto acc_release = [&](uint32_t bar) {
+    tc_fence_before();
+    mbar_arrive(&mi->acc_free[bar]);
+  };
+  for (;;) {
+    ok = mbar_wait(&mi->sched_full[slot], sphase, abort_flag) && ok;
+    compute_sync();  // also orders the previous tile's last shared-memory reads before this tile's writes
+    if (*abort_flag) break;
+    const int s_lo = mi->tile[slot][0], nsets = mi->tile[slot][1], base = mi->tile[slot][2], rows = mi->tile[slot][3];
+    mbar_arrive(&mi->sched_empty[slot]);
+    if (++slot == 2) { slot = 0; sphase ^= 1u; }
+    if (nsets < 0) break;
+    const bool live = 32 * (warp & 3) < rows;  // this warp's 32 tile rows hold at least one voxel
+    // the attention pads its key blocks up to 15 rows past the tile: those K / V rows must be real bf16
+    const bool live_kv = 32 * (warp & 3) < rows + 16;
+    if (tid < kTM) { mi->rowvox[tid] = -1; mi->row_lo[tid] = (short)tid; mi->row_hi[tid] = (short)(tid + 1); }
+    compute_sync();
+    phase_row_list(a.table, a.rowoff, a.n, g.tau, s_lo, nsets, base, rows, mi, status);
+    compute_sync();
+    phase_gather<C>(a.x, mi->rowvox, rows, sm + g.off_a);
+    fence_proxy_async();
+    mbar_arrive(&mi->a_ready);  // X is in place
 
-      // ---- chunks 0..2: K, V, Q epilogues: + bias, to bf16, into the operand layout ----
-      for (int c = 0; c < 3; ++c) {
-        const uint32_t bar = (c == 1) ? 1u : 0u;
-        acc_wait(bar);
-        if (c == 2 ? live : live_kv) {
-          float rr[QC];
-          tmem_ld_row(tmem + lane_addr + (c == 1 ? COL_B : 0u) + hq * QC, rr);
-          tmem_wait_ld();
-          acc_release(bar);  // the accumulator is in registers now
-          const float* bias = p.b_qkv ? p.b_qkv + (c == 0 ? 1 : c == 1 ? 2 : 0) * C + hq * QC : nullptr;
-          unsigned char* dst = sm + (c == 2 ? g.off_a : g.off_kv + (uint32_t)c * (NKB * kTM * 128));
-#pragma unroll
-          for (int q = 0; q < QC / 8; ++q) {
-            float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
-            if (bias) { b0 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q); b1 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q + 1); }
-            *reinterpret_cast<uint4*>(dst + swz(row, ((hq * QC) >> 3) + q)) =
-                make_uint4(pack_bf16(rr[8 * q] + b0.x, rr[8 * q + 1] + b0.y), pack_bf16(rr[8 * q + 2] + b0.z, rr[8 * q + 3] + b0.w),
-                           pack_bf16(rr[8 * q + 4] + b1.x, rr[8 * q + 5] + b1.y), pack_bf16(rr[8 * q + 6] + b1.z, rr[8 * q + 7] + b1.w));
-          }
-        } else {
-          acc_release(bar);
-        }
-      }
-      compute_sync();
-      // ---- attention inside each set ----
-      if (BLOCKED)
-        attend_blocked<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->row_lo, mi->row_hi, rows, g.heads, warp, lane);
+    // ---- chunks 0..2: K, V, Q epilogues: + bias, to bf16, into the operand layout ----
+    for (int c = 0; c < 3; ++c) {
+      const uint32_t bar = (c == 1) ? 1u : 0u;
+      acc_wait(bar);
+      if (c == 2 ? live : live_kv)
+        phase_epi_bf16<QC, false>(tmem + lane_addr + (c == 1 ? COL_B : 0u) + hq * QC, &mi->acc_free[bar],
+                                  p.b_qkv ? p.b_qkv + (c == 0 ? 1 : c == 1 ? 2 : 0) * C + hq * QC : nullptr,
+                                  sm + (c == 2 ? g.off_a : g.off_kv + (uint32_t)c * (NKB * kTM * 128)), row,
+                                  (hq * QC) >> 3);
       else
-        attend_tile<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->set_lo, nsets, g.heads, warp, lane);
-      fence_proxy_async();
-      mbar_arrive(&mi->a_ready);  // attention output is the A operand of the output projection
-      compute_sync();             // every warp is done with K and V: their region becomes fp32 staging
-      if (g.mode != 0) {
-        // x rows (fp32) for the first residual: asynchronous 16-byte copies global -> shared, all of a
-        // warp's rows in flight at once, no registers involved
-        for (int r = warp; r < rows; r += kComputeWarps) {
-          const int v = mi->rowvox[r];
-          for (int c4 = lane; c4 < C4; c4 += 32) {
-            const uint32_t dst = sbase + g.off_kv + stage_off<C>(r, c4);
-            if (v >= 0)
-              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst),
-                           "l"(reinterpret_cast<const float4*>(a.x + (size_t)v * C) + c4) : "memory");
-            else
-              *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(r, c4)) = make_float4(0.f, 0.f, 0.f, 0.f);
-          }
-        }
-        asm volatile("cp.async.wait_all;" ::: "memory");
+        acc_release(bar);
+    }
+    compute_sync();
+    // ---- attention inside each set ----
+    if (BLOCKED)
+      attend_blocked<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->row_lo, mi->row_hi, rows, g.heads, warp, lane);
+    else
+      attend_tile<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->set_lo, nsets, g.heads, warp, lane);
+    fence_proxy_async();
+    mbar_arrive(&mi->a_ready);  // attention output is the A operand of the output projection
+    compute_sync();             // every warp is done with K and V: their region becomes fp32 staging
+    if (g.mode != 0) {
+      phase_stage_x<C>(a.x, mi->rowvox, rows, sm + g.off_kv, sbase + g.off_kv);
+      compute_sync();
+    }
+    // ---- chunk 3: output projection epilogue: Z + b_o (+ x, LayerNorm) ----
+    {
+      acc_wait(0u);
+      LnArgs ln;
+      ln.bias = p.b_o;
+      ln.gain = g.mode != 0 ? p.ln1_g : nullptr;
+      ln.shift = p.ln1_b;
+      ln.eps = p.ln_eps;
+      phase_epi_o<C, QC>(tmem + lane_addr + hq * QC, &mi->acc_free[0], ln, g.mode != 0, g.mode != 2, sm + g.off_kv,
+                         sm + g.off_a, tmem + lane_addr + COL_PARK + hq * QC, mi, rows);
+      if (g.mode != 2) {  // final result of this call
         compute_sync();
-      }
-      // ---- chunk 3: output projection epilogue: Z + b_o (+ x, LayerNorm) ----
-      {
-        acc_wait(0u);
-        float t[QC];
-        float sum = 0.f;
-        {
-          tmem_ld_row(tmem + lane_addr + hq * QC, t);
-          tmem_wait_ld();
-          acc_release(0u);
-#pragma unroll
-          for (int q = 0; q < QC / 4; ++q) {
-            float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f), b4 = x4;
-            if (g.mode != 0 && row < rows)
-              x4 = *reinterpret_cast<const float4*>(sm + g.off_kv + stage_off<C>(row, hq * (QC / 4) + q));
-            if (p.b_o) b4 = __ldg(reinterpret_cast<const float4*>(p.b_o + hq * QC) + q);
-            t[4 * q] += x4.x + b4.x;
-            t[4 * q + 1] += x4.y + b4.y;
-            t[4 * q + 2] += x4.z + b4.z;
-            t[4 * q + 3] += x4.w + b4.w;
-            sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
-          }
-        }
-        if (g.mode != 0 && p.ln1_g) layer_norm(t, sum, p.ln1_g, p.ln1_b);
-        if (!mlp) {
-          // final result of this call: stage it (the x staging is dead once every thread has its t)
-          compute_sync();
-#pragma unroll
-          for (int i4 = 0; i4 < QC / 4; ++i4)
-            *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(row, hq * (QC / 4) + i4)) =
-                make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
-          store_rows(rows);
-          continue;
-        }
-        // x1: bf16 A operand of MLP-1 in shared memory, fp32 copy parked in TMEM for the second residual
-        tmem_st_row(tmem + lane_addr + COL_PARK + hq * QC, t);
-        tmem_wait_st();
-#pragma unroll
-        for (int q = 0; q < QC / 8; ++q)
-          *reinterpret_cast<uint4*>(sm + g.off_a + swz(row, ((hq * QC) >> 3) + q)) =
-              make_uint4(pack_bf16(t[8 * q], t[8 * q + 1]), pack_bf16(t[8 * q + 2], t[8 * q + 3]),
-                         pack_bf16(t[8 * q + 4], t[8 * q + 5]), pack_bf16(t[8 * q + 6], t[8 * q + 7]));
-        tc_fence_before();
-        fence_proxy_async();
-        mbar_arrive(&mi->a_ready);  // x1 (bf16) is the A operand of MLP-1
-      }
-      // ---- MLP-1 pieces: H = gelu(x1 W_1^T + b_1) as the A operand of MLP-2 ----
-      for (int c = 0; c < g.n_f1; ++c) {
-        const uint32_t bar = (uint32_t)c & 1u;
-        acc_wait(bar);
-        if (live) {
-          const int qw = g.NF >> 2;  // columns per thread: 32 or 16
-          float rr[32];
-          const uint32_t src = tmem + lane_addr + bar * (uint32_t)g.NF + hq * qw;
-          tmem_ld16_at<0>(src, rr);
-          if (qw > 16) tmem_ld16_at<16>(src + 16, rr);
-          tmem_wait_ld();
-          acc_release(bar);
-          const int col0 = c * g.NF + hq * qw;  // first hidden column of this thread
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            if (8 * q < qw) {
-              float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
-              if (p.b_1) { b0 = __ldg(reinterpret_cast<const float4*>(p.b_1 + col0) + 2 * q); b1 = __ldg(reinterpret_cast<const float4*>(p.b_1 + col0) + 2 * q + 1); }
-              *reinterpret_cast<uint4*>(sm + g.off_kv + swz(row, (col0 >> 3) + q)) =
-                  make_uint4(pack_bf16(gelu_fast(rr[8 * q] + b0.x), gelu_fast(rr[8 * q + 1] + b0.y)),
-                             pack_bf16(gelu_fast(rr[8 * q + 2] + b0.z), gelu_fast(rr[8 * q + 3] + b0.w)),
-                             pack_bf16(gelu_fast(rr[8 * q + 4] + b1.x), gelu_fast(rr[8 * q + 5] + b1.y)),
-                             pack_bf16(gelu_fast(rr[8 * q + 6] + b1.z), gelu_fast(rr[8 * q + 7] + b1.w)));
-            }
-          }
-        } else {
-          acc_release(bar);
-        }
+        phase_store_rows<C>(a.y, mi->rowvox, rows, sm + g.off_kv);
+        continue;
       }
       fence_proxy_async();
-      mbar_arrive(&mi->a_ready);  // H is in place
-      // ---- MLP-2 epilogue: y = LN2(x1 + M) ----
-      {
-        const uint32_t bar = (uint32_t)g.n_f1 & 1u;
-        acc_wait(bar);
-        float t[QC];
-        float sum = 0.f;
-        {
-          tmem_ld_row(tmem + lane_addr + hq * QC, t);
-          tmem_wait_ld();
-          acc_release(bar);
-          // + parked x1 and bias, 16 columns at a time (keeps the register footprint at one row quarter)
-          auto add_park = [&](auto off) {
-            constexpr int OFF = decltype(off)::value;
-            float rp[16];
-            tmem_ld16_at<0>(tmem + lane_addr + COL_PARK + hq * QC + OFF, rp);
-            tmem_wait_ld();
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (p.b_2) b4 = __ldg(reinterpret_cast<const float4*>(p.b_2 + hq * QC + OFF) + q);
-              t[OFF + 4 * q] += rp[4 * q] + b4.x;
-              t[OFF + 4 * q + 1] += rp[4 * q + 1] + b4.y;
-              t[OFF + 4 * q + 2] += rp[4 * q + 2] + b4.z;
-              t[OFF + 4 * q + 3] += rp[4 * q + 3] + b4.w;
-              sum += (t[OFF + 4 * q] + t[OFF + 4 * q + 1]) + (t[OFF + 4 * q + 2] + t[OFF + 4 * q + 3]);
-            }
-          };
-          add_park(std::integral_constant<int, 0>{});
-          if constexpr (QC > 16) add_park(std::integral_constant<int, 16>{});
-          if constexpr (QC > 32) add_park(std::integral_constant<int, 32>{});
-        }
-        if (p.ln2_g) layer_norm(t, sum, p.ln2_g, p.ln2_b);
-        // the MLP-2 MMAs have read H: its region takes the fp32 output rows
-#pragma unroll
-        for (int i4 = 0; i4 < QC / 4; ++i4)
-          *reinterpret_cast<float4*>(sm + g.off_kv + stage_off<C>(row, hq * (QC / 4) + i4)) =
-              make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
-        store_rows(rows);
+      mbar_arrive(&mi->a_ready);  // x1 (bf16) is the A operand of MLP-1
+    }
+    // ---- MLP-1 pieces: H = gelu(x1 W_1^T + b_1) as the A operand of MLP-2 ----
+    for (int c = 0; c < g.n_f1; ++c) {
+      const uint32_t bar = (uint32_t)c & 1u;
+      acc_wait(bar);
+      if (live) {
+        const int qw = g.NF >> 2;             // columns per thread: 32 or 16
+        const int col0 = c * g.NF + hq * qw;  // first hidden column of this thread
+        const uint32_t src = tmem + lane_addr + bar * (uint32_t)g.NF + hq * qw;
+        if (qw == 32)
+          phase_epi_bf16<32, true>(src, &mi->acc_free[bar], p.b_1 ? p.b_1 + col0 : nullptr, sm + g.off_kv, row, col0 >> 3);
+        else
+          phase_epi_bf16<16, true>(src, &mi->acc_free[bar], p.b_1 ? p.b_1 + col0 : nullptr, sm + g.off_kv, row, col0 >> 3);
+      } else {
+        acc_release(bar);
       }
     }
-    if (!ok || *abort_flag) {
-      if (tid == 0) atomicOr(status, DSVT_STATUS_TIMEOUT);
+    fence_proxy_async();
+    mbar_arrive(&mi->a_ready);  // H is in place
+    // ---- MLP-2 epilogue: y = LN2(x1 + M) ----
+    {
+      const uint32_t bar = (uint32_t)g.n_f1 & 1u;
+      acc_wait(bar);
+      LnArgs ln;
+      ln.bias = p.b_2;
+      ln.gain = p.ln2_g;
+      ln.shift = p.ln2_b;
+      ln.eps = p.ln_eps;
+      phase_epi_f2<C, QC>(tmem + lane_addr + hq * QC, &mi->acc_free[bar], ln, sm + g.off_kv,
+                          tmem + lane_addr + COL_PARK + hq * QC, mi);
+      compute_sync();
+      phase_store_rows<C>(a.y, mi->rowvox, rows, sm + g.off_kv);
     }
+  }
+  if (!ok || *abort_flag) {
+    if (tid == 0) atomicOr(status, DSVT_STATUS_TIMEOUT);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
