@@ -851,14 +851,16 @@ struct LnArgs {
 // LayerNorm over the row that four threads share: t holds this thread's QC values.
 template <int C, int QC>
 __device__ __forceinline__ void layer_norm_rows(float (&t)[QC], float sum, const LnArgs& ln, Misc* mi, int row, int hq) {
+  // the four threads of a row sit in warps q, q + 4, q + 8, q + 12: they meet at a barrier of their own
+  const int quarter_bar = 2 + ((threadIdx.x >> 5) & 3);
   mi->red[0][hq][row] = sum;
-  compute_sync();
+  asm volatile("bar.sync %0, 128;" ::"r"(quarter_bar) : "memory");
   const float mean = (mi->red[0][0][row] + mi->red[0][1][row] + mi->red[0][2][row] + mi->red[0][3][row]) * (1.0f / (float)C);
   float sq = 0.f;
 #pragma unroll
   for (int i = 0; i < QC; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
   mi->red[1][hq][row] = sq;
-  compute_sync();
+  asm volatile("bar.sync %0, 128;" ::"r"(quarter_bar) : "memory");
   const float var = (mi->red[1][0][row] + mi->red[1][1][row] + mi->red[1][2][row] + mi->red[1][3][row]) * (1.0f / (float)C);
   const float inv = rsqrtf(var + ln.eps);
 #pragma unroll
