@@ -48,7 +48,7 @@ struct TcGeom {
   int NF;       // MLP-1 chunk width (128 or 64)
   int n_f1;     // hidden / NF
   int mode;     // 0: attention only, 1: attention + residual + LN1, 2: full layer
-  uint32_t off_a, off_kv, off_stage, off_misc;  // byte offsets from the 1024-aligned base
+  uint32_t off_a, off_kv, off_stage, off_misc, off_par;  // byte offsets from the 1024-aligned base
 };
 
 struct Misc {  // small shared state behind the big regions
@@ -59,7 +59,6 @@ struct Misc {  // small shared state behind the big regions
   int rowvox[kTM];
   int set_lo[kTM + 1];
   short row_lo[kTM], row_hi[kTM];  // tile-row range of the set each row belongs to
-  float red[2][4][kTM];  // [exchange][column quarter][row]
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -785,10 +784,10 @@ __device__ __noinline__ void phase_gather(const float* __restrict__ x, const int
   }
 }
 
-// Epilogue of a projection chunk: QC accumulator columns + bias -> bf16 into an operand tile.
+// Epilogue of a projection chunk: QC accumulator columns + bias (in shared memory) -> bf16 into an operand tile.
 // GELU = true applies gelu first (MLP-1).  c8 = first 16-byte chunk of this thread in the destination.
 template <int QC, bool GELU>
-__device__ __noinline__ void phase_epi_bf16(uint32_t taddr, unsigned long long* acc_free, const float* __restrict__ bias,
+__device__ __noinline__ void phase_epi_bf16(uint32_t taddr, unsigned long long* acc_free, const float* bias,
                                             unsigned char* dst, int row, int c8) {
   float rr[QC];
   tmem_ld_row(taddr, rr);
@@ -797,8 +796,7 @@ __device__ __noinline__ void phase_epi_bf16(uint32_t taddr, unsigned long long* 
   mbar_arrive(acc_free);  // the accumulator is in registers now
 #pragma unroll
   for (int q = 0; q < QC / 8; ++q) {
-    float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
-    if (bias) { b0 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q); b1 = __ldg(reinterpret_cast<const float4*>(bias) + 2 * q + 1); }
+    const float4 b0 = *reinterpret_cast<const float4*>(bias + 8 * q), b1 = *reinterpret_cast<const float4*>(bias + 8 * q + 4);
     float v[8] = {rr[8 * q] + b0.x, rr[8 * q + 1] + b0.y, rr[8 * q + 2] + b0.z, rr[8 * q + 3] + b0.w,
                   rr[8 * q + 4] + b1.x, rr[8 * q + 5] + b1.y, rr[8 * q + 6] + b1.z, rr[8 * q + 7] + b1.w};
     if (GELU) {
@@ -843,31 +841,34 @@ __device__ __noinline__ void phase_store_rows(float* __restrict__ y, const int* 
   }
 }
 
-struct LnArgs {
-  const float *bias, *gain, *shift;  // projection bias, LayerNorm gain (NULL: no LayerNorm) and shift
-  float eps;
+// Per-layer vectors staged in shared memory (float offsets into the parameter block).
+template <int C>
+struct ParOff {
+  static constexpr int b_qkv = 0, b_o = 3 * C, b_2 = 4 * C, ln1_g = 5 * C, ln1_b = 6 * C, ln2_g = 7 * C, ln2_b = 8 * C,
+                       b_1 = 9 * C;  // b_1 has `hidden` entries and comes last
 };
 
-// LayerNorm over the row that four threads share: t holds this thread's QC values.
-template <int C, int QC>
-__device__ __forceinline__ void layer_norm_rows(float (&t)[QC], float sum, const LnArgs& ln, Misc* mi, int row, int hq) {
+// LayerNorm over the row that four threads share: t holds this thread's QC values.  The partial sums are
+// exchanged through 4-byte slots that the caller picks: slot(which, quarter) for the two rounds.
+template <int C, int QC, class Slot>
+__device__ __forceinline__ void layer_norm_rows(float (&t)[QC], float sum, const float* gain, const float* shift, float eps,
+                                                int hq, Slot slot) {
   // the four threads of a row sit in warps q, q + 4, q + 8, q + 12: they meet at a barrier of their own
   const int quarter_bar = 2 + ((threadIdx.x >> 5) & 3);
-  mi->red[0][hq][row] = sum;
+  *slot(0, hq) = sum;
   asm volatile("bar.sync %0, 128;" ::"r"(quarter_bar) : "memory");
-  const float mean = (mi->red[0][0][row] + mi->red[0][1][row] + mi->red[0][2][row] + mi->red[0][3][row]) * (1.0f / (float)C);
+  const float mean = ((*slot(0, 0) + *slot(0, 1)) + (*slot(0, 2) + *slot(0, 3))) * (1.0f / (float)C);
   float sq = 0.f;
 #pragma unroll
   for (int i = 0; i < QC; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
-  mi->red[1][hq][row] = sq;
+  *slot(1, hq) = sq;
   asm volatile("bar.sync %0, 128;" ::"r"(quarter_bar) : "memory");
-  const float var = (mi->red[1][0][row] + mi->red[1][1][row] + mi->red[1][2][row] + mi->red[1][3][row]) * (1.0f / (float)C);
-  const float inv = rsqrtf(var + ln.eps);
+  const float var = ((*slot(1, 0) + *slot(1, 1)) + (*slot(1, 2) + *slot(1, 3))) * (1.0f / (float)C);
+  const float inv = rsqrtf(var + eps);
 #pragma unroll
   for (int i4 = 0; i4 < QC / 4; ++i4) {
-    const float4 g4 = __ldg(reinterpret_cast<const float4*>(ln.gain + hq * QC) + i4);
-    float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (ln.shift) b4 = __ldg(reinterpret_cast<const float4*>(ln.shift + hq * QC) + i4);
+    const float4 g4 = *reinterpret_cast<const float4*>(gain + hq * QC + 4 * i4);
+    const float4 b4 = *reinterpret_cast<const float4*>(shift + hq * QC + 4 * i4);
     t[4 * i4] = t[4 * i4] * inv * g4.x + b4.x;
     t[4 * i4 + 1] = t[4 * i4 + 1] * inv * g4.y + b4.y;
     t[4 * i4 + 2] = t[4 * i4 + 2] * inv * g4.z + b4.z;
@@ -877,10 +878,11 @@ __device__ __forceinline__ void layer_norm_rows(float (&t)[QC], float sum, const
 
 // Output-projection epilogue: t = Z + b_o (+ staged x); LayerNorm; then either the fp32 rows go to the staging
 // area (final result of the call: to_stage) or x1 goes to TMEM (fp32 park) and to the A operand (bf16).
+// par: the parameter block in shared memory; do_ln: apply LayerNorm 1.
 template <int C, int QC>
-__device__ __noinline__ void phase_epi_o(uint32_t taddr, unsigned long long* acc_free, LnArgs ln, bool add_x, bool to_stage,
-                                         unsigned char* stage, unsigned char* a_tile, uint32_t park_addr, Misc* mi,
-                                         int rows) {
+__device__ __noinline__ void phase_epi_o(uint32_t taddr, unsigned long long* acc_free, const float* par, float eps, bool do_ln,
+                                         bool add_x, bool to_stage, unsigned char* stage, unsigned char* a_tile,
+                                         uint32_t park_addr, int rows) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = 32 * (warp & 3) + lane, hq = warp >> 2;
   float t[QC];
@@ -891,18 +893,24 @@ __device__ __noinline__ void phase_epi_o(uint32_t taddr, unsigned long long* acc
   mbar_arrive(acc_free);
 #pragma unroll
   for (int q = 0; q < QC / 4; ++q) {
-    float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f), b4 = x4;
+    float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f);
     if (add_x && row < rows) x4 = *reinterpret_cast<const float4*>(stage + stage_off<C>(row, hq * (QC / 4) + q));
-    if (ln.bias) b4 = __ldg(reinterpret_cast<const float4*>(ln.bias + hq * QC) + q);
+    const float4 b4 = *reinterpret_cast<const float4*>(par + ParOff<C>::b_o + hq * QC + 4 * q);
     t[4 * q] += x4.x + b4.x;
     t[4 * q + 1] += x4.y + b4.y;
     t[4 * q + 2] += x4.z + b4.z;
     t[4 * q + 3] += x4.w + b4.w;
     sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
   }
-  if (ln.gain) layer_norm_rows<C, QC>(t, sum, ln, mi, row, hq);
+  if (do_ln) {
+    // exchange slots: the first two words of each thread's own (already consumed) x staging chunk
+    auto slot = [&](int which, int quarter) {
+      return reinterpret_cast<float*>(stage + stage_off<C>(row, quarter * (QC / 4))) + which;
+    };
+    layer_norm_rows<C, QC>(t, sum, par + ParOff<C>::ln1_g, par + ParOff<C>::ln1_b, eps, hq, slot);
+  }
   if (to_stage) {
-    compute_sync();  // the x staging is dead once every thread has its t
+    compute_sync();  // the x staging (and the exchange slots in it) is dead once every thread has its t
 #pragma unroll
     for (int i4 = 0; i4 < QC / 4; ++i4)
       *reinterpret_cast<float4*>(stage + stage_off<C>(row, hq * (QC / 4) + i4)) =
@@ -919,10 +927,11 @@ __device__ __noinline__ void phase_epi_o(uint32_t taddr, unsigned long long* acc
   tc_fence_before();
 }
 
-// MLP-2 epilogue: t = M + b_2 + parked x1; LayerNorm; fp32 rows to the staging area.
+// MLP-2 epilogue: t = M + b_2 + parked x1; LayerNorm; fp32 rows to the staging area.  The exchange slots
+// live in the A operand tile, which nobody uses between MLP-1 and the next tile's gather.
 template <int C, int QC>
-__device__ __noinline__ void phase_epi_f2(uint32_t taddr, unsigned long long* acc_free, LnArgs ln, unsigned char* stage,
-                                          uint32_t park_addr, Misc* mi) {
+__device__ __noinline__ void phase_epi_f2(uint32_t taddr, unsigned long long* acc_free, const float* par, float eps, bool do_ln,
+                                          unsigned char* stage, unsigned char* a_tile, uint32_t park_addr) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = 32 * (warp & 3) + lane, hq = warp >> 2;
   float t[QC];
@@ -937,8 +946,7 @@ __device__ __noinline__ void phase_epi_f2(uint32_t taddr, unsigned long long* ac
     tmem_wait_ld();
 #pragma unroll
     for (int q = 0; q < QC / 4; ++q) {
-      float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (ln.bias) b4 = __ldg(reinterpret_cast<const float4*>(ln.bias + hq * QC) + q);
+      const float4 b4 = *reinterpret_cast<const float4*>(par + ParOff<C>::b_2 + hq * QC + 4 * q);
       t[4 * q] += rp[4 * q] + b4.x;
       t[4 * q + 1] += rp[4 * q + 1] + b4.y;
       t[4 * q + 2] += rp[4 * q + 2] + b4.z;
@@ -946,7 +954,10 @@ __device__ __noinline__ void phase_epi_f2(uint32_t taddr, unsigned long long* ac
       sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
     }
   }
-  if (ln.gain) layer_norm_rows<C, QC>(t, sum, ln, mi, row, hq);
+  if (do_ln) {
+    auto slot = [&](int which, int quarter) { return reinterpret_cast<float*>(a_tile) + (which * 4 + quarter) * kTM + row; };
+    layer_norm_rows<C, QC>(t, sum, par + ParOff<C>::ln2_g, par + ParOff<C>::ln2_b, eps, hq, slot);
+  }
   // the MLP-2 MMAs have read H: its region takes the fp32 output rows
 #pragma unroll
   for (int i4 = 0; i4 < QC / 4; ++i4)
@@ -965,6 +976,7 @@ __device__ __forceinline__ void compute_role(const dsvt_fused_args& a, const TcG
   unsigned char* sm = rc.sm;
   const uint32_t sbase = rc.sbase, tmem = rc.tmem;
   Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
+  const float* par = reinterpret_cast<const float*>(sm + g.off_par);  // biases and LayerNorm vectors
   const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &mi->abort_flag;
@@ -1010,7 +1022,7 @@ __device__ __forceinline__ void compute_role(const dsvt_fused_args& a, const TcG
       acc_wait(bar);
       if (c == 2 ? live : live_kv)
         phase_epi_bf16<QC, false>(tmem + lane_addr + (c == 1 ? COL_B : 0u) + hq * QC, &mi->acc_free[bar],
-                                  p.b_qkv ? p.b_qkv + (c == 0 ? 1 : c == 1 ? 2 : 0) * C + hq * QC : nullptr,
+                                  par + ParOff<C>::b_qkv + (c == 0 ? 1 : c == 1 ? 2 : 0) * C + hq * QC,
                                   sm + (c == 2 ? g.off_a : g.off_kv + (uint32_t)c * (NKB * kTM * 128)), row,
                                   (hq * QC) >> 3);
       else
@@ -1032,13 +1044,8 @@ __device__ __forceinline__ void compute_role(const dsvt_fused_args& a, const TcG
     // ---- chunk 3: output projection epilogue: Z + b_o (+ x, LayerNorm) ----
     {
       acc_wait(0u);
-      LnArgs ln;
-      ln.bias = p.b_o;
-      ln.gain = g.mode != 0 ? p.ln1_g : nullptr;
-      ln.shift = p.ln1_b;
-      ln.eps = p.ln_eps;
-      phase_epi_o<C, QC>(tmem + lane_addr + hq * QC, &mi->acc_free[0], ln, g.mode != 0, g.mode != 2, sm + g.off_kv,
-                         sm + g.off_a, tmem + lane_addr + COL_PARK + hq * QC, mi, rows);
+      phase_epi_o<C, QC>(tmem + lane_addr + hq * QC, &mi->acc_free[0], par, p.ln_eps, g.mode != 0 && p.ln1_g != nullptr,
+                         g.mode != 0, g.mode != 2, sm + g.off_kv, sm + g.off_a, tmem + lane_addr + COL_PARK + hq * QC, rows);
       if (g.mode != 2) {  // final result of this call
         compute_sync();
         phase_store_rows<C>(a.y, mi->rowvox, rows, sm + g.off_kv);
@@ -1056,9 +1063,9 @@ __device__ __forceinline__ void compute_role(const dsvt_fused_args& a, const TcG
         const int col0 = c * g.NF + hq * qw;  // first hidden column of this thread
         const uint32_t src = tmem + lane_addr + bar * (uint32_t)g.NF + hq * qw;
         if (qw == 32)
-          phase_epi_bf16<32, true>(src, &mi->acc_free[bar], p.b_1 ? p.b_1 + col0 : nullptr, sm + g.off_kv, row, col0 >> 3);
+          phase_epi_bf16<32, true>(src, &mi->acc_free[bar], par + ParOff<C>::b_1 + col0, sm + g.off_kv, row, col0 >> 3);
         else
-          phase_epi_bf16<16, true>(src, &mi->acc_free[bar], p.b_1 ? p.b_1 + col0 : nullptr, sm + g.off_kv, row, col0 >> 3);
+          phase_epi_bf16<16, true>(src, &mi->acc_free[bar], par + ParOff<C>::b_1 + col0, sm + g.off_kv, row, col0 >> 3);
       } else {
         acc_release(bar);
       }
@@ -1069,13 +1076,8 @@ __device__ __forceinline__ void compute_role(const dsvt_fused_args& a, const TcG
     {
       const uint32_t bar = (uint32_t)g.n_f1 & 1u;
       acc_wait(bar);
-      LnArgs ln;
-      ln.bias = p.b_2;
-      ln.gain = p.ln2_g;
-      ln.shift = p.ln2_b;
-      ln.eps = p.ln_eps;
-      phase_epi_f2<C, QC>(tmem + lane_addr + hq * QC, &mi->acc_free[bar], ln, sm + g.off_kv,
-                          tmem + lane_addr + COL_PARK + hq * QC, mi);
+      phase_epi_f2<C, QC>(tmem + lane_addr + hq * QC, &mi->acc_free[bar], par, p.ln_eps, p.ln2_g != nullptr, sm + g.off_kv,
+                          sm + g.off_a, tmem + lane_addr + COL_PARK + hq * QC);
       compute_sync();
       phase_store_rows<C>(a.y, mi->rowvox, rows, sm + g.off_kv);
     }
@@ -1121,6 +1123,17 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   for (uint32_t i = tid; i < ((uint32_t)kTM * 2 * C * 2 + kStages * (uint32_t)C * 128u) / 16; i += kThreads)
     reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_proxy_async();  // the TMA writes that follow must not be overtaken by these generic stores
+  {  // biases and LayerNorm vectors -> shared memory (absent vectors read as zeros)
+    float* par = reinterpret_cast<float*>(sm + g.off_par);
+    const dsvt_layer_params& p = a.p;
+    const float* src[9] = {p.b_qkv, p.b_qkv ? p.b_qkv + C : nullptr, p.b_qkv ? p.b_qkv + 2 * C : nullptr, p.b_o, p.b_2,
+                           p.ln1_g, p.ln1_b, p.ln2_g, p.ln2_b};
+    for (int i = tid; i < 9 * C; i += kThreads) {
+      const float* v = src[i / C];
+      par[i] = v ? __ldg(v + i % C) : 0.f;
+    }
+    for (int i = tid; i < g.hidden; i += kThreads) par[9 * C + i] = p.b_1 ? __ldg(p.b_1 + i) : 0.f;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -1232,7 +1245,8 @@ int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a) {
   g.off_kv = a_bytes;
   g.off_stage = g.off_kv + (uint32_t)kTM * 2 * C * 2;  // K + V (bf16) = fp32 staging = MLP hidden (<= 2C) bytes
   g.off_misc = g.off_stage + kStages * (uint32_t)C * 128u;
-  const size_t smem = (size_t)g.off_misc + sizeof(Misc) + 1024;
+  g.off_par = g.off_misc + (uint32_t)((sizeof(Misc) + 15) / 16 * 16);
+  const size_t smem = (size_t)g.off_par + (size_t)(9 * C + g.hidden) * sizeof(float) + 1024;
   if (smem > 227 * 1024) return DSVT_ERR_UNSUPPORTED;
   TcMaps maps;
   bool okm = make_weight_map(&maps.qkv, p.W_qkv, 3 * C, C, C) && make_weight_map(&maps.o, p.W_o, C, C, C);
