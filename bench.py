@@ -44,27 +44,50 @@ class ClockSampler:
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
-        self.proc, self.idx = None, gpu_index
+        self.proc, self.idx, self.rows, self.thread = None, gpu_index, [], None
 
-    def start(self):
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), line))
+
+    def start(self, wait_s: float = 5.0):
+        """Starts nvidia-smi and returns once its first sample has arrived (or after wait_s)."""
+        import threading
+
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.QUERY,
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
-                                         stderr=subprocess.DEVNULL, text=True)
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True, bufsize=1)
         except OSError:
             self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+        t0 = time.perf_counter()
+        while not self.rows and time.perf_counter() - t0 < wait_s and self.proc.poll() is None:
+            time.sleep(0.01)
 
-    def stop(self):
+    def stop(self, t_begin: float, t_end: float):
+        """Summary of the samples taken in [t_begin, t_end] (perf_counter times of the timed region); if the
+        region was shorter than one sampling period, of the samples closest to it."""
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
+        time.sleep(0.06)  # one more sampling period, so that a short region is bracketed
         self.proc.terminate()
         try:
-            out, _ = self.proc.communicate(timeout=10)
+            self.proc.wait(timeout=10)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-            out, _ = self.proc.communicate()
+        if self.thread is not None:
+            self.thread.join(timeout=5)
+        inside = [r for r in self.rows if t_begin <= r[0] <= t_end]
+        note = "all samples inside the timed region"
+        if not inside and self.rows:
+            mid = 0.5 * (t_begin + t_end)
+            inside = sorted(self.rows, key=lambda r: abs(r[0] - mid))[:2]
+            note = "timed region shorter than the 50 ms sampling period: the two samples closest to it"
         sm, mx, reasons = [], [], set()
-        for line in out.strip().splitlines():
+        for _, line in inside:
             f = [t.strip() for t in line.split(",")]
             if len(f) < 9:
                 continue
@@ -76,7 +99,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "note": note}
 
 
 def _dist_env():
@@ -211,6 +234,7 @@ def run_ours(args):
     sampler.start()
     launches0 = ctx.launch_count()
     barrier()
+    t_begin = time.perf_counter()
     for k in range(args.steps):
         flush.zero_()
         e = ev[k]
@@ -223,8 +247,9 @@ def run_ours(args):
             src = y
             e[2 + b].record(stream)
     barrier()
+    t_end = time.perf_counter()
     launches = ctx.launch_count() - launches0
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_begin, t_end)
     t_step = np.array([e[0].elapsed_time(e[1 + nb]) for e in ev])  # ms
     t_part = np.array([e[0].elapsed_time(e[1]) for e in ev])
     t_blocks = np.array([[e[1 + b].elapsed_time(e[2 + b]) for b in range(nb)] for e in ev])
@@ -305,7 +330,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2)

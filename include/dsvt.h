@@ -86,7 +86,12 @@ int64_t dsvt_launch_count(const dsvt_ctx* ctx);
  *   grid        cells per axis (x, y, z); window = (L, W, H); windows start at cell 0 and do not
  *               cross frames.  Window id = ((b*nWx + x/L)*nWy + y/W)*nWz + z/H, nW* = ceil(grid/window).
  *   axis        0: X main order, voxels of a window ordered by (x, y, z) of their in-window
- *               offsets; 1: Y main order, ordered by (y, x, z).  Equal keys keep index order.
+ *               offsets; 1: Y main order, ordered by (y, x, z).  Voxels occupy distinct cells (the
+ *               output of voxelisation).  Two voxels in one cell are an input error: every voxel
+ *               still lands in exactly one set of its window, but the later arrivals are ranked
+ *               behind the window's other voxels and DSVT_STATUS_DUPLICATE_CELL is raised (calls
+ *               whose key space exceeds the context's 64 Mi-key bitmap fall back to a stable sort,
+ *               which keeps equal keys in index order and raises nothing).
  *   set_table   out, int32 [cap_sets][set_size]: row s = the voxel indices of one set, slot k holding
  *               the voxel of inner-window rank floor((j*set_size + k) * N / (S*set_size)) (exact
  *               integer floor), j = the set's number inside its window.  Rows are ordered by
@@ -113,6 +118,19 @@ int dsvt_partition(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batc
                    const int32_t window[3], int32_t set_size, int32_t axis, int32_t* set_table, int32_t cap_sets,
                    int32_t* num_sets, int32_t* set_rowoff, int32_t* perm, int32_t* win_start, int32_t* win_count,
                    int32_t* win_setoff);
+
+/*
+ * Both rotated partitions of one DSVT block (Sec. 3.2, "Rotated set attention": X main order for
+ * the first layer, Y main order for the second) in one pass: the two axes share the window ids,
+ * the per-window counts and the launches.  Arguments as for dsvt_partition; set_table, num_sets,
+ * set_rowoff and perm are HOST arrays of two device pointers, entry 0 for axis 0 and entry 1 for
+ * axis 1 (set_rowoff, perm or their entries may be NULL; both num_sets entries are required and
+ * receive the same value).  The results equal those of two dsvt_partition calls.
+ */
+int dsvt_partition_rotated(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch, const int32_t grid[3],
+                           const int32_t window[3], int32_t set_size, int32_t* const set_table[2],
+                           int32_t cap_sets, int32_t* const num_sets[2], int32_t* const set_rowoff[2],
+                           int32_t* const perm[2], int32_t* win_start, int32_t* win_count, int32_t* win_setoff);
 
 /*
  * dsvt_partition without any allocation.  (The paper has no counterpart: this is a deployment

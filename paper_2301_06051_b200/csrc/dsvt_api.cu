@@ -40,6 +40,10 @@ void carve(dsvt_ctx* c, unsigned char* base, size_t* total) {
   c->rowoff_a = k.take<int32_t>(2 * nv + 3);
   c->rowoff_b = k.take<int32_t>(2 * nv + 3);
   c->region_key = k.take<int32_t>(nv);
+  c->bm_words = (size_t)1 << 21;  // 64 Mi keys per sort axis
+  c->bm_zero = k.take<int32_t>(2 * (nw + 1) + 2 * c->bm_words);
+  c->bm_wordrank = k.take<int32_t>(2 * c->bm_words);
+  c->bm_dup = k.take<int32_t>(nv);
   *total = align_up(k.off, 256);
 }
 

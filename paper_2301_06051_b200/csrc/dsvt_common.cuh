@@ -28,6 +28,11 @@ struct dsvt_ctx {
   int32_t* rowoff_a;    // [2 max_voxels + 3] row offsets + tile plan derived from a caller table
   int32_t* rowoff_b;    // [2 max_voxels + 3]
   int32_t* region_key;  // [max_voxels] pooling: dense region id of each output row
+  // partition, bitmap route (bm_words == 0: route not available)
+  size_t bm_words;       // bitmap capacity per sort axis, in 32-bit words
+  int32_t* bm_zero;      // [2 (max_windows + 1) + 2 bm_words] window counts, duplicate counts, bitmaps
+  int32_t* bm_wordrank;  // [2 bm_words] popcount prefix of each bitmap word inside its window
+  int32_t* bm_dup;       // [max_voxels] -1, or the voxel's ticket among the duplicates of its window
   // pooling: dense cell -> voxel map, grown on demand
   int32_t* cell_map;
   size_t cell_map_entries;

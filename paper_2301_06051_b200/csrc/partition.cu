@@ -212,11 +212,9 @@ __global__ void __launch_bounds__(kSortThreads) radix_scatter_kernel(const uint3
 
 // ---- per-window scans (Eq. 2) ------------------------------------------------------------------
 // Single block.  win_start = exclusive scan of N_w; win_setoff = exclusive scan of S_w = ceil(N_w / tau).
-__global__ void __launch_bounds__(kScanThreads) window_scan_kernel(const int32_t* __restrict__ win_count,
-                                                                   int32_t num_windows, int32_t tau,
-                                                                   int32_t* win_start, int32_t* win_setoff,
-                                                                   int32_t cap_sets, int32_t* num_sets,
-                                                                   int32_t* status) {
+__device__ __forceinline__ void window_scan_body(const int32_t* __restrict__ win_count, int32_t num_windows,
+                                                 int32_t tau, int32_t* win_start, int32_t* win_setoff, int32_t cap_sets,
+                                                 int32_t* num_sets0, int32_t* num_sets1, int32_t* status) {
   __shared__ int warp_tot[33];
   int carry_n = 0, carry_s = 0;
   for (int base = 0; base < num_windows; base += kScanTile) {
@@ -253,19 +251,34 @@ __global__ void __launch_bounds__(kScanThreads) window_scan_kernel(const int32_t
       atomicOr(status, DSVT_STATUS_TABLE_OVERFLOW);
       carry_s = cap_sets;
     }
-    *num_sets = carry_s;
+    *num_sets0 = carry_s;
+    if (num_sets1) *num_sets1 = carry_s;
   }
 }
 
+__global__ void __launch_bounds__(kScanThreads) window_scan_kernel(const int32_t* __restrict__ win_count,
+                                                                   int32_t num_windows, int32_t tau,
+                                                                   int32_t* win_start, int32_t* win_setoff,
+                                                                   int32_t cap_sets, int32_t* num_sets,
+                                                                   int32_t* status) {
+  window_scan_body(win_count, num_windows, tau, win_start, win_setoff, cap_sets, num_sets, nullptr, status);
+}
+
 // ---- set table fill (Eq. 3, Eq. 4's rank -> voxel id) -------------------------------------------
-// One warp per set.
-__global__ void table_fill_kernel(const int32_t* __restrict__ sorted_vox, const int32_t* __restrict__ win_count,
+// One warp per set; grid row y fills the table of sort axis slot y.
+struct FillAxis {
+  const int32_t* sorted_vox;
+  const int32_t* num_sets;
+  int32_t* table;
+  int32_t* rowoff;
+};
+__global__ void table_fill_kernel(FillAxis ax0, FillAxis ax1, const int32_t* __restrict__ win_count,
                                   const int32_t* __restrict__ win_start, const int32_t* __restrict__ win_setoff,
-                                  int32_t num_windows, int32_t tau, const int32_t* __restrict__ num_sets,
-                                  int32_t* __restrict__ table, int32_t* __restrict__ rowoff) {
+                                  int32_t num_windows, int32_t tau) {
+  const FillAxis ax = blockIdx.y ? ax1 : ax0;
   const int lane = threadIdx.x & 31;
   const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int S_all = *num_sets;
+  const int S_all = *ax.num_sets;
   if (s >= S_all) return;
   // last window w with win_setoff[w] <= s; it is non-empty because win_setoff[w + 1] > s
   int lo = 0, hi = num_windows;  // invariant: win_setoff[lo] <= s < win_setoff[hi]
@@ -281,11 +294,11 @@ __global__ void table_fill_kernel(const int32_t* __restrict__ sorted_vox, const 
   const uint64_t den = Sw * (uint64_t)tau;
   for (int k = lane; k < tau; k += 32) {
     const uint64_t q = ((j * (uint64_t)tau + (uint64_t)k) * N) / den;  // Eq. 3, exact integer floor
-    table[(size_t)s * tau + k] = sorted_vox[start + (int)q];
+    ax.table[(size_t)s * tau + k] = ax.sorted_vox[start + (int)q];
   }
-  if (rowoff && lane == 0) {
-    rowoff[s] = start + (int)((j * N) / Sw);  // first rank of set j (proof of Theorem A.2)
-    if (s == S_all - 1) rowoff[S_all] = start + (int)(((j + 1) * N) / Sw);
+  if (ax.rowoff && lane == 0) {
+    ax.rowoff[s] = start + (int)((j * N) / Sw);  // first rank of set j (proof of Theorem A.2)
+    if (s == S_all - 1) ax.rowoff[S_all] = start + (int)(((j + 1) * N) / Sw);
   }
 }
 
@@ -316,10 +329,13 @@ __global__ void table_unique_count_kernel(const int32_t* __restrict__ table, int
 // row segments).  The greedy chain 0 -> next(0) -> next(next(0)) ... is found by pointer doubling, all
 // sets in parallel: single block, arrays in shared memory.
 constexpr int kPlanMaxSets = 24576;
-__global__ void __launch_bounds__(kScanThreads) tile_plan_kernel(const int32_t* __restrict__ rowoff,
+__global__ void __launch_bounds__(kScanThreads) tile_plan_kernel(int32_t* rowoff0, int32_t* rowoff1,
                                                                  const int32_t* __restrict__ num_sets, int32_t cap_sets,
-                                                                 int32_t smax, int32_t max_rows, int32_t* __restrict__ plan) {
+                                                                 int32_t smax, int32_t max_rows) {
   extern __shared__ int plan_smem[];
+  int32_t* rowoff = blockIdx.x ? rowoff1 : rowoff0;  // one block per buffer: offsets, then the plan
+  if (!rowoff) return;
+  int32_t* plan = rowoff + cap_sets + 1;
   __shared__ int warp_tot[33];
   int* cur = plan_smem;
   int* nxt = cur + (smax + 1);
@@ -366,6 +382,116 @@ __global__ void __launch_bounds__(kScanThreads) tile_plan_kernel(const int32_t* 
   for (int s = s0; s < s1; ++s)
     if (mark[s]) plan[1 + off++] = s;
   if (tid == 0) { plan[0] = total; plan[1 + total] = S; }
+}
+
+// ---- bitmap route: ranks by population count instead of sorting --------------------------------
+// When the key space (windows x padded cells per window) fits a bitmap, the inner-window rank of a
+// voxel (Eq. 1 followed by the sort) is the number of occupied cells of its window with a smaller
+// key: each window owns wpw whole 32-bit words of the bitmap, wordrank holds the exclusive popcount
+// prefix of the words inside their window, and a voxel's rank is wordrank[word] plus the set bits
+// below its own.  Both sort axes are handled by the same launches (they share windows and counts).
+struct BmAxis {
+  uint32_t* keys;      // [n] window * Vp + inner-window key
+  uint32_t* bitmap;    // [num_windows * wpw], cleared by the caller
+  int32_t* wordrank;   // [num_windows * wpw]
+  int32_t* sorted;     // [n] voxel ids in (window, inner-window) order
+  int32_t axis;        // 0: X main order, 1: Y main order
+};
+struct BmJob {
+  BmAxis ax[2];
+  int32_t naxes;
+};
+
+__global__ void bm_mark_kernel(const int4* __restrict__ coords, int32_t n, PartGeom g, uint32_t Vp, BmJob job,
+                               int32_t* __restrict__ win_count, int32_t* __restrict__ dup_count,
+                               int32_t* __restrict__ dup, int32_t* __restrict__ status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  int4 c = coords[i];  // (b, x, y, z)
+  const bool bad =
+      c.x < 0 || c.x >= g.batch || c.y < 0 || c.y >= g.gx || c.z < 0 || c.z >= g.gy || c.w < 0 || c.w >= g.gz;
+  if (bad) {
+    atomicOr(status, DSVT_STATUS_BAD_COORD);
+    c.x = min(max(c.x, 0), g.batch - 1);
+    c.y = min(max(c.y, 0), g.gx - 1);
+    c.z = min(max(c.z, 0), g.gy - 1);
+    c.w = min(max(c.w, 0), g.gz - 1);
+  }
+  const int wx = c.y / g.L, wy = c.z / g.W, wz = c.w / g.H;
+  const int xi = c.y - wx * g.L, yi = c.z - wy * g.W, zi = c.w - wz * g.H;
+  const uint32_t win = (uint32_t)(((c.x * g.nWx + wx) * g.nWy + wy) * g.nWz + wz);
+  atomicAdd(&win_count[win], 1);
+  int ticket = -1;
+#pragma unroll
+  for (int a = 0; a < 2; ++a) {
+    if (a < job.naxes) {
+      const uint32_t inner =
+          job.ax[a].axis == 0 ? (uint32_t)((xi * g.W + yi) * g.H + zi) : (uint32_t)((yi * g.L + xi) * g.H + zi);
+      const uint32_t key = win * Vp + inner;
+      job.ax[a].keys[i] = key;
+      const uint32_t bit = 1u << (key & 31);
+      const uint32_t old = atomicOr(&job.ax[a].bitmap[key >> 5], bit);
+      if (a == 0 && (old & bit)) {  // cell already taken: this voxel goes behind the window's distinct cells
+        ticket = atomicAdd(&dup_count[win], 1);
+        atomicOr(status, DSVT_STATUS_DUPLICATE_CELL);
+      }
+    }
+  }
+  dup[i] = ticket;
+}
+
+// Block 0: the per-window scans (Eq. 2).  Other blocks: wordrank, one warp per (axis, window).
+__global__ void __launch_bounds__(kScanThreads) bm_scan_kernel(const int32_t* __restrict__ win_count,
+                                                               int32_t num_windows, int32_t tau, int32_t* win_start,
+                                                               int32_t* win_setoff, int32_t cap_sets,
+                                                               int32_t* num_sets0, int32_t* num_sets1, BmJob job,
+                                                               int32_t wpw, int32_t* status) {
+  if (blockIdx.x == 0) {
+    window_scan_body(win_count, num_windows, tau, win_start, win_setoff, cap_sets, num_sets0, num_sets1, status);
+    return;
+  }
+  const int lane = threadIdx.x & 31;
+  const int64_t items = (int64_t)job.naxes * num_windows;
+  const int64_t stride = (int64_t)(gridDim.x - 1) * (kScanThreads / 32);
+  for (int64_t it = (int64_t)(blockIdx.x - 1) * (kScanThreads / 32) + (threadIdx.x >> 5); it < items; it += stride) {
+    const int a = it >= num_windows ? 1 : 0;
+    const int w = (int)(it - (int64_t)a * num_windows);
+    if (win_count[w] == 0) continue;
+    const uint32_t* bm = a ? job.ax[1].bitmap : job.ax[0].bitmap;
+    int32_t* wr = a ? job.ax[1].wordrank : job.ax[0].wordrank;
+    const size_t base = (size_t)w * wpw;
+    int carry = 0;
+    for (int c0 = 0; c0 < wpw; c0 += 32) {
+      const int k = c0 + lane;
+      const int v = k < wpw ? __popc(bm[base + k]) : 0;
+      const int incl = warp_incl_scan(v);
+      if (k < wpw) wr[base + k] = carry + incl - v;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+  }
+}
+
+__global__ void bm_place_kernel(int32_t n, BmJob job, int32_t wpw, const int32_t* __restrict__ dup,
+                                const int32_t* __restrict__ win_start) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int ticket = dup[i];
+#pragma unroll
+  for (int a = 0; a < 2; ++a) {
+    if (a < job.naxes) {
+      const uint32_t key = job.ax[a].keys[i];
+      const uint32_t word = key >> 5;
+      const uint32_t win = word / (uint32_t)wpw;
+      int r;
+      if (ticket < 0) {
+        r = job.ax[a].wordrank[word] + __popc(job.ax[a].bitmap[word] & ((1u << (key & 31)) - 1u));
+      } else {
+        const size_t last = (size_t)win * wpw + (wpw - 1);
+        r = job.ax[a].wordrank[last] + __popc(job.ax[a].bitmap[last]) + ticket;
+      }
+      job.ax[a].sorted[win_start[win] + r] = i;
+    }
+  }
 }
 
 }  // namespace
@@ -420,8 +546,9 @@ int dsvt_launch_rowoff_from_table(dsvt_ctx* ctx, const int32_t* table, int32_t c
   return dsvt_launch_scan_i32(ctx, rowoff, rowoff, cap_sets, nullptr);
 }
 
-// Tile plan behind the row offsets: set_rowoff + cap_sets + 1 (see include/dsvt.h).
-int dsvt_launch_tile_plan(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap_sets, int32_t* set_rowoff) {
+// Tile plans behind the row offsets of one or two buffers: set_rowoff + cap_sets + 1 (see include/dsvt.h).
+static int launch_tile_plans(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap_sets, int32_t* set_rowoff,
+                             int32_t* set_rowoff1) {
   const int32_t smax = cap_sets < kPlanMaxSets ? cap_sets : kPlanMaxSets;
   const size_t smem = (size_t)(smax + 1) * 8 + (size_t)smax + 16;
   static bool attr_set = false;
@@ -430,10 +557,14 @@ int dsvt_launch_tile_plan(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap_se
                                             (int)((size_t)(kPlanMaxSets + 1) * 8 + kPlanMaxSets + 16)));
     attr_set = true;
   }
-  tile_plan_kernel<<<1, kScanThreads, smem, ctx->stream>>>(set_rowoff, num_sets, cap_sets, smax, 128,
-                                                          set_rowoff + cap_sets + 1);
+  tile_plan_kernel<<<set_rowoff1 ? 2 : 1, kScanThreads, smem, ctx->stream>>>(set_rowoff, set_rowoff1, num_sets,
+                                                                            cap_sets, smax, 128);
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
+}
+
+int dsvt_launch_tile_plan(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap_sets, int32_t* set_rowoff) {
+  return launch_tile_plans(ctx, num_sets, cap_sets, set_rowoff, nullptr);
 }
 
 static int key_bits_for(uint64_t max_key) {
@@ -442,69 +573,204 @@ static int key_bits_for(uint64_t max_key) {
   return b;
 }
 
-extern "C" int dsvt_partition(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch, const int32_t grid[3],
-                              const int32_t window[3], int32_t set_size, int32_t axis, int32_t* set_table,
-                              int32_t cap_sets, int32_t* num_sets, int32_t* set_rowoff, int32_t* perm,
-                              int32_t* win_start, int32_t* win_count, int32_t* win_setoff) {
-  if (!ctx || !grid || !window || !num_sets || n < 0 || batch < 1 || set_size < 1 || cap_sets < 0 ||
-      (axis != 0 && axis != 1))
-    return DSVT_ERR_INVALID_ARG;
+namespace {
+
+struct PartOut {  // device outputs of one sort axis
+  int32_t axis;
+  int32_t* set_table;
+  int32_t* num_sets;
+  int32_t* set_rowoff;
+  int32_t* perm;
+};
+
+struct PartCall {
+  const int32_t* coords;
+  int32_t n, set_size, cap_sets, nw;
+  PartGeom g;
+  uint64_t V;
+  int32_t *win_start, *win_count, *win_setoff;  // optional outputs
+};
+
+int validate(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch, const int32_t grid[3],
+             const int32_t window[3], int32_t set_size, int32_t cap_sets, PartCall* pc) {
+  if (!ctx || !grid || !window || n < 0 || batch < 1 || set_size < 1 || cap_sets < 0) return DSVT_ERR_INVALID_ARG;
   for (int a = 0; a < 3; ++a)
     if (grid[a] < 1 || window[a] < 1) return DSVT_ERR_INVALID_ARG;
-  if (n > 0 && (!coords || !set_table)) return DSVT_ERR_INVALID_ARG;
+  if (n > 0 && !coords) return DSVT_ERR_INVALID_ARG;
   if (((uintptr_t)coords & 15) != 0) return DSVT_ERR_INVALID_ARG;
-  PartGeom g;
+  PartGeom& g = pc->g;
   g.batch = batch; g.gx = grid[0]; g.gy = grid[1]; g.gz = grid[2];
   g.L = window[0]; g.W = window[1]; g.H = window[2];
   g.nWx = (int32_t)dsvt_ceil_div(grid[0], window[0]);
   g.nWy = (int32_t)dsvt_ceil_div(grid[1], window[1]);
   g.nWz = (int32_t)dsvt_ceil_div(grid[2], window[2]);
-  g.axis = axis;
+  g.axis = 0;
   const uint64_t V = (uint64_t)window[0] * window[1] * window[2];
   const uint64_t num_windows = (uint64_t)batch * g.nWx * g.nWy * g.nWz;
   if (V >= (1ull << 31) || num_windows >= (1ull << 31) || num_windows * V > 0xFFFFFFFFull) return DSVT_ERR_UNSUPPORTED;
   g.V = (uint32_t)V;
   if (n > ctx->max_voxels || (int64_t)num_windows > ctx->max_windows) return DSVT_ERR_CAPACITY;
-  const int32_t nw = (int32_t)num_windows;
-  cudaStream_t st = ctx->stream;
+  pc->coords = coords; pc->n = n; pc->set_size = set_size; pc->cap_sets = cap_sets;
+  pc->nw = (int32_t)num_windows;
+  pc->V = V;
+  return DSVT_OK;
+}
 
+// upper bound of the number of sets: floor(n / tau) + (non-empty windows), at most min(cap_sets, n)
+int64_t sets_bound(const PartCall& pc) {
+  int64_t b = (int64_t)pc.n / pc.set_size + (int64_t)(pc.nw < pc.n ? pc.nw : pc.n);
+  if (b > pc.n) b = pc.n;
+  if (b > pc.cap_sets) b = pc.cap_sets;
+  return b;
+}
+
+int copy_window_arrays(dsvt_ctx* ctx, const PartCall& pc, const int32_t* counts) {
+  cudaStream_t st = ctx->stream;
+  const size_t nw = (size_t)pc.nw;
+  if (pc.win_count)
+    DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(pc.win_count, counts, sizeof(int32_t) * nw, cudaMemcpyDeviceToDevice, st));
+  if (pc.win_start)
+    DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(pc.win_start, ctx->win_start, sizeof(int32_t) * (nw + 1), cudaMemcpyDeviceToDevice, st));
+  if (pc.win_setoff)
+    DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(pc.win_setoff, ctx->win_setoff, sizeof(int32_t) * (nw + 1), cudaMemcpyDeviceToDevice, st));
+  return DSVT_OK;
+}
+
+// Sorting route: one axis per call; works for any key space below 2^32.
+int partition_sorted(dsvt_ctx* ctx, const PartCall& pc, const PartOut& o) {
+  cudaStream_t st = ctx->stream;
+  const int32_t n = pc.n, nw = pc.nw, cap_sets = pc.cap_sets;
+  PartGeom g = pc.g;
+  g.axis = o.axis;
   DSVT_CUDA_TRY(ctx, cudaMemsetAsync(ctx->win_count, 0, sizeof(int32_t) * (size_t)(nw + 1), st));
   int fin = 0;
   if (n > 0) {
-    window_key_kernel<<<(unsigned)dsvt_ceil_div(n, 256), 256, 0, st>>>((const int4*)coords, n, g, ctx->keys[0],
+    window_key_kernel<<<(unsigned)dsvt_ceil_div(n, 256), 256, 0, st>>>((const int4*)pc.coords, n, g, ctx->keys[0],
                                                                        ctx->vals[0], ctx->win_count, ctx->status);
     DSVT_LAUNCHED(ctx);
-    int rc = dsvt_launch_sort_pairs(ctx, n, key_bits_for(num_windows * V - 1), &fin);
+    int rc = dsvt_launch_sort_pairs(ctx, n, key_bits_for((uint64_t)nw * pc.V - 1), &fin);
     if (rc != DSVT_OK) return rc;
   }
-  window_scan_kernel<<<1, kScanThreads, 0, st>>>(ctx->win_count, nw, set_size, ctx->win_start, ctx->win_setoff,
-                                                 cap_sets, num_sets, ctx->status);
+  window_scan_kernel<<<1, kScanThreads, 0, st>>>(ctx->win_count, nw, pc.set_size, ctx->win_start, ctx->win_setoff,
+                                                 cap_sets, o.num_sets, ctx->status);
   DSVT_LAUNCHED(ctx);
   if (n > 0) {
-    // number of sets <= floor(n / tau) + (non-empty windows) <= min(cap_sets, n)
-    int64_t s_bound = (int64_t)n / set_size + (int64_t)(nw < n ? nw : n);
-    if (s_bound > n) s_bound = n;
-    if (s_bound > cap_sets) s_bound = cap_sets;
+    const int64_t s_bound = sets_bound(pc);
     if (s_bound > 0) {
-      table_fill_kernel<<<(unsigned)dsvt_ceil_div(s_bound, 8), 256, 0, st>>>(ctx->vals[fin], ctx->win_count,
-                                                                             ctx->win_start, ctx->win_setoff, nw,
-                                                                             set_size, num_sets, set_table, set_rowoff);
+      FillAxis f{ctx->vals[fin], o.num_sets, o.set_table, o.set_rowoff};
+      table_fill_kernel<<<(unsigned)dsvt_ceil_div(s_bound, 8), 256, 0, st>>>(f, f, ctx->win_count, ctx->win_start,
+                                                                             ctx->win_setoff, nw, pc.set_size);
       DSVT_LAUNCHED(ctx);
     }
-    if (set_rowoff && s_bound > 0) {
-      int rc = dsvt_launch_tile_plan(ctx, num_sets, cap_sets, set_rowoff);
+    if (o.set_rowoff && s_bound > 0) {
+      int rc = dsvt_launch_tile_plan(ctx, o.num_sets, cap_sets, o.set_rowoff);
       if (rc != DSVT_OK) return rc;
     }
-    if (perm)
-      DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(perm, ctx->vals[fin], sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToDevice, st));
+    if (o.perm)
+      DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(o.perm, ctx->vals[fin], sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToDevice, st));
   }
-  if (set_rowoff && (n == 0 || cap_sets == 0))  // no sets: row offset 0, empty tile plan
-    DSVT_CUDA_TRY(ctx, cudaMemsetAsync(set_rowoff, 0, sizeof(int32_t) * (size_t)(2 * (size_t)cap_sets + 3), st));
-  if (win_count)
-    DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(win_count, ctx->win_count, sizeof(int32_t) * (size_t)nw, cudaMemcpyDeviceToDevice, st));
-  if (win_start)
-    DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(win_start, ctx->win_start, sizeof(int32_t) * (size_t)(nw + 1), cudaMemcpyDeviceToDevice, st));
-  if (win_setoff)
-    DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(win_setoff, ctx->win_setoff, sizeof(int32_t) * (size_t)(nw + 1), cudaMemcpyDeviceToDevice, st));
-  return DSVT_OK;
+  if (o.set_rowoff && (n == 0 || cap_sets == 0))  // no sets: row offset 0, empty tile plan
+    DSVT_CUDA_TRY(ctx, cudaMemsetAsync(o.set_rowoff, 0, sizeof(int32_t) * (size_t)(2 * (size_t)cap_sets + 3), st));
+  return copy_window_arrays(ctx, pc, ctx->win_count);
+}
+
+// Words of bitmap per window, or 0 if the bitmap route cannot take this call.
+int32_t bitmap_words_per_window(const dsvt_ctx* ctx, const PartCall& pc) {
+  if (ctx->bm_words == 0 || pc.n == 0 || pc.cap_sets == 0) return 0;
+  const uint64_t wpw = (pc.V + 31) / 32;
+  if ((uint64_t)pc.nw * wpw > ctx->bm_words || (uint64_t)pc.nw * wpw * 32 > 0xFFFFFFFFull) return 0;
+  return (int32_t)wpw;
+}
+
+// Bitmap route: one or both axes in six launches.
+int partition_bitmap(dsvt_ctx* ctx, const PartCall& pc, int32_t wpw, int naxes, const PartOut* o) {
+  cudaStream_t st = ctx->stream;
+  const int32_t n = pc.n, nw = pc.nw;
+  const size_t words = (size_t)nw * wpw;
+  // cleared region: [win_count nw + 1 | dup_count nw + 1 | bitmap of axis slot 0 | bitmap of axis slot 1]
+  int32_t* counts = ctx->bm_zero;
+  int32_t* dup_count = counts + (nw + 1);
+  uint32_t* bitmap0 = reinterpret_cast<uint32_t*>(dup_count + (nw + 1));
+  DSVT_CUDA_TRY(ctx, cudaMemsetAsync(counts, 0, sizeof(int32_t) * (2 * (size_t)(nw + 1) + (size_t)naxes * words), st));
+  BmJob job;
+  job.naxes = naxes;
+  for (int a = 0; a < 2; ++a) {
+    const int b = a < naxes ? a : 0;
+    job.ax[a].keys = ctx->keys[b];
+    job.ax[a].bitmap = bitmap0 + (size_t)b * words;
+    job.ax[a].wordrank = ctx->bm_wordrank + (size_t)b * words;
+    job.ax[a].sorted = ctx->vals[b];
+    job.ax[a].axis = o[b].axis;
+  }
+  const unsigned vox_blocks = (unsigned)dsvt_ceil_div(n, 256);
+  bm_mark_kernel<<<vox_blocks, 256, 0, st>>>((const int4*)pc.coords, n, pc.g, (uint32_t)wpw * 32u, job, counts,
+                                             dup_count, ctx->bm_dup, ctx->status);
+  DSVT_LAUNCHED(ctx);
+  int64_t rank_blocks = dsvt_ceil_div((int64_t)naxes * nw, kScanThreads / 32);
+  if (rank_blocks > 2 * (int64_t)ctx->sm_count) rank_blocks = 2 * (int64_t)ctx->sm_count;
+  bm_scan_kernel<<<(unsigned)(1 + rank_blocks), kScanThreads, 0, st>>>(
+      counts, nw, pc.set_size, ctx->win_start, ctx->win_setoff, pc.cap_sets, o[0].num_sets,
+      naxes > 1 ? o[1].num_sets : nullptr, job, wpw, ctx->status);
+  DSVT_LAUNCHED(ctx);
+  bm_place_kernel<<<vox_blocks, 256, 0, st>>>(n, job, wpw, ctx->bm_dup, ctx->win_start);
+  DSVT_LAUNCHED(ctx);
+  const int64_t s_bound = sets_bound(pc);
+  if (s_bound > 0) {
+    FillAxis f0{ctx->vals[0], o[0].num_sets, o[0].set_table, o[0].set_rowoff};
+    FillAxis f1 = f0;
+    if (naxes > 1) f1 = FillAxis{ctx->vals[1], o[1].num_sets, o[1].set_table, o[1].set_rowoff};
+    table_fill_kernel<<<dim3((unsigned)dsvt_ceil_div(s_bound, 8), (unsigned)naxes), 256, 0, st>>>(
+        f0, f1, counts, ctx->win_start, ctx->win_setoff, nw, pc.set_size);
+    DSVT_LAUNCHED(ctx);
+    int32_t* r0 = o[0].set_rowoff;
+    int32_t* r1 = naxes > 1 ? o[1].set_rowoff : nullptr;
+    if (!r0) { r0 = r1; r1 = nullptr; }
+    if (r0) {
+      int rc = launch_tile_plans(ctx, o[0].num_sets, pc.cap_sets, r0, r1);
+      if (rc != DSVT_OK) return rc;
+    }
+  }
+  for (int a = 0; a < naxes; ++a)
+    if (o[a].perm)
+      DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(o[a].perm, ctx->vals[a], sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToDevice, st));
+  return copy_window_arrays(ctx, pc, counts);
+}
+
+}  // namespace
+
+extern "C" int dsvt_partition(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch, const int32_t grid[3],
+                              const int32_t window[3], int32_t set_size, int32_t axis, int32_t* set_table,
+                              int32_t cap_sets, int32_t* num_sets, int32_t* set_rowoff, int32_t* perm,
+                              int32_t* win_start, int32_t* win_count, int32_t* win_setoff) {
+  if (!num_sets || (axis != 0 && axis != 1)) return DSVT_ERR_INVALID_ARG;
+  PartCall pc;
+  int rc = validate(ctx, coords, n, batch, grid, window, set_size, cap_sets, &pc);
+  if (rc != DSVT_OK) return rc;
+  if (n > 0 && !set_table) return DSVT_ERR_INVALID_ARG;
+  pc.win_start = win_start; pc.win_count = win_count; pc.win_setoff = win_setoff;
+  const PartOut o{axis, set_table, num_sets, set_rowoff, perm};
+  const int32_t wpw = bitmap_words_per_window(ctx, pc);
+  if (wpw > 0) return partition_bitmap(ctx, pc, wpw, 1, &o);
+  return partition_sorted(ctx, pc, o);
+}
+
+extern "C" int dsvt_partition_rotated(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch,
+                                      const int32_t grid[3], const int32_t window[3], int32_t set_size,
+                                      int32_t* const set_table[2], int32_t cap_sets, int32_t* const num_sets[2],
+                                      int32_t* const set_rowoff[2], int32_t* const perm[2], int32_t* win_start,
+                                      int32_t* win_count, int32_t* win_setoff) {
+  if (!set_table || !num_sets || !num_sets[0] || !num_sets[1]) return DSVT_ERR_INVALID_ARG;
+  PartCall pc;
+  int rc = validate(ctx, coords, n, batch, grid, window, set_size, cap_sets, &pc);
+  if (rc != DSVT_OK) return rc;
+  if (n > 0 && (!set_table[0] || !set_table[1])) return DSVT_ERR_INVALID_ARG;
+  pc.win_start = win_start; pc.win_count = win_count; pc.win_setoff = win_setoff;
+  PartOut o[2];
+  for (int a = 0; a < 2; ++a)
+    o[a] = PartOut{a, set_table[a], num_sets[a], set_rowoff ? set_rowoff[a] : nullptr, perm ? perm[a] : nullptr};
+  const int32_t wpw = bitmap_words_per_window(ctx, pc);
+  if (wpw > 0) return partition_bitmap(ctx, pc, wpw, 2, o);
+  rc = partition_sorted(ctx, pc, o[0]);
+  if (rc != DSVT_OK) return rc;
+  return partition_sorted(ctx, pc, o[1]);
 }

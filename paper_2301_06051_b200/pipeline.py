@@ -1,7 +1,7 @@
 """Sequencing of the C-ABI calls for a whole backbone pass (no arithmetic here).
 
 A DSVT backbone is a stack of blocks; all blocks of a stage share the two rotated set tables of their
-frame, so a pass is: dsvt_partition (X axis), dsvt_partition (Y axis), then one dsvt_block per block,
+frame, so a pass is: dsvt_partition_rotated (X and Y axis tables), then one dsvt_block per block,
 and optionally dsvt_pool followed by a second stage on the pooled grid.
 """
 from __future__ import annotations
@@ -30,8 +30,7 @@ class Stage:
         ]
 
     def partition(self, coords: torch.Tensor):
-        for axis in (0, 1):
-            self.ctx.partition(coords, self.batch, self.grid, self.window, self.set_size, axis, out=self.tables[axis])
+        self.ctx.partition_rotated(coords, self.batch, self.grid, self.window, self.set_size, out=tuple(self.tables))
 
     def forward(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
         """Partition (both axes) then every block; the result ends up in y."""

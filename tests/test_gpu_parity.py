@@ -25,37 +25,47 @@ def _nwin(batch, grid, window):
 # ------------------------------------------------------------------------------------------------
 # partition: bit-exact
 # ------------------------------------------------------------------------------------------------
-def _check_partition(gpu, oracle, coords, batch, grid, window, tau, ctx=None):
-    n = coords.shape[0]
-    ctx = ctx or gpu.Context(max(n, 1), _nwin(batch, grid, window), 64)
-    dc = dev(coords)
-    for axis in (0, 1):
-        t = ctx.partition(dc, batch, grid, window, tau, axis, extras=True)
-        assert ctx.status_sync() == 0
-        ref = oracle.partition(coords, batch, grid, window, tau, axis)
-        tbl, ro = table_np(t)
-        assert tbl.shape == ref.set_table.shape, (axis, tbl.shape, ref.set_table.shape)
-        assert np.array_equal(tbl, ref.set_table), axis
-        assert np.array_equal(ro, rowoff_of(ref.set_table)), axis
-        # tile plan behind the row offsets: greedy packing of whole sets into tiles of at most 128 rows
-        plan = t.set_rowoff[t.cap_sets + 1:].cpu().numpy()
-        S = tbl.shape[0]
-        starts, s = [], 0
-        while s < S:
-            starts.append(s)
-            e = s + 1
-            while e < S and ro[e + 1] - ro[s] <= 128:
-                e += 1
-            s = e
-        if S <= 24576:
-            assert plan[0] == len(starts), axis
-            assert np.array_equal(plan[1:1 + len(starts)], np.array(starts, dtype=np.int32)) and plan[1 + len(starts)] == S
-        else:
-            assert plan[0] == -1
+def _compare_table(t, ref, n, axis, extras=True):
+    tbl, ro = table_np(t)
+    assert tbl.shape == ref.set_table.shape, (axis, tbl.shape, ref.set_table.shape)
+    assert np.array_equal(tbl, ref.set_table), axis
+    assert np.array_equal(ro, rowoff_of(ref.set_table)), axis
+    # tile plan behind the row offsets: greedy packing of whole sets into tiles of at most 128 rows
+    plan = t.set_rowoff[t.cap_sets + 1:].cpu().numpy()
+    S = tbl.shape[0]
+    starts, s = [], 0
+    while s < S:
+        starts.append(s)
+        e = s + 1
+        while e < S and ro[e + 1] - ro[s] <= 128:
+            e += 1
+        s = e
+    if S <= 24576:
+        assert plan[0] == len(starts), axis
+        assert np.array_equal(plan[1:1 + len(starts)], np.array(starts, dtype=np.int32)) and plan[1 + len(starts)] == S
+    else:
+        assert plan[0] == -1
+    if extras:
         assert np.array_equal(t.perm[:n].cpu().numpy(), ref.perm)
         assert np.array_equal(t.win_count.cpu().numpy(), ref.win_count)
         assert np.array_equal(t.win_start.cpu().numpy(), ref.win_start)
         assert np.array_equal(t.win_setoff.cpu().numpy(), ref.win_setoff)
+
+
+def _check_partition(gpu, oracle, coords, batch, grid, window, tau, ctx=None):
+    """dsvt_partition per axis and dsvt_partition_rotated, both against the oracle."""
+    n = coords.shape[0]
+    ctx = ctx or gpu.Context(max(n, 1), _nwin(batch, grid, window), 64)
+    dc = dev(coords)
+    refs = [oracle.partition(coords, batch, grid, window, tau, axis) for axis in (0, 1)]
+    for axis in (0, 1):
+        t = ctx.partition(dc, batch, grid, window, tau, axis, extras=True)
+        assert ctx.status_sync() == 0
+        _compare_table(t, refs[axis], n, axis)
+    both = ctx.partition_rotated(dc, batch, grid, window, tau)
+    assert ctx.status_sync() == 0
+    for axis in (0, 1):
+        _compare_table(both[axis], refs[axis], n, axis, extras=False)
     return ctx
 
 
@@ -79,11 +89,49 @@ def test_partition_bit_exact_small_and_edge_cases(gpu, oracle, grid, window, bat
     _check_partition(gpu, oracle, di.unique_cells(rng, n, grid, batch), batch, grid, window, tau)
 
 
+def test_partition_sorting_route_on_a_key_space_beyond_the_bitmap(gpu, oracle):
+    """8400 x 8400 cells in 12 x 12 windows: 490000 windows x 160 padded cells exceed the context's
+    64 Mi-key bitmap, so the call takes the radix-sort route; results are the same."""
+    grid, window, n, tau = (8400, 8400, 1), (12, 12, 1), 6000, 36
+    rng = np.random.default_rng(99)
+    # clustered cells so that windows hold several voxels
+    centre = rng.integers(100, 8300, size=(40, 2))
+    pts = centre[rng.integers(0, 40, size=4 * n)] + rng.integers(-30, 31, size=(4 * n, 2))
+    _, first = np.unique(pts[:, 0] * 8400 + pts[:, 1], return_index=True)
+    pts = pts[np.sort(first)][:n]
+    coords = np.zeros((pts.shape[0], 4), dtype=np.int32)
+    coords[:, 1:3] = pts
+    _check_partition(gpu, oracle, coords, 1, grid, window, tau)
+
+
+def test_partition_flags_duplicate_cells_and_still_places_every_voxel(gpu):
+    rng = np.random.default_rng(5)
+    grid, window, tau = (24, 24, 1), (12, 12, 1), 5
+    coords = di.unique_cells(rng, 200, grid, 1)
+    coords = np.concatenate([coords, coords[:30], coords[:10]])  # 40 extra voxels in occupied cells
+    n = coords.shape[0]
+    ctx = gpu.Context(n, 4, 64)
+    both = ctx.partition_rotated(dev(coords), 1, grid, window, tau)
+    assert ctx.status_sync() & gpu.STATUS_DUPLICATE_CELL
+    wid = (coords[:, 1] // 12) * 2 + coords[:, 2] // 12
+    for t in both:
+        tbl, ro = table_np(t)
+        assert ro[-1] == n
+        seen = np.zeros(n, dtype=np.int64)
+        for row in tbl:
+            u = np.unique(row)
+            seen[u] += 1
+            assert len(set(wid[u].tolist())) == 1
+        assert np.all(seen == 1)
+
+
 def test_partition_empty_and_errors(gpu):
     ctx = gpu.Context(100, 64, 64)
     empty = torch.zeros((0, 4), dtype=torch.int32, device="cuda")
     t = ctx.partition(empty, 1, (8, 8, 1), (4, 4, 1), 3, 0, extras=True)
     assert int(t.num_sets.item()) == 0 and int(t.win_start.sum().item()) == 0 and ctx.status_sync() == 0
+    both = ctx.partition_rotated(empty, 1, (8, 8, 1), (4, 4, 1), 3)
+    assert int(both[0].num_sets.item()) == 0 and int(both[1].num_sets.item()) == 0 and ctx.status_sync() == 0
     ok = dev(np.array([[0, 1, 1, 0], [0, 2, 2, 0], [0, 7, 7, 0]], dtype=np.int32))
     with pytest.raises(gpu.DsvtError):
         ctx.partition(ok, 1, (8, 8, 1), (4, 4, 1), 3, 2)  # bad axis
