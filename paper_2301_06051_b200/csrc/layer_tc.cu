@@ -48,18 +48,33 @@ struct TcGeom {
   int NF;       // MLP-1 chunk width (128 or 64)
   int n_f1;     // hidden / NF
   int mode;     // 0: attention only, 1: attention + residual + LN1, 2: full layer
-  uint32_t off_a, off_kv, off_stage, off_misc, off_par;  // byte offsets from the 1024-aligned base
+  uint32_t off_a, off_kv, off_stage, off_par;  // byte offsets from the 1024-aligned base
 };
 
-struct Misc {  // small shared state behind the big regions
+struct Misc {  // small shared state beside the big regions
   unsigned long long full[kStages], empty[kStages], acc_full[2], acc_free[2], a_ready, sched_full[2], sched_empty[2];
   uint32_t tmem_base;
   int abort_flag;
   int tile[2][4];  // ring of tiles: first set, number of sets (< 0: no more tiles), first row, rows
+  // launch constants, written once before the roles start: the phase functions read them from here
+  // instead of taking them as arguments, so that nothing has to stay in registers across their calls
+  const float* x;
+  float* y;
+  const int32_t* table;
+  const int32_t* rowoff;
+  int32_t* status;
+  unsigned char* sm;   // 1024-aligned base of the dynamic shared memory (generic address)
+  uint32_t sbase;      // the same as a shared-space address
+  uint32_t off_a, off_kv, off_par;
+  int n, tau, heads, mode, NF, n_f1, ln1, ln2;
+  float eps;
+  // the tile the compute warps are working on
+  int s_lo, nsets, base, rows;
   int rowvox[kTM];
-  int set_lo[kTM + 1];
+  short set_lo[kTM + 1];
   short row_lo[kTM], row_hi[kTM];  // tile-row range of the set each row belongs to
 };
+__shared__ Misc s_mi;
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -291,10 +306,14 @@ struct TcMaps {
 // Attention of one tile with mma.sync: one warp per (set, head, 16-query block).
 // D = head dim (16 / 24 / 32), NT = key blocks of 8 a set can have.
 // ---------------------------------------------------------------------------------------------
-template <int D, int NT>
-__device__ __noinline__ void attend_tile(uint32_t a_base, uint32_t k_base, uint32_t v_base, const int* set_lo,
-                                            int nsets, int heads, int warp, int lane) {
+template <int C, int D, int NT>
+__device__ __noinline__ void attend_tile() {
   constexpr int DC = D / 8;  // 16-byte chunks per head
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t a_base = s_mi.sbase + s_mi.off_a, k_base = s_mi.sbase + s_mi.off_kv;
+  const uint32_t v_base = k_base + (C / 64) * (kTM * 128);
+  const short* set_lo = s_mi.set_lo;
+  const int nsets = s_mi.nsets, heads = s_mi.heads;
   const int g = lane >> 2, t4 = lane & 3;
   const float sc = 1.4426950408889634f * rsqrtf((float)D);  // log2(e) / sqrt(d)
   int item = 0;
@@ -403,10 +422,15 @@ __device__ __noinline__ void attend_tile(uint32_t a_base, uint32_t k_base, uint3
 // many tiny sets cost one item per 16 rows instead of one per set.
 // NTB = key blocks of 8 a row block can need: ceil((2 tau + 14) / 8).
 // ---------------------------------------------------------------------------------------------
-template <int D, int NTB>
-__device__ __noinline__ void attend_blocked(uint32_t a_base, uint32_t k_base, uint32_t v_base, const short* row_lo,
-                                            const short* row_hi, int rows, int heads, int warp, int lane) {
+template <int C, int D, int NTB>
+__device__ __noinline__ void attend_blocked() {
   constexpr int DC = D / 8;  // 16-byte chunks per head
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t a_base = s_mi.sbase + s_mi.off_a, k_base = s_mi.sbase + s_mi.off_kv;
+  const uint32_t v_base = k_base + (C / 64) * (kTM * 128);
+  const short* row_lo = s_mi.row_lo;
+  const short* row_hi = s_mi.row_hi;
+  const int rows = s_mi.rows, heads = s_mi.heads;
   constexpr int PW = 4;      // key blocks of 8 per pass (running softmax across passes keeps registers low)
   const int t4 = lane & 3;
   const float sc = 1.4426950408889634f * rsqrtf((float)D);  // log2(e) / sqrt(d)
@@ -562,7 +586,7 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
   constexpr uint32_t STAGE_BYTES = C * 128;
   unsigned char* sm = rc.sm;
   const uint32_t sbase = rc.sbase, tmem = rc.tmem;
-  Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
+  Misc* mi = &s_mi;
   const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &mi->abort_flag;
@@ -662,7 +686,7 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
   constexpr uint32_t STAGE_BYTES = C * 128;
   unsigned char* sm = rc.sm;
   const uint32_t sbase = rc.sbase, tmem = rc.tmem;
-  Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
+  Misc* mi = &s_mi;
   const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &mi->abort_flag;
@@ -718,14 +742,16 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
 }
 
 // ================= compute warps ========================================================================
-// Each phase of a tile is a separate (not inlined) function with a handful of scalar arguments, so that each
-// gets a register allocation of its own and the tile loop keeps only a few values alive across them.
+// Each phase of a tile is a separate (not inlined) function that takes at most a few scalars and reads the
+// rest from s_mi, so that each gets a register allocation of its own and the tile loop keeps almost nothing
+// alive across the calls.
 
 // Distinct slots of each set -> tile rows (Eq. 4), per-row set ranges, per-set first rows.
-__device__ __noinline__ void phase_row_list(const int32_t* __restrict__ table, const int32_t* __restrict__ rowoff, int n,
-                                            int tau, int s_lo, int nsets, int base, int rows, Misc* mi,
-                                            int32_t* __restrict__ status) {
+__device__ __noinline__ void phase_row_list() {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int32_t* __restrict__ table = s_mi.table;
+  const int32_t* __restrict__ rowoff = s_mi.rowoff;
+  const int n = s_mi.n, tau = s_mi.tau, s_lo = s_mi.s_lo, nsets = s_mi.nsets, base = s_mi.base;
   for (int si = warp; si < nsets; si += kComputeWarps) {
     const int s = s_lo + si;
     const int32_t* trow = table + (size_t)s * tau;
@@ -739,34 +765,37 @@ __device__ __noinline__ void phase_row_list(const int32_t* __restrict__ table, c
       const unsigned bal = __ballot_sync(0xffffffffu, uniq);
       const int pos = cnt + __popc(bal & ((1u << lane) - 1u));
       if (uniq && pos < cap && lb >= 0 && lb + pos < kTM) {
-        if (v < 0 || v >= n) { atomicOr(status, DSVT_STATUS_BAD_INDEX); v = -1; }
-        mi->rowvox[lb + pos] = v;
+        if (v < 0 || v >= n) { atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX); v = -1; }
+        s_mi.rowvox[lb + pos] = v;
       }
       cnt += __popc(bal);
     }
     if (lb >= 0)
       for (int i = lane; i < cap && lb + i < kTM; i += 32) {
-        mi->row_lo[lb + i] = (short)lb;
-        mi->row_hi[lb + i] = (short)min(lb + cap, kTM);
+        s_mi.row_lo[lb + i] = (short)lb;
+        s_mi.row_hi[lb + i] = (short)min(lb + cap, kTM);
       }
     if (lane == 0) {
-      mi->set_lo[si] = min(max(lb, 0), kTM);
-      if (cnt != cap) atomicOr(status, DSVT_STATUS_BAD_INDEX);
+      s_mi.set_lo[si] = (short)min(max(lb, 0), kTM);
+      if (cnt != cap) atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX);
     }
   }
-  if (tid == 0) mi->set_lo[nsets] = rows;
+  if (tid == 0) s_mi.set_lo[nsets] = (short)s_mi.rows;
 }
 
 // Gather: fp32 rows -> bf16 A operand (four rows in flight per warp); all 128 rows are written.
 template <int C>
-__device__ __noinline__ void phase_gather(const float* __restrict__ x, const int* rowvox, int rows, unsigned char* a_tile) {
+__device__ __noinline__ void phase_gather() {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float* __restrict__ x = s_mi.x;
+  unsigned char* a_tile = s_mi.sm + s_mi.off_a;
+  const int rows = s_mi.rows;
   for (int r0 = warp; r0 < kTM; r0 += 4 * kComputeWarps) {
     float4 f[4][2];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int r = r0 + kComputeWarps * u;
-      const int v = r < rows ? rowvox[r] : -1;
+      const int v = r < rows ? s_mi.rowvox[r] : -1;
       f[u][0] = f[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (v >= 0 && lane < (C >> 3)) {
         const float4* src = reinterpret_cast<const float4*>(x + (size_t)v * C) + 2 * lane;
@@ -784,16 +813,33 @@ __device__ __noinline__ void phase_gather(const float* __restrict__ x, const int
   }
 }
 
-// Epilogue of a projection chunk: QC accumulator columns + bias (in shared memory) -> bf16 into an operand tile.
-// GELU = true applies gelu first (MLP-1).  c8 = first 16-byte chunk of this thread in the destination.
+// Epilogue of a projection chunk: QC accumulator columns per thread + bias -> bf16 into an operand tile.
+// Four threads per tile row: warp w owns TMEM lanes 32 (w % 4) .. + 31 and column quarter w / 4.
+//   tcol      first TMEM column of the chunk's accumulator
+//   bar       accumulator barrier pair to release
+//   bias_off  float offset of the chunk's bias in the parameter block
+//   dst_off   byte offset of the destination operand tile from the shared-memory base
+//   c8_0      16-byte chunk index of the chunk's first column in the destination rows
+//   need      number of leading tile rows whose results are needed (warps wholly past it only release)
+// GELU = true applies gelu first (MLP-1).
 template <int QC, bool GELU>
-__device__ __noinline__ void phase_epi_bf16(uint32_t taddr, unsigned long long* acc_free, const float* bias,
-                                            unsigned char* dst, int row, int c8) {
+__device__ __noinline__ void phase_epi_bf16(uint32_t tcol, int bar, int bias_off, uint32_t dst_off, int c8_0, int need) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = 32 * (warp & 3) + lane, hq = warp >> 2;
+  if (32 * (warp & 3) >= need) {
+    tc_fence_before();
+    mbar_arrive(&s_mi.acc_free[bar]);
+    return;
+  }
+  const uint32_t taddr = s_mi.tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + tcol + hq * QC;
+  const float* bias = reinterpret_cast<const float*>(s_mi.sm + s_mi.off_par) + bias_off + hq * QC;
+  unsigned char* dst = s_mi.sm + dst_off;
+  const int c8 = c8_0 + ((hq * QC) >> 3);
   float rr[QC];
   tmem_ld_row(taddr, rr);
   tmem_wait_ld();
   tc_fence_before();
-  mbar_arrive(acc_free);  // the accumulator is in registers now
+  mbar_arrive(&s_mi.acc_free[bar]);  // the accumulator is in registers now
 #pragma unroll
   for (int q = 0; q < QC / 8; ++q) {
     const float4 b0 = *reinterpret_cast<const float4*>(bias + 8 * q), b1 = *reinterpret_cast<const float4*>(bias + 8 * q + 4);
@@ -810,12 +856,15 @@ __device__ __noinline__ void phase_epi_bf16(uint32_t taddr, unsigned long long* 
 
 // x rows (fp32) for the first residual: asynchronous 16-byte copies global -> shared staging.
 template <int C>
-__device__ __noinline__ void phase_stage_x(const float* __restrict__ x, const int* rowvox, int rows, unsigned char* stage,
-                                           uint32_t stage_saddr) {
+__device__ __noinline__ void phase_stage_x() {
   constexpr int C4 = C / 4;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float* __restrict__ x = s_mi.x;
+  unsigned char* stage = s_mi.sm + s_mi.off_kv;
+  const uint32_t stage_saddr = s_mi.sbase + s_mi.off_kv;
+  const int rows = s_mi.rows;
   for (int r = warp; r < rows; r += kComputeWarps) {
-    const int v = rowvox[r];
+    const int v = s_mi.rowvox[r];
     for (int c4 = lane; c4 < C4; c4 += 32) {
       const uint32_t off = stage_off<C>(r, c4);
       if (v >= 0)
@@ -830,11 +879,14 @@ __device__ __noinline__ void phase_stage_x(const float* __restrict__ x, const in
 
 // fp32 rows staged in shared memory -> coalesced global rows.
 template <int C>
-__device__ __noinline__ void phase_store_rows(float* __restrict__ y, const int* rowvox, int rows, const unsigned char* stage) {
+__device__ __noinline__ void phase_store_rows() {
   constexpr int C4 = C / 4;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float* __restrict__ y = s_mi.y;
+  const unsigned char* stage = s_mi.sm + s_mi.off_kv;
+  const int rows = s_mi.rows;
   for (int r = warp; r < rows; r += kComputeWarps) {
-    const int v = rowvox[r];
+    const int v = s_mi.rowvox[r];
     if (v < 0) continue;
     for (int c4 = lane; c4 < C4; c4 += 32)
       reinterpret_cast<float4*>(y + (size_t)v * C)[c4] = *reinterpret_cast<const float4*>(stage + stage_off<C>(r, c4));
@@ -876,25 +928,29 @@ __device__ __forceinline__ void layer_norm_rows(float (&t)[QC], float sum, const
   }
 }
 
-// Output-projection epilogue: t = Z + b_o (+ staged x); LayerNorm; then either the fp32 rows go to the staging
-// area (final result of the call: to_stage) or x1 goes to TMEM (fp32 park) and to the A operand (bf16).
-// par: the parameter block in shared memory; do_ln: apply LayerNorm 1.
+// Output-projection epilogue: t = Z + b_o (+ staged x); LayerNorm 1; then either the fp32 rows go to the
+// staging area (mode 0 / 1: final result of the call) or x1 goes to TMEM (fp32 park) and to the A operand
+// (bf16).  The accumulator is buffer A (column 0, barrier pair 0).
 template <int C, int QC>
-__device__ __noinline__ void phase_epi_o(uint32_t taddr, unsigned long long* acc_free, const float* par, float eps, bool do_ln,
-                                         bool add_x, bool to_stage, unsigned char* stage, unsigned char* a_tile,
-                                         uint32_t park_addr, int rows) {
+__device__ __noinline__ void phase_epi_o() {
+  constexpr uint32_t COL_PARK = kTmemCols - C;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = 32 * (warp & 3) + lane, hq = warp >> 2;
+  const uint32_t taddr = s_mi.tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + hq * QC;
+  const float* par = reinterpret_cast<const float*>(s_mi.sm + s_mi.off_par);
+  unsigned char* stage = s_mi.sm + s_mi.off_kv;
+  const int mode = s_mi.mode;
+  const bool add_x = mode != 0 && row < s_mi.rows;
   float t[QC];
   float sum = 0.f;
   tmem_ld_row(taddr, t);
   tmem_wait_ld();
   tc_fence_before();
-  mbar_arrive(acc_free);
+  mbar_arrive(&s_mi.acc_free[0]);
 #pragma unroll
   for (int q = 0; q < QC / 4; ++q) {
     float4 x4 = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (add_x && row < rows) x4 = *reinterpret_cast<const float4*>(stage + stage_off<C>(row, hq * (QC / 4) + q));
+    if (add_x) x4 = *reinterpret_cast<const float4*>(stage + stage_off<C>(row, hq * (QC / 4) + q));
     const float4 b4 = *reinterpret_cast<const float4*>(par + ParOff<C>::b_o + hq * QC + 4 * q);
     t[4 * q] += x4.x + b4.x;
     t[4 * q + 1] += x4.y + b4.y;
@@ -902,14 +958,14 @@ __device__ __noinline__ void phase_epi_o(uint32_t taddr, unsigned long long* acc
     t[4 * q + 3] += x4.w + b4.w;
     sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
   }
-  if (do_ln) {
+  if (mode != 0 && s_mi.ln1) {
     // exchange slots: the first two words of each thread's own (already consumed) x staging chunk
     auto slot = [&](int which, int quarter) {
       return reinterpret_cast<float*>(stage + stage_off<C>(row, quarter * (QC / 4))) + which;
     };
-    layer_norm_rows<C, QC>(t, sum, par + ParOff<C>::ln1_g, par + ParOff<C>::ln1_b, eps, hq, slot);
+    layer_norm_rows<C, QC>(t, sum, par + ParOff<C>::ln1_g, par + ParOff<C>::ln1_b, s_mi.eps, hq, slot);
   }
-  if (to_stage) {
+  if (mode != 2) {
     compute_sync();  // the x staging (and the exchange slots in it) is dead once every thread has its t
 #pragma unroll
     for (int i4 = 0; i4 < QC / 4; ++i4)
@@ -917,8 +973,9 @@ __device__ __noinline__ void phase_epi_o(uint32_t taddr, unsigned long long* acc
           make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
     return;
   }
-  tmem_st_row(park_addr, t);
+  tmem_st_row(taddr + COL_PARK, t);
   tmem_wait_st();
+  unsigned char* a_tile = s_mi.sm + s_mi.off_a;
 #pragma unroll
   for (int q = 0; q < QC / 8; ++q)
     *reinterpret_cast<uint4*>(a_tile + swz(row, ((hq * QC) >> 3) + q)) =
@@ -927,38 +984,46 @@ __device__ __noinline__ void phase_epi_o(uint32_t taddr, unsigned long long* acc
   tc_fence_before();
 }
 
-// MLP-2 epilogue: t = M + b_2 + parked x1; LayerNorm; fp32 rows to the staging area.  The exchange slots
+// MLP-2 epilogue: t = M + b_2 + parked x1; LayerNorm 2; fp32 rows to the staging area.  The exchange slots
 // live in the A operand tile, which nobody uses between MLP-1 and the next tile's gather.
+// tcol / bar: the accumulator's first TMEM column and barrier pair.
 template <int C, int QC>
-__device__ __noinline__ void phase_epi_f2(uint32_t taddr, unsigned long long* acc_free, const float* par, float eps, bool do_ln,
-                                          unsigned char* stage, unsigned char* a_tile, uint32_t park_addr) {
+__device__ __noinline__ void phase_epi_f2(uint32_t tcol, int bar) {
+  constexpr uint32_t COL_PARK = kTmemCols - C;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = 32 * (warp & 3) + lane, hq = warp >> 2;
+  const uint32_t lane_addr = s_mi.tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + hq * QC;
+  const float* par = reinterpret_cast<const float*>(s_mi.sm + s_mi.off_par);
   float t[QC];
   float sum = 0.f;
-  tmem_ld_row(taddr, t);
+  tmem_ld_row(lane_addr + tcol, t);
   tmem_wait_ld();
   tc_fence_before();
-  mbar_arrive(acc_free);
-  {
-    float rp[QC];
-    tmem_ld_row(park_addr, rp);
+  mbar_arrive(&s_mi.acc_free[bar]);
+  // the parked x1 comes in pieces of 16 columns, so that only one piece is live beside t
+#pragma unroll
+  for (int q16 = 0; q16 < QC / 16; ++q16) {
+    float rp[16];
+    tmem_ld_row(lane_addr + COL_PARK + 16 * q16, rp);
     tmem_wait_ld();
 #pragma unroll
-    for (int q = 0; q < QC / 4; ++q) {
-      const float4 b4 = *reinterpret_cast<const float4*>(par + ParOff<C>::b_2 + hq * QC + 4 * q);
-      t[4 * q] += rp[4 * q] + b4.x;
-      t[4 * q + 1] += rp[4 * q + 1] + b4.y;
-      t[4 * q + 2] += rp[4 * q + 2] + b4.z;
-      t[4 * q + 3] += rp[4 * q + 3] + b4.w;
-      sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
+    for (int q = 0; q < 4; ++q) {
+      const float4 b4 = *reinterpret_cast<const float4*>(par + ParOff<C>::b_2 + hq * QC + 16 * q16 + 4 * q);
+      float* tt = &t[16 * q16 + 4 * q];
+      tt[0] += rp[4 * q] + b4.x;
+      tt[1] += rp[4 * q + 1] + b4.y;
+      tt[2] += rp[4 * q + 2] + b4.z;
+      tt[3] += rp[4 * q + 3] + b4.w;
+      sum += (tt[0] + tt[1]) + (tt[2] + tt[3]);
     }
   }
-  if (do_ln) {
-    auto slot = [&](int which, int quarter) { return reinterpret_cast<float*>(a_tile) + (which * 4 + quarter) * kTM + row; };
-    layer_norm_rows<C, QC>(t, sum, par + ParOff<C>::ln2_g, par + ParOff<C>::ln2_b, eps, hq, slot);
+  if (s_mi.ln2) {
+    float* xch = reinterpret_cast<float*>(s_mi.sm + s_mi.off_a);
+    auto slot = [&](int which, int quarter) { return xch + (which * 4 + quarter) * kTM + row; };
+    layer_norm_rows<C, QC>(t, sum, par + ParOff<C>::ln2_g, par + ParOff<C>::ln2_b, s_mi.eps, hq, slot);
   }
   // the MLP-2 MMAs have read H: its region takes the fp32 output rows
+  unsigned char* stage = s_mi.sm + s_mi.off_kv;
 #pragma unroll
   for (int i4 = 0; i4 < QC / 4; ++i4)
     *reinterpret_cast<float4*>(stage + stage_off<C>(row, hq * (QC / 4) + i4)) =
@@ -966,124 +1031,101 @@ __device__ __noinline__ void phase_epi_f2(uint32_t taddr, unsigned long long* ac
 }
 
 template <int C, int D, int NT, bool BLOCKED>
-__device__ __forceinline__ void compute_role(const dsvt_fused_args& a, const TcGeom& g, int32_t* __restrict__ status,
-                                             const RoleCtx rc) {
+__device__ __forceinline__ void compute_role() {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
   constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
   constexpr uint32_t COL_B = C;      // second accumulator buffer
-  constexpr uint32_t COL_PARK = kTmemCols - C;  // parked fp32 x1
-  const dsvt_layer_params& p = a.p;
-  unsigned char* sm = rc.sm;
-  const uint32_t sbase = rc.sbase, tmem = rc.tmem;
-  Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
-  const float* par = reinterpret_cast<const float*>(sm + g.off_par);  // biases and LayerNorm vectors
-  const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  volatile int* abort_flag = &mi->abort_flag;
-  // epilogues: four threads per tile row; warp w owns TMEM lanes 32 (w % 4) .. + 31 and column quarter w / 4
-  const int row = 32 * (warp & 3) + lane;
-  const int hq = warp >> 2;
-  const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+  volatile int* abort_flag = &s_mi.abort_flag;
   uint32_t uses[2] = {0u, 0u};
   int slot = 0;
   uint32_t sphase = 0;
   bool ok = true;
   auto acc_wait = [&](uint32_t bar) {
-    ok = mbar_wait(&mi->acc_full[bar], uses[bar] & 1u, abort_flag) && ok;
+    ok = mbar_wait(&s_mi.acc_full[bar], uses[bar] & 1u, abort_flag) && ok;
     ++uses[bar];
     tc_fence_after();
   };
-  auto acc_release = [&](uint32_t bar) {
-    tc_fence_before();
-    mbar_arrive(&mi->acc_free[bar]);
-  };
   for (;;) {
-    ok = mbar_wait(&mi->sched_full[slot], sphase, abort_flag) && ok;
+    ok = mbar_wait(&s_mi.sched_full[slot], sphase, abort_flag) && ok;
     compute_sync();  // also orders the previous tile's last shared-memory reads before this tile's writes
     if (*abort_flag) break;
-    const int s_lo = mi->tile[slot][0], nsets = mi->tile[slot][1], base = mi->tile[slot][2], rows = mi->tile[slot][3];
-    mbar_arrive(&mi->sched_empty[slot]);
+    const int nsets = s_mi.tile[slot][1], rows = s_mi.tile[slot][3];
+    if (threadIdx.x == 0) {
+      s_mi.s_lo = s_mi.tile[slot][0];
+      s_mi.nsets = nsets;
+      s_mi.base = s_mi.tile[slot][2];
+      s_mi.rows = rows;
+    }
+    mbar_arrive(&s_mi.sched_empty[slot]);
     if (++slot == 2) { slot = 0; sphase ^= 1u; }
     if (nsets < 0) break;
-    const bool live = 32 * (warp & 3) < rows;  // this warp's 32 tile rows hold at least one voxel
-    // the attention pads its key blocks up to 15 rows past the tile: those K / V rows must be real bf16
-    const bool live_kv = 32 * (warp & 3) < rows + 16;
-    if (tid < kTM) { mi->rowvox[tid] = -1; mi->row_lo[tid] = (short)tid; mi->row_hi[tid] = (short)(tid + 1); }
+    if (threadIdx.x < kTM) {
+      s_mi.rowvox[threadIdx.x] = -1;
+      s_mi.row_lo[threadIdx.x] = (short)threadIdx.x;
+      s_mi.row_hi[threadIdx.x] = (short)(threadIdx.x + 1);
+    }
     compute_sync();
-    phase_row_list(a.table, a.rowoff, a.n, g.tau, s_lo, nsets, base, rows, mi, status);
+    phase_row_list();
     compute_sync();
-    phase_gather<C>(a.x, mi->rowvox, rows, sm + g.off_a);
+    phase_gather<C>();
     fence_proxy_async();
-    mbar_arrive(&mi->a_ready);  // X is in place
+    mbar_arrive(&s_mi.a_ready);  // X is in place
 
     // ---- chunks 0..2: K, V, Q epilogues: + bias, to bf16, into the operand layout ----
-    for (int c = 0; c < 3; ++c) {
-      const uint32_t bar = (c == 1) ? 1u : 0u;
-      acc_wait(bar);
-      if (c == 2 ? live : live_kv)
-        phase_epi_bf16<QC, false>(tmem + lane_addr + (c == 1 ? COL_B : 0u) + hq * QC, &mi->acc_free[bar],
-                                  par + ParOff<C>::b_qkv + (c == 0 ? 1 : c == 1 ? 2 : 0) * C + hq * QC,
-                                  sm + (c == 2 ? g.off_a : g.off_kv + (uint32_t)c * (NKB * kTM * 128)), row,
-                                  (hq * QC) >> 3);
-      else
-        acc_release(bar);
-    }
+    // (the attention pads its key blocks up to 15 rows past the tile: those K / V rows must be real bf16)
+    acc_wait(0u);
+    phase_epi_bf16<QC, false>(0u, 0, ParOff<C>::b_qkv + C, s_mi.off_kv, 0, rows + 16);
+    acc_wait(1u);
+    phase_epi_bf16<QC, false>(COL_B, 1, ParOff<C>::b_qkv + 2 * C, s_mi.off_kv + NKB * kTM * 128, 0, rows + 16);
+    acc_wait(0u);
+    phase_epi_bf16<QC, false>(0u, 0, ParOff<C>::b_qkv, s_mi.off_a, 0, rows);
     compute_sync();
     // ---- attention inside each set ----
     if (BLOCKED)
-      attend_blocked<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->row_lo, mi->row_hi, rows, g.heads, warp, lane);
+      attend_blocked<C, D, NT>();
     else
-      attend_tile<D, NT>(a_base, kv_base, kv_base + NKB * (kTM * 128), mi->set_lo, nsets, g.heads, warp, lane);
+      attend_tile<C, D, NT>();
     fence_proxy_async();
-    mbar_arrive(&mi->a_ready);  // attention output is the A operand of the output projection
-    compute_sync();             // every warp is done with K and V: their region becomes fp32 staging
-    if (g.mode != 0) {
-      phase_stage_x<C>(a.x, mi->rowvox, rows, sm + g.off_kv, sbase + g.off_kv);
+    mbar_arrive(&s_mi.a_ready);  // attention output is the A operand of the output projection
+    compute_sync();              // every warp is done with K and V: their region becomes fp32 staging
+    const int mode = s_mi.mode;
+    if (mode != 0) {
+      phase_stage_x<C>();
       compute_sync();
     }
     // ---- chunk 3: output projection epilogue: Z + b_o (+ x, LayerNorm) ----
-    {
-      acc_wait(0u);
-      phase_epi_o<C, QC>(tmem + lane_addr + hq * QC, &mi->acc_free[0], par, p.ln_eps, g.mode != 0 && p.ln1_g != nullptr,
-                         g.mode != 0, g.mode != 2, sm + g.off_kv, sm + g.off_a, tmem + lane_addr + COL_PARK + hq * QC, rows);
-      if (g.mode != 2) {  // final result of this call
-        compute_sync();
-        phase_store_rows<C>(a.y, mi->rowvox, rows, sm + g.off_kv);
-        continue;
-      }
-      fence_proxy_async();
-      mbar_arrive(&mi->a_ready);  // x1 (bf16) is the A operand of MLP-1
-    }
-    // ---- MLP-1 pieces: H = gelu(x1 W_1^T + b_1) as the A operand of MLP-2 ----
-    for (int c = 0; c < g.n_f1; ++c) {
-      const uint32_t bar = (uint32_t)c & 1u;
-      acc_wait(bar);
-      if (live) {
-        const int qw = g.NF >> 2;             // columns per thread: 32 or 16
-        const int col0 = c * g.NF + hq * qw;  // first hidden column of this thread
-        const uint32_t src = tmem + lane_addr + bar * (uint32_t)g.NF + hq * qw;
-        if (qw == 32)
-          phase_epi_bf16<32, true>(src, &mi->acc_free[bar], par + ParOff<C>::b_1 + col0, sm + g.off_kv, row, col0 >> 3);
-        else
-          phase_epi_bf16<16, true>(src, &mi->acc_free[bar], par + ParOff<C>::b_1 + col0, sm + g.off_kv, row, col0 >> 3);
-      } else {
-        acc_release(bar);
-      }
+    acc_wait(0u);
+    phase_epi_o<C, QC>();
+    if (mode != 2) {  // final result of this call
+      compute_sync();
+      phase_store_rows<C>();
+      continue;
     }
     fence_proxy_async();
-    mbar_arrive(&mi->a_ready);  // H is in place
+    mbar_arrive(&s_mi.a_ready);  // x1 (bf16) is the A operand of MLP-1
+    // ---- MLP-1 pieces: H = gelu(x1 W_1^T + b_1) as the A operand of MLP-2 ----
+    const int n_f1 = s_mi.n_f1, NF = s_mi.NF;
+    for (int c = 0; c < n_f1; ++c) {
+      const int bar = c & 1;
+      acc_wait((uint32_t)bar);
+      if (NF == 128)
+        phase_epi_bf16<32, true>((uint32_t)(bar * NF), bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
+      else
+        phase_epi_bf16<16, true>((uint32_t)(bar * NF), bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
+    }
+    fence_proxy_async();
+    mbar_arrive(&s_mi.a_ready);  // H is in place
     // ---- MLP-2 epilogue: y = LN2(x1 + M) ----
     {
-      const uint32_t bar = (uint32_t)g.n_f1 & 1u;
-      acc_wait(bar);
-      phase_epi_f2<C, QC>(tmem + lane_addr + hq * QC, &mi->acc_free[bar], par, p.ln_eps, p.ln2_g != nullptr, sm + g.off_kv,
-                          sm + g.off_a, tmem + lane_addr + COL_PARK + hq * QC);
+      const int bar = n_f1 & 1;
+      acc_wait((uint32_t)bar);
+      phase_epi_f2<C, QC>(0u, bar);
       compute_sync();
-      phase_store_rows<C>(a.y, mi->rowvox, rows, sm + g.off_kv);
+      phase_store_rows<C>();
     }
   }
   if (!ok || *abort_flag) {
-    if (tid == 0) atomicOr(status, DSVT_STATUS_TIMEOUT);
+    if (threadIdx.x == 0) atomicOr(s_mi.status, DSVT_STATUS_TIMEOUT);
   }
 }
 
@@ -1098,7 +1140,7 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   unsigned char* sm = smem_raw + pad;
-  Misc* mi = reinterpret_cast<Misc*>(sm + g.off_misc);
+  Misc* mi = &s_mi;
   const int tid = threadIdx.x, warp = tid >> 5;
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(&mi->full[i], 1); mbar_init(&mi->empty[i], 1); }
@@ -1110,6 +1152,13 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
     }
     mbar_init(&mi->a_ready, kComputeThreads);
     mi->abort_flag = 0;
+    mi->x = a.x; mi->y = a.y; mi->table = a.table; mi->rowoff = a.rowoff; mi->status = status;
+    mi->sm = sm; mi->sbase = raw + pad;
+    mi->off_a = g.off_a; mi->off_kv = g.off_kv; mi->off_par = g.off_par;
+    mi->n = a.n; mi->tau = g.tau; mi->heads = g.heads; mi->mode = g.mode; mi->NF = g.NF; mi->n_f1 = g.n_f1;
+    mi->ln1 = a.p.ln1_g != nullptr; mi->ln2 = a.p.ln2_g != nullptr;
+    mi->eps = a.p.ln_eps;
+    mi->s_lo = mi->nsets = mi->base = mi->rows = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kMmaWarp) {
@@ -1151,7 +1200,7 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
     if ((tid & 31) == 0) mma_role<C>(a, g, rc);
     __syncwarp();
   } else {
-    compute_role<C, D, NT, BLOCKED>(a, g, status, rc);
+    compute_role<C, D, NT, BLOCKED>();
   }
   // ---- teardown: everyone meets here, then the allocating warp returns the TMEM columns ----
   tc_fence_before();
@@ -1244,10 +1293,9 @@ int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a) {
   g.off_a = 0;
   g.off_kv = a_bytes;
   g.off_stage = g.off_kv + (uint32_t)kTM * 2 * C * 2;  // K + V (bf16) = fp32 staging = MLP hidden (<= 2C) bytes
-  g.off_misc = g.off_stage + kStages * (uint32_t)C * 128u;
-  g.off_par = g.off_misc + (uint32_t)((sizeof(Misc) + 15) / 16 * 16);
+  g.off_par = g.off_stage + kStages * (uint32_t)C * 128u;
   const size_t smem = (size_t)g.off_par + (size_t)(9 * C + g.hidden) * sizeof(float) + 1024;
-  if (smem > 227 * 1024) return DSVT_ERR_UNSUPPORTED;
+  if (smem + sizeof(Misc) + 16 > 227 * 1024) return DSVT_ERR_UNSUPPORTED;  // s_mi is static shared memory
   TcMaps maps;
   bool okm = make_weight_map(&maps.qkv, p.W_qkv, 3 * C, C, C) && make_weight_map(&maps.o, p.W_o, C, C, C);
   if (g.hidden > 0)
