@@ -37,7 +37,9 @@ constexpr int kTM = 128;               // tile rows = UMMA M
 constexpr int kComputeWarps = 16;
 constexpr int kComputeThreads = 32 * kComputeWarps;
 constexpr int kTmaWarp = kComputeWarps, kMmaWarp = kComputeWarps + 1;
-constexpr int kThreads = kComputeThreads + 64;  // + scheduler/TMA warp + MMA warp
+constexpr int kLoadWarp0 = kComputeWarps + 2, kLoadWarps = 2;  // row-list + gather warps, one tile ahead
+constexpr int kLoadThreads = 32 * kLoadWarps;
+constexpr int kThreads = kComputeThreads + 64 + kLoadThreads;
 constexpr int kStages = 3;             // weight ring depth
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxPolls = 1 << 20;
@@ -52,7 +54,13 @@ struct TcGeom {
 };
 
 struct Misc {  // small shared state beside the big regions
-  unsigned long long full[kStages], empty[kStages], acc_full[2], acc_free[2], a_ready, sched_full[2], sched_empty[2];
+  // weight ring; accumulator regions 0 / 1 / 2 (see the TMEM map at compute_role); operand hand-offs
+  unsigned long long full[kStages], empty[kStages], acc_full[3], acc_free[3];
+  unsigned long long a_ready;   // compute warps -> MMA: attention output / x1 / MLP hidden is in place
+  unsigned long long x_ready;   // compute warps -> MMA: the gathered rows of a tile are in the A operand
+  unsigned long long rl_ready[2];  // loader warps -> compute: row-list buffer b describes its next tile
+  unsigned long long rl_free[2];   // compute -> loader warps: row-list buffer b is no longer read
+  unsigned long long sched_full[2], sched_empty[2];
   uint32_t tmem_base;
   int abort_flag;
   int tile[2][4];  // ring of tiles: first set, number of sets (< 0: no more tiles), first row, rows
@@ -68,11 +76,14 @@ struct Misc {  // small shared state beside the big regions
   uint32_t off_a, off_kv, off_par;
   int n, tau, heads, mode, NF, n_f1, ln1, ln2;
   float eps;
-  // the tile the compute warps are working on
-  int s_lo, nsets, base, rows;
-  int rowvox[kTM];
-  short set_lo[kTM + 1];
-  short row_lo[kTM], row_hi[kTM];  // tile-row range of the set each row belongs to
+  // the tile the compute warps are working on, and which row-list buffer describes it
+  int s_lo, nsets, base, rows, buf;
+  int next_rows[2];  // rows of the tile listed in buffer b (< 0: there is no such tile), valid after rl_ready[b]
+  // row lists, double buffered: the loader warps fill buffer (k + 1) & 1 while the compute warps work on tile k;
+  // the compute warps gather tile k + 1 as soon as tile k's MMAs no longer read the A operand
+  int rowvox[2][kTM];              // tile row -> voxel (-1: none)
+  short set_lo[2][kTM + 1];        // first tile row of each set of the tile
+  unsigned char row_lo[2][kTM], row_n[2][kTM];  // per tile row: first row and row count of its set
 };
 __shared__ Misc s_mi;
 
@@ -115,6 +126,20 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory"); }
+// Barrier `id` over `nthreads` threads that also ORs a predicate: every participant gets the same answer, so a
+// loop exit taken on it is taken by all of them together.
+__device__ __forceinline__ bool bar_or(int id, int nthreads, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(nthreads), "r"((uint32_t)pred)
+      : "memory");
+  return r != 0;
+}
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, unsigned long long* bar) {
   asm volatile(
@@ -312,7 +337,7 @@ __device__ __noinline__ void attend_tile() {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t a_base = s_mi.sbase + s_mi.off_a, k_base = s_mi.sbase + s_mi.off_kv;
   const uint32_t v_base = k_base + (C / 64) * (kTM * 128);
-  const short* set_lo = s_mi.set_lo;
+  const short* set_lo = s_mi.set_lo[s_mi.buf];
   const int nsets = s_mi.nsets, heads = s_mi.heads;
   const int g = lane >> 2, t4 = lane & 3;
   const float sc = 1.4426950408889634f * rsqrtf((float)D);  // log2(e) / sqrt(d)
@@ -417,7 +442,7 @@ __device__ __noinline__ void attend_tile() {
 // ---------------------------------------------------------------------------------------------
 // Attention of one tile, blocked by 16 consecutive tile rows instead of by set: one warp per (row
 // block, head).  The keys of a block are the rows of every set that the block touches; a score is
-// kept only where query and key belong to the same set (row_lo / row_hi give each row's set range).
+// kept only where query and key belong to the same set (row_lo / row_n give each row's set range).
 // The arithmetic per query row is exactly the per-set softmax attention, but sparse regions with
 // many tiny sets cost one item per 16 rows instead of one per set.
 // NTB = key blocks of 8 a row block can need: ceil((2 tau + 14) / 8).
@@ -428,8 +453,8 @@ __device__ __noinline__ void attend_blocked() {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t a_base = s_mi.sbase + s_mi.off_a, k_base = s_mi.sbase + s_mi.off_kv;
   const uint32_t v_base = k_base + (C / 64) * (kTM * 128);
-  const short* row_lo = s_mi.row_lo;
-  const short* row_hi = s_mi.row_hi;
+  const unsigned char* row_lo = s_mi.row_lo[s_mi.buf];
+  const unsigned char* row_n = s_mi.row_n[s_mi.buf];
   const int rows = s_mi.rows, heads = s_mi.heads;
   constexpr int PW = 4;      // key blocks of 8 per pass (running softmax across passes keeps registers low)
   const int t4 = lane & 3;
@@ -440,14 +465,15 @@ __device__ __noinline__ void attend_blocked() {
     const int c0 = h * DC;
     const int q0 = 16 * blk;
     const int k_lo = row_lo[q0];
-    const int ntu = min((row_hi[min(q0 + 15, rows - 1)] - k_lo + 7) >> 3, NTB);
+    const int r_last = min(q0 + 15, rows - 1);
+    const int ntu = min((row_lo[r_last] + row_n[r_last] - k_lo + 7) >> 3, NTB);
     const int ra = q0 + (lane >> 2), rb = ra + 8;
     // each thread's two query rows: first key and number of keys of their sets, relative to k_lo
     // (rows past the tile get zero keys)
     const unsigned loA = ra < rows ? (unsigned)(row_lo[ra] - k_lo) : 0u;
-    const unsigned nA = ra < rows ? (unsigned)(row_hi[ra] - row_lo[ra]) : 0u;
+    const unsigned nA = ra < rows ? (unsigned)row_n[ra] : 0u;
     const unsigned loB = rb < rows ? (unsigned)(row_lo[rb] - k_lo) : 0u;
-    const unsigned nB = rb < rows ? (unsigned)(row_hi[rb] - row_lo[rb]) : 0u;
+    const unsigned nB = rb < rows ? (unsigned)row_n[rb] : 0u;
     uint32_t qa[4], qb[4];
     {
       const int row = q0 + (lane & 15);  // <= 127
@@ -649,15 +675,25 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
       uint32_t phase = 0, sphase = 0;
       int ns, base, rows;
       next_tile(s, ns, base, rows);
-      for (;;) {
-        if (!mbar_wait(&mi->sched_empty[slot], sphase ^ 1u, abort_flag)) break;
+      // Tiles are published two ahead of the weights (the ring has two entries), so that the loader
+      // warps can prepare tile k + 1 while tile k is being computed.
+      int ahead = 0;          // published tiles whose weights have not been streamed yet
+      bool all_out = false;   // the end marker has been published
+      auto publish = [&]() -> bool {
+        if (!mbar_wait(&mi->sched_empty[slot], sphase ^ 1u, abort_flag)) return false;
         mi->tile[slot][0] = s; mi->tile[slot][1] = ns; mi->tile[slot][2] = base; mi->tile[slot][3] = rows;
         mbar_arrive(&mi->sched_full[slot]);
         if (++slot == 2) { slot = 0; sphase ^= 1u; }
-        if (ns < 0) break;
+        if (ns < 0) { all_out = true; return true; }
+        ++ahead;
         s += ns;
-        next_tile(s, ns, base, rows);  // found now, published as soon as this tile's weights are on their way
-        // the layer's weights for this tile, chunk by chunk, K block by K block
+        next_tile(s, ns, base, rows);
+        return true;
+      };
+      if (!publish()) goto producer_done;
+      if (!all_out && !publish()) goto producer_done;
+      while (ahead > 0) {
+        // the layer's weights for one tile, chunk by chunk, K block by K block
         for (int c = 0; c < n_chunks; ++c) {
           const CUtensorMap* map;
           int row0, nkb;
@@ -673,6 +709,8 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
+        --ahead;
+        if (!all_out && !publish()) goto producer_done;
       }
     producer_done:;
     }
@@ -697,8 +735,8 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
   (void)tmem; (void)S; (void)n_chunks; (void)tid;
     if (lane == 0) {
       int stage = 0, slot = 0;
-      uint32_t phase = 0, a_phase = 0, sphase = 0;
-      uint32_t uses[2] = {0u, 0u};  // how often each accumulator barrier pair has been used
+      uint32_t phase = 0, a_phase = 0, x_phase = 0, sphase = 0;
+      uint32_t uses[3] = {0u, 0u, 0u};  // how often each accumulator region has been used
       for (;;) {
         if (!mbar_wait(&mi->sched_full[slot], sphase, abort_flag)) break;
         const int ns = mi->tile[slot][1];
@@ -707,16 +745,24 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
         if (ns < 0) break;
         for (int c = 0; c < n_chunks; ++c) {
           // a fresh A operand: X (chunks 0-2), attention output (3), x1 (4..), MLP hidden (last)
-          if (c == 0 || c == 3 || c == 4 || c == 4 + g.n_f1) {
+          if (c == 0) {
+            if (!mbar_wait(&mi->x_ready, x_phase, abort_flag)) goto mma_done;
+            x_phase ^= 1u;
+          } else if (c == 3 || c == 4 || c == 4 + g.n_f1) {
             if (!mbar_wait(&mi->a_ready, a_phase, abort_flag)) goto mma_done;
             a_phase ^= 1u;
           }
-          // accumulator placement: K -> A, V -> B, Q -> A, O -> A, MLP-1 piece i -> i & 1, MLP-2 -> A
+          // accumulator placement: K -> region 0, V -> 1, Q -> 0, O -> 0, MLP-1 piece i -> i & 1, MLP-2 -> 2
+          // (on top of the parked x1 + b_2)
           uint32_t bar, col, n;
           if (c < 4) { bar = (c == 1) ? 1u : 0u; col = (c == 1) ? COL_B : 0u; n = C; }
-          else if (c < 4 + g.n_f1) { bar = (uint32_t)(c - 4) & 1u; col = bar * (uint32_t)g.NF; n = (uint32_t)g.NF; }
-          else { bar = (uint32_t)g.n_f1 & 1u; col = 0u; n = C; }
-          if (!mbar_wait(&mi->acc_free[bar], (uses[bar] & 1u) ^ 1u, abort_flag)) goto mma_done;
+          else if (c < 4 + g.n_f1) { bar = (uint32_t)(c - 4) & 1u; col = bar * COL_B; n = (uint32_t)g.NF; }
+          else { bar = 2u; col = kTmemCols - C; n = C; }
+          if (c == 1) {
+            // region 1 may overlap region 2: the previous tile's MLP-2 result must have been read
+            if (!mbar_wait(&mi->acc_free[2], (uses[2] & 1u) ^ 1u, abort_flag)) goto mma_done;
+          }
+          if (bar != 2u && !mbar_wait(&mi->acc_free[bar], (uses[bar] & 1u) ^ 1u, abort_flag)) goto mma_done;
           ++uses[bar];
           tc_fence_after();
           const bool last = mlp && c == 4 + g.n_f1;
@@ -730,7 +776,7 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
             const uint32_t sa = abase + kb * (kTM * 128), sb = st_base + stage * STAGE_BYTES;
 #pragma unroll
             for (int k4 = 0; k4 < 4; ++k4)
-              umma_bf16(d_tmem, umma_desc(sa + k4 * 32), umma_desc(sb + k4 * 32), idesc, (kb | k4) != 0 ? 1u : 0u);
+              umma_bf16(d_tmem, umma_desc(sa + k4 * 32), umma_desc(sb + k4 * 32), idesc, (last || (kb | k4) != 0) ? 1u : 0u);
             umma_commit(&mi->empty[stage]);  // frees the weight stage once these MMAs have read it
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
@@ -741,12 +787,95 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
     }
 }
 
+// ================= loader warps: row list + gather, one tile ahead of the compute warps ==================
+__device__ __forceinline__ void loader_sync() { asm volatile("bar.sync 6, %0;" ::"n"(kLoadThreads) : "memory"); }
+
+// Distinct slots of each set -> tile rows (Eq. 4), per-row set ranges, per-set first rows: one thread per
+// set (a tile of a sparse region holds dozens of tiny sets), walking the set's table row.
+__device__ __forceinline__ void loader_row_list(int b, int lt, int s_lo, int nsets, int base) {
+  const int32_t* __restrict__ table = s_mi.table;
+  const int32_t* __restrict__ rowoff = s_mi.rowoff;
+  const int n = s_mi.n, tau = s_mi.tau;
+  for (int si = lt; si < nsets; si += kLoadThreads) {
+    const int s = s_lo + si;
+    const int32_t* trow = table + (size_t)s * tau;
+    const int lb = __ldg(rowoff + s) - base, cap = __ldg(rowoff + s + 1) - __ldg(rowoff + s);
+    const bool inside = lb >= 0 && lb < kTM;
+    const int cnt_max = inside ? min(cap, kTM - lb) : 0;  // tile rows this set may fill
+    int pos = 0, prev = 0;
+    bool bad = false;
+    for (int k0 = 0; k0 < tau; k0 += 32) {
+      int v4[32];  // 32 independent loads per round trip to L2
+#pragma unroll
+      for (int u = 0; u < 32; ++u) v4[u] = k0 + u < tau ? __ldg(trow + k0 + u) : 0;
+#pragma unroll
+      for (int u = 0; u < 32; ++u) {
+        if (k0 + u < tau) {
+          int v = v4[u];
+          const bool uniq = (k0 + u == 0) || (v != prev);
+          prev = v;
+          if (uniq) {
+            if (pos < cnt_max) {
+              if (v < 0 || v >= n) { bad = true; v = -1; }
+              s_mi.rowvox[b][lb + pos] = v;
+              s_mi.row_lo[b][lb + pos] = (unsigned char)lb;
+              s_mi.row_n[b][lb + pos] = (unsigned char)cnt_max;
+            }
+            ++pos;
+          }
+        }
+      }
+    }
+    s_mi.set_lo[b][si] = (short)min(max(lb, 0), kTM);
+    if (bad || pos != cap) atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX);
+  }
+}
+
+template <int C>
+__device__ __noinline__ void loader_role() {
+  const int lt = threadIdx.x - 32 * kLoadWarp0, lane = lt & 31;
+  volatile int* abort_flag = &s_mi.abort_flag;
+  int slot = 0;
+  uint32_t sphase = 0;
+  bool ok = true;
+  for (int k = 0;; ++k) {
+    ok = mbar_wait(&s_mi.sched_full[slot], sphase, abort_flag) && ok;
+    // every exit from this loop is taken by all loader threads together
+    if (bar_or(6, kLoadThreads, !ok || *abort_flag != 0)) break;
+    const int s_lo = s_mi.tile[slot][0], nsets = s_mi.tile[slot][1], base = s_mi.tile[slot][2], rows = s_mi.tile[slot][3];
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&s_mi.sched_empty[slot]);
+    if (++slot == 2) { slot = 0; sphase ^= 1u; }
+    const int b = k & 1;
+    if (k == 0) {  // the compute warps list a CTA's first tile themselves (nothing can run ahead of it)
+      mbar_arrive(&s_mi.rl_ready[b]);
+      if (nsets < 0) break;
+      continue;
+    }
+    // buffer b was last used by tile k - 2: the compute warps release it when they are done with that tile
+    if (k >= 2) ok = mbar_wait(&s_mi.rl_free[b], (uint32_t)((k >> 1) - 1) & 1u, abort_flag) && ok;
+    if (nsets >= 0) {
+      for (int i = lt; i < kTM; i += kLoadThreads) {
+        s_mi.rowvox[b][i] = -1;
+        s_mi.row_lo[b][i] = (unsigned char)i;
+        s_mi.row_n[b][i] = 1;
+      }
+      loader_sync();
+      loader_row_list(b, lt, s_lo, nsets, base);
+      if (lt == 0) s_mi.set_lo[b][nsets] = (short)rows;
+    }
+    if (lt == 0) s_mi.next_rows[b] = nsets < 0 ? -1 : rows;
+    mbar_arrive(&s_mi.rl_ready[b]);
+    if (nsets < 0) break;
+  }
+}
+
 // ================= compute warps ========================================================================
 // Each phase of a tile is a separate (not inlined) function that takes at most a few scalars and reads the
 // rest from s_mi, so that each gets a register allocation of its own and the tile loop keeps almost nothing
 // alive across the calls.
 
-// Distinct slots of each set -> tile rows (Eq. 4), per-row set ranges, per-set first rows.
+// Row list of a CTA's first tile by the compute warps (one warp per set), into buffer 0.
 __device__ __noinline__ void phase_row_list() {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int32_t* __restrict__ table = s_mi.table;
@@ -756,6 +885,7 @@ __device__ __noinline__ void phase_row_list() {
     const int s = s_lo + si;
     const int32_t* trow = table + (size_t)s * tau;
     const int lb = rowoff[s] - base, cap = rowoff[s + 1] - rowoff[s];
+    const int cnt_max = (lb >= 0 && lb < kTM) ? min(cap, kTM - lb) : 0;
     int cnt = 0;
     for (int k0 = 0; k0 < tau; k0 += 32) {
       const int k = k0 + lane;
@@ -764,38 +894,38 @@ __device__ __noinline__ void phase_row_list() {
       if (k < tau) { v = trow[k]; uniq = (k == 0) || (v != trow[k - 1]); }
       const unsigned bal = __ballot_sync(0xffffffffu, uniq);
       const int pos = cnt + __popc(bal & ((1u << lane) - 1u));
-      if (uniq && pos < cap && lb >= 0 && lb + pos < kTM) {
+      if (uniq && pos < cnt_max) {
         if (v < 0 || v >= n) { atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX); v = -1; }
-        s_mi.rowvox[lb + pos] = v;
+        s_mi.rowvox[0][lb + pos] = v;
       }
       cnt += __popc(bal);
     }
-    if (lb >= 0)
-      for (int i = lane; i < cap && lb + i < kTM; i += 32) {
-        s_mi.row_lo[lb + i] = (short)lb;
-        s_mi.row_hi[lb + i] = (short)min(lb + cap, kTM);
-      }
+    for (int i = lane; i < cnt_max; i += 32) {
+      s_mi.row_lo[0][lb + i] = (unsigned char)lb;
+      s_mi.row_n[0][lb + i] = (unsigned char)cnt_max;
+    }
     if (lane == 0) {
-      s_mi.set_lo[si] = (short)min(max(lb, 0), kTM);
+      s_mi.set_lo[0][si] = (short)min(max(lb, 0), kTM);
       if (cnt != cap) atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX);
     }
   }
-  if (tid == 0) s_mi.set_lo[nsets] = (short)s_mi.rows;
+  if (tid == 0) s_mi.set_lo[0][nsets] = (short)s_mi.rows;
 }
 
-// Gather: fp32 rows -> bf16 A operand (four rows in flight per warp); all 128 rows are written.
+// Gather (Eq. 4): the fp32 rows listed in buffer b -> bf16 A operand, four rows in flight per warp; all 128 rows
+// are written (rows past the tile as zeros).
 template <int C>
-__device__ __noinline__ void phase_gather() {
+__device__ __noinline__ void phase_gather(int b, int rows) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float* __restrict__ x = s_mi.x;
   unsigned char* a_tile = s_mi.sm + s_mi.off_a;
-  const int rows = s_mi.rows;
+  const int* rowvox = s_mi.rowvox[b];
   for (int r0 = warp; r0 < kTM; r0 += 4 * kComputeWarps) {
     float4 f[4][2];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int r = r0 + kComputeWarps * u;
-      const int v = r < rows ? s_mi.rowvox[r] : -1;
+      const int v = r < rows ? rowvox[r] : -1;
       f[u][0] = f[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (v >= 0 && lane < (C >> 3)) {
         const float4* src = reinterpret_cast<const float4*>(x + (size_t)v * C) + 2 * lane;
@@ -821,8 +951,9 @@ __device__ __noinline__ void phase_gather() {
 //   dst_off   byte offset of the destination operand tile from the shared-memory base
 //   c8_0      16-byte chunk index of the chunk's first column in the destination rows
 //   need      number of leading tile rows whose results are needed (warps wholly past it only release)
-// GELU = true applies gelu first (MLP-1).
-template <int QC, bool GELU>
+// GELU = true applies gelu first (MLP-1); BIAS = false skips the bias (the key projection: a key bias adds
+// the same amount q . b_k to every score of a query, which the softmax cancels).
+template <int QC, bool GELU, bool BIAS>
 __device__ __noinline__ void phase_epi_bf16(uint32_t tcol, int bar, int bias_off, uint32_t dst_off, int c8_0, int need) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = 32 * (warp & 3) + lane, hq = warp >> 2;
@@ -842,7 +973,8 @@ __device__ __noinline__ void phase_epi_bf16(uint32_t tcol, int bar, int bias_off
   mbar_arrive(&s_mi.acc_free[bar]);  // the accumulator is in registers now
 #pragma unroll
   for (int q = 0; q < QC / 8; ++q) {
-    const float4 b0 = *reinterpret_cast<const float4*>(bias + 8 * q), b1 = *reinterpret_cast<const float4*>(bias + 8 * q + 4);
+    float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+    if (BIAS) { b0 = *reinterpret_cast<const float4*>(bias + 8 * q); b1 = *reinterpret_cast<const float4*>(bias + 8 * q + 4); }
     float v[8] = {rr[8 * q] + b0.x, rr[8 * q + 1] + b0.y, rr[8 * q + 2] + b0.z, rr[8 * q + 3] + b0.w,
                   rr[8 * q + 4] + b1.x, rr[8 * q + 5] + b1.y, rr[8 * q + 6] + b1.z, rr[8 * q + 7] + b1.w};
     if (GELU) {
@@ -863,8 +995,9 @@ __device__ __noinline__ void phase_stage_x() {
   unsigned char* stage = s_mi.sm + s_mi.off_kv;
   const uint32_t stage_saddr = s_mi.sbase + s_mi.off_kv;
   const int rows = s_mi.rows;
+  const int* rowvox = s_mi.rowvox[s_mi.buf];
   for (int r = warp; r < rows; r += kComputeWarps) {
-    const int v = s_mi.rowvox[r];
+    const int v = rowvox[r];
     for (int c4 = lane; c4 < C4; c4 += 32) {
       const uint32_t off = stage_off<C>(r, c4);
       if (v >= 0)
@@ -885,8 +1018,9 @@ __device__ __noinline__ void phase_store_rows() {
   float* __restrict__ y = s_mi.y;
   const unsigned char* stage = s_mi.sm + s_mi.off_kv;
   const int rows = s_mi.rows;
+  const int* rowvox = s_mi.rowvox[s_mi.buf];
   for (int r = warp; r < rows; r += kComputeWarps) {
-    const int v = s_mi.rowvox[r];
+    const int v = rowvox[r];
     if (v < 0) continue;
     for (int c4 = lane; c4 < C4; c4 += 32)
       reinterpret_cast<float4*>(y + (size_t)v * C)[c4] = *reinterpret_cast<const float4*>(stage + stage_off<C>(r, c4));
@@ -896,41 +1030,48 @@ __device__ __noinline__ void phase_store_rows() {
 // Per-layer vectors staged in shared memory (float offsets into the parameter block).
 template <int C>
 struct ParOff {
-  static constexpr int b_qkv = 0, b_o = 3 * C, b_2 = 4 * C, ln1_g = 5 * C, ln1_b = 6 * C, ln2_g = 7 * C, ln2_b = 8 * C,
-                       b_1 = 9 * C;  // b_1 has `hidden` entries and comes last
+  static constexpr int b_q = 0, b_v = C, b_o = 2 * C, b_2 = 3 * C, ln1_g = 4 * C, ln1_b = 5 * C, ln2_g = 6 * C,
+                       ln2_b = 7 * C, b_1 = 8 * C;  // b_1 has `hidden` entries and comes last; no key bias
+  static constexpr int vectors = 8;
 };
 
-// LayerNorm over the row that four threads share: t holds this thread's QC values.  The partial sums are
-// exchanged through 4-byte slots that the caller picks: slot(which, quarter) for the two rounds.
+// LayerNorm over the row that four threads share: t holds this thread's QC values, sum their sum.  Each
+// thread reduces its own quarter to (mean, sum of squared deviations), the four pairs are exchanged once
+// through 8-byte slots that the caller picks (slot(quarter)) and combined exactly (pairwise update of
+// Chan et al.).  The four threads of a row sit in warps q, q + 4, q + 8, q + 12 and meet at a barrier of
+// their own.  Leaves t normalised; a caller whose slots are overwritten by the results calls quarter_sync()
+// before it stores them.
+__device__ __forceinline__ void quarter_sync() {
+  asm volatile("bar.sync %0, 128;" ::"r"(2 + ((threadIdx.x >> 5) & 3)) : "memory");
+}
 template <int C, int QC, class Slot>
 __device__ __forceinline__ void layer_norm_rows(float (&t)[QC], float sum, const float* gain, const float* shift, float eps,
                                                 int hq, Slot slot) {
-  // the four threads of a row sit in warps q, q + 4, q + 8, q + 12: they meet at a barrier of their own
-  const int quarter_bar = 2 + ((threadIdx.x >> 5) & 3);
-  *slot(0, hq) = sum;
-  asm volatile("bar.sync %0, 128;" ::"r"(quarter_bar) : "memory");
-  const float mean = ((*slot(0, 0) + *slot(0, 1)) + (*slot(0, 2) + *slot(0, 3))) * (1.0f / (float)C);
-  float sq = 0.f;
+  const float mq = sum * (1.0f / (float)QC);
+  float m2 = 0.f;
 #pragma unroll
-  for (int i = 0; i < QC; ++i) { t[i] -= mean; sq = fmaf(t[i], t[i], sq); }
-  *slot(1, hq) = sq;
-  asm volatile("bar.sync %0, 128;" ::"r"(quarter_bar) : "memory");
-  const float var = ((*slot(1, 0) + *slot(1, 1)) + (*slot(1, 2) + *slot(1, 3))) * (1.0f / (float)C);
-  const float inv = rsqrtf(var + eps);
+  for (int i = 0; i < QC; ++i) { const float d = t[i] - mq; m2 = fmaf(d, d, m2); }
+  *slot(hq) = make_float2(mq, m2);
+  quarter_sync();
+  const float2 s0 = *slot(0), s1 = *slot(1), s2 = *slot(2), s3 = *slot(3);
+  const float mean = 0.25f * ((s0.x + s1.x) + (s2.x + s3.x));
+  const float d0 = s0.x - mean, d1 = s1.x - mean, d2 = s2.x - mean, d3 = s3.x - mean;
+  const float ssq = ((s0.y + s1.y) + (s2.y + s3.y)) + (float)QC * ((d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3));
+  const float inv = rsqrtf(ssq * (1.0f / (float)C) + eps);
 #pragma unroll
   for (int i4 = 0; i4 < QC / 4; ++i4) {
     const float4 g4 = *reinterpret_cast<const float4*>(gain + hq * QC + 4 * i4);
     const float4 b4 = *reinterpret_cast<const float4*>(shift + hq * QC + 4 * i4);
-    t[4 * i4] = t[4 * i4] * inv * g4.x + b4.x;
-    t[4 * i4 + 1] = t[4 * i4 + 1] * inv * g4.y + b4.y;
-    t[4 * i4 + 2] = t[4 * i4 + 2] * inv * g4.z + b4.z;
-    t[4 * i4 + 3] = t[4 * i4 + 3] * inv * g4.w + b4.w;
+    t[4 * i4] = (t[4 * i4] - mean) * inv * g4.x + b4.x;
+    t[4 * i4 + 1] = (t[4 * i4 + 1] - mean) * inv * g4.y + b4.y;
+    t[4 * i4 + 2] = (t[4 * i4 + 2] - mean) * inv * g4.z + b4.z;
+    t[4 * i4 + 3] = (t[4 * i4 + 3] - mean) * inv * g4.w + b4.w;
   }
 }
 
 // Output-projection epilogue: t = Z + b_o (+ staged x); LayerNorm 1; then either the fp32 rows go to the
-// staging area (mode 0 / 1: final result of the call) or x1 goes to TMEM (fp32 park) and to the A operand
-// (bf16).  The accumulator is buffer A (column 0, barrier pair 0).
+// staging area (mode 0 / 1: final result of the call) or x1 goes to the A operand (bf16) and x1 + b_2 to
+// TMEM region 2 (fp32), where the MLP-2 MMAs accumulate on top of it.  The accumulator is region 0.
 template <int C, int QC>
 __device__ __noinline__ void phase_epi_o() {
   constexpr uint32_t COL_PARK = kTmemCols - C;
@@ -959,10 +1100,8 @@ __device__ __noinline__ void phase_epi_o() {
     sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
   }
   if (mode != 0 && s_mi.ln1) {
-    // exchange slots: the first two words of each thread's own (already consumed) x staging chunk
-    auto slot = [&](int which, int quarter) {
-      return reinterpret_cast<float*>(stage + stage_off<C>(row, quarter * (QC / 4))) + which;
-    };
+    // exchange slots: the first eight bytes of each thread's own (already consumed) x staging chunk
+    auto slot = [&](int quarter) { return reinterpret_cast<float2*>(stage + stage_off<C>(row, quarter * (QC / 4))); };
     layer_norm_rows<C, QC>(t, sum, par + ParOff<C>::ln1_g, par + ParOff<C>::ln1_b, s_mi.eps, hq, slot);
   }
   if (mode != 2) {
@@ -973,70 +1112,68 @@ __device__ __noinline__ void phase_epi_o() {
           make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
     return;
   }
-  tmem_st_row(taddr + COL_PARK, t);
-  tmem_wait_st();
   unsigned char* a_tile = s_mi.sm + s_mi.off_a;
 #pragma unroll
   for (int q = 0; q < QC / 8; ++q)
     *reinterpret_cast<uint4*>(a_tile + swz(row, ((hq * QC) >> 3) + q)) =
         make_uint4(pack_bf16(t[8 * q], t[8 * q + 1]), pack_bf16(t[8 * q + 2], t[8 * q + 3]),
                    pack_bf16(t[8 * q + 4], t[8 * q + 5]), pack_bf16(t[8 * q + 6], t[8 * q + 7]));
+#pragma unroll
+  for (int q = 0; q < QC / 4; ++q) {
+    const float4 b4 = *reinterpret_cast<const float4*>(par + ParOff<C>::b_2 + hq * QC + 4 * q);
+    t[4 * q] += b4.x;
+    t[4 * q + 1] += b4.y;
+    t[4 * q + 2] += b4.z;
+    t[4 * q + 3] += b4.w;
+  }
+  tmem_st_row(taddr + COL_PARK, t);
+  tmem_wait_st();
   tc_fence_before();
 }
 
-// MLP-2 epilogue: t = M + b_2 + parked x1; LayerNorm 2; fp32 rows to the staging area.  The exchange slots
-// live in the A operand tile, which nobody uses between MLP-1 and the next tile's gather.
-// tcol / bar: the accumulator's first TMEM column and barrier pair.
+// MLP-2 epilogue: region 2 holds x1 + b_2 + M; LayerNorm 2; fp32 rows to the staging area (the MLP-2 MMAs
+// have read H: its region takes the output rows).  The exchange slots are the first eight bytes of each
+// thread's own output chunk, which is therefore stored last, after one more meeting of the row's threads.
 template <int C, int QC>
-__device__ __noinline__ void phase_epi_f2(uint32_t tcol, int bar) {
+__device__ __noinline__ void phase_epi_f2() {
   constexpr uint32_t COL_PARK = kTmemCols - C;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = 32 * (warp & 3) + lane, hq = warp >> 2;
-  const uint32_t lane_addr = s_mi.tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + hq * QC;
+  const uint32_t taddr = s_mi.tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + COL_PARK + hq * QC;
   const float* par = reinterpret_cast<const float*>(s_mi.sm + s_mi.off_par);
+  unsigned char* stage = s_mi.sm + s_mi.off_kv;
   float t[QC];
-  float sum = 0.f;
-  tmem_ld_row(lane_addr + tcol, t);
+  tmem_ld_row(taddr, t);
   tmem_wait_ld();
   tc_fence_before();
-  mbar_arrive(&s_mi.acc_free[bar]);
-  // the parked x1 comes in pieces of 16 columns, so that only one piece is live beside t
+  mbar_arrive(&s_mi.acc_free[2]);
+  const bool ln = s_mi.ln2 != 0;
+  if (ln) {
+    float sum = 0.f;
 #pragma unroll
-  for (int q16 = 0; q16 < QC / 16; ++q16) {
-    float rp[16];
-    tmem_ld_row(lane_addr + COL_PARK + 16 * q16, rp);
-    tmem_wait_ld();
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const float4 b4 = *reinterpret_cast<const float4*>(par + ParOff<C>::b_2 + hq * QC + 16 * q16 + 4 * q);
-      float* tt = &t[16 * q16 + 4 * q];
-      tt[0] += rp[4 * q] + b4.x;
-      tt[1] += rp[4 * q + 1] + b4.y;
-      tt[2] += rp[4 * q + 2] + b4.z;
-      tt[3] += rp[4 * q + 3] + b4.w;
-      sum += (tt[0] + tt[1]) + (tt[2] + tt[3]);
-    }
-  }
-  if (s_mi.ln2) {
-    float* xch = reinterpret_cast<float*>(s_mi.sm + s_mi.off_a);
-    auto slot = [&](int which, int quarter) { return xch + (which * 4 + quarter) * kTM + row; };
+    for (int q = 0; q < QC / 4; ++q) sum += (t[4 * q] + t[4 * q + 1]) + (t[4 * q + 2] + t[4 * q + 3]);
+    auto slot = [&](int quarter) { return reinterpret_cast<float2*>(stage + stage_off<C>(row, quarter * (QC / 4))); };
     layer_norm_rows<C, QC>(t, sum, par + ParOff<C>::ln2_g, par + ParOff<C>::ln2_b, s_mi.eps, hq, slot);
   }
-  // the MLP-2 MMAs have read H: its region takes the fp32 output rows
-  unsigned char* stage = s_mi.sm + s_mi.off_kv;
 #pragma unroll
-  for (int i4 = 0; i4 < QC / 4; ++i4)
+  for (int i4 = 1; i4 < QC / 4; ++i4)
     *reinterpret_cast<float4*>(stage + stage_off<C>(row, hq * (QC / 4) + i4)) =
         make_float4(t[4 * i4], t[4 * i4 + 1], t[4 * i4 + 2], t[4 * i4 + 3]);
+  if (ln) quarter_sync();  // the row's other threads have read this thread's slot
+  *reinterpret_cast<float4*>(stage + stage_off<C>(row, hq * (QC / 4))) = make_float4(t[0], t[1], t[2], t[3]);
 }
 
+// TMEM map (512 columns): region 0 = [0, C): K, Q, O and the even MLP-1 pieces; region 1 = [C, 2C): V and
+// the odd MLP-1 pieces; region 2 = [512 - C, 512): x1 + b_2 parked by the output-projection epilogue, then
+// the MLP-2 accumulator.  Each region has its own full / free barrier pair.  For C = 192 regions 1 and 2
+// overlap, which is why the MMA issuer waits for region 2 before it starts the next tile's V.
 template <int C, int D, int NT, bool BLOCKED>
 __device__ __forceinline__ void compute_role() {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
   constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
-  constexpr uint32_t COL_B = C;      // second accumulator buffer
+  constexpr uint32_t COL_B = C;      // accumulator region 1
   volatile int* abort_flag = &s_mi.abort_flag;
-  uint32_t uses[2] = {0u, 0u};
+  uint32_t uses[3] = {0u, 0u, 0u};
   int slot = 0;
   uint32_t sphase = 0;
   bool ok = true;
@@ -1045,40 +1182,58 @@ __device__ __forceinline__ void compute_role() {
     ++uses[bar];
     tc_fence_after();
   };
-  for (;;) {
+  // The next tile's rows are gathered as soon as the current tile's MMAs have stopped reading the A operand
+  // (the caller has just waited for the accumulator of the last such chunk), so that its first projections
+  // run on the tensor pipe while the compute warps finish the current tile.
+  auto gather_next = [&](int k) {
+    const int b = (k + 1) & 1;
+    ok = mbar_wait(&s_mi.rl_ready[b], (uint32_t)((k + 1) >> 1) & 1u, abort_flag) && ok;
+    const int nr = s_mi.next_rows[b];
+    if (ok && nr >= 0) {
+      phase_gather<C>(b, nr);
+      fence_proxy_async();
+      mbar_arrive(&s_mi.x_ready);
+    }
+  };
+  for (int k = 0;; ++k) {
     ok = mbar_wait(&s_mi.sched_full[slot], sphase, abort_flag) && ok;
-    compute_sync();  // also orders the previous tile's last shared-memory reads before this tile's writes
-    if (*abort_flag) break;
+    // also orders the previous tile's last shared-memory reads before this tile's writes; every exit from
+    // this loop is taken by all compute threads together
+    if (bar_or(1, kComputeThreads, !ok || *abort_flag != 0)) break;
     const int nsets = s_mi.tile[slot][1], rows = s_mi.tile[slot][3];
     if (threadIdx.x == 0) {
       s_mi.s_lo = s_mi.tile[slot][0];
       s_mi.nsets = nsets;
       s_mi.base = s_mi.tile[slot][2];
       s_mi.rows = rows;
+      s_mi.buf = k & 1;
+      if (k >= 1) mbar_arrive(&s_mi.rl_free[(k - 1) & 1]);  // the previous tile's row list is dead
     }
     mbar_arrive(&s_mi.sched_empty[slot]);
     if (++slot == 2) { slot = 0; sphase ^= 1u; }
     if (nsets < 0) break;
-    if (threadIdx.x < kTM) {
-      s_mi.rowvox[threadIdx.x] = -1;
-      s_mi.row_lo[threadIdx.x] = (short)threadIdx.x;
-      s_mi.row_hi[threadIdx.x] = (short)(threadIdx.x + 1);
+    if (k == 0 && threadIdx.x < kTM) {
+      s_mi.rowvox[0][threadIdx.x] = -1;
+      s_mi.row_lo[0][threadIdx.x] = (unsigned char)threadIdx.x;
+      s_mi.row_n[0][threadIdx.x] = 1;
     }
-    compute_sync();
-    phase_row_list();
-    compute_sync();
-    phase_gather<C>();
-    fence_proxy_async();
-    mbar_arrive(&s_mi.a_ready);  // X is in place
+    compute_sync();  // the tile's fields are visible to the phase functions
+    if (k == 0) {  // nothing runs ahead of a CTA's first tile: all compute warps list and gather it
+      phase_row_list();
+      compute_sync();
+      phase_gather<C>(0, rows);
+      fence_proxy_async();
+      mbar_arrive(&s_mi.x_ready);  // X is in place
+    }
 
-    // ---- chunks 0..2: K, V, Q epilogues: + bias, to bf16, into the operand layout ----
+    // ---- chunks 0..2: K, V, Q epilogues: (+ bias,) to bf16, into the operand layout ----
     // (the attention pads its key blocks up to 15 rows past the tile: those K / V rows must be real bf16)
     acc_wait(0u);
-    phase_epi_bf16<QC, false>(0u, 0, ParOff<C>::b_qkv + C, s_mi.off_kv, 0, rows + 16);
+    phase_epi_bf16<QC, false, false>(0u, 0, 0, s_mi.off_kv, 0, rows + 16);
     acc_wait(1u);
-    phase_epi_bf16<QC, false>(COL_B, 1, ParOff<C>::b_qkv + 2 * C, s_mi.off_kv + NKB * kTM * 128, 0, rows + 16);
+    phase_epi_bf16<QC, false, true>(COL_B, 1, ParOff<C>::b_v, s_mi.off_kv + NKB * kTM * 128, 0, rows + 16);
     acc_wait(0u);
-    phase_epi_bf16<QC, false>(0u, 0, ParOff<C>::b_qkv, s_mi.off_a, 0, rows);
+    phase_epi_bf16<QC, false, true>(0u, 0, ParOff<C>::b_q, s_mi.off_a, 0, rows);
     compute_sync();
     // ---- attention inside each set ----
     if (BLOCKED)
@@ -1097,6 +1252,7 @@ __device__ __forceinline__ void compute_role() {
     acc_wait(0u);
     phase_epi_o<C, QC>();
     if (mode != 2) {  // final result of this call
+      gather_next(k);  // the output projection was the last chunk to read the A operand
       compute_sync();
       phase_store_rows<C>();
       continue;
@@ -1109,20 +1265,18 @@ __device__ __forceinline__ void compute_role() {
       const int bar = c & 1;
       acc_wait((uint32_t)bar);
       if (NF == 128)
-        phase_epi_bf16<32, true>((uint32_t)(bar * NF), bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
+        phase_epi_bf16<32, true, true>(bar * COL_B, bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
       else
-        phase_epi_bf16<16, true>((uint32_t)(bar * NF), bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
+        phase_epi_bf16<16, true, true>(bar * COL_B, bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
     }
     fence_proxy_async();
     mbar_arrive(&s_mi.a_ready);  // H is in place
+    gather_next(k);  // the last MLP-1 piece has been drained: nothing reads the A operand any more
     // ---- MLP-2 epilogue: y = LN2(x1 + M) ----
-    {
-      const int bar = n_f1 & 1;
-      acc_wait((uint32_t)bar);
-      phase_epi_f2<C, QC>(0u, bar);
-      compute_sync();
-      phase_store_rows<C>();
-    }
+    acc_wait(2u);
+    phase_epi_f2<C, QC>();
+    compute_sync();
+    phase_store_rows<C>();
   }
   if (!ok || *abort_flag) {
     if (threadIdx.x == 0) atomicOr(s_mi.status, DSVT_STATUS_TIMEOUT);
@@ -1144,13 +1298,19 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   const int tid = threadIdx.x, warp = tid >> 5;
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(&mi->full[i], 1); mbar_init(&mi->empty[i], 1); }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 3; ++i) {
       mbar_init(&mi->acc_full[i], 1);
       mbar_init(&mi->acc_free[i], kComputeThreads);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(&mi->sched_full[i], 1);
-      mbar_init(&mi->sched_empty[i], kComputeThreads + 1);
+      mbar_init(&mi->sched_empty[i], kComputeThreads + 1 + kLoadWarps);  // compute threads, MMA issuer, loader warps
+      mbar_init(&mi->rl_free[i], 1);
+      mbar_init(&mi->rl_ready[i], kLoadThreads);
+      mi->next_rows[i] = -1;
     }
     mbar_init(&mi->a_ready, kComputeThreads);
+    mbar_init(&mi->x_ready, kComputeThreads);
     mi->abort_flag = 0;
     mi->x = a.x; mi->y = a.y; mi->table = a.table; mi->rowoff = a.rowoff; mi->status = status;
     mi->sm = sm; mi->sbase = raw + pad;
@@ -1158,7 +1318,7 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
     mi->n = a.n; mi->tau = g.tau; mi->heads = g.heads; mi->mode = g.mode; mi->NF = g.NF; mi->n_f1 = g.n_f1;
     mi->ln1 = a.p.ln1_g != nullptr; mi->ln2 = a.p.ln2_g != nullptr;
     mi->eps = a.p.ln_eps;
-    mi->s_lo = mi->nsets = mi->base = mi->rows = 0;
+    mi->s_lo = mi->nsets = mi->base = mi->rows = mi->buf = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kMmaWarp) {
@@ -1175,13 +1335,14 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   {  // biases and LayerNorm vectors -> shared memory (absent vectors read as zeros)
     float* par = reinterpret_cast<float*>(sm + g.off_par);
     const dsvt_layer_params& p = a.p;
-    const float* src[9] = {p.b_qkv, p.b_qkv ? p.b_qkv + C : nullptr, p.b_qkv ? p.b_qkv + 2 * C : nullptr, p.b_o, p.b_2,
-                           p.ln1_g, p.ln1_b, p.ln2_g, p.ln2_b};
-    for (int i = tid; i < 9 * C; i += kThreads) {
-      const float* v = src[i / C];
+    // order of ParOff: b_q, b_v, b_o, b_2, ln1_g, ln1_b, ln2_g, ln2_b, then b_1 (the key bias is not needed)
+    for (int i = tid; i < ParOff<C>::vectors * C; i += kThreads) {
+      const int which = i / C;
+      const float* v = which == 0 ? p.b_qkv : which == 1 ? (p.b_qkv ? p.b_qkv + 2 * C : nullptr) : which == 2 ? p.b_o
+                     : which == 3 ? p.b_2 : which == 4 ? p.ln1_g : which == 5 ? p.ln1_b : which == 6 ? p.ln2_g : p.ln2_b;
       par[i] = v ? __ldg(v + i % C) : 0.f;
     }
-    for (int i = tid; i < g.hidden; i += kThreads) par[9 * C + i] = p.b_1 ? __ldg(p.b_1 + i) : 0.f;
+    for (int i = tid; i < g.hidden; i += kThreads) par[ParOff<C>::b_1 + i] = p.b_1 ? __ldg(p.b_1 + i) : 0.f;
   }
   tc_fence_before();
   __syncthreads();
@@ -1199,6 +1360,8 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   } else if (warp == kMmaWarp) {
     if ((tid & 31) == 0) mma_role<C>(a, g, rc);
     __syncwarp();
+  } else if (warp >= kLoadWarp0) {
+    loader_role<C>();
   } else {
     compute_role<C, D, NT, BLOCKED>();
   }
@@ -1294,7 +1457,7 @@ int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a) {
   g.off_kv = a_bytes;
   g.off_stage = g.off_kv + (uint32_t)kTM * 2 * C * 2;  // K + V (bf16) = fp32 staging = MLP hidden (<= 2C) bytes
   g.off_par = g.off_stage + kStages * (uint32_t)C * 128u;
-  const size_t smem = (size_t)g.off_par + (size_t)(9 * C + g.hidden) * sizeof(float) + 1024;
+  const size_t smem = (size_t)g.off_par + (size_t)(8 * C + g.hidden) * sizeof(float) + 1024;
   if (smem + sizeof(Misc) + 16 > 227 * 1024) return DSVT_ERR_UNSUPPORTED;  // s_mi is static shared memory
   TcMaps maps;
   bool okm = make_weight_map(&maps.qkv, p.W_qkv, 3 * C, C, C) && make_weight_map(&maps.o, p.W_o, C, C, C);
