@@ -37,6 +37,11 @@ def _peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one fused-layer launch at configuration 2, from the ncu capture
+# summarised in profiles/layer_tc_kernel_config2.md (25.69 MB read + 0.06 MB written: the output stays in L2).
+LAYER_DRAM_BYTES_PER_LAUNCH = 25.75e6
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -320,7 +325,8 @@ def run_ours(args):
         "roofline": {"kernel": "fused DSVT layer", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                      "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"], "peak_source": peaks["source"],
-                     "flops_per_launch": flops_per_launch, "ms_per_launch": layer_ms, "traffic": None},
+                     "flops_per_launch": flops_per_launch, "ms_per_launch": layer_ms,
+                     "traffic": LAYER_DRAM_BYTES_PER_LAUNCH if args.config == 2 else None},
         "cpu_baseline": cpu,
     }))
     if world > 1:
