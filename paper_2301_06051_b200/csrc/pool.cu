@@ -181,6 +181,340 @@ __global__ void __launch_bounds__(kThreads, 1) pool_attn_kernel(PoolArgs a) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Tensor-core version of the fused kernel for bfloat16 weights (mma.sync.m16n8k16, fp32 accumulation).
+// Tile = up to 128 padded slot rows = TR regions.  Shared memory: X (padded slots, bf16, the A operand
+// of the key / value projections), K, V (bf16), P (Eq. 6 maxima, bf16, later the attention output), a
+// two-stage ring of 64-column weight blocks.  All operand tiles use the 128-byte-swizzled K-major layout
+// (64 bf16 per 128-byte row, 8-row groups of 1024 bytes, chunk index XOR row & 7), which ldmatrix reads
+// without bank conflicts.  The fp32 queries and the fp32 output rows reuse X's space once X is dead.
+// ---------------------------------------------------------------------------------------------------
+namespace mma_pool {
+constexpr int kT = 512, kW = kT / 32;
+constexpr int kRows = 128;  // slot rows per tile
+constexpr int kRegs = 64;   // regions per tile at most
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// byte offset of 16-byte chunk c8 of `row` in a tile whose 64-column blocks hold rows_pb rows each
+__device__ __forceinline__ uint32_t swz(int row, int c8, int rows_pb) {
+  return (uint32_t)((c8 >> 3) * (rows_pb * 128) + (row >> 3) * 1024 + (row & 7) * 128 + (((c8 & 7) ^ (row & 7)) << 4));
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+__device__ __forceinline__ float bf16_at(const unsigned char* tile, int row, int col, int rows_pb) {
+  const unsigned short u = *reinterpret_cast<const unsigned short*>(tile + swz(row, col >> 3, rows_pb) + (col & 7) * 2);
+  return __uint_as_float((uint32_t)u << 16);
+}
+
+constexpr int kStages = 4;  // weight ring: 64-column blocks, prefetched three ahead
+constexpr int kMaxHeads = 8;
+
+struct Layout {  // byte offsets into dynamic shared memory (1024-aligned base)
+  uint32_t x, kv, p, w, probs, rowvox, total;
+};
+__host__ __device__ inline Layout make_layout(int C) {
+  Layout L;
+  L.x = 0;                                   // padded slot rows (bf16 A operand); at the end the fp32 output rows
+  L.kv = L.x + kRows * C * 2;                // keys, later values (bf16)
+  L.p = L.kv + kRows * C * 2;                // Eq. 6 maxima -> queries (in place) -> attention output (bf16)
+  L.w = L.p + kRegs * C * 2;
+  L.probs = L.w + kStages * (uint32_t)C * 128;
+  L.rowvox = L.probs + 2 * kRows * kMaxHeads * 4;  // (regions x padded slots) < 2 x 128 per head
+  L.total = L.rowvox + kRows * 4;
+  return L;
+}
+
+// The weight blocks of a CTA form one stream: tile after tile, W_q, W_k, W_v, W_o, each in C / 64 blocks of
+// 64 input columns.  Block g lives in stage g mod 4 and is requested three steps before it is used.
+struct WeightStream {
+  const __nv_bfloat16* W[4];
+  int C, nkb;
+  long long total;   // blocks this CTA will consume
+  long long next;    // next block to consume
+  uint32_t base, stage_bytes;
+
+  __device__ __forceinline__ void request(long long g) {
+    if (g < total) {
+      const int kb = (int)(g % nkb);
+      const __nv_bfloat16* w = W[(g / nkb) & 3];
+      const uint32_t stage = base + (uint32_t)(g % kStages) * stage_bytes;
+      for (int i = threadIdx.x; i < C * 8; i += kT) {
+        const int n = i >> 3, c = i & 7;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage + swz(n, c, 0)),
+                     "l"(w + (size_t)n * C + kb * 64 + c * 8) : "memory");
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");  // one group per step, empty or not
+  }
+  __device__ __forceinline__ void prologue() {
+    for (int g = 0; g < kStages - 1; ++g) request(g);
+  }
+  // Makes the next block usable by every thread and returns its stage; requests the block three ahead.
+  __device__ __forceinline__ uint32_t acquire() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(kStages - 2) : "memory");
+    __syncthreads();  // the block is visible to all; everyone is done with the block before it
+    request(next + kStages - 1);
+    const uint32_t stage = base + (uint32_t)(next % kStages) * stage_bytes;
+    ++next;
+    return stage;
+  }
+};
+
+// epi(row, col, v0, v1) receives out(row, col) and out(row, col + 1), out = A W^T + bias, for row < 16 mt_count.
+// A: swizzled bf16 tile with rows_pb rows per 64-column block; W: the stream's next C / 64 blocks.  Work
+// item = (16-row tile, 32 output columns); all A reads are complete before the first epi call.
+template <class Epi>
+__device__ __forceinline__ void gemm(uint32_t a_base, int rows_pb, int mt_count, WeightStream& ws, const float* bias,
+                                     Epi epi) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int C = ws.C, ng = C >> 5, items = mt_count * ng;
+  float acc[3][4][4];
+#pragma unroll
+  for (int ii = 0; ii < 3; ++ii) {
+    const int item = warp + kW * ii;
+    const int g = item < items ? item % ng : 0;
+#pragma unroll
+    for (int nb = 0; nb < 4; ++nb) {
+      const int col = g * 32 + nb * 8 + 2 * (lane & 3);
+      const float b0 = bias ? __ldg(bias + col) : 0.f, b1 = bias ? __ldg(bias + col + 1) : 0.f;
+      acc[ii][nb][0] = b0; acc[ii][nb][1] = b1; acc[ii][nb][2] = b0; acc[ii][nb][3] = b1;
+    }
+  }
+  for (int kb = 0; kb < ws.nkb; ++kb) {
+    const uint32_t wb = ws.acquire();
+#pragma unroll
+    for (int ii = 0; ii < 3; ++ii) {
+      const int item = warp + kW * ii;
+      if (item < items) {
+        const int mt = item / ng, g = item - mt * ng;
+        uint32_t af[4][4];
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          ldsm_x4(a_base + swz(16 * mt + (lane & 15), kb * 8 + ks * 2 + (lane >> 4), rows_pb), af[ks]);
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb) {
+          const int n0 = g * 32 + nb * 8;
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t bf[4];
+            ldsm_x4(wb + swz(n0 + (lane & 7), half * 4 + (lane >> 3), 0), bf);
+            mma_16816(acc[ii][nb], af[2 * half], bf[0], bf[1]);
+            mma_16816(acc[ii][nb], af[2 * half + 1], bf[2], bf[3]);
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();  // every warp has read its A fragments: the epilogue may overwrite A in place
+#pragma unroll
+  for (int ii = 0; ii < 3; ++ii) {
+    const int item = warp + kW * ii;
+    if (item < items) {
+      const int mt = item / ng, g = item - mt * ng;
+#pragma unroll
+      for (int nb = 0; nb < 4; ++nb) {
+        const int row = 16 * mt + (lane >> 2), col = g * 32 + nb * 8 + 2 * (lane & 3);
+        epi(row, col, acc[ii][nb][0], acc[ii][nb][1]);
+        epi(row + 8, col, acc[ii][nb][2], acc[ii][nb][3]);
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void unpack8(const uint4 u, float (&f)[8]) {
+  f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xFFFF0000u);
+  f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xFFFF0000u);
+  f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xFFFF0000u);
+  f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xFFFF0000u);
+}
+
+__global__ void __launch_bounds__(kT, 1) pool_attn_mma_kernel(PoolArgs a) {
+  extern __shared__ unsigned char pool_smem_raw[];
+  const uint32_t raw = smem_u32(pool_smem_raw);
+  unsigned char* sm = pool_smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+  const uint32_t sb = smem_u32(sm);
+  const int C = a.C, ns = a.nslots, TR = a.TR, heads = a.heads;
+  const Layout L = make_layout(C);
+  int* rowvox = reinterpret_cast<int*>(sm + L.rowvox);
+  float* probs = reinterpret_cast<float*>(sm + L.probs);  // [region][head][padded slot]
+  float* outf = reinterpret_cast<float*>(sm + L.x);       // fp32 output rows [kRegs][C], once X is dead
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int C4 = C >> 2, d = C / heads;
+  const float scale = 1.0f / sqrtf((float)d);
+  const int m = min(*a.num_out, a.cap_m);
+  const int num_tiles = (m + TR - 1) / TR;
+  int nsp = 1;
+  while (nsp < ns) nsp <<= 1;
+  const int hpg = 32 / nsp;  // heads per pass of a warp
+
+  WeightStream ws;
+  ws.W[0] = reinterpret_cast<const __nv_bfloat16*>(a.W_q);
+  ws.W[1] = reinterpret_cast<const __nv_bfloat16*>(a.W_k);
+  ws.W[2] = reinterpret_cast<const __nv_bfloat16*>(a.W_v);
+  ws.W[3] = reinterpret_cast<const __nv_bfloat16*>(a.W_o);
+  ws.C = C; ws.nkb = C >> 6;
+  const long long my_tiles = blockIdx.x < num_tiles ? (num_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+  ws.total = my_tiles * 4 * ws.nkb;
+  ws.next = 0;
+  ws.base = sb + L.w;
+  ws.stage_bytes = (uint32_t)C * 128;
+  ws.prologue();
+
+  for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+    __syncthreads();
+    const int r_lo = t * TR, nr = min(TR, m - r_lo), rows = nr * ns;
+    const int mt_rows = (rows + 15) >> 4, mt_reg = (nr + 15) >> 4;
+    for (int r = tid; r < kRows; r += kT) {
+      int v = -1;
+      if (r < rows) {
+        const int ri = r / ns;
+        v = a.cell_map[(size_t)a.region_key[r_lo + ri] * ns + (r - ri * ns)];
+      }
+      rowvox[r] = v;
+    }
+    __syncthreads();
+    // padded slot rows (+ slot term) -> X as bf16; Eq. 6 maxima -> P as bf16.  One warp per region, the loads
+    // of four slots in flight together.
+    for (int ri = warp; ri < (mt_reg << 4); ri += kW) {
+      for (int c4 = lane; c4 < C4; c4 += 32) {
+        float4 mx = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ri < nr) {
+          mx = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+          for (int s0 = 0; s0 < ns; s0 += 4) {
+            float4 f[4];
+            int vv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              vv[u] = s0 + u < ns ? rowvox[ri * ns + s0 + u] : -1;
+              f[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (vv[u] >= 0) f[u] = __ldg(reinterpret_cast<const float4*>(a.feats + (size_t)vv[u] * C) + c4);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              if (s0 + u < ns) {
+                const int s = s0 + u, r = ri * ns + s;
+                if (!a.mask_empty || vv[u] >= 0) {
+                  mx.x = fmaxf(mx.x, f[u].x); mx.y = fmaxf(mx.y, f[u].y); mx.z = fmaxf(mx.z, f[u].z); mx.w = fmaxf(mx.w, f[u].w);
+                }
+                if (a.slot_pe) {
+                  const float4 e = __ldg(reinterpret_cast<const float4*>(a.slot_pe + (size_t)s * C) + c4);
+                  f[u].x += e.x; f[u].y += e.y; f[u].z += e.z; f[u].w += e.w;
+                }
+                *reinterpret_cast<uint2*>(sm + L.x + swz(r, c4 >> 1, kRows) + (c4 & 1) * 8) =
+                    make_uint2(pack_bf16(f[u].x, f[u].y), pack_bf16(f[u].z, f[u].w));
+              }
+            }
+          }
+        }
+        *reinterpret_cast<uint2*>(sm + L.p + swz(ri, c4 >> 1, kRegs) + (c4 & 1) * 8) =
+            make_uint2(pack_bf16(mx.x, mx.y), pack_bf16(mx.z, mx.w));
+      }
+    }
+    // rows between the last slot row and the end of its 16-row tile: zeros
+    for (int idx = tid; idx < ((mt_rows << 4) - rows) * (C >> 3); idx += kT) {
+      const int r = rows + idx / (C >> 3), c8 = idx % (C >> 3);
+      *reinterpret_cast<uint4*>(sm + L.x + swz(r, c8, kRows)) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    __syncthreads();
+    // Eq. 7.  Queries from P, in place (bf16); keys from the padded slots.
+    gemm(sb + L.p, kRegs, mt_reg, ws, a.b_q, [&](int row, int col, float v0, float v1) {
+      *reinterpret_cast<uint32_t*>(sm + L.p + swz(row, col >> 3, kRegs) + (col & 7) * 2) = pack_bf16(v0, v1);
+    });
+    gemm(sb + L.x, kRows, mt_rows, ws, a.b_k, [&](int row, int col, float v0, float v1) {
+      *reinterpret_cast<uint32_t*>(sm + L.kv + swz(row, col >> 3, kRows) + (col & 7) * 2) = pack_bf16(v0, v1);
+    });
+    __syncthreads();
+    // scores and softmax: one warp per region, lane = (head of the current group, slot)
+    for (int ri = warp; ri < nr; ri += kW) {
+      const int s = lane & (nsp - 1), hh = lane / nsp;
+      for (int h0 = 0; h0 < heads; h0 += hpg) {
+        const int h = h0 + hh;
+        const bool use = h < heads && s < ns && (!a.mask_empty || rowvox[ri * ns + s] >= 0);
+        float lg = -INFINITY;
+        if (use) {
+          float acc = 0.f;
+          if ((d & 7) == 0) {
+            for (int j = 0; j < (d >> 3); ++j) {
+              float q[8], k[8];
+              unpack8(*reinterpret_cast<const uint4*>(sm + L.p + swz(ri, ((h * d) >> 3) + j, kRegs)), q);
+              unpack8(*reinterpret_cast<const uint4*>(sm + L.kv + swz(ri * ns + s, ((h * d) >> 3) + j, kRows)), k);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) acc = fmaf(q[e], k[e], acc);
+            }
+          } else {
+            for (int c = 0; c < d; ++c)
+              acc = fmaf(bf16_at(sm + L.p, ri, h * d + c, kRegs), bf16_at(sm + L.kv, ri * ns + s, h * d + c, kRows), acc);
+          }
+          lg = acc * scale;
+        }
+        float mx = lg;
+        for (int o = nsp >> 1; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float e = use ? expf(lg - mx) : 0.f;
+        float sum = e;
+        for (int o = nsp >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (h < heads) probs[(ri * heads + h) * nsp + s] = sum > 0.f ? e / sum : 0.f;
+      }
+    }
+    // values into the keys' space
+    gemm(sb + L.x, kRows, mt_rows, ws, a.b_v, [&](int row, int col, float v0, float v1) {
+      *reinterpret_cast<uint32_t*>(sm + L.kv + swz(row, col >> 3, kRows) + (col & 7) * 2) = pack_bf16(v0, v1);
+    });
+    __syncthreads();
+    // attention output (bf16) over the queries: one thread per (region, 8-channel chunk) (or per channel)
+    if ((d & 7) == 0) {
+      const int cpr = C >> 3;
+      for (int idx = tid; idx < (mt_reg << 4) * cpr; idx += kT) {
+        const int ri = idx / cpr, c8 = idx - ri * cpr;
+        float o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (ri < nr) {
+          const int h = (c8 << 3) / d;
+          const float* pr = probs + (ri * heads + h) * nsp;
+          for (int s2 = 0; s2 < ns; ++s2) {
+            float v[8];
+            unpack8(*reinterpret_cast<const uint4*>(sm + L.kv + swz(ri * ns + s2, c8, kRows)), v);
+            const float ps = pr[s2];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o[e] = fmaf(ps, v[e], o[e]);
+          }
+        }
+        *reinterpret_cast<uint4*>(sm + L.p + swz(ri, c8, kRegs)) =
+            make_uint4(pack_bf16(o[0], o[1]), pack_bf16(o[2], o[3]), pack_bf16(o[4], o[5]), pack_bf16(o[6], o[7]));
+      }
+    } else {
+      for (int idx = tid; idx < (mt_reg << 4) * C; idx += kT) {
+        const int ri = idx / C, c = idx - ri * C;
+        float o = 0.f;
+        if (ri < nr) {
+          const float* pr = probs + (ri * heads + c / d) * nsp;
+          for (int s2 = 0; s2 < ns; ++s2) o = fmaf(pr[s2], bf16_at(sm + L.kv, ri * ns + s2, c, kRows), o);
+        }
+        *reinterpret_cast<__nv_bfloat16*>(sm + L.p + swz(ri, c >> 3, kRegs) + (c & 7) * 2) = __float2bfloat16_rn(o);
+      }
+    }
+    __syncthreads();
+    gemm(sb + L.p, kRegs, mt_reg, ws, a.b_o, [&](int row, int col, float v0, float v1) {
+      *reinterpret_cast<float2*>(outf + (size_t)row * C + col) = make_float2(v0, v1);  // X is dead
+    });
+    __syncthreads();
+    for (int r = warp; r < nr; r += kW)
+      for (int c4 = lane; c4 < C4; c4 += 32)
+        reinterpret_cast<float4*>(a.out_feats + (size_t)(r_lo + r) * C)[c4] = *reinterpret_cast<const float4*>(outf + (size_t)r * C + 4 * c4);
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+}  // namespace mma_pool
+
 size_t pool_smem_bytes(int TM, int C, int LDQ) {
   return ((size_t)TM * C + (size_t)TM * LDQ + kKC * kNC) * 4 + (size_t)TM * 4 + 16;
 }
@@ -270,6 +604,22 @@ extern "C" int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feat
   a.W_q = W_q; a.W_k = W_k; a.W_v = W_v; a.W_o = W_o;
   a.b_q = b_q; a.b_k = b_k; a.b_v = b_v; a.b_o = b_o; a.slot_pe = slot_pe;
   a.out_feats = out_feats; a.C = C; a.heads = heads; a.nslots = (int32_t)nslots; a.mask_empty = mask_empty ? 1 : 0;
+  // bfloat16 weights, C in {64, 128, 192}, head dim <= 32: the tensor-core kernel
+  if (precision == DSVT_BF16_FP32ACC && (C == 64 || C == 128 || C == 192) && heads <= mma_pool::kMaxHeads) {
+    a.TM = mma_pool::kRows;
+    a.LDQ = 0;
+    a.TR = (int32_t)(mma_pool::kRows / nslots);
+    if (a.TR > mma_pool::kRegs) a.TR = mma_pool::kRegs;
+    const size_t smem = (size_t)mma_pool::make_layout(C).total + 1024;
+    int64_t tiles = dsvt_ceil_div(n < cap_m ? n : cap_m, a.TR);
+    int64_t gridn = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+    if (gridn < 1) gridn = 1;
+    cudaError_t e = cudaFuncSetAttribute(mma_pool::pool_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
+    mma_pool::pool_attn_mma_kernel<<<(unsigned)gridn, mma_pool::kT, smem, st>>>(a);
+    DSVT_LAUNCHED(ctx);
+    return DSVT_OK;
+  }
   a.LDQ = 3 * C + (36 - (3 * C) % 32) % 32;
   static const int kTiles[] = {128, 96, 64, 48, 32};
   a.TM = 0;

@@ -1,0 +1,90 @@
+"""Per-configuration device timings of the path: partition (both axes), blocks, pooling, whole backbone.
+
+    python -m paper_2301_06051_b200.timings [--configs 1 2 3 4 5] [--steps 20]
+
+One JSON line per configuration.  Times are CUDA-event medians over `steps` passes on synthetic frames that are
+resident in HBM; a 256 MiB write flushes L2 before every pass.  bench.py measures the headline configuration under
+its full contract; this tool is the per-configuration table.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+import torch
+
+import dsvt_inputs as di
+from . import api, pipeline
+
+
+def time_config(cid: int, steps: int, device: int = 0):
+    cfg = di.make_config(cid)
+    dev = torch.device("cuda", device)
+    bb = pipeline.Backbone(cfg, device=device)
+    coords = torch.from_numpy(cfg["coords"]).to(dev)
+    x = torch.from_numpy(cfg["feats"]).to(dev)
+    y = torch.empty_like(x)
+    flush = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    rec = []
+
+    def mark(tag):
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        rec[-1].append((tag, e))
+
+    def run_stage(stage, c, src, dst, tag):
+        stage.partition(c)
+        mark(tag + "partition")
+        for blk in stage.blocks:
+            bb.ctx.block(src, stage.tables[0], stage.tables[1], blk, dst)
+            src = dst
+        mark(tag + "blocks")
+
+    m = cfg["n"]
+    for it in range(3 + steps):
+        flush.zero_()
+        rec.append([])
+        mark("start")
+        run_stage(bb.stage1, coords, x, y, "s1_")
+        if bb.stage2:
+            oc, of, num, _, _ = bb.ctx.pool(coords, y, cfg["batch"], cfg["grid"], bb.pool_shape, bb.pool_w)
+            mark("pool")
+            m = int(num.item())  # the pooled voxel count sizes the second stage's tensors
+            mark("readback")
+            run_stage(bb.stage2, oc[:m], of[:m], of[:m], "s2_")
+    torch.cuda.synchronize(dev)
+    if bb.ctx.status_sync() != 0:
+        raise SystemExit("device status word is not clean")
+    spans = {}
+    for r in rec[3:]:
+        for (t0, e0), (t1, e1) in zip(r[:-1], r[1:]):
+            spans.setdefault(t1, []).append(e0.elapsed_time(e1))
+        spans.setdefault("backbone", []).append(r[0][1].elapsed_time(r[-1][1]))
+    med = {k: float(np.median(v)) for k, v in spans.items()}
+    nb1 = len(bb.stage1.blocks)
+    out = {"config": cid, "name": cfg["name"], "voxels": cfg["n"], "precision": cfg["precision"],
+           "sets": int(bb.stage1.tables[0].num_sets.item()),
+           "t_partition_ms": med["s1_partition"], "t_block_ms": med["s1_blocks"] / nb1,
+           "voxels_per_s_per_block": cfg["n"] / (med["s1_blocks"] / nb1 * 1e-3),
+           "t_backbone_ms": med["backbone"], "frames_per_s": cfg["batch"] / (med["backbone"] * 1e-3)}
+    if bb.stage2:
+        nb2 = len(bb.stage2.blocks)
+        out.update({"t_pool_ms": med["pool"], "pooled_voxels": m, "t_partition2_ms": med["s2_partition"],
+                    "t_block2_ms": med["s2_blocks"] / nb2})
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser(description=__doc__)
+    ap.add_argument("--configs", type=int, nargs="+", default=list(di.CONFIG_IDS))
+    ap.add_argument("--steps", type=int, default=20)
+    args = ap.parse_args()
+    api.load()
+    for cid in args.configs:
+        print(json.dumps(time_config(cid, args.steps)), flush=True)
+
+
+if __name__ == "__main__":
+    main()

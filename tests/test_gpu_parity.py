@@ -324,6 +324,9 @@ def test_in_place_and_repeatability(gpu):
     ((40, 40, 1), (3, 3, 1), 1, 900, 64, 8, True, False),
     ((100, 100, 1), (2, 2, 1), 1, 4000, 192, 8, False, True),
     ((20, 20, 16), (2, 2, 4), 1, 3000, 192, 8, True, True),
+    ((60, 60, 1), (2, 2, 1), 2, 5000, 128, 8, True, True),     # several tiles per CTA, ragged last tile
+    ((30, 30, 4), (3, 3, 2), 1, 2500, 64, 4, False, True),      # 18 slots per region
+    ((50, 50, 1), (2, 1, 1), 1, 2000, 128, 4, False, True),     # 2 slots: 64 regions per tile
 ])
 def test_pool_matches_oracle(gpu, oracle, grid, pool, batch, n, C, heads, with_pe, bf16, mask_empty):
     rng = np.random.default_rng(n + C)
