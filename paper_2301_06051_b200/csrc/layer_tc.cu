@@ -2,20 +2,23 @@
 // accumulation: gather (Eq. 4) -> QKV projection -> per-set multi-head attention (Eq. 5) -> output
 // projection -> residual + LayerNorm -> MLP with GELU -> residual + LayerNorm -> scatter (App. B.1.1).
 //
-// One persistent CTA per SM.  The distinct voxel rows of the frame are cut into one contiguous
-// segment per CTA (equal row counts, cut at set boundaries); inside its segment a CTA packs whole
-// sets greedily into tiles of at most 128 rows (the UMMA M).
+// One persistent CTA per SM.  Whole sets are packed greedily into tiles of at most 128 distinct rows (the
+// UMMA M); the tile plan comes from the partition (tile t goes to CTA t mod gridDim.x), or, without a
+// plan, each CTA cuts its own contiguous row segment into tiles.
 //
-// Roles: warps 0-7 compute (gather, TMEM epilogues, attention); warp 8 is the scheduler and TMA
-// producer: it finds the next tile (binary searches in the row-offset array), publishes it through a
-// two-entry ring, and streams the layer's weight matrices through a shared-memory ring with TMA (no
-// cluster multicast); warp 9 allocates TMEM and issues the tcgen05.mma instructions.
+// Roles (640 threads): warps 0-15 compute (gather, TMEM epilogues, attention); warp 16 is the scheduler
+// and TMA producer: it publishes tiles through a two-entry ring, two ahead, and streams the layer's
+// weight matrices through a three-stage shared-memory ring with plain (single-CTA) TMA loads; warp 17
+// allocates TMEM and issues the tcgen05.mma instructions; warps 18-19 build the next tile's row list
+// while the current tile is computed.  The compute warps gather the next tile's rows as soon as the
+// current tile's MMAs have stopped reading the A operand, so that its first projections overlap the
+// current tile's tail.
 //
-// The four projections of a layer are chunks of at most 192 output columns (K, V, Q, O, MLP-1 in
-// pieces of 128 or 64 hidden columns, MLP-2).  Accumulators alternate between two TMEM buffers so the
-// tensor pipe works on one chunk while the compute warps drain the previous one.  The fp32 residual
-// stream never leaves the chip inside a layer: x is staged in shared memory for the first residual,
-// and x1 = LN1(x + attention) is parked in spare TMEM columns until the second residual.
+// The projections of a layer are chunks of at most 192 output columns (K, V, Q, O, MLP-1 in pieces of
+// 128 or 64 hidden columns, MLP-2), accumulated in three TMEM regions (map at compute_role) so the
+// tensor pipe works on one chunk while the compute warps drain another.  The fp32 residual stream never
+// leaves the chip inside a layer: x is staged in shared memory for the first residual, and
+// x1 + b_2 = LN1(x + attention) + b_2 is parked in TMEM, where MLP-2 accumulates on top of it.
 //
 // Every operand tile in shared memory uses the K-major 128-byte-swizzled layout that tcgen05.mma and
 // TMA share: 64 bf16 columns per 128-byte row, 8-row groups of 1024 bytes, 16-byte chunk index XORed
@@ -162,51 +165,6 @@ __device__ __forceinline__ void umma_commit(unsigned long long* bar) {
 }
 
 // 32 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
-        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
-        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
-        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
-        "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
-      : "memory");
-}
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // 16 fp32 columns of this thread's TMEM lane into / from elements [OFF, OFF + 16) of a register array
 // (compile-time offsets keep the array in registers).
@@ -244,24 +202,6 @@ __device__ __forceinline__ void tmem_st_row(uint32_t taddr, const float (&v)[N])
   if constexpr (N > 32) tmem_st16_at<32>(taddr + 32, v);
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
-        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
-        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
-        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
-        "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])),
-        "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
-        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])),
-        "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])),
-        "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])),
-        "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
-      : "memory");
-  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-}
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -613,7 +553,6 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
   constexpr uint32_t COL_B = C;      // second accumulator buffer
   constexpr uint32_t STAGE_BYTES = C * 128;
-  unsigned char* sm = rc.sm;
   const uint32_t sbase = rc.sbase, tmem = rc.tmem;
   Misc* mi = &s_mi;
   const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
@@ -725,7 +664,6 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
   constexpr uint32_t COL_B = C;      // second accumulator buffer
   constexpr uint32_t STAGE_BYTES = C * 128;
-  unsigned char* sm = rc.sm;
   const uint32_t sbase = rc.sbase, tmem = rc.tmem;
   Misc* mi = &s_mi;
   const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
