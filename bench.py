@@ -136,6 +136,12 @@ def job_throughput(world: int, units_per_rank: float, ms_per_step: float) -> flo
     return world * units_per_rank / (ms_per_step * 1e-3)
 
 
+def workload_name(cid: int, cfg) -> str:
+    """The `config.workload` string: the same for both arms."""
+    return "config %d (%s): %d voxels, grid %s, window %s, set size %d, C=%d, %d blocks x 2 layers" % (
+        cid, cfg["name"], cfg["n"], cfg["grid"], cfg["window"], cfg["set_size"], cfg["C"], len(cfg["blocks"]))
+
+
 def run_reference(args):
     """The CPU oracle as it stands, on a bounded sample of the same workload (rank 0 only)."""
     rank, _, world = _dist_env()
@@ -175,7 +181,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "voxels/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "config %d (%s), CPU oracle on a bounded sample" % (args.config, cfg["name"])},
+        "config": {"workload": workload_name(args.config, cfg), "sample": sample},
         "cpu_baseline": {"value": value, "unit": "voxels/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "voxels/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -311,8 +317,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": "voxels/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if cfg["precision"] == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": "config %d (%s): %d voxels, grid %s, window %s, set size %d, C=%d, %d blocks x 2 layers"
-                   % (args.config, cfg["name"], n, cfg["grid"], cfg["window"], cfg["set_size"], C, nb),
+        "config": {"workload": workload_name(args.config, cfg),
                    "l2": "L2 flushed by a %d MiB write before every step" % (L2_FLUSH_BYTES >> 20),
                    "num_sets": S, "pad_ratio": pad, "frames_per_rank": 1},
         "frames_per_sec": world / (ms_per_step * 1e-3),
