@@ -539,8 +539,34 @@ struct RoleCtx {
   unsigned char* sm;  // 1024-aligned shared-memory base (generic address) and its shared-space address
   uint32_t sbase;
   uint32_t tmem;      // TMEM base address of the CTA's allocation
-  int S, R;           // number of sets, number of distinct rows
+  // read by the scheduler thread while the other threads set up shared memory (see prefetch_first_tile)
+  int S;              // number of sets
+  int n_plan;         // tiles in the plan (< 0: no plan)
+  int pre_ok;         // the CTA's first plan tile below is valid
+  int pre_s, pre_ns, pre_base, pre_rows;
 };
+
+// The scheduler thread's first global reads (set count, plan header, the CTA's first tile and its row range)
+// are issued at kernel entry, so that their two round trips overlap the shared-memory set-up.
+__device__ __forceinline__ void prefetch_first_tile(const dsvt_fused_args& a, RoleCtx& rc) {
+  const int32_t* plan = a.rowoff + a.cap_sets + 1;
+  const int n_plan = plan[0];
+  const int S = min(*a.num_sets, a.cap_sets);
+  // in bounds for every block index: the grid has at most cap_sets CTAs and the plan cap_sets + 2 entries
+  const int f = plan[1 + blockIdx.x], l = plan[2 + blockIdx.x];
+  rc.n_plan = n_plan;
+  rc.S = S;
+  rc.pre_ok = 0;
+  rc.pre_s = rc.pre_ns = rc.pre_base = rc.pre_rows = 0;
+  if (n_plan >= 0 && (int)blockIdx.x < n_plan && f >= 0 && l > f && l <= S && l - f <= kTM) {
+    const int base = a.rowoff[f], rows = a.rowoff[l] - base;
+    if (rows > 0 && rows <= kTM) {
+      rc.pre_ok = 1;
+      rc.pre_s = f; rc.pre_ns = l - f; rc.pre_base = base; rc.pre_rows = rows;
+    }
+  }
+}
+
 
 // The scheduler and the MMA issuer are separate (not inlined) functions so that their polling loops get
 // their own, spill-free register allocation; the compute role is inlined into the kernel, where the
@@ -558,20 +584,21 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
   const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &mi->abort_flag;
-  const int S = rc.S, R = rc.R;
+  const int S = rc.S;
   const bool mlp = g.mode == 2;
   const int n_chunks = 4 + (mlp ? g.n_f1 + 1 : 0);
-  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp; (void)R;
+  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp;
   (void)tmem; (void)S; (void)n_chunks; (void)tid;
     if (lane == 0) {
       // Tiles come from the plan behind the row offsets (greedy packing of the whole frame, tile t goes to
       // CTA t mod G); without a plan each CTA packs its own segment, the sets whose first row lies in
       // [b R / G, (b + 1) R / G).
       const int32_t* plan = a.rowoff + a.cap_sets + 1;
-      const int n_plan = plan[0];
+      const int n_plan = rc.n_plan;
       int t_next = blockIdx.x;
       int s = 0, s_end = 0;
       if (n_plan < 0) {
+        const int R = S > 0 ? a.rowoff[S] : 0;
         const int row_lo = (int)(((long long)blockIdx.x * R) / gridDim.x);
         const int row_hi = (int)(((long long)(blockIdx.x + 1) * R) / gridDim.x);
         int lo = 0, hi = S;
@@ -616,7 +643,12 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
       int stage = 0, slot = 0;
       uint32_t phase = 0, sphase = 0;
       int ns, base, rows;
-      next_tile(s, ns, base, rows);
+      if (rc.pre_ok) {  // the first tile was looked up at kernel entry
+        s = rc.pre_s; ns = rc.pre_ns; base = rc.pre_base; rows = rc.pre_rows;
+        t_next += gridDim.x;
+      } else {
+        next_tile(s, ns, base, rows);
+      }
       // Tiles are published two ahead of the weights (the ring has two entries), so that the loader
       // warps can prepare tile k + 1 while tile k is being computed.
       int ahead = 0;          // published tiles whose weights have not been streamed yet
@@ -669,11 +701,10 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
   const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &mi->abort_flag;
-  const int S = rc.S, R = rc.R;
   const bool mlp = g.mode == 2;
   const int n_chunks = 4 + (mlp ? g.n_f1 + 1 : 0);
-  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp; (void)R;
-  (void)tmem; (void)S; (void)n_chunks; (void)tid;
+  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp;
+  (void)tmem; (void)n_chunks; (void)tid;
     if (lane == 0) {
       int stage = 0, slot = 0;
       uint32_t phase = 0, a_phase = 0, x_phase = 0, sphase = 0;
@@ -1242,6 +1273,9 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   unsigned char* sm = smem_raw + pad;
   Misc* mi = &s_mi;
   const int tid = threadIdx.x, warp = tid >> 5;
+  RoleCtx rc;
+  rc.S = rc.n_plan = rc.pre_ok = rc.pre_s = rc.pre_ns = rc.pre_base = rc.pre_rows = 0;
+  if (tid == 32 * kTmaWarp) prefetch_first_tile(a, rc);
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(&mi->full[i], 1); mbar_init(&mi->empty[i], 1); }
     for (int i = 0; i < 3; ++i) {
@@ -1293,12 +1327,9 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  RoleCtx rc;
   rc.sm = sm;
   rc.sbase = raw + pad;
   rc.tmem = mi->tmem_base;
-  rc.S = min(*a.num_sets, a.cap_sets);
-  rc.R = rc.S > 0 ? a.rowoff[rc.S] : 0;
 
   if (warp == kTmaWarp) {
     if ((tid & 31) == 0) producer_role<C>(a, g, maps, status, rc);
