@@ -29,6 +29,7 @@
 // Every wait on an mbarrier is bounded; a wait that gives up raises DSVT_STATUS_TIMEOUT and all roles
 // leave their loops.
 #include <cuda.h>
+#include <limits.h>
 
 #include <type_traits>
 
@@ -544,6 +545,10 @@ struct RoleCtx {
   int n_plan;         // tiles in the plan (< 0: no plan)
   int pre_ok;         // the CTA's first plan tile below is valid
   int pre_s, pre_ns, pre_base, pre_rows;
+  // copies of the kernel parameters the two single-thread roles use (registers instead of parameter-space loads)
+  const int32_t* rowoff;
+  int cap_sets, mode, n_f1, NF, nkb_h;
+  uint32_t off_a, off_kv, off_stage;
 };
 
 // The scheduler thread's first global reads (set count, plan header, the CTA's first tile and its row range)
@@ -581,31 +586,31 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
   constexpr uint32_t STAGE_BYTES = C * 128;
   const uint32_t sbase = rc.sbase, tmem = rc.tmem;
   Misc* mi = &s_mi;
-  const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
+  const uint32_t a_base = sbase + rc.off_a, kv_base = sbase + rc.off_kv, st_base = sbase + rc.off_stage;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &mi->abort_flag;
   const int S = rc.S;
-  const bool mlp = g.mode == 2;
-  const int n_chunks = 4 + (mlp ? g.n_f1 + 1 : 0);
+  const bool mlp = rc.mode == 2;
+  const int n_chunks = 4 + (mlp ? rc.n_f1 + 1 : 0);
   (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp;
   (void)tmem; (void)S; (void)n_chunks; (void)tid;
     if (lane == 0) {
       // Tiles come from the plan behind the row offsets (greedy packing of the whole frame, tile t goes to
       // CTA t mod G); without a plan each CTA packs its own segment, the sets whose first row lies in
       // [b R / G, (b + 1) R / G).
-      const int32_t* plan = a.rowoff + a.cap_sets + 1;
+      const int32_t* plan = rc.rowoff + rc.cap_sets + 1;
       const int n_plan = rc.n_plan;
       int t_next = blockIdx.x;
       int s = 0, s_end = 0;
       if (n_plan < 0) {
-        const int R = S > 0 ? a.rowoff[S] : 0;
+        const int R = S > 0 ? rc.rowoff[S] : 0;
         const int row_lo = (int)(((long long)blockIdx.x * R) / gridDim.x);
         const int row_hi = (int)(((long long)(blockIdx.x + 1) * R) / gridDim.x);
         int lo = 0, hi = S;
-        while (lo < hi) { const int m = (lo + hi) >> 1; if (a.rowoff[m] < row_lo) lo = m + 1; else hi = m; }
+        while (lo < hi) { const int m = (lo + hi) >> 1; if (rc.rowoff[m] < row_lo) lo = m + 1; else hi = m; }
         s = lo;
         hi = S;
-        while (lo < hi) { const int m = (lo + hi) >> 1; if (a.rowoff[m] < row_hi) lo = m + 1; else hi = m; }
+        while (lo < hi) { const int m = (lo + hi) >> 1; if (rc.rowoff[m] < row_hi) lo = m + 1; else hi = m; }
         s_end = lo;
       }
       // next tile: first set s0, ns sets (< 0: none left), first row, rows
@@ -616,8 +621,8 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
             const int f = plan[1 + t_next], l = plan[2 + t_next];
             t_next += gridDim.x;
             if (f < 0 || l <= f || l > S) { atomicOr(status, DSVT_STATUS_BAD_INDEX); continue; }
-            base = a.rowoff[f];
-            rows = a.rowoff[l] - base;
+            base = rc.rowoff[f];
+            rows = rc.rowoff[l] - base;
             if (rows <= 0 || rows > kTM || l - f > kTM) { atomicOr(status, DSVT_STATUS_BAD_INDEX); continue; }
             s0 = f;
             ns = l - f;
@@ -626,17 +631,17 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
           return;
         }
         while (s0 < s_end) {
-          base = a.rowoff[s0];
-          const int first = a.rowoff[s0 + 1] - base;
+          base = rc.rowoff[s0];
+          const int first = rc.rowoff[s0 + 1] - base;
           if (first <= 0 || first > kTM) {  // offsets that do not describe a set: skip it
             atomicOr(status, DSVT_STATUS_BAD_INDEX);
             ++s0;
             continue;
           }
           int l2 = s0 + 1, h2 = s_end;  // last e in (s0, s_end] with rowoff[e] - base <= 128
-          while (l2 < h2) { const int m = (l2 + h2 + 1) >> 1; if (a.rowoff[m] - base <= kTM) l2 = m; else h2 = m - 1; }
+          while (l2 < h2) { const int m = (l2 + h2 + 1) >> 1; if (rc.rowoff[m] - base <= kTM) l2 = m; else h2 = m - 1; }
           ns = l2 - s0;
-          rows = a.rowoff[l2] - base;
+          rows = rc.rowoff[l2] - base;
           return;
         }
       };
@@ -674,8 +679,8 @@ __device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeo
           uint32_t bytes = STAGE_BYTES;
           if (c < 3) { map = &maps.qkv; row0 = (c == 0 ? 1 : c == 1 ? 2 : 0) * C; nkb = NKB; }   // K, V, Q
           else if (c == 3) { map = &maps.o; row0 = 0; nkb = NKB; }
-          else if (c < 4 + g.n_f1) { map = &maps.w1; row0 = (c - 4) * g.NF; nkb = NKB; bytes = (uint32_t)g.NF * 128u; }
-          else { map = &maps.w2; row0 = 0; nkb = g.nkb_h; }
+          else if (c < 4 + rc.n_f1) { map = &maps.w1; row0 = (c - 4) * rc.NF; nkb = NKB; bytes = (uint32_t)rc.NF * 128u; }
+          else { map = &maps.w2; row0 = 0; nkb = rc.nkb_h; }
           for (int kb = 0; kb < nkb; ++kb) {
             if (!mbar_wait(&mi->empty[stage], phase ^ 1u, abort_flag)) goto producer_done;
             mbar_expect_tx(&mi->full[stage], bytes);
@@ -698,11 +703,11 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
   constexpr uint32_t STAGE_BYTES = C * 128;
   const uint32_t sbase = rc.sbase, tmem = rc.tmem;
   Misc* mi = &s_mi;
-  const uint32_t a_base = sbase + g.off_a, kv_base = sbase + g.off_kv, st_base = sbase + g.off_stage;
+  const uint32_t a_base = sbase + rc.off_a, kv_base = sbase + rc.off_kv, st_base = sbase + rc.off_stage;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &mi->abort_flag;
-  const bool mlp = g.mode == 2;
-  const int n_chunks = 4 + (mlp ? g.n_f1 + 1 : 0);
+  const bool mlp = rc.mode == 2;
+  const int n_chunks = 4 + (mlp ? rc.n_f1 + 1 : 0);
   (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp;
   (void)tmem; (void)n_chunks; (void)tid;
     if (lane == 0) {
@@ -720,7 +725,7 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
           if (c == 0) {
             if (!mbar_wait(&mi->x_ready, x_phase, abort_flag)) goto mma_done;
             x_phase ^= 1u;
-          } else if (c == 3 || c == 4 || c == 4 + g.n_f1) {
+          } else if (c == 3 || c == 4 || c == 4 + rc.n_f1) {
             if (!mbar_wait(&mi->a_ready, a_phase, abort_flag)) goto mma_done;
             a_phase ^= 1u;
           }
@@ -728,7 +733,7 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
           // (on top of the parked x1 + b_2)
           uint32_t bar, col, n;
           if (c < 4) { bar = (c == 1) ? 1u : 0u; col = (c == 1) ? COL_B : 0u; n = C; }
-          else if (c < 4 + g.n_f1) { bar = (uint32_t)(c - 4) & 1u; col = bar * COL_B; n = (uint32_t)g.NF; }
+          else if (c < 4 + rc.n_f1) { bar = (uint32_t)(c - 4) & 1u; col = bar * COL_B; n = (uint32_t)rc.NF; }
           else { bar = 2u; col = kTmemCols - C; n = C; }
           if (c == 1) {
             // region 1 may overlap region 2: the previous tile's MLP-2 result must have been read
@@ -737,9 +742,9 @@ __device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g,
           if (bar != 2u && !mbar_wait(&mi->acc_free[bar], (uses[bar] & 1u) ^ 1u, abort_flag)) goto mma_done;
           ++uses[bar];
           tc_fence_after();
-          const bool last = mlp && c == 4 + g.n_f1;
+          const bool last = mlp && c == 4 + rc.n_f1;
           const uint32_t abase = last ? kv_base : a_base;
-          const int nkb = last ? g.nkb_h : NKB;
+          const int nkb = last ? rc.nkb_h : NKB;
           const uint32_t idesc = umma_idesc((int)n);
           const uint32_t d_tmem = tmem + col;
           for (int kb = 0; kb < nkb; ++kb) {
@@ -1276,6 +1281,29 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   RoleCtx rc;
   rc.S = rc.n_plan = rc.pre_ok = rc.pre_s = rc.pre_ns = rc.pre_base = rc.pre_rows = 0;
   if (tid == 32 * kTmaWarp) prefetch_first_tile(a, rc);
+  // (the scheduler warp takes no part in the set-up loops: its first thread is busy with the plan look-ups)
+  const bool setup = warp != kTmaWarp;
+  const int stid = warp > kTmaWarp ? tid - 32 : tid;  // dense index of the threads that take part
+  constexpr int kSetupThreads = kThreads - 32;
+  // biases and LayerNorm vectors (absent vectors read as zeros): the loads are issued first, the values go to
+  // shared memory at the end of the set-up.  Order of ParOff: b_q, b_v, b_o, b_2, ln1_g, ln1_b, ln2_g, ln2_b,
+  // then b_1 (the key bias is not needed).
+  constexpr int kParSlots = (ParOff<C>::vectors * C + 2 * C + kSetupThreads - 1) / kSetupThreads;
+  const int n_par = ParOff<C>::vectors * C + g.hidden;
+  float pv[kParSlots];
+#pragma unroll
+  for (int j = 0; j < kParSlots; ++j) {
+    const int i = stid + j * kSetupThreads;
+    pv[j] = 0.f;
+    if (setup && i < n_par) {
+      const dsvt_layer_params& p = a.p;
+      const int which = i / C;
+      const float* v = which == 0 ? p.b_qkv : which == 1 ? (p.b_qkv ? p.b_qkv + 2 * C : nullptr) : which == 2 ? p.b_o
+                     : which == 3 ? p.b_2 : which == 4 ? p.ln1_g : which == 5 ? p.ln1_b : which == 6 ? p.ln2_g
+                     : which == 7 ? p.ln2_b : (p.b_1 ? p.b_1 - ParOff<C>::b_1 + which * C : nullptr);
+      if (v) pv[j] = __ldg(v + i % C);
+    }
+  }
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { mbar_init(&mi->full[i], 1); mbar_init(&mi->empty[i], 1); }
     for (int i = 0; i < 3; ++i) {
@@ -1309,20 +1337,17 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   // rows of K / V past the end of a tile are read (and masked) by the attention: never let them hold
   // uninitialised bit patterns
   // (the weight ring behind it as well: key blocks that run past row 127 read a little of it)
-  for (uint32_t i = tid; i < ((uint32_t)kTM * 2 * C * 2 + kStages * (uint32_t)C * 128u) / 16; i += kThreads)
-    reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
+  if (setup)
+    for (uint32_t i = stid; i < ((uint32_t)kTM * 2 * C * 2 + kStages * (uint32_t)C * 128u) / 16; i += kSetupThreads)
+      reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_proxy_async();  // the TMA writes that follow must not be overtaken by these generic stores
-  {  // biases and LayerNorm vectors -> shared memory (absent vectors read as zeros)
+  {
     float* par = reinterpret_cast<float*>(sm + g.off_par);
-    const dsvt_layer_params& p = a.p;
-    // order of ParOff: b_q, b_v, b_o, b_2, ln1_g, ln1_b, ln2_g, ln2_b, then b_1 (the key bias is not needed)
-    for (int i = tid; i < ParOff<C>::vectors * C; i += kThreads) {
-      const int which = i / C;
-      const float* v = which == 0 ? p.b_qkv : which == 1 ? (p.b_qkv ? p.b_qkv + 2 * C : nullptr) : which == 2 ? p.b_o
-                     : which == 3 ? p.b_2 : which == 4 ? p.ln1_g : which == 5 ? p.ln1_b : which == 6 ? p.ln2_g : p.ln2_b;
-      par[i] = v ? __ldg(v + i % C) : 0.f;
+#pragma unroll
+    for (int j = 0; j < kParSlots; ++j) {
+      const int i = stid + j * kSetupThreads;
+      if (setup && i < n_par) par[i] = pv[j];
     }
-    for (int i = tid; i < g.hidden; i += kThreads) par[ParOff<C>::b_1 + i] = p.b_1 ? __ldg(p.b_1 + i) : 0.f;
   }
   tc_fence_before();
   __syncthreads();
@@ -1330,6 +1355,9 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   rc.sm = sm;
   rc.sbase = raw + pad;
   rc.tmem = mi->tmem_base;
+  rc.rowoff = a.rowoff; rc.cap_sets = a.cap_sets;
+  rc.mode = g.mode; rc.n_f1 = g.n_f1; rc.NF = g.NF; rc.nkb_h = g.nkb_h;
+  rc.off_a = g.off_a; rc.off_kv = g.off_kv; rc.off_stage = g.off_stage;
 
   if (warp == kTmaWarp) {
     if ((tid & 31) == 0) producer_role<C>(a, g, maps, status, rc);
