@@ -82,6 +82,7 @@ struct Misc {  // small shared state beside the big regions
   float eps;
   // the tile the compute warps are working on, and which row-list buffer describes it
   int s_lo, nsets, base, rows, buf;
+  int pre0;  // the CTA's first tile was listed and gathered during the kernel's set-up
   int next_rows[2];  // rows of the tile listed in buffer b (< 0: there is no such tile), valid after rl_ready[b]
   // row lists, double buffered: the loader warps fill buffer (k + 1) & 1 while the compute warps work on tile k;
   // the compute warps gather tile k + 1 as soon as tile k's MMAs no longer read the A operand
@@ -1194,17 +1195,21 @@ __device__ __forceinline__ void compute_role() {
     mbar_arrive(&s_mi.sched_empty[slot]);
     if (++slot == 2) { slot = 0; sphase ^= 1u; }
     if (nsets < 0) break;
-    if (k == 0 && threadIdx.x < kTM) {
+    const bool listed = k != 0 || s_mi.pre0 != 0;  // (pre0 is not written after the kernel's set-up)
+    if (!listed && threadIdx.x < kTM) {
       s_mi.rowvox[0][threadIdx.x] = -1;
       s_mi.row_lo[0][threadIdx.x] = (unsigned char)threadIdx.x;
       s_mi.row_n[0][threadIdx.x] = 1;
     }
     compute_sync();  // the tile's fields are visible to the phase functions
-    if (k == 0) {  // nothing runs ahead of a CTA's first tile: all compute warps list and gather it
-      phase_row_list();
-      compute_sync();
-      phase_gather<C>(0, rows);
-      fence_proxy_async();
+    if (k == 0) {  // nothing runs ahead of a CTA's first tile: the compute warps list and gather it themselves,
+                   // as a rule already during the kernel's set-up
+      if (!listed) {
+        phase_row_list();
+        compute_sync();
+        phase_gather<C>(0, rows);
+        fence_proxy_async();
+      }
       mbar_arrive(&s_mi.x_ready);  // X is in place
     }
 
@@ -1304,7 +1309,18 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
       if (v) pv[j] = __ldg(v + i % C);
     }
   }
-  if (tid == 0) {
+  if (tid == 0) {  // launch constants for the phase functions
+    mi->abort_flag = 0;
+    mi->x = a.x; mi->y = a.y; mi->table = a.table; mi->rowoff = a.rowoff; mi->status = status;
+    mi->sm = sm; mi->sbase = raw + pad;
+    mi->off_a = g.off_a; mi->off_kv = g.off_kv; mi->off_par = g.off_par;
+    mi->n = a.n; mi->tau = g.tau; mi->heads = g.heads; mi->mode = g.mode; mi->NF = g.NF; mi->n_f1 = g.n_f1;
+    mi->ln1 = a.p.ln1_g != nullptr; mi->ln2 = a.p.ln2_g != nullptr;
+    mi->eps = a.p.ln_eps;
+    mi->s_lo = mi->nsets = mi->base = mi->rows = mi->buf = mi->pre0 = 0;
+    mi->next_rows[0] = mi->next_rows[1] = -1;
+  }
+  if (tid == 32 * kLoadWarp0) {  // barriers
     for (int i = 0; i < kStages; ++i) { mbar_init(&mi->full[i], 1); mbar_init(&mi->empty[i], 1); }
     for (int i = 0; i < 3; ++i) {
       mbar_init(&mi->acc_full[i], 1);
@@ -1315,24 +1331,44 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
       mbar_init(&mi->sched_empty[i], kComputeThreads + 1 + kLoadWarps);  // compute threads, MMA issuer, loader warps
       mbar_init(&mi->rl_free[i], 1);
       mbar_init(&mi->rl_ready[i], kLoadThreads);
-      mi->next_rows[i] = -1;
     }
     mbar_init(&mi->a_ready, kComputeThreads);
     mbar_init(&mi->x_ready, kComputeThreads);
-    mi->abort_flag = 0;
-    mi->x = a.x; mi->y = a.y; mi->table = a.table; mi->rowoff = a.rowoff; mi->status = status;
-    mi->sm = sm; mi->sbase = raw + pad;
-    mi->off_a = g.off_a; mi->off_kv = g.off_kv; mi->off_par = g.off_par;
-    mi->n = a.n; mi->tau = g.tau; mi->heads = g.heads; mi->mode = g.mode; mi->NF = g.NF; mi->n_f1 = g.n_f1;
-    mi->ln1 = a.p.ln1_g != nullptr; mi->ln2 = a.p.ln2_g != nullptr;
-    mi->eps = a.p.ln_eps;
-    mi->s_lo = mi->nsets = mi->base = mi->rows = mi->buf = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&mi->tmem_base)),
                  "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // The compute warps look up the CTA's first tile themselves (the same plan entries the scheduler reads) and
+  // list and gather it right here, under the rest of the set-up; the A operand is not touched by the loops below.
+  if (warp < kComputeWarps) {
+    const int32_t* plan = a.rowoff + a.cap_sets + 1;
+    const int n_plan = plan[0];
+    const int S = min(*a.num_sets, a.cap_sets);
+    const int f = plan[1 + blockIdx.x], l = plan[2 + blockIdx.x];  // in bounds: see prefetch_first_tile
+    bool pre = n_plan >= 0 && (int)blockIdx.x < n_plan && f >= 0 && l > f && l <= S && l - f <= kTM;
+    int base = 0, rows = 0;
+    if (pre) {
+      base = a.rowoff[f];
+      rows = a.rowoff[l] - base;
+      pre = rows > 0 && rows <= kTM;
+    }
+    compute_sync();  // thread 0's constants are in place
+    if (pre) {
+      if (tid == 0) { mi->s_lo = f; mi->nsets = l - f; mi->base = base; mi->rows = rows; mi->buf = 0; mi->pre0 = 1; }
+      if (tid < kTM) {
+        mi->rowvox[0][tid] = -1;
+        mi->row_lo[0][tid] = (unsigned char)tid;
+        mi->row_n[0][tid] = 1;
+      }
+      compute_sync();
+      phase_row_list();
+      compute_sync();
+      phase_gather<C>(0, rows);
+      fence_proxy_async();
+    }
   }
   // rows of K / V past the end of a tile are read (and masked) by the attention: never let them hold
   // uninitialised bit patterns
