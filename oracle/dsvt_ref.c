@@ -104,14 +104,21 @@ static int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
  * win_count[num_windows], win_start[num_windows+1], win_setoff[num_windows+1]
  * over ALL windows (empty ones have count 0), num_windows = batch*nWx*nWy*nWz.
  */
-int dsvt_ref_partition(const int32_t* coords, int32_t n, int32_t batch, const int32_t* grid, const int32_t* window,
-                       int32_t set_size, int32_t axis, int32_t* set_table, int32_t cap_sets, int32_t* num_sets,
-                       int32_t* perm, int32_t* win_start, int32_t* win_count, int32_t* win_setoff) {
+/* Window partition displaced by `shift` cells (Sec. 3.2, "Hybrid window partition": the windows are re-cut
+ * between consecutive blocks with the window shifting of Swin, and with another window size).  A voxel at
+ * cell (x, y, z) lies in the window that holds cell (x + shift_x, y + shift_y, z + shift_z) of the unshifted
+ * cut; 0 <= shift < window per axis, so the first window of every axis is the partial one and there are
+ * ceil((grid + shift) / window) windows per axis.  Everything else is dsvt_ref_partition. */
+int dsvt_ref_partition_shifted(const int32_t* coords, int32_t n, int32_t batch, const int32_t* grid,
+                               const int32_t* window, const int32_t* shift, int32_t set_size, int32_t axis,
+                               int32_t* set_table, int32_t cap_sets, int32_t* num_sets, int32_t* perm,
+                               int32_t* win_start, int32_t* win_count, int32_t* win_setoff) {
   if (n < 0 || batch < 1 || set_size < 1 || (axis != 0 && axis != 1)) return REF_ERR_ARG;
   for (int a = 0; a < 3; ++a)
-    if (grid[a] < 1 || window[a] < 1) return REF_ERR_ARG;
+    if (grid[a] < 1 || window[a] < 1 || shift[a] < 0 || shift[a] >= window[a]) return REF_ERR_ARG;
   const int64_t L = window[0], W = window[1], H = window[2];
-  const int64_t nWx = ceil_div64(grid[0], L), nWy = ceil_div64(grid[1], W), nWz = ceil_div64(grid[2], H);
+  const int64_t nWx = ceil_div64((int64_t)grid[0] + shift[0], L), nWy = ceil_div64((int64_t)grid[1] + shift[1], W),
+                nWz = ceil_div64((int64_t)grid[2] + shift[2], H);
   const int64_t num_windows = (int64_t)batch * nWx * nWy * nWz;
 
   ref_key* keys = (ref_key*)malloc(sizeof(ref_key) * (size_t)(n > 0 ? n : 1));
@@ -124,8 +131,9 @@ int dsvt_ref_partition(const int32_t* coords, int32_t n, int32_t batch, const in
       free(keys); free(cnt);
       return REF_ERR_BAD_INPUT;
     }
-    const int64_t wx = x / L, wy = y / W, wz = z / H;
-    const int64_t xi = x - wx * L, yi = y - wy * W, zi = z - wz * H;
+    const int64_t xs = x + shift[0], ys = y + shift[1], zs = z + shift[2];
+    const int64_t wx = xs / L, wy = ys / W, wz = zs / H;
+    const int64_t xi = xs - wx * L, yi = ys - wy * W, zi = zs - wz * H;
     keys[i].win = ((b * nWx + wx) * nWy + wy) * nWz + wz;
     keys[i].inner = axis == 0 ? (xi * W + yi) * H + zi : (yi * L + xi) * H + zi;
     keys[i].idx = i;
@@ -163,6 +171,14 @@ int dsvt_ref_partition(const int32_t* coords, int32_t n, int32_t batch, const in
   free(keys);
   free(cnt);
   return rc;
+}
+
+int dsvt_ref_partition(const int32_t* coords, int32_t n, int32_t batch, const int32_t* grid, const int32_t* window,
+                       int32_t set_size, int32_t axis, int32_t* set_table, int32_t cap_sets, int32_t* num_sets,
+                       int32_t* perm, int32_t* win_start, int32_t* win_count, int32_t* win_setoff) {
+  const int32_t no_shift[3] = {0, 0, 0};
+  return dsvt_ref_partition_shifted(coords, n, batch, grid, window, no_shift, set_size, axis, set_table, cap_sets,
+                                    num_sets, perm, win_start, win_count, win_setoff);
 }
 
 /* ------------------------------------------------------------------ */

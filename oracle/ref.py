@@ -91,14 +91,16 @@ class Partition:
         return int(self.set_table.shape[0])
 
 
-def num_windows(batch, grid, window) -> int:
-    return int(batch) * int(np.prod([-(-int(g) // int(w)) for g, w in zip(grid, window)]))
+def num_windows(batch, grid, window, shift=(0, 0, 0)) -> int:
+    return int(batch) * int(np.prod([-(-(int(g) + int(s)) // int(w)) for g, w, s in zip(grid, window, shift)]))
 
 
-def partition(coords, batch, grid, window, set_size, axis, cap_sets: Optional[int] = None) -> Partition:
+def partition(coords, batch, grid, window, set_size, axis, cap_sets: Optional[int] = None,
+              shift=(0, 0, 0)) -> Partition:
+    """Set partition for one sort axis; `shift` displaces the window cut (hybrid window partition, Sec. 3.2)."""
     coords = _i32(coords).reshape(-1, 4)
     n = coords.shape[0]
-    nw = num_windows(batch, grid, window)
+    nw = num_windows(batch, grid, window, shift)
     cap = int(cap_sets) if cap_sets is not None else max(n, 1)
     table = np.full((cap, set_size), -1, dtype=np.int32)
     ns = np.zeros(1, dtype=np.int32)
@@ -108,13 +110,14 @@ def partition(coords, batch, grid, window, set_size, axis, cap_sets: Optional[in
     wo = np.zeros(nw + 1, dtype=np.int32)
     g = _i32(grid)
     w = _i32(window)
-    rc = lib().dsvt_ref_partition(
-        _p(coords, C.c_int32), C.c_int32(n), C.c_int32(batch), _p(g, C.c_int32), _p(w, C.c_int32),
+    sh = _i32(shift)
+    rc = lib().dsvt_ref_partition_shifted(
+        _p(coords, C.c_int32), C.c_int32(n), C.c_int32(batch), _p(g, C.c_int32), _p(w, C.c_int32), _p(sh, C.c_int32),
         C.c_int32(set_size), C.c_int32(axis), _p(table, C.c_int32), C.c_int32(cap), _p(ns, C.c_int32),
         _p(perm, C.c_int32), _p(ws, C.c_int32), _p(wc, C.c_int32), _p(wo, C.c_int32),
     )
     if rc != 0:
-        raise ValueError("dsvt_ref_partition rc=%d" % rc)
+        raise ValueError("dsvt_ref_partition_shifted rc=%d" % rc)
     return Partition(table[: ns[0]].copy(), perm[:n].copy(), ws, wc[:nw].copy(), wo)
 
 

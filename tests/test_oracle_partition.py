@@ -30,9 +30,9 @@ def test_eq3_hand_worked_rows(oracle):
         assert np.array_equal(got, want), (N, tau, got, want)
 
 
-def _read_tiny_grid():
+def _read_tiny_grid(name="tiny_grid.txt"):
     sect, data = None, {"coords": [], "axis0": [], "axis1": []}
-    for line in open(os.path.join(GOLD, "tiny_grid.txt")):
+    for line in open(os.path.join(GOLD, name)):
         line = line.strip()
         if not line or line.startswith("#"):
             continue
@@ -55,6 +55,47 @@ def test_tiny_grid_hand_worked_tables(oracle):
     py = oracle.partition(g["coords"], 1, (8, 4, 1), (4, 4, 1), 3, 1).perm
     assert list(px) == [4, 1, 2, 6, 5, 0, 8, 7, 3]
     assert list(py) == [4, 2, 0, 1, 5, 6, 8, 7, 3]
+
+
+def test_tiny_grid_shifted_hand_worked_tables(oracle):
+    """Window cut displaced by (2, 0, 0): hand-worked tables, counts and orders."""
+    g = _read_tiny_grid("tiny_grid_shift.txt")
+    for axis in (0, 1):
+        p = oracle.partition(g["coords"], 1, (8, 4, 1), (4, 4, 1), 3, axis, shift=(2, 0, 0))
+        assert np.array_equal(p.set_table, g["axis%d" % axis]), axis
+        assert list(p.win_count) == [4, 5, 0]
+        assert list(p.win_start) == [0, 4, 9, 9]
+        assert list(p.win_setoff) == [0, 2, 4, 4]
+    assert list(oracle.partition(g["coords"], 1, (8, 4, 1), (4, 4, 1), 3, 0, shift=(2, 0, 0)).perm) == [4, 1, 2, 6, 5, 0, 8, 7, 3]
+    assert list(oracle.partition(g["coords"], 1, (8, 4, 1), (4, 4, 1), 3, 1, shift=(2, 0, 0)).perm) == [4, 2, 1, 6, 7, 0, 5, 8, 3]
+
+
+@pytest.mark.parametrize("grid,window,shift,batch,n,tau", [
+    ((20, 17, 1), (6, 5, 1), (3, 2, 0), 1, 200, 7),
+    ((9, 9, 6), (4, 4, 3), (2, 1, 1), 2, 500, 10),
+    ((64, 64, 1), (24, 24, 1), (12, 12, 0), 1, 2000, 36),
+])
+def test_shifted_partition_is_the_plain_partition_of_translated_voxels(oracle, grid, window, shift, batch, n, tau):
+    """Displacing the window cut by s is the same as moving every voxel by +s on a grid that is s cells larger:
+    this reduces the shifted partition to the unshifted one, which the tests above pin on its own; also the
+    brute-force restatement with the shift written out."""
+    rng = np.random.default_rng(11)
+    coords = di.unique_cells(rng, n, grid, batch)
+    moved = coords.copy()
+    moved[:, 1:] += np.array(shift, dtype=np.int32)
+    big = tuple(g + s for g, s in zip(grid, shift))
+    for axis in (0, 1):
+        p = oracle.partition(coords, batch, grid, window, tau, axis, shift=shift)
+        q = oracle.partition(moved, batch, big, window, tau, axis)
+        assert np.array_equal(p.set_table, q.set_table)
+        assert np.array_equal(p.perm, q.perm)
+        assert np.array_equal(p.win_count, q.win_count) and np.array_equal(p.win_setoff, q.win_setoff)
+        assert np.array_equal(p.set_table, _brute_partition(moved, batch, big, window, tau, axis))
+    # a shift of zero is the plain partition; a shift outside [0, window) is refused
+    assert np.array_equal(oracle.partition(coords, batch, grid, window, tau, 0, shift=(0, 0, 0)).set_table,
+                          oracle.partition(coords, batch, grid, window, tau, 0).set_table)
+    with pytest.raises(ValueError):
+        oracle.partition(coords, batch, grid, window, tau, 0, shift=(window[0], 0, 0))
 
 
 @pytest.mark.parametrize("tau", [3, 24, 36, 48, 60, 90])
