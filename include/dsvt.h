@@ -133,6 +133,22 @@ int dsvt_partition_rotated(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int3
                            int32_t* const perm[2], int32_t* win_start, int32_t* win_count, int32_t* win_setoff);
 
 /*
+ * dsvt_partition_rotated with the window cut displaced by `shift` cells: Sec. 3.2, "Hybrid window partition"
+ * (the windows are re-cut between consecutive blocks with the window shifting of Swin, and with another
+ * window size; `window` is a per-call argument anyway).  A voxel at cell (x, y, z) lies in the window that
+ * holds cell (x + shift[0], y + shift[1], z + shift[2]) of the unshifted cut: window id =
+ * ((b*nWx + (x+sx)/L)*nWy + (y+sy)/W)*nWz + (z+sz)/H with nW* = ceil((grid + shift) / window), in-window
+ * offsets ((x+sx) mod L, ...).  0 <= shift[a] < window[a] (else DSVT_ERR_INVALID_ARG); shift NULL = no shift.
+ * The window arrays have batch*nWx*nWy*nWz (+ 1) entries, and that count must fit max_windows.  Everything
+ * else is dsvt_partition_rotated.
+ */
+int dsvt_partition_shifted(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch, const int32_t grid[3],
+                           const int32_t window[3], const int32_t shift[3], int32_t set_size,
+                           int32_t* const set_table[2], int32_t cap_sets, int32_t* const num_sets[2],
+                           int32_t* const set_rowoff[2], int32_t* const perm[2], int32_t* win_start,
+                           int32_t* win_count, int32_t* win_setoff);
+
+/*
  * dsvt_partition without any allocation.  (The paper has no counterpart: this is a deployment
  * variant of dsvt_partition, computing exactly the same table.)
  *

@@ -23,7 +23,7 @@ STATUS_BAD_COORD, STATUS_TABLE_OVERFLOW, STATUS_BAD_INDEX, STATUS_DUPLICATE_CELL
 
 EXPORTS = [
     "dsvt_create", "dsvt_destroy", "dsvt_status_sync", "dsvt_last_cuda_error", "dsvt_error_string",
-    "dsvt_launch_count", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_layer", "dsvt_block", "dsvt_pool",
+    "dsvt_launch_count", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_layer", "dsvt_block", "dsvt_pool",
 ]
 
 _lib = None
@@ -68,6 +68,7 @@ def load():
     lib.dsvt_launch_count.restype = i64
     lib.dsvt_partition.argtypes = [vp, vp, i32, i32, p3, p3, i32, i32, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.dsvt_partition_rotated.argtypes = [vp, vp, i32, i32, p3, p3, i32, vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.dsvt_partition_shifted.argtypes = [vp, vp, i32, i32, p3, p3, p3, i32, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.dsvt_partition_noalloc.argtypes = [vp, vp, i32, i32, p3, p3, i32, i32, vp, i32, vp, vp, vp, C.POINTER(i32)]
     lib.dsvt_set_attention.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, i32, vp, vp, vp, vp, i32, vp, C.c_int, vp]
     lib.dsvt_layer.argtypes = [vp, vp, i32, vp, i32, vp, vp, C.POINTER(LayerParams), vp]
@@ -229,8 +230,9 @@ class Context:
 
     # ---- dsvt_partition_rotated ----
     def partition_rotated(self, coords: torch.Tensor, batch: int, grid, window, set_size: int,
-                          cap_sets: Optional[int] = None, out=None):
-        """Both sort axes in one call; returns (X-axis SetTable, Y-axis SetTable)."""
+                          cap_sets: Optional[int] = None, out=None, shift=None):
+        """Both sort axes in one call; returns (X-axis SetTable, Y-axis SetTable).  `shift` displaces the window
+        cut (dsvt_partition_shifted); None calls dsvt_partition_rotated."""
         n = int(coords.shape[0])
         if out is None:
             cap = int(cap_sets) if cap_sets is not None else max(n, 1)
@@ -242,12 +244,16 @@ class Context:
         t0, t1 = out
         assert t0.cap_sets == t1.cap_sets and t0.set_size == t1.set_size == set_size
         pair = lambda a, b: (C.c_void_p * 2)(_ptr(a), _ptr(b))
-        rc = self.lib.dsvt_partition_rotated(self._h, _ptr(coords), n, int(batch), _i3(grid), _i3(window),
-                                             int(set_size), pair(t0.set_table, t1.set_table), t0.cap_sets,
-                                             pair(t0.num_sets, t1.num_sets), pair(t0.set_rowoff, t1.set_rowoff),
-                                             pair(t0.perm, t1.perm), _ptr(t0.win_start), _ptr(t0.win_count),
-                                             _ptr(t0.win_setoff))
-        self._check(rc, "dsvt_partition_rotated")
+        tail = (int(set_size), pair(t0.set_table, t1.set_table), t0.cap_sets, pair(t0.num_sets, t1.num_sets),
+                pair(t0.set_rowoff, t1.set_rowoff), pair(t0.perm, t1.perm), _ptr(t0.win_start), _ptr(t0.win_count),
+                _ptr(t0.win_setoff))
+        if shift is None:
+            rc = self.lib.dsvt_partition_rotated(self._h, _ptr(coords), n, int(batch), _i3(grid), _i3(window), *tail)
+            self._check(rc, "dsvt_partition_rotated")
+        else:
+            rc = self.lib.dsvt_partition_shifted(self._h, _ptr(coords), n, int(batch), _i3(grid), _i3(window),
+                                                 _i3(shift), *tail)
+            self._check(rc, "dsvt_partition_shifted")
         return out
 
     # ---- dsvt_set_attention ----

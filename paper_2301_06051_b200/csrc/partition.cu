@@ -113,6 +113,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_add_kernel(int32_t* out, in
 // ---- window keys -----------------------------------------------------------------------------
 struct PartGeom {
   int32_t batch, gx, gy, gz, L, W, H, nWx, nWy, nWz, axis;
+  int32_t sx, sy, sz;  // displacement of the window cut (hybrid window partition): cell x sits at x + sx
   uint32_t V;
 };
 
@@ -131,8 +132,9 @@ __global__ void window_key_kernel(const int4* __restrict__ coords, int32_t n, Pa
     c.z = min(max(c.z, 0), g.gy - 1);
     c.w = min(max(c.w, 0), g.gz - 1);
   }
-  const int wx = c.y / g.L, wy = c.z / g.W, wz = c.w / g.H;
-  const int xi = c.y - wx * g.L, yi = c.z - wy * g.W, zi = c.w - wz * g.H;
+  const int xs = c.y + g.sx, ys = c.z + g.sy, zs = c.w + g.sz;
+  const int wx = xs / g.L, wy = ys / g.W, wz = zs / g.H;
+  const int xi = xs - wx * g.L, yi = ys - wy * g.W, zi = zs - wz * g.H;
   const uint32_t win = (uint32_t)(((c.x * g.nWx + wx) * g.nWy + wy) * g.nWz + wz);
   const uint32_t inner =
       g.axis == 0 ? (uint32_t)((xi * g.W + yi) * g.H + zi) : (uint32_t)((yi * g.L + xi) * g.H + zi);
@@ -417,8 +419,9 @@ __global__ void bm_mark_kernel(const int4* __restrict__ coords, int32_t n, PartG
     c.z = min(max(c.z, 0), g.gy - 1);
     c.w = min(max(c.w, 0), g.gz - 1);
   }
-  const int wx = c.y / g.L, wy = c.z / g.W, wz = c.w / g.H;
-  const int xi = c.y - wx * g.L, yi = c.z - wy * g.W, zi = c.w - wz * g.H;
+  const int xs = c.y + g.sx, ys = c.z + g.sy, zs = c.w + g.sz;
+  const int wx = xs / g.L, wy = ys / g.W, wz = zs / g.H;
+  const int xi = xs - wx * g.L, yi = ys - wy * g.W, zi = zs - wz * g.H;
   const uint32_t win = (uint32_t)(((c.x * g.nWx + wx) * g.nWy + wy) * g.nWz + wz);
   atomicAdd(&win_count[win], 1);
   int ticket = -1;
@@ -592,18 +595,22 @@ struct PartCall {
 };
 
 int validate(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch, const int32_t grid[3],
-             const int32_t window[3], int32_t set_size, int32_t cap_sets, PartCall* pc) {
+             const int32_t window[3], const int32_t shift[3], int32_t set_size, int32_t cap_sets, PartCall* pc) {
   if (!ctx || !grid || !window || n < 0 || batch < 1 || set_size < 1 || cap_sets < 0) return DSVT_ERR_INVALID_ARG;
-  for (int a = 0; a < 3; ++a)
+  for (int a = 0; a < 3; ++a) {
     if (grid[a] < 1 || window[a] < 1) return DSVT_ERR_INVALID_ARG;
+    if (shift && (shift[a] < 0 || shift[a] >= window[a])) return DSVT_ERR_INVALID_ARG;
+    if ((int64_t)grid[a] + window[a] >= (1ll << 31)) return DSVT_ERR_UNSUPPORTED;
+  }
   if (n > 0 && !coords) return DSVT_ERR_INVALID_ARG;
   if (((uintptr_t)coords & 15) != 0) return DSVT_ERR_INVALID_ARG;
   PartGeom& g = pc->g;
   g.batch = batch; g.gx = grid[0]; g.gy = grid[1]; g.gz = grid[2];
   g.L = window[0]; g.W = window[1]; g.H = window[2];
-  g.nWx = (int32_t)dsvt_ceil_div(grid[0], window[0]);
-  g.nWy = (int32_t)dsvt_ceil_div(grid[1], window[1]);
-  g.nWz = (int32_t)dsvt_ceil_div(grid[2], window[2]);
+  g.sx = shift ? shift[0] : 0; g.sy = shift ? shift[1] : 0; g.sz = shift ? shift[2] : 0;
+  g.nWx = (int32_t)dsvt_ceil_div((int64_t)grid[0] + g.sx, window[0]);
+  g.nWy = (int32_t)dsvt_ceil_div((int64_t)grid[1] + g.sy, window[1]);
+  g.nWz = (int32_t)dsvt_ceil_div((int64_t)grid[2] + g.sz, window[2]);
   g.axis = 0;
   const uint64_t V = (uint64_t)window[0] * window[1] * window[2];
   const uint64_t num_windows = (uint64_t)batch * g.nWx * g.nWy * g.nWz;
@@ -744,7 +751,7 @@ extern "C" int dsvt_partition(dsvt_ctx* ctx, const int32_t* coords, int32_t n, i
                               int32_t* win_start, int32_t* win_count, int32_t* win_setoff) {
   if (!num_sets || (axis != 0 && axis != 1)) return DSVT_ERR_INVALID_ARG;
   PartCall pc;
-  int rc = validate(ctx, coords, n, batch, grid, window, set_size, cap_sets, &pc);
+  int rc = validate(ctx, coords, n, batch, grid, window, nullptr, set_size, cap_sets, &pc);
   if (rc != DSVT_OK) return rc;
   if (n > 0 && !set_table) return DSVT_ERR_INVALID_ARG;
   pc.win_start = win_start; pc.win_count = win_count; pc.win_setoff = win_setoff;
@@ -759,9 +766,19 @@ extern "C" int dsvt_partition_rotated(dsvt_ctx* ctx, const int32_t* coords, int3
                                       int32_t* const set_table[2], int32_t cap_sets, int32_t* const num_sets[2],
                                       int32_t* const set_rowoff[2], int32_t* const perm[2], int32_t* win_start,
                                       int32_t* win_count, int32_t* win_setoff) {
+  return dsvt_partition_shifted(ctx, coords, n, batch, grid, window, nullptr, set_size, set_table, cap_sets, num_sets,
+                                set_rowoff, perm, win_start, win_count, win_setoff);
+}
+
+extern "C" int dsvt_partition_shifted(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch,
+                                      const int32_t grid[3], const int32_t window[3], const int32_t shift[3],
+                                      int32_t set_size, int32_t* const set_table[2], int32_t cap_sets,
+                                      int32_t* const num_sets[2], int32_t* const set_rowoff[2],
+                                      int32_t* const perm[2], int32_t* win_start, int32_t* win_count,
+                                      int32_t* win_setoff) {
   if (!set_table || !num_sets || !num_sets[0] || !num_sets[1]) return DSVT_ERR_INVALID_ARG;
   PartCall pc;
-  int rc = validate(ctx, coords, n, batch, grid, window, set_size, cap_sets, &pc);
+  int rc = validate(ctx, coords, n, batch, grid, window, shift, set_size, cap_sets, &pc);
   if (rc != DSVT_OK) return rc;
   if (n > 0 && (!set_table[0] || !set_table[1])) return DSVT_ERR_INVALID_ARG;
   pc.win_start = win_start; pc.win_count = win_count; pc.win_setoff = win_setoff;

@@ -2,7 +2,8 @@
 
 A DSVT backbone is a stack of blocks; all blocks of a stage share the two rotated set tables of their
 frame, so a pass is: dsvt_partition_rotated (X and Y axis tables), then one dsvt_block per block,
-and optionally dsvt_pool followed by a second stage on the pooled grid.
+and optionally dsvt_pool followed by a second stage on the pooled grid.  With hybrid windows a stage holds one
+pair of tables per distinct (window, shift) and calls dsvt_partition_shifted for the displaced cuts.
 """
 from __future__ import annotations
 
@@ -14,30 +15,45 @@ from . import api
 
 
 class Stage:
-    """Blocks that share one grid / window shape: two set tables + per-block weights."""
+    """Blocks on one grid.  By default all blocks share one window shape and the two rotated set tables of the
+    frame; `block_windows` gives each block its own (window, shift) instead (hybrid window partition: another
+    window size and a displaced cut between consecutive blocks), with one pair of tables per distinct entry."""
 
     def __init__(self, ctx: api.Context, blocks: Sequence[Sequence[Dict]], batch: int, grid, window, set_size: int,
-                 precision: int, max_voxels: int):
+                 precision: int, max_voxels: int, block_windows: Optional[Sequence] = None):
         self.ctx, self.batch, self.grid, self.window, self.set_size = ctx, batch, tuple(grid), tuple(window), set_size
         dev = ctx.device
         self.blocks = [[api.device_weights(l, precision, dev) for l in blk] for blk in blocks]
         cap = max(int(max_voxels), 1)
-        self.tables = [
-            api.SetTable(torch.empty((cap, set_size), dtype=torch.int32, device=dev),
-                         torch.zeros(1, dtype=torch.int32, device=dev),
-                         torch.empty(2 * cap + 3, dtype=torch.int32, device=dev), cap, set_size)
-            for _ in range(2)
-        ]
+
+        def new_tables():
+            return [api.SetTable(torch.empty((cap, set_size), dtype=torch.int32, device=dev),
+                                 torch.zeros(1, dtype=torch.int32, device=dev),
+                                 torch.empty(2 * cap + 3, dtype=torch.int32, device=dev), cap, set_size)
+                    for _ in range(2)]
+
+        specs = [(self.window, None)] * len(self.blocks) if block_windows is None else [
+            (tuple(w), None if sh is None else tuple(sh)) for w, sh in block_windows]
+        assert len(specs) == len(self.blocks)
+        self.specs = specs
+        self.tables_of = {}
+        for sp in specs:
+            if sp not in self.tables_of:
+                self.tables_of[sp] = new_tables()
+        self.tables = self.tables_of[specs[0]] if specs else new_tables()  # the first block's pair
 
     def partition(self, coords: torch.Tensor):
-        self.ctx.partition_rotated(coords, self.batch, self.grid, self.window, self.set_size, out=tuple(self.tables))
+        for (window, shift), tables in self.tables_of.items():
+            self.ctx.partition_rotated(coords, self.batch, self.grid, window, self.set_size, out=tuple(tables),
+                                       shift=shift)
 
     def forward(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
-        """Partition (both axes) then every block; the result ends up in y."""
+        """Partition (both axes of every distinct window cut) then every block; the result ends up in y."""
         self.partition(coords)
         src = x
-        for blk in self.blocks:
-            self.ctx.block(src, self.tables[0], self.tables[1], blk, y)
+        for blk, sp in zip(self.blocks, self.specs):
+            t = self.tables_of[sp]
+            self.ctx.block(src, t[0], t[1], blk, y)
             src = y
         return y
 
@@ -51,13 +67,22 @@ class Backbone:
         self.precision = api.BF16_FP32ACC if cfg["precision"] == "bf16" else api.FP32
         grid, window = cfg["grid"], cfg["window"]
         nwin = cfg["batch"] * (-(-grid[0] // window[0])) * (-(-grid[1] // window[1])) * (-(-grid[2] // window[2]))
+        bw = cfg.get("block_windows")
+        if bw:  # displaced or larger windows: the largest window count of any cut
+            for w, sh in bw:
+                sh = sh or (0, 0, 0)
+                cnt = cfg["batch"]
+                for a in range(3):
+                    cnt *= -(-(grid[a] + sh[a]) // w[a])
+                nwin = max(nwin, cnt)
         max_windows = nwin
         self.pool_shape = cfg.get("pool_shape")
         if self.pool_shape:
             pg = [-(-grid[a] // self.pool_shape[a]) for a in range(3)]
             max_windows = max(max_windows, cfg["batch"] * pg[0] * pg[1] * pg[2])
         self.ctx = api.Context(n, max_windows, cfg["C"], device)
-        self.stage1 = Stage(self.ctx, cfg["blocks"], cfg["batch"], grid, window, cfg["set_size"], self.precision, n)
+        self.stage1 = Stage(self.ctx, cfg["blocks"], cfg["batch"], grid, window, cfg["set_size"], self.precision, n,
+                            block_windows=bw)
         self.stage2 = None
         if self.pool_shape:
             self.pool_w = api.device_weights(cfg["pool"], self.precision, self.ctx.device)

@@ -18,9 +18,15 @@ import dsvt_inputs as di
 from . import api, pipeline
 
 
-def time_config(cid: int, steps: int, device: int = 0):
+def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False):
     cfg = di.make_config(cid)
     dev = torch.device("cuda", device)
+    if hybrid:
+        # hybrid window partition (Sec. 3.2): every second block works on windows twice as large in x and y,
+        # cut with a displacement of one original window
+        w = cfg["window"]
+        big = (2 * w[0], 2 * w[1], w[2])
+        cfg["block_windows"] = [(w, None) if i % 2 == 0 else (big, (w[0], w[1], 0)) for i in range(len(cfg["blocks"]))]
     bb = pipeline.Backbone(cfg, device=device)
     coords = torch.from_numpy(cfg["coords"]).to(dev)
     x = torch.from_numpy(cfg["feats"]).to(dev)
@@ -64,7 +70,7 @@ def time_config(cid: int, steps: int, device: int = 0):
         spans.setdefault("backbone", []).append(r[0][1].elapsed_time(r[-1][1]))
     med = {k: float(np.median(v)) for k, v in spans.items()}
     nb1 = len(bb.stage1.blocks)
-    out = {"config": cid, "name": cfg["name"], "voxels": cfg["n"], "precision": cfg["precision"],
+    out = {"config": cid, "name": cfg["name"] + (" + hybrid windows" if hybrid else ""), "voxels": cfg["n"], "precision": cfg["precision"],
            "sets": int(bb.stage1.tables[0].num_sets.item()),
            "t_partition_ms": med["s1_partition"], "t_block_ms": med["s1_blocks"] / nb1,
            "voxels_per_s_per_block": cfg["n"] / (med["s1_blocks"] / nb1 * 1e-3),
@@ -80,10 +86,12 @@ def main():
     ap = argparse.ArgumentParser(description=__doc__)
     ap.add_argument("--configs", type=int, nargs="+", default=list(di.CONFIG_IDS))
     ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--hybrid", action="store_true",
+                    help="alternate the configuration's windows with doubled, displaced ones (single-stage configurations)")
     args = ap.parse_args()
     api.load()
     for cid in args.configs:
-        print(json.dumps(time_config(cid, args.steps)), flush=True)
+        print(json.dumps(time_config(cid, args.steps, hybrid=args.hybrid)), flush=True)
 
 
 if __name__ == "__main__":

@@ -89,6 +89,55 @@ def test_partition_bit_exact_small_and_edge_cases(gpu, oracle, grid, window, bat
     _check_partition(gpu, oracle, di.unique_cells(rng, n, grid, batch), batch, grid, window, tau)
 
 
+@pytest.mark.parametrize("grid,window,shift,batch,n,tau", [
+    ((20, 17, 1), (6, 5, 1), (3, 2, 0), 1, 200, 7),
+    ((9, 9, 6), (4, 4, 3), (2, 1, 1), 2, 500, 10),
+    ((468, 468, 1), (24, 24, 1), (12, 12, 0), 1, 32000, 36),   # the hybrid partner of the 12 x 12 windows
+    ((64, 64, 8), (12, 12, 8), (6, 6, 0), 1, 9000, 48),
+])
+def test_partition_shifted_bit_exact(gpu, oracle, grid, window, shift, batch, n, tau):
+    """dsvt_partition_shifted (displaced window cut, hybrid window partition) against the oracle."""
+    rng = np.random.default_rng(n + tau)
+    if grid == (468, 468, 1):
+        coords = di.make_config(2, with_feats=False)["coords"]  # the LiDAR-shaped frame of configuration 2
+    else:
+        coords = di.unique_cells(rng, n, grid, batch)
+    nwin = batch * int(np.prod([-(-(g + s) // w) for g, w, s in zip(grid, window, shift)]))
+    ctx = gpu.Context(n, nwin, 64)
+    both = ctx.partition_rotated(dev(coords), batch, grid, window, tau, shift=shift)
+    assert ctx.status_sync() == 0
+    for axis in (0, 1):
+        ref = oracle.partition(coords, batch, grid, window, tau, axis, shift=shift)
+        _compare_table(both[axis], ref, n, axis, extras=False)
+    with pytest.raises(gpu.DsvtError):
+        ctx.partition_rotated(dev(coords), batch, grid, window, tau, shift=(window[0], 0, 0))
+
+
+def test_hybrid_window_backbone_matches_oracle(gpu, oracle):
+    """Four blocks that alternate 12 x 12 windows with 24 x 24 windows displaced by (12, 12) (hybrid window
+    partition, Sec. 3.2), whole small frame, bf16 weights: pipeline.Stage against the oracle block by block."""
+    from paper_2301_06051_b200 import pipeline
+
+    cfg = di.random_case(21, 3000, (96, 96, 1), (12, 12, 1), 36, 192, 8, hidden=384, layernorm=True, bf16=True,
+                         n_blocks=4)
+    specs = [((12, 12, 1), None), ((24, 24, 1), (12, 12, 0))] * 2
+    nwin = int(np.prod([-(-(96 + 12) // 12)] * 2))
+    ctx = gpu.Context(cfg["n"], nwin, 192)
+    stage = pipeline.Stage(ctx, cfg["blocks"], 1, cfg["grid"], cfg["window"], 36, gpu.BF16_FP32ACC, cfg["n"],
+                           block_windows=specs)
+    x = dev(cfg["feats"])
+    y = torch.empty_like(x)
+    stage.forward(dev(cfg["coords"]), x, y)
+    assert ctx.status_sync() == 0
+    want = cfg["feats"].astype(np.float64)
+    for blk, (window, shift) in zip(cfg["blocks"], specs):
+        sh = shift or (0, 0, 0)
+        t0 = oracle.partition(cfg["coords"], 1, cfg["grid"], window, 36, 0, shift=sh).set_table
+        t1 = oracle.partition(cfg["coords"], 1, cfg["grid"], window, 36, 1, shift=sh).set_table
+        want = oracle.block(want, t0, t1, blk)
+    check_close(y.cpu().numpy(), want, "bf16", "hybrid-window backbone")
+
+
 def test_partition_sorting_route_on_a_key_space_beyond_the_bitmap(gpu, oracle):
     """8400 x 8400 cells in 12 x 12 windows: 490000 windows x 160 padded cells exceed the context's
     64 Mi-key bitmap, so the call takes the radix-sort route; results are the same."""
