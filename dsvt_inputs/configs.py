@@ -125,14 +125,14 @@ def _first_unique(keys: np.ndarray, limit: int) -> np.ndarray:
     return first[:limit]
 
 
-def lidar_pillars(rng, n: int, grid_xy: int = 468) -> np.ndarray:
+def lidar_pillars(rng, n: int, grid_xy: int = 468, half_range: float = HALF_RANGE, cell: float = CELL) -> np.ndarray:
     """Exactly n distinct (x, y) cells of a LiDAR-shaped frame, in draw order.  int64 [n][2]."""
     cells = np.zeros((0, 2), dtype=np.int64)
     while True:
         px, py, _ = _lidar_points(rng, 2 * n)
-        ok = (np.abs(px) < HALF_RANGE) & (np.abs(py) < HALF_RANGE)
-        cx = np.floor((px[ok] + HALF_RANGE) / CELL).astype(np.int64)
-        cy = np.floor((py[ok] + HALF_RANGE) / CELL).astype(np.int64)
+        ok = (np.abs(px) < half_range) & (np.abs(py) < half_range)
+        cx = np.floor((px[ok] + half_range) / cell).astype(np.int64)
+        cy = np.floor((py[ok] + half_range) / cell).astype(np.int64)
         ok2 = (cx >= 0) & (cx < grid_xy) & (cy >= 0) & (cy < grid_xy)
         cells = np.concatenate([cells, np.stack([cx[ok2], cy[ok2]], axis=1)], axis=0)
         keep = _first_unique(cells[:, 0] * grid_xy + cells[:, 1], n)
@@ -228,7 +228,7 @@ def _coords4(b, xy_or_xyz: np.ndarray) -> np.ndarray:
 # the five configurations
 # ---------------------------------------------------------------------------
 def make_config(cid: int, n_override: Optional[int] = None, with_feats: bool = True) -> Dict:
-    """Configuration `cid` (1..5) as a dict.
+    """Configuration `cid` (1..5, and 6 = the nuScenes-shaped extra) as a dict.
 
     Keys: id, name, batch, grid, window, set_size, C, heads, hidden, precision
     ('fp32' | 'bf16'), coords int32 [n][4], feats float32 [n][C], blocks (list of
@@ -268,8 +268,16 @@ def make_config(cid: int, n_override: Optional[int] = None, with_feats: bool = T
                    heads=8, hidden=384, layernorm=True, precision="bf16", n_blocks=2,
                    pool_shape=(2, 2, 1), n_blocks_after_pool=2)
         cfg["coords"] = _coords4(0, skewed_pillars(rng, n))
+    elif cid == 6:
+        # the paper's second workload shape (Appendix B.1.2: windows 30 x 30 x 1, set size 90, 128 channels, 8 heads,
+        # 256 hidden channels).  The paper does not state the pillar size there: 0.3 m cells over +-54 m (360 x 360)
+        # and 30 000 pillars are this generator's choice.  Not one of the five measured configurations.
+        n = n_override or 30_000
+        cfg.update(name="nuscenes_pillars", batch=1, grid=(360, 360, 1), window=(30, 30, 1), set_size=90, C=128,
+                   heads=8, hidden=256, layernorm=True, precision="bf16", n_blocks=4)
+        cfg["coords"] = _coords4(0, lidar_pillars(rng, n, 360, 54.0, 0.3))
     else:
-        raise ValueError("config id must be 1..5")
+        raise ValueError("config id must be 1..6")
     n = cfg["coords"].shape[0]
     cfg["n"] = n
     C = cfg["C"]

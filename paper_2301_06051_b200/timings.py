@@ -84,7 +84,8 @@ def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False):
 
 def main():
     ap = argparse.ArgumentParser(description=__doc__)
-    ap.add_argument("--configs", type=int, nargs="+", default=list(di.CONFIG_IDS))
+    ap.add_argument("--configs", type=int, nargs="+", default=list(di.CONFIG_IDS),
+                    help="1..5; 6 = the nuScenes-shaped extra (windows 30 x 30, set size 90, C=128)")
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--hybrid", action="store_true",
                     help="alternate the configuration's windows with doubled, displaced ones (single-stage configurations)")

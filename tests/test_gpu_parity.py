@@ -69,7 +69,7 @@ def _check_partition(gpu, oracle, coords, batch, grid, window, tau, ctx=None):
     return ctx
 
 
-@pytest.mark.parametrize("cid", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("cid", [1, 2, 3, 4, 5, 6])
 def test_partition_bit_exact_on_every_config(gpu, oracle, cid):
     cfg = di.make_config(cid, with_feats=False)
     _check_partition(gpu, oracle, cfg["coords"], cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"])
@@ -339,9 +339,10 @@ def _sample_windows(oracle, cfg, coords, n_target, seed, win=None):
     return np.sort(np.unique(np.concatenate(sel)))
 
 
-@pytest.mark.parametrize("cid,n_sample", [(2, 2500), (3, 2500), (4, 2500)])
+@pytest.mark.parametrize("cid,n_sample", [(2, 2500), (3, 2500), (4, 2500), (6, 2500)])
 def test_backbone_full_size_bf16_on_sampled_windows(gpu, oracle, cid, n_sample):
-    """Configs 2-4 at full size (four blocks, bf16 weights).  The backbone is window-local (both
+    """Configs 2-4 (and the nuScenes-shaped extra, 6: windows 30 x 30, set size 90, C=128) at full size (four
+    blocks, bf16 weights).  The backbone is window-local (both
     layers of every block use the same windows), so the oracle recomputes whole sampled windows."""
     cfg = di.make_config(cid)
     got = _run_blocks_gpu(gpu, cfg, cfg["blocks"], cfg["coords"], cfg["feats"])
