@@ -228,7 +228,7 @@ def _coords4(b, xy_or_xyz: np.ndarray) -> np.ndarray:
 # the five configurations
 # ---------------------------------------------------------------------------
 def make_config(cid: int, n_override: Optional[int] = None, with_feats: bool = True) -> Dict:
-    """Configuration `cid` (1..5, and 6 = the nuScenes-shaped extra) as a dict.
+    """Configuration `cid` (1..5; 6 = the nuScenes-shaped extra; 7 = the DSVT-V stage layout: `stages`, `pools`) as a dict.
 
     Keys: id, name, batch, grid, window, set_size, C, heads, hidden, precision
     ('fp32' | 'bf16'), coords int32 [n][4], feats float32 [n][C], blocks (list of
@@ -276,8 +276,17 @@ def make_config(cid: int, n_override: Optional[int] = None, with_feats: bool = T
         cfg.update(name="nuscenes_pillars", batch=1, grid=(360, 360, 1), window=(30, 30, 1), set_size=90, C=128,
                    heads=8, hidden=256, layernorm=True, precision="bf16", n_blocks=4)
         cfg["coords"] = _coords4(0, lidar_pillars(rng, n, 360, 54.0, 0.3))
+    elif cid == 7:
+        # the voxel variant's stage layout (Appendix B.1.1, DSVT-V): four stages of one block each, windows of
+        # 32 / 8 / 2 / 1 cells along z (12 x 12 in x, y), attention-style pooling along z with strides 4, 4, 2
+        # between them, set size 48.  Same voxel generator as configuration 3.  Not one of the five measured
+        # configurations.
+        n = n_override or 120_000
+        cfg.update(name="dsvt_v_stages", batch=1, grid=(468, 468, 32), window=(12, 12, 32), set_size=48, C=192,
+                   heads=8, hidden=384, layernorm=True, precision="bf16", n_blocks=1)
+        cfg["coords"] = _coords4(0, lidar_voxels(rng, n))
     else:
-        raise ValueError("config id must be 1..6")
+        raise ValueError("config id must be 1..7")
     n = cfg["coords"].shape[0]
     cfg["n"] = n
     C = cfg["C"]
@@ -288,6 +297,15 @@ def make_config(cid: int, n_override: Optional[int] = None, with_feats: bool = T
         [make_layer(wrng, C, cfg["heads"], cfg["hidden"], cfg["layernorm"], bf16) for _ in range(2)]
         for _ in range(cfg["n_blocks"])
     ]
+    if cid == 7:
+        z_windows, strides = (32, 8, 2, 1), (4, 4, 2)
+        cfg["stages"] = [{"window": (12, 12, z_windows[0]), "blocks": cfg["blocks"]}]
+        cfg["pools"] = []
+        for i, st in enumerate(strides):
+            cfg["pools"].append({"shape": (1, 1, st), "weights": make_pool_weights(wrng, C, cfg["heads"], bf16)})
+            cfg["stages"].append({"window": (12, 12, z_windows[i + 1]),
+                                  "blocks": [[make_layer(wrng, C, cfg["heads"], cfg["hidden"], True, bf16)
+                                              for _ in range(2)]]})
     if cid == 5:
         cfg["pool"] = make_pool_weights(wrng, C, cfg["heads"], bf16)
         cfg["blocks_after_pool"] = [

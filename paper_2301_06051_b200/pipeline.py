@@ -101,3 +101,52 @@ class Backbone:
         oc, of = oc[:m], of[:m]
         self.stage2.forward(oc, of, of)
         return oc, of, num
+
+
+class StagedBackbone:
+    """Any number of stages with attention-style pooling between them (the voxel variant's layout: windows that
+    shrink along z while pooling reduces the z extent).  cfg["stages"][i] = {"window", "blocks"}; cfg["pools"][i] =
+    {"shape", "weights"} maps stage i's grid to stage i + 1's."""
+
+    def __init__(self, cfg: Dict, device: int = 0):
+        self.cfg = cfg
+        n = int(cfg["n"])
+        self.precision = api.BF16_FP32ACC if cfg["precision"] == "bf16" else api.FP32
+        grids = [tuple(cfg["grid"])]
+        for pl in cfg["pools"]:
+            grids.append(tuple(-(-grids[-1][a] // pl["shape"][a]) for a in range(3)))
+        self.grids = grids
+        max_windows = 1
+        for g, st in zip(grids, cfg["stages"]):
+            w = st["window"]
+            max_windows = max(max_windows, cfg["batch"] * (-(-g[0] // w[0])) * (-(-g[1] // w[1])) * (-(-g[2] // w[2])))
+        for g in grids[1:]:  # pooling works on one region per cell of the next grid
+            max_windows = max(max_windows, cfg["batch"] * g[0] * g[1] * g[2])
+        self.ctx = api.Context(n, max_windows, cfg["C"], device)
+        self.stages = [Stage(self.ctx, st["blocks"], cfg["batch"], g, st["window"], cfg["set_size"], self.precision, n)
+                       for g, st in zip(grids, cfg["stages"])]
+        self.pool_w = [api.device_weights(pl["weights"], self.precision, self.ctx.device) for pl in cfg["pools"]]
+
+    def forward(self, coords: torch.Tensor, x: torch.Tensor, on_step=None):
+        """Returns (coords, feats) of the last stage.  on_step(tag), if given, is called after every call group."""
+        feats = x
+        for i, stage in enumerate(self.stages):
+            y = torch.empty_like(feats)
+            stage.partition(coords)
+            if on_step:
+                on_step("s%d_partition" % i)
+            src = feats
+            for blk in stage.blocks:
+                self.ctx.block(src, stage.tables[0], stage.tables[1], blk, y)
+                src = y
+            if on_step:
+                on_step("s%d_blocks" % i)
+            feats = y
+            if i < len(self.pool_w):
+                oc, of, num, _, _ = self.ctx.pool(coords, feats, self.cfg["batch"], self.grids[i],
+                                                  self.cfg["pools"][i]["shape"], self.pool_w[i])
+                m = int(num.item())  # the pooled voxel count sizes the next stage's tensors
+                coords, feats = oc[:m], of[:m]
+                if on_step:
+                    on_step("s%d_pool" % i)
+        return coords, feats

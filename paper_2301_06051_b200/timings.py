@@ -18,8 +18,46 @@ import dsvt_inputs as di
 from . import api, pipeline
 
 
+def time_staged(cfg, steps: int, device: int = 0):
+    """Configurations with a `stages` list (the voxel variant's layout)."""
+    dev = torch.device("cuda", device)
+    bb = pipeline.StagedBackbone(cfg, device=device)
+    coords = torch.from_numpy(cfg["coords"]).to(dev)
+    x = torch.from_numpy(cfg["feats"]).to(dev)
+    flush = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    rec = []
+    for it in range(3 + steps):
+        flush.zero_()
+        marks = []
+
+        def on_step(tag):
+            e = torch.cuda.Event(enable_timing=True)
+            e.record(stream)
+            marks.append((tag, e))
+
+        on_step("start")
+        oc, of = bb.forward(coords, x, on_step)
+        rec.append(marks)
+    torch.cuda.synchronize(dev)
+    if bb.ctx.status_sync() != 0:
+        raise SystemExit("device status word is not clean")
+    spans = {}
+    for r in rec[3:]:
+        for (t0, e0), (t1, e1) in zip(r[:-1], r[1:]):
+            spans.setdefault(t1, []).append(e0.elapsed_time(e1))
+        spans.setdefault("backbone", []).append(r[0][1].elapsed_time(r[-1][1]))
+    out = {"config": cfg["id"], "name": cfg["name"], "voxels": cfg["n"], "precision": cfg["precision"],
+           "voxels_out": int(oc.shape[0])}
+    out.update({"t_%s_ms" % k: float(np.median(v)) for k, v in spans.items()})
+    out["frames_per_s"] = cfg["batch"] / (out["t_backbone_ms"] * 1e-3)
+    return out
+
+
 def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False):
     cfg = di.make_config(cid)
+    if cfg.get("stages"):
+        return time_staged(cfg, steps, device)
     dev = torch.device("cuda", device)
     if hybrid:
         # hybrid window partition (Sec. 3.2): every second block works on windows twice as large in x and y,
@@ -85,7 +123,7 @@ def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False):
 def main():
     ap = argparse.ArgumentParser(description=__doc__)
     ap.add_argument("--configs", type=int, nargs="+", default=list(di.CONFIG_IDS),
-                    help="1..5; 6 = the nuScenes-shaped extra (windows 30 x 30, set size 90, C=128)")
+                    help="1..5; 6 = the nuScenes-shaped extra (windows 30 x 30, set size 90, C=128); 7 = DSVT-V stage layout")
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--hybrid", action="store_true",
                     help="alternate the configuration's windows with doubled, displaced ones (single-stage configurations)")

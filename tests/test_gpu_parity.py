@@ -443,3 +443,36 @@ def test_config5_blocks_pool_blocks_on_sampled_windows(gpu, oracle):
     rows = np.array([pos[k] for k in key(pooled.coords).tolist()])
     assert np.all(np.diff(key(oc)) > 0)  # ascending pooled coordinates
     check_close(of[rows], want, "bf16", "config 5 chain, %d pooled voxels" % rows.shape[0])
+
+
+def test_dsvt_v_stage_layout_on_sampled_windows(gpu, oracle):
+    """The voxel variant's layout at full size (configuration 7: four one-block stages, z windows 32 / 8 / 2 / 1,
+    pooling along z by 4, 4, 2, set size 48).  Pooling along z keeps the 12 x 12 footprint of a window, so the whole
+    chain is local to a footprint and the oracle recomputes sampled footprints."""
+    from paper_2301_06051_b200 import pipeline
+
+    cfg = di.make_config(7)
+    bb = pipeline.StagedBackbone(cfg)
+    oc, of = bb.forward(dev(cfg["coords"]), dev(cfg["feats"]))
+    assert bb.ctx.status_sync() == 0
+    oc, of = oc.cpu().numpy(), of.cpu().numpy()
+    assert np.all(np.isfinite(of))
+    sel = _sample_windows(oracle, cfg, cfg["coords"], 2500, 7)
+    cs, fs = cfg["coords"][sel], cfg["feats"][sel].astype(np.float64)
+    grid = tuple(cfg["grid"])
+    for i, st in enumerate(cfg["stages"]):
+        c_i = dict(cfg, grid=grid, window=st["window"])
+        fs = _run_blocks_oracle(oracle, c_i, st["blocks"], cs, fs)
+        if i < len(cfg["pools"]):
+            pl = cfg["pools"][i]
+            pw = pl["weights"]
+            pooled = oracle.pool(cs, fs, 1, grid, pl["shape"], pw["W_q"], pw["W_k"], pw["W_v"], pw["W_o"],
+                                 pw["b_q"], pw["b_k"], pw["b_v"], pw["b_o"], cfg["heads"])
+            cs, fs = pooled.coords, pooled.feats
+            grid = tuple(-(-grid[a] // pl["shape"][a]) for a in range(3))
+    assert grid == (468, 468, 1)
+    key = lambda c: (c[:, 1].astype(np.int64) * 468 + c[:, 2])
+    assert np.all(np.diff(key(oc)) > 0)  # ascending pooled coordinates
+    pos = {k: i for i, k in enumerate(key(oc).tolist())}
+    rows = np.array([pos[k] for k in key(cs).tolist()])
+    check_close(of[rows], fs, "bf16", "DSVT-V stage layout, %d output voxels" % rows.shape[0])
