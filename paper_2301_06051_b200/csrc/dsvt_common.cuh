@@ -84,3 +84,6 @@ int dsvt_launch_layer_fma(dsvt_ctx* ctx, const dsvt_fused_args& a);
 // tcgen05 path: bfloat16 weights, C in {64, 128, 192}, head dim in {16, 24, 32}, set size <= 96.
 bool dsvt_layer_tc_supported(const dsvt_fused_args& a);
 int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a);
+// CUtensorMap (128 bytes, 64-byte aligned) of a row-major bf16 matrix [rows][cols]: boxes of 64 columns x box_rows
+// rows, 128-byte swizzle.  Returns false if the driver cannot encode it.
+bool dsvt_make_weight_map(void* tensor_map, const void* w, int rows, int cols, int box_rows);

@@ -1470,6 +1470,12 @@ int launch_tc_nt(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const
 
 }  // namespace
 
+// Tensor map of a row-major bf16 matrix [rows][cols] for boxes of 64 columns x box_rows rows with the 128-byte
+// swizzle (the layout every operand tile here uses); false if the driver entry point is missing or refuses.
+bool dsvt_make_weight_map(void* tensor_map, const void* w, int rows, int cols, int box_rows) {
+  return make_weight_map(reinterpret_cast<CUtensorMap*>(tensor_map), w, rows, cols, box_rows);
+}
+
 // Shapes the tensor-core kernel covers; everything else goes to the FMA kernel.
 bool dsvt_layer_tc_supported(const dsvt_fused_args& a) {
   const dsvt_layer_params& p = a.p;

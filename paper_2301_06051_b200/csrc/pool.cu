@@ -1,6 +1,8 @@
 // Attention-style 3D pooling (Eq. 6, Eq. 7): dense cell map -> region ranks -> fused
 // pad / max-pool / cross-attention kernel.  The region bookkeeping is exact integer work; the
 // attention runs on the fp32 FMA pipes with float or bfloat16 weights.
+#include <cuda.h>
+
 #include "dsvt_common.cuh"
 #include "fma_tile.cuh"
 
@@ -221,7 +223,7 @@ constexpr int kStages = 4;  // weight ring: 64-column blocks, prefetched three a
 constexpr int kMaxHeads = 8;
 
 struct Layout {  // byte offsets into dynamic shared memory (1024-aligned base)
-  uint32_t x, kv, p, w, probs, rowvox, total;
+  uint32_t x, kv, p, w, probs, rowvox, bars, total;
 };
 __host__ __device__ inline Layout make_layout(int C) {
   Layout L;
@@ -231,43 +233,59 @@ __host__ __device__ inline Layout make_layout(int C) {
   L.w = L.p + kRegs * C * 2;
   L.probs = L.w + kStages * (uint32_t)C * 128;
   L.rowvox = L.probs + 2 * kRows * kMaxHeads * 4;  // (regions x padded slots) < 2 x 128 per head
-  L.total = L.rowvox + kRows * 4;
+  L.bars = L.rowvox + kRows * 4;             // kStages mbarriers + the error flag
+  L.total = L.bars + kStages * 8 + 8;
   return L;
 }
 
+struct PoolMaps {
+  CUtensorMap w[4];  // W_q, W_k, W_v, W_o: boxes of 64 input columns x C rows, 128-byte swizzle
+};
+constexpr int kMaxPolls = 1 << 20;
+
 // The weight blocks of a CTA form one stream: tile after tile, W_q, W_k, W_v, W_o, each in C / 64 blocks of
-// 64 input columns.  Block g lives in stage g mod 4 and is requested three steps before it is used.
+// 64 input columns.  Block g lives in stage g mod 4 and is requested three steps before it is used, by one
+// thread, as a TMA load that completes on the stage's mbarrier.  Every wait is bounded (error flag).
 struct WeightStream {
-  const __nv_bfloat16* W[4];
+  const PoolMaps* maps;
+  unsigned long long* full;  // [kStages] in shared memory
+  int* error;                // shared flag: a wait gave up
   int C, nkb;
   long long total;   // blocks this CTA will consume
   long long next;    // next block to consume
   uint32_t base, stage_bytes;
 
   __device__ __forceinline__ void request(long long g) {
-    if (g < total) {
-      const int kb = (int)(g % nkb);
-      const __nv_bfloat16* w = W[(g / nkb) & 3];
-      const uint32_t stage = base + (uint32_t)(g % kStages) * stage_bytes;
-      for (int i = threadIdx.x; i < C * 8; i += kT) {
-        const int n = i >> 3, c = i & 7;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage + swz(n, c, 0)),
-                     "l"(w + (size_t)n * C + kb * 64 + c * 8) : "memory");
-      }
+    if (g < total && threadIdx.x == 0) {
+      const int kb = (int)(g % nkb), st = (int)(g % kStages);
+      const uint32_t bar = smem_u32(&full[st]);
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(stage_bytes) : "memory");
+      asm volatile(
+          "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+          ::"r"(base + (uint32_t)st * stage_bytes), "l"((uint64_t)&maps->w[(g / nkb) & 3]), "r"(bar), "r"(kb * 64), "r"(0)
+          : "memory");
     }
-    asm volatile("cp.async.commit_group;" ::: "memory");  // one group per step, empty or not
   }
   __device__ __forceinline__ void prologue() {
     for (int g = 0; g < kStages - 1; ++g) request(g);
   }
   // Makes the next block usable by every thread and returns its stage; requests the block three ahead.
   __device__ __forceinline__ uint32_t acquire() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(kStages - 2) : "memory");
-    __syncthreads();  // the block is visible to all; everyone is done with the block before it
+    const int st = (int)(next % kStages);
+    const uint32_t bar = smem_u32(&full[st]), parity = (uint32_t)((next / kStages) & 1);
+    bool ok = false;
+    for (int i = 0; i < kMaxPolls && !ok; ++i) {
+      uint32_t done;
+      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                   : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+      ok = done != 0;
+      if (!ok && (i & 255) == 255 && *reinterpret_cast<volatile int*>(error)) break;
+    }
+    if (!ok) *reinterpret_cast<volatile int*>(error) = 1;
+    __syncthreads();  // everyone is done with the block before it: its stage may be overwritten
     request(next + kStages - 1);
-    const uint32_t stage = base + (uint32_t)(next % kStages) * stage_bytes;
     ++next;
-    return stage;
+    return base + (uint32_t)st * stage_bytes;
   }
 };
 
@@ -339,7 +357,9 @@ __device__ __forceinline__ void unpack8(const uint4 u, float (&f)[8]) {
   f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xFFFF0000u);
 }
 
-__global__ void __launch_bounds__(kT, 1) pool_attn_mma_kernel(PoolArgs a) {
+__global__ void __launch_bounds__(kT, 1) pool_attn_mma_kernel(const __grid_constant__ PoolArgs a,
+                                                              const __grid_constant__ PoolMaps maps,
+                                                              int32_t* __restrict__ status) {
   extern __shared__ unsigned char pool_smem_raw[];
   const uint32_t raw = smem_u32(pool_smem_raw);
   unsigned char* sm = pool_smem_raw + ((1024u - (raw & 1023u)) & 1023u);
@@ -359,10 +379,16 @@ __global__ void __launch_bounds__(kT, 1) pool_attn_mma_kernel(PoolArgs a) {
   const int hpg = 32 / nsp;  // heads per pass of a warp
 
   WeightStream ws;
-  ws.W[0] = reinterpret_cast<const __nv_bfloat16*>(a.W_q);
-  ws.W[1] = reinterpret_cast<const __nv_bfloat16*>(a.W_k);
-  ws.W[2] = reinterpret_cast<const __nv_bfloat16*>(a.W_v);
-  ws.W[3] = reinterpret_cast<const __nv_bfloat16*>(a.W_o);
+  ws.maps = &maps;
+  ws.full = reinterpret_cast<unsigned long long*>(sm + L.bars);
+  ws.error = reinterpret_cast<int*>(sm + L.bars + kStages * 8);
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&ws.full[i])) : "memory");
+    *ws.error = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
   ws.C = C; ws.nkb = C >> 6;
   const long long my_tiles = blockIdx.x < num_tiles ? (num_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
   ws.total = my_tiles * 4 * ws.nkb;
@@ -511,7 +537,7 @@ __global__ void __launch_bounds__(kT, 1) pool_attn_mma_kernel(PoolArgs a) {
       for (int c4 = lane; c4 < C4; c4 += 32)
         reinterpret_cast<float4*>(a.out_feats + (size_t)(r_lo + r) * C)[c4] = *reinterpret_cast<const float4*>(outf + (size_t)r * C + 4 * c4);
   }
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  if (tid == 0 && *ws.error) atomicOr(status, DSVT_STATUS_TIMEOUT);
 }
 }  // namespace mma_pool
 
@@ -616,7 +642,11 @@ extern "C" int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feat
     if (gridn < 1) gridn = 1;
     cudaError_t e = cudaFuncSetAttribute(mma_pool::pool_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
-    mma_pool::pool_attn_mma_kernel<<<(unsigned)gridn, mma_pool::kT, smem, st>>>(a);
+    mma_pool::PoolMaps maps;
+    const void* wm[4] = {W_q, W_k, W_v, W_o};
+    for (int i = 0; i < 4; ++i)
+      if (!dsvt_make_weight_map(&maps.w[i], wm[i], C, C, C)) return DSVT_ERR_CUDA;
+    mma_pool::pool_attn_mma_kernel<<<(unsigned)gridn, mma_pool::kT, smem, st>>>(a, maps, ctx->status);
     DSVT_LAUNCHED(ctx);
     return DSVT_OK;
   }
