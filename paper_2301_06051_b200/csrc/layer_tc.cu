@@ -782,12 +782,12 @@ __device__ __forceinline__ void loader_row_list(int b, int lt, int s_lo, int nse
     const int cnt_max = inside ? min(cap, kTM - lb) : 0;  // tile rows this set may fill
     int pos = 0, prev = 0;
     bool bad = false;
-    for (int k0 = 0; k0 < tau; k0 += 32) {
-      int v4[32];  // 32 independent loads per round trip to L2
+    for (int k0 = 0; k0 < tau; k0 += 8) {
+      int v4[8];  // eight independent loads per round trip to L2 (the loader warps run a whole tile ahead)
 #pragma unroll
-      for (int u = 0; u < 32; ++u) v4[u] = k0 + u < tau ? __ldg(trow + k0 + u) : 0;
+      for (int u = 0; u < 8; ++u) v4[u] = k0 + u < tau ? __ldg(trow + k0 + u) : 0;
 #pragma unroll
-      for (int u = 0; u < 32; ++u) {
+      for (int u = 0; u < 8; ++u) {
         if (k0 + u < tau) {
           int v = v4[u];
           const bool uniq = (k0 + u == 0) || (v != prev);
