@@ -38,8 +38,8 @@ def _peaks():
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-layer launch at configuration 2, from the ncu capture
-# summarised in profiles/layer_tc_kernel_config2.md (25.68 MB read + 0.08 MB written: the output stays in L2).
-LAYER_DRAM_BYTES_PER_LAUNCH = 25.76e6
+# summarised in profiles/layer_tc_kernel_config2.md (25.63 MB read + 0.06 MB written: the output stays in L2).
+LAYER_DRAM_BYTES_PER_LAUNCH = 25.69e6
 
 
 class ClockSampler:
