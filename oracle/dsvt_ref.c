@@ -197,13 +197,57 @@ static void ref_linear(const double* W, const double* b, const double* x, int ou
 }
 
 /*
+ * Relative position bias, the mechanism of the Swin transformer that the text after Eq. 5 points to
+ * for PE(.): a learned scalar per head and per coordinate offset between query and key, added to
+ * the scaled logit.  Voxels of one set lie in one window of extent (L, W, H), so an offset component
+ * lies in [-(L-1), L-1] etc.; the table holds (2L-1)(2W-1)(2H-1) entries per head and the entry for
+ * offset (dx, dy, dz) = coords[query] - coords[key] sits at
+ *   ((dx + L-1) * (2W-1) + (dy + W-1)) * (2H-1) + (dz + H-1).
+ */
+typedef struct {
+  const double* table;   /* [heads][(2L-1)(2W-1)(2H-1)] */
+  const int32_t* coords; /* [n][4] = (b, x, y, z) */
+  int32_t ext[3];        /* L, W, H */
+} ref_rel_bias;
+
+static size_t ref_rel_bias_len(const ref_rel_bias* rb) {
+  return (size_t)(2 * rb->ext[0] - 1) * (size_t)(2 * rb->ext[1] - 1) * (size_t)(2 * rb->ext[2] - 1);
+}
+
+static size_t ref_rel_bias_index(const ref_rel_bias* rb, int32_t query, int32_t key) {
+  const int32_t* cq = rb->coords + (size_t)query * 4;
+  const int32_t* ck = rb->coords + (size_t)key * 4;
+  const int dx = cq[1] - ck[1], dy = cq[2] - ck[2], dz = cq[3] - ck[3];
+  const int L = rb->ext[0], W = rb->ext[1], H = rb->ext[2];
+  return ((size_t)(dx + L - 1) * (size_t)(2 * W - 1) + (size_t)(dy + W - 1)) * (size_t)(2 * H - 1) + (size_t)(dz + H - 1);
+}
+
+/* 1 iff every pair of members of every table row has an offset the table covers */
+static int ref_rel_bias_covers(const ref_rel_bias* rb, const int32_t* set_table, int32_t num_sets, int32_t tau) {
+  for (int32_t s = 0; s < num_sets; ++s) {
+    const int32_t* rows = set_table + (size_t)s * tau;
+    int32_t lo[3], hi[3];
+    for (int a = 0; a < 3; ++a) lo[a] = hi[a] = rb->coords[(size_t)rows[0] * 4 + 1 + a];
+    for (int k = 1; k < tau; ++k)
+      for (int a = 0; a < 3; ++a) {
+        const int32_t v = rb->coords[(size_t)rows[k] * 4 + 1 + a];
+        if (v < lo[a]) lo[a] = v;
+        if (v > hi[a]) hi[a] = v;
+      }
+    for (int a = 0; a < 3; ++a)
+      if (hi[a] - lo[a] > rb->ext[a] - 1) return 0;
+  }
+  return 1;
+}
+
+/*
  * One set: rows[tau] voxel indices.  Slot k is a masked key iff k > 0 and
  * rows[k] == rows[k-1].  Z[tau][C] receives the projected attention output of
  * every slot; keep[k] says whether slot k is a non-duplicate.
  */
 static void ref_attend_one_set(const double* feats, const double* pe, int C, const int32_t* rows, int tau,
                                const double* W_qkv, const double* b_qkv, const double* W_o, const double* b_o,
-                               int heads, double* Z, int* keep, double* work) {
+                               int heads, const ref_rel_bias* rb, double* Z, int* keep, double* work) {
   const int d = C / heads;
   double* Q = work;                       /* [tau][C] */
   double* K = Q + (size_t)tau * C;        /* [tau][C] */
@@ -229,6 +273,7 @@ static void ref_attend_one_set(const double* feats, const double* pe, int C, con
         double s = 0.0;
         for (int c = 0; c < d; ++c) s += Q[(size_t)a * C + h * d + c] * K[(size_t)b * C + h * d + c];
         logit[b] = s * scale;
+        if (rb) logit[b] += rb->table[(size_t)h * ref_rel_bias_len(rb) + ref_rel_bias_index(rb, rows[a], rows[b])];
         if (logit[b] > mx) mx = logit[b];
       }
       double den = 0.0;
@@ -252,12 +297,22 @@ static size_t ref_attend_work_doubles(int tau, int C) { return (size_t)4 * tau *
  * table row.  Rows of `out` for voxels in no table row are left untouched.
  * `covered` (optional, int32[n]) is set to 1 for written voxels.
  */
-int dsvt_ref_set_attention(const double* feats, int32_t n, int32_t C, const int32_t* set_table, int32_t num_sets,
-                           int32_t set_size, const double* W_qkv, const double* b_qkv, const double* W_o,
-                           const double* b_o, int32_t heads, const double* pe, double* out, int32_t* covered) {
+int dsvt_ref_set_attention_rpb(const double* feats, int32_t n, int32_t C, const int32_t* set_table,
+                               int32_t num_sets, int32_t set_size, const double* W_qkv, const double* b_qkv,
+                               const double* W_o, const double* b_o, int32_t heads, const double* pe,
+                               const double* rpb, const int32_t* coords, const int32_t* rpb_extent, double* out,
+                               int32_t* covered) {
   if (n < 0 || C < 1 || heads < 1 || C % heads != 0 || set_size < 1 || num_sets < 0) return REF_ERR_ARG;
   for (int64_t i = 0; i < (int64_t)num_sets * set_size; ++i)
     if (set_table[i] < 0 || set_table[i] >= n) return REF_ERR_BAD_INPUT;
+  ref_rel_bias rbv, *rb = NULL;
+  if (rpb) {
+    if (!coords || !rpb_extent || rpb_extent[0] < 1 || rpb_extent[1] < 1 || rpb_extent[2] < 1) return REF_ERR_ARG;
+    rbv.table = rpb; rbv.coords = coords;
+    rbv.ext[0] = rpb_extent[0]; rbv.ext[1] = rpb_extent[1]; rbv.ext[2] = rpb_extent[2];
+    if (!ref_rel_bias_covers(&rbv, set_table, num_sets, set_size)) return REF_ERR_BAD_INPUT;
+    rb = &rbv;
+  }
   int s;
 #pragma omp parallel for schedule(dynamic, 4) num_threads(g_threads)
   for (s = 0; s < num_sets; ++s) {
@@ -266,7 +321,7 @@ int dsvt_ref_set_attention(const double* feats, int32_t n, int32_t C, const int3
     int* keep = (int*)malloc(sizeof(int) * (size_t)tau);
     double* Z = work + ref_attend_work_doubles(tau, C);
     const int32_t* rows = set_table + (size_t)s * tau;
-    ref_attend_one_set(feats, pe, C, rows, tau, W_qkv, b_qkv, W_o, b_o, heads, Z, keep, work);
+    ref_attend_one_set(feats, pe, C, rows, tau, W_qkv, b_qkv, W_o, b_o, heads, rb, Z, keep, work);
     for (int k = 0; k < tau; ++k)
       if (keep[k]) {
         memcpy(out + (size_t)rows[k] * C, Z + (size_t)k * C, sizeof(double) * (size_t)C);
@@ -276,6 +331,13 @@ int dsvt_ref_set_attention(const double* feats, int32_t n, int32_t C, const int3
     free(keep);
   }
   return REF_OK;
+}
+
+int dsvt_ref_set_attention(const double* feats, int32_t n, int32_t C, const int32_t* set_table, int32_t num_sets,
+                           int32_t set_size, const double* W_qkv, const double* b_qkv, const double* W_o,
+                           const double* b_o, int32_t heads, const double* pe, double* out, int32_t* covered) {
+  return dsvt_ref_set_attention_rpb(feats, n, C, set_table, num_sets, set_size, W_qkv, b_qkv, W_o, b_o, heads, pe,
+                                    NULL, NULL, NULL, out, covered);
 }
 
 /* ------------------------------------------------------------------ */
@@ -291,6 +353,9 @@ typedef struct {
   const double *ln1_g, *ln1_b; /* NULL gain: no LayerNorm after the attention */
   const double *ln2_g, *ln2_b; /* NULL gain: no LayerNorm after the MLP */
   const double* pe;            /* [n][C] or NULL */
+  const double* rpb;           /* relative position bias [heads][(2L-1)(2W-1)(2H-1)] or NULL */
+  const int32_t* coords;       /* [n][4], read when rpb is given */
+  int32_t rpb_extent[3];       /* L, W, H */
 } dsvt_ref_layer_params;
 
 /* LayerNorm over C channels, biased variance. */
@@ -317,8 +382,8 @@ int dsvt_ref_layer(const double* x, int32_t n, const int32_t* set_table, int32_t
   const int C = p->C, Hd = p->hidden;
   double* Z = (double*)calloc((size_t)(n > 0 ? n : 1) * C, sizeof(double));
   int32_t* covered = (int32_t*)calloc((size_t)(n > 0 ? n : 1), sizeof(int32_t));
-  int rc = dsvt_ref_set_attention(x, n, C, set_table, num_sets, p->set_size, p->W_qkv, p->b_qkv, p->W_o, p->b_o,
-                                  p->heads, p->pe, Z, covered);
+  int rc = dsvt_ref_set_attention_rpb(x, n, C, set_table, num_sets, p->set_size, p->W_qkv, p->b_qkv, p->W_o, p->b_o,
+                                      p->heads, p->pe, p->rpb, p->coords, p->rpb_extent, Z, covered);
   if (rc != REF_OK) { free(Z); free(covered); return rc; }
   int i;
 #pragma omp parallel for schedule(static) num_threads(g_threads)
@@ -491,4 +556,39 @@ int dsvt_ref_pool(const int32_t* coords, const double* feats, int32_t n, int32_t
   free(slot);
   free(rstart);
   return bad ? REF_ERR_BAD_INPUT : REF_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* BEV projection (Sec. 3.1: the backbone's voxel features are         */
+/* projected to a bird's-eye-view feature map)                         */
+/* ------------------------------------------------------------------ */
+/*
+ * Dense map of the grid's (x, y) plane; the z cells of a column are stacked into channels:
+ * channel c*Z + z of cell (b, y, x) = feats[i][c] of the voxel i at (b, x, y, z); cells without a voxel are 0.
+ * channels_last == 0: out[b][c*Z + z][y][x]  (the image's rows run along y, its columns along x);
+ * channels_last == 1: out[b][y][x][c*Z + z].
+ * Two voxels in one cell are an input error.
+ */
+int dsvt_ref_bev_scatter(const int32_t* coords, const double* feats, int32_t n, int32_t C, int32_t batch,
+                         const int32_t* grid, int32_t channels_last, double* out) {
+  if (n < 0 || C < 1 || batch < 1 || grid[0] < 1 || grid[1] < 1 || grid[2] < 1) return REF_ERR_ARG;
+  const int64_t X = grid[0], Y = grid[1], Z = grid[2], CH = (int64_t)C * Z;
+  const int64_t total = (int64_t)batch * CH * Y * X;
+  unsigned char* seen = (unsigned char*)calloc((size_t)((int64_t)batch * X * Y * Z), 1);
+  for (int64_t i = 0; i < total; ++i) out[i] = 0.0;
+  for (int32_t i = 0; i < n; ++i) {
+    const int64_t b = coords[4 * (size_t)i], x = coords[4 * (size_t)i + 1], y = coords[4 * (size_t)i + 2],
+                  z = coords[4 * (size_t)i + 3];
+    if (b < 0 || b >= batch || x < 0 || x >= X || y < 0 || y >= Y || z < 0 || z >= Z) { free(seen); return REF_ERR_BAD_INPUT; }
+    const int64_t cell = ((b * X + x) * Y + y) * Z + z;
+    if (seen[cell]) { free(seen); return REF_ERR_BAD_INPUT; }
+    seen[cell] = 1;
+    for (int64_t c = 0; c < C; ++c) {
+      const int64_t ch = c * Z + z;
+      const int64_t o = channels_last ? ((b * Y + y) * X + x) * CH + ch : ((b * CH + ch) * Y + y) * X + x;
+      out[o] = feats[(size_t)i * C + c];
+    }
+  }
+  free(seen);
+  return REF_OK;
 }

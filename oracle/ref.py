@@ -121,8 +121,18 @@ def partition(coords, batch, grid, window, set_size, axis, cap_sets: Optional[in
     return Partition(table[: ns[0]].copy(), perm[:n].copy(), ws, wc[:nw].copy(), wo)
 
 
-def set_attention(feats, set_table, W_qkv, b_qkv, W_o, b_o, heads, pe=None, out=None):
-    """Returns (out [n, C] float64, covered [n] int32)."""
+def rel_bias_len(extent) -> int:
+    """Entries per head of a relative position bias table for windows of extent (L, W, H)."""
+    L, W, H = (int(v) for v in extent)
+    return (2 * L - 1) * (2 * W - 1) * (2 * H - 1)
+
+
+def set_attention(feats, set_table, W_qkv, b_qkv, W_o, b_o, heads, pe=None, out=None, rpb=None, coords=None,
+                  rpb_extent=None):
+    """Returns (out [n, C] float64, covered [n] int32).
+
+    rpb: optional relative position bias [heads, rel_bias_len(rpb_extent)], added to the scaled logits and indexed
+    by coords[query] - coords[key]; needs coords [n, 4] and rpb_extent = (L, W, H)."""
     feats = _f64(feats)
     n, Cc = feats.shape
     table = _i32(set_table)
@@ -130,13 +140,19 @@ def set_attention(feats, set_table, W_qkv, b_qkv, W_o, b_o, heads, pe=None, out=
     out = np.zeros((n, Cc), dtype=np.float64) if out is None else out
     covered = np.zeros(max(n, 1), dtype=np.int32)
     Wq, bq, Wo, bo, pe = _f64(W_qkv), _f64(b_qkv), _f64(W_o), _f64(b_o), _f64(pe)
-    rc = lib().dsvt_ref_set_attention(
+    rpb = _f64(rpb)
+    cc = None if rpb is None else _i32(coords).reshape(-1, 4)
+    ext = None if rpb is None else _i32(rpb_extent)
+    if rpb is not None and rpb.shape != (heads, rel_bias_len(ext)):
+        raise ValueError("rpb must be [heads, (2L-1)(2W-1)(2H-1)]")
+    rc = lib().dsvt_ref_set_attention_rpb(
         _p(feats, C.c_double), C.c_int32(n), C.c_int32(Cc), _p(table, C.c_int32), C.c_int32(S), C.c_int32(tau),
         _p(Wq, C.c_double), _p(bq, C.c_double), _p(Wo, C.c_double), _p(bo, C.c_double), C.c_int32(heads),
-        _p(pe, C.c_double), _p(out, C.c_double), _p(covered, C.c_int32),
+        _p(pe, C.c_double), _p(rpb, C.c_double), _p(cc, C.c_int32), _p(ext, C.c_int32), _p(out, C.c_double),
+        _p(covered, C.c_int32),
     )
     if rc != 0:
-        raise ValueError("dsvt_ref_set_attention rc=%d" % rc)
+        raise ValueError("dsvt_ref_set_attention_rpb rc=%d" % rc)
     return out, covered[:n]
 
 
@@ -151,14 +167,16 @@ class _LayerParams(C.Structure):
         ("ln1_g", C.POINTER(C.c_double)), ("ln1_b", C.POINTER(C.c_double)),
         ("ln2_g", C.POINTER(C.c_double)), ("ln2_b", C.POINTER(C.c_double)),
         ("pe", C.POINTER(C.c_double)),
+        ("rpb", C.POINTER(C.c_double)), ("coords", C.POINTER(C.c_int32)), ("rpb_extent", C.c_int32 * 3),
     ]
 
 
 _WEIGHT_KEYS = ["W_qkv", "b_qkv", "W_o", "b_o", "W_1", "b_1", "W_2", "b_2", "ln1_g", "ln1_b", "ln2_g", "ln2_b"]
 
 
-def _pack_layer(layer: dict, set_size: int, pe=None):
-    """layer: dict with C, heads, hidden, ln_eps and the arrays of _WEIGHT_KEYS (None allowed)."""
+def _pack_layer(layer: dict, set_size: int, pe=None, coords=None):
+    """layer: dict with C, heads, hidden, ln_eps and the arrays of _WEIGHT_KEYS (None allowed); optional "rpb"
+    [heads, rel_bias_len(rpb_extent)] with "rpb_extent" = (L, W, H), which needs coords [n, 4]."""
     keep = {}
     p = _LayerParams()
     p.C, p.heads, p.hidden, p.set_size = int(layer["C"]), int(layer["heads"]), int(layer.get("hidden", 0)), int(set_size)
@@ -169,14 +187,25 @@ def _pack_layer(layer: dict, set_size: int, pe=None):
         setattr(p, k, _p(a, C.c_double))
     keep["pe"] = _f64(pe)
     p.pe = _p(keep["pe"], C.c_double)
+    keep["rpb"] = _f64(layer.get("rpb"))
+    if keep["rpb"] is not None:
+        if coords is None:
+            raise ValueError("a layer with a relative position bias needs coords")
+        ext = [int(v) for v in layer["rpb_extent"]]
+        if keep["rpb"].shape != (p.heads, rel_bias_len(ext)):
+            raise ValueError("rpb must be [heads, (2L-1)(2W-1)(2H-1)]")
+        keep["coords"] = _i32(coords).reshape(-1, 4)
+        p.rpb = _p(keep["rpb"], C.c_double)
+        p.coords = _p(keep["coords"], C.c_int32)
+        p.rpb_extent = (C.c_int32 * 3)(*ext)
     return p, keep
 
 
-def layer(x, set_table, layer_params: dict, pe=None):
+def layer(x, set_table, layer_params: dict, pe=None, coords=None):
     x = _f64(x)
     n, Cc = x.shape
     table = _i32(set_table)
-    p, keep = _pack_layer(layer_params, table.shape[1], pe)
+    p, keep = _pack_layer(layer_params, table.shape[1], pe, coords)
     y = np.zeros_like(x)
     rc = lib().dsvt_ref_layer(_p(x, C.c_double), C.c_int32(n), _p(table, C.c_int32), C.c_int32(table.shape[0]),
                               C.byref(p), _p(y, C.c_double))
@@ -185,7 +214,7 @@ def layer(x, set_table, layer_params: dict, pe=None):
     return y
 
 
-def block(x, table0, table1, layers, pe=None):
+def block(x, table0, table1, layers, pe=None, coords=None):
     """layers: sequence of two layer dicts (X-axis layer, Y-axis layer)."""
     x = _f64(x)
     n, Cc = x.shape
@@ -193,7 +222,7 @@ def block(x, table0, table1, layers, pe=None):
     arr = (_LayerParams * 2)()
     keeps = []
     for i in range(2):
-        p, keep = _pack_layer(layers[i], t0.shape[1], pe)
+        p, keep = _pack_layer(layers[i], t0.shape[1], pe, coords)
         arr[i] = p
         keeps.append(keep)
     y = np.zeros_like(x)
@@ -233,3 +262,20 @@ def pool(coords, feats, batch, grid, pool_shape, W_q, W_k, W_v, W_o, b_q, b_k, b
     if rc != 0:
         raise ValueError("dsvt_ref_pool rc=%d" % rc)
     return Pooled(oc[: m[0]].copy(), of[: m[0]].copy(), reg[:n].copy(), slot[:n].copy())
+
+
+def bev_scatter(coords, feats, batch, grid, channels_last=False) -> np.ndarray:
+    """Dense bird's-eye-view map: [batch, C*Z, Y, X] (or [batch, Y, X, C*Z] when channels_last), zeros where no voxel."""
+    coords = _i32(coords).reshape(-1, 4)
+    feats = _f64(feats)
+    n, Cc = feats.shape
+    g = _i32(grid)
+    X, Y, Z = (int(v) for v in g)
+    shape = (batch, Y, X, Cc * Z) if channels_last else (batch, Cc * Z, Y, X)
+    out = np.empty(shape, dtype=np.float64)
+    rc = lib().dsvt_ref_bev_scatter(_p(coords, C.c_int32), _p(feats, C.c_double), C.c_int32(n), C.c_int32(Cc),
+                                    C.c_int32(batch), _p(g, C.c_int32), C.c_int32(1 if channels_last else 0),
+                                    _p(out, C.c_double))
+    if rc != 0:
+        raise ValueError("dsvt_ref_bev_scatter rc=%d" % rc)
+    return out
