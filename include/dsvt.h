@@ -3,7 +3,8 @@
  *
  * The library implements the hot path of the DSVT 3D backbone (arXiv 2301.06051):
  * rotated set partitioning (Sec. 3.2, Eq. 1-3), batched set attention (Eq. 4-5), the DSVT
- * layer and block (Eq. 5, Appendix B.1.1) and the attention-style 3D pooling (Eq. 6-7).
+ * layer and block (Eq. 5, Appendix B.1.1), the attention-style 3D pooling (Eq. 6-7) and the
+ * projection of the voxel features to a bird's-eye-view map (Sec. 3.1).
  *
  * Conventions that hold for every call unless a comment says otherwise:
  *   - Every data pointer is a DEVICE pointer owned by the caller.  The library reads / writes it
@@ -203,6 +204,17 @@ int dsvt_set_attention(dsvt_ctx* ctx, const float* feats, int32_t n, int32_t C, 
                        const void* W_qkv, const float* b_qkv, const void* W_o, const float* b_o, int32_t heads,
                        const float* pe, int precision, float* out);
 
+/*
+ * dsvt_set_attention with a relative position bias on the logits (see dsvt_layer_params for the
+ * table layout and the meaning of rpb, coords and rpb_extent; rpb_extent is a HOST pointer).
+ * rpb == NULL gives dsvt_set_attention exactly.
+ */
+int dsvt_set_attention_rpb(dsvt_ctx* ctx, const float* feats, int32_t n, int32_t C, const int32_t* set_table,
+                           int32_t cap_sets, const int32_t* num_sets, const int32_t* set_rowoff, int32_t set_size,
+                           const void* W_qkv, const float* b_qkv, const void* W_o, const float* b_o, int32_t heads,
+                           const float* pe, const float* rpb, const int32_t* coords, const int32_t rpb_extent[3],
+                           int precision, float* out);
+
 /* Parameters of one DSVT layer (Appendix B.1.1).  hidden == 0 drops the MLP; ln1_g == NULL /
  * ln2_g == NULL drops the corresponding LayerNorm.  hidden <= 2C. */
 typedef struct dsvt_layer_params {
@@ -215,6 +227,16 @@ typedef struct dsvt_layer_params {
   const float *b_qkv, *b_o, *b_1, *b_2;       /* each may be NULL (= 0) */
   const float *ln1_g, *ln1_b, *ln2_g, *ln2_b; /* float [C]; *_b may be NULL */
   const float* pe;                            /* float [n][C] or NULL */
+  /* Relative position bias, the Swin transformer's mechanism that the text after Eq. 5 names for
+   * PE(.): rpb float [heads][(2L-1)(2W-1)(2H-1)] or NULL.  The scaled logit of (query, key) in head
+   * h gets rpb[h][((dx+L-1)(2W-1) + (dy+W-1))(2H-1) + (dz+H-1)] added, with (dx, dy, dz) =
+   * coords[query] - coords[key].  coords: int32 [n][4] = (b, x, y, z), required with rpb.
+   * rpb_extent = (L, W, H): the window extent the table covers, at least the window the set
+   * table was cut with.  A set whose members are spread wider raises DSVT_STATUS_BAD_INDEX and
+   * its out-of-table pairs read a clamped entry. */
+  const float* rpb;
+  const int32_t* coords;
+  int32_t rpb_extent[3];
 } dsvt_layer_params;
 
 /*
@@ -256,6 +278,24 @@ int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feats, int32_t 
               const void* W_o, const float* b_q, const float* b_k, const float* b_v, const float* b_o,
               const float* slot_pe, int32_t heads, int32_t mask_empty, int precision, int32_t* out_coords,
               float* out_feats, int32_t cap_m, int32_t* num_out, int32_t* region_of, int32_t* slot_of);
+
+/*
+ * Projection of the backbone's voxel features to a dense bird's-eye-view map (Sec. 3.1).  The z
+ * cells of a column are stacked into channels: channel c*Z + z of cell (b, y, x) is feats[i][c] of
+ * the voxel i at (b, x, y, z), and 0 where the grid holds no voxel; (X, Y, Z) = grid.
+ *
+ *   coords  int32 [n][4] = (b, x, y, z); feats float [n][C], 16-byte aligned, C % 4 == 0.
+ *   out     float, 16-byte aligned, written in full:
+ *           channels_last == 0: [batch][C*Z][Y][X] (rows of the image run along y, columns along x);
+ *           channels_last == 1: [batch][Y][X][C*Z].
+ *
+ * A voxel outside the grid is skipped with DSVT_STATUS_BAD_COORD; of two voxels in one cell one is
+ * kept and DSVT_STATUS_DUPLICATE_CELL is raised.  batch*X*Y*Z must be below 2^31.  The call may
+ * grow the context's dense cell map (one cudaMalloc, after a stream synchronise) the first time a
+ * grid of that size is seen.
+ */
+int dsvt_bev_scatter(dsvt_ctx* ctx, const int32_t* coords, const float* feats, int32_t n, int32_t C, int32_t batch,
+                     const int32_t grid[3], int32_t channels_last, float* out);
 
 #ifdef __cplusplus
 }

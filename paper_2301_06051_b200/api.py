@@ -23,7 +23,8 @@ STATUS_BAD_COORD, STATUS_TABLE_OVERFLOW, STATUS_BAD_INDEX, STATUS_DUPLICATE_CELL
 
 EXPORTS = [
     "dsvt_create", "dsvt_destroy", "dsvt_status_sync", "dsvt_last_cuda_error", "dsvt_error_string",
-    "dsvt_launch_count", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_layer", "dsvt_block", "dsvt_pool",
+    "dsvt_launch_count", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_set_attention_rpb", "dsvt_layer", "dsvt_block", "dsvt_pool",
+    "dsvt_bev_scatter",
 ]
 
 _lib = None
@@ -45,6 +46,7 @@ class LayerParams(C.Structure):
         ("b_qkv", C.c_void_p), ("b_o", C.c_void_p), ("b_1", C.c_void_p), ("b_2", C.c_void_p),
         ("ln1_g", C.c_void_p), ("ln1_b", C.c_void_p), ("ln2_g", C.c_void_p), ("ln2_b", C.c_void_p),
         ("pe", C.c_void_p),
+        ("rpb", C.c_void_p), ("coords", C.c_void_p), ("rpb_extent", C.c_int32 * 3),
     ]
 
 
@@ -71,6 +73,9 @@ def load():
     lib.dsvt_partition_shifted.argtypes = [vp, vp, i32, i32, p3, p3, p3, i32, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.dsvt_partition_noalloc.argtypes = [vp, vp, i32, i32, p3, p3, i32, i32, vp, i32, vp, vp, vp, C.POINTER(i32)]
     lib.dsvt_set_attention.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, i32, vp, vp, vp, vp, i32, vp, C.c_int, vp]
+    lib.dsvt_set_attention_rpb.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, p3,
+                                           C.c_int, vp]
+    lib.dsvt_bev_scatter.argtypes = [vp, vp, vp, i32, i32, i32, p3, i32, vp]
     lib.dsvt_layer.argtypes = [vp, vp, i32, vp, i32, vp, vp, C.POINTER(LayerParams), vp]
     lib.dsvt_block.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, i32, vp, vp, C.POINTER(LayerParams), vp]
     lib.dsvt_pool.argtypes = [vp, vp, vp, i32, i32, i32, p3, p3, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32,
@@ -98,7 +103,7 @@ def device_weights(layer: Dict, precision: int, device) -> Dict:
     the chosen precision expects: matrices float32 or bfloat16, everything else float32."""
     import numpy as np
 
-    out: Dict = {k: layer[k] for k in ("C", "heads", "hidden") if k in layer}
+    out: Dict = {k: layer[k] for k in ("C", "heads", "hidden", "rpb_extent") if k in layer}
     out["ln_eps"] = float(layer.get("ln_eps", 1e-5))
     out["precision"] = precision
     for k, v in layer.items():
@@ -113,7 +118,10 @@ def device_weights(layer: Dict, precision: int, device) -> Dict:
     return out
 
 
-def layer_params(w: Dict, set_size: int, pe: Optional[torch.Tensor] = None) -> LayerParams:
+def layer_params(w: Dict, set_size: int, pe: Optional[torch.Tensor] = None,
+                 coords: Optional[torch.Tensor] = None) -> LayerParams:
+    """w may hold "rpb" (float tensor [heads, (2L-1)(2W-1)(2H-1)]) and "rpb_extent" = (L, W, H); then coords
+    (int32 [n, 4]) is required."""
     p = LayerParams()
     p.C, p.heads, p.hidden, p.set_size = int(w["C"]), int(w["heads"]), int(w.get("hidden", 0)), int(set_size)
     p.precision = int(w["precision"])
@@ -121,6 +129,12 @@ def layer_params(w: Dict, set_size: int, pe: Optional[torch.Tensor] = None) -> L
     for k in ("W_qkv", "W_o", "W_1", "W_2", "b_qkv", "b_o", "b_1", "b_2", "ln1_g", "ln1_b", "ln2_g", "ln2_b"):
         setattr(p, k, _ptr(w.get(k)))
     p.pe = _ptr(pe)
+    if w.get("rpb") is not None:
+        if coords is None:
+            raise ValueError("a layer with a relative position bias needs coords")
+        p.rpb = _ptr(w["rpb"])
+        p.coords = _ptr(coords)
+        p.rpb_extent = _i3(w["rpb_extent"])
     return p
 
 
@@ -258,8 +272,17 @@ class Context:
 
     # ---- dsvt_set_attention ----
     def set_attention(self, feats: torch.Tensor, table: SetTable, w: Dict, out: torch.Tensor,
-                      pe: Optional[torch.Tensor] = None, use_rowoff: bool = True) -> torch.Tensor:
+                      pe: Optional[torch.Tensor] = None, use_rowoff: bool = True,
+                      coords: Optional[torch.Tensor] = None) -> torch.Tensor:
         n, Cc = int(feats.shape[0]), int(feats.shape[1])
+        if w.get("rpb") is not None:  # dsvt_set_attention_rpb
+            rc = self.lib.dsvt_set_attention_rpb(
+                self._h, _ptr(feats), n, Cc, _ptr(table.set_table), table.cap_sets, _ptr(table.num_sets),
+                _ptr(table.set_rowoff) if use_rowoff else None, table.set_size, _ptr(w["W_qkv"]), _ptr(w.get("b_qkv")),
+                _ptr(w["W_o"]), _ptr(w.get("b_o")), int(w["heads"]), _ptr(pe), _ptr(w["rpb"]), _ptr(coords),
+                _i3(w["rpb_extent"]), int(w["precision"]), _ptr(out))
+            self._check(rc, "dsvt_set_attention_rpb")
+            return out
         rc = self.lib.dsvt_set_attention(self._h, _ptr(feats), n, Cc, _ptr(table.set_table), table.cap_sets,
                                          _ptr(table.num_sets), _ptr(table.set_rowoff) if use_rowoff else None,
                                          table.set_size, _ptr(w["W_qkv"]), _ptr(w.get("b_qkv")), _ptr(w["W_o"]),
@@ -269,8 +292,8 @@ class Context:
 
     # ---- dsvt_layer ----
     def layer(self, x: torch.Tensor, table: SetTable, w: Dict, y: torch.Tensor, pe: Optional[torch.Tensor] = None,
-              use_rowoff: bool = True) -> torch.Tensor:
-        p = layer_params(w, table.set_size, pe)
+              use_rowoff: bool = True, coords: Optional[torch.Tensor] = None) -> torch.Tensor:
+        p = layer_params(w, table.set_size, pe, coords)
         rc = self.lib.dsvt_layer(self._h, _ptr(x), int(x.shape[0]), _ptr(table.set_table), table.cap_sets,
                                  _ptr(table.num_sets), _ptr(table.set_rowoff) if use_rowoff else None, C.byref(p),
                                  _ptr(y))
@@ -279,13 +302,29 @@ class Context:
 
     # ---- dsvt_block ----
     def block(self, x: torch.Tensor, t0: SetTable, t1: SetTable, ws: Sequence[Dict], y: torch.Tensor,
-              pe: Optional[torch.Tensor] = None) -> torch.Tensor:
-        arr = (LayerParams * 2)(layer_params(ws[0], t0.set_size, pe), layer_params(ws[1], t1.set_size, pe))
+              pe: Optional[torch.Tensor] = None, coords: Optional[torch.Tensor] = None) -> torch.Tensor:
+        arr = (LayerParams * 2)(layer_params(ws[0], t0.set_size, pe, coords),
+                                layer_params(ws[1], t1.set_size, pe, coords))
         rc = self.lib.dsvt_block(self._h, _ptr(x), int(x.shape[0]), _ptr(t0.set_table), t0.cap_sets,
                                  _ptr(t0.num_sets), _ptr(t0.set_rowoff), _ptr(t1.set_table), t1.cap_sets,
                                  _ptr(t1.num_sets), _ptr(t1.set_rowoff), arr, _ptr(y))
         self._check(rc, "dsvt_block")
         return y
+
+    # ---- dsvt_bev_scatter ----
+    def bev_scatter(self, coords: torch.Tensor, feats: torch.Tensor, batch: int, grid, channels_last: bool = False,
+                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Dense BEV map [batch, C*Z, Y, X] (or [batch, Y, X, C*Z] when channels_last), written in full."""
+        n, Cc = int(feats.shape[0]), int(feats.shape[1])
+        X, Y, Z = (int(v) for v in grid)
+        shape = (batch, Y, X, Cc * Z) if channels_last else (batch, Cc * Z, Y, X)
+        if out is None:
+            out = torch.empty(shape, dtype=torch.float32, device=self.device)
+        assert tuple(out.shape) == shape and out.dtype == torch.float32
+        rc = self.lib.dsvt_bev_scatter(self._h, _ptr(coords), _ptr(feats), n, Cc, int(batch), _i3(grid),
+                                       1 if channels_last else 0, _ptr(out))
+        self._check(rc, "dsvt_bev_scatter")
+        return out
 
     # ---- dsvt_pool ----
     def pool(self, coords: torch.Tensor, feats: torch.Tensor, batch: int, grid, pool_shape, w: Dict,

@@ -57,9 +57,18 @@ int check_layer_shape(const dsvt_ctx* ctx, const dsvt_layer_params& p, bool atte
     if (p.hidden % 8 != 0 || p.hidden > 2 * p.C) return DSVT_ERR_UNSUPPORTED;
   }
   if (p.C > ctx->max_channels) return DSVT_ERR_CAPACITY;
-  const void* ptrs[] = {p.W_qkv, p.W_o, p.W_1, p.W_2, p.b_qkv, p.b_o, p.b_1, p.b_2, p.pe};
+  const void* ptrs[] = {p.W_qkv, p.W_o, p.W_1, p.W_2, p.b_qkv, p.b_o, p.b_1, p.b_2, p.pe, p.coords};
   for (const void* q : ptrs)
     if (((uintptr_t)q & 15) != 0) return DSVT_ERR_INVALID_ARG;
+  if (p.rpb) {
+    if (!p.coords || ((uintptr_t)p.rpb & 3) != 0) return DSVT_ERR_INVALID_ARG;
+    int64_t len = p.heads;
+    for (int a = 0; a < 3; ++a) {
+      if (p.rpb_extent[a] < 1 || p.rpb_extent[a] > (1 << 12)) return DSVT_ERR_INVALID_ARG;
+      len *= 2 * p.rpb_extent[a] - 1;
+      if (len >= (1ll << 30)) return DSVT_ERR_UNSUPPORTED;
+    }
+  }
   return DSVT_OK;
 }
 
@@ -182,12 +191,27 @@ extern "C" int dsvt_set_attention(dsvt_ctx* ctx, const float* feats, int32_t n, 
                                   int32_t cap_sets, const int32_t* num_sets, const int32_t* set_rowoff,
                                   int32_t set_size, const void* W_qkv, const float* b_qkv, const void* W_o,
                                   const float* b_o, int32_t heads, const float* pe, int precision, float* out) {
+  return dsvt_set_attention_rpb(ctx, feats, n, C, set_table, cap_sets, num_sets, set_rowoff, set_size, W_qkv, b_qkv,
+                                W_o, b_o, heads, pe, nullptr, nullptr, nullptr, precision, out);
+}
+
+extern "C" int dsvt_set_attention_rpb(dsvt_ctx* ctx, const float* feats, int32_t n, int32_t C,
+                                      const int32_t* set_table, int32_t cap_sets, const int32_t* num_sets,
+                                      const int32_t* set_rowoff, int32_t set_size, const void* W_qkv,
+                                      const float* b_qkv, const void* W_o, const float* b_o, int32_t heads,
+                                      const float* pe, const float* rpb, const int32_t* coords,
+                                      const int32_t rpb_extent[3], int precision, float* out) {
   int rc = check_common(ctx, feats, out, n, set_table, cap_sets, num_sets);
   if (rc != DSVT_OK) return rc;
   if (n > 0 && feats == out) return DSVT_ERR_INVALID_ARG;
   dsvt_layer_params p = {};
   p.C = C; p.heads = heads; p.hidden = 0; p.set_size = set_size; p.precision = precision; p.ln_eps = 0.f;
   p.W_qkv = W_qkv; p.W_o = W_o; p.b_qkv = b_qkv; p.b_o = b_o; p.pe = pe;
+  if (rpb) {
+    if (!rpb_extent) return DSVT_ERR_INVALID_ARG;
+    p.rpb = rpb; p.coords = coords;
+    for (int a = 0; a < 3; ++a) p.rpb_extent[a] = rpb_extent[a];
+  }
   rc = check_layer_shape(ctx, p, true);
   if (rc != DSVT_OK) return rc;
   return run_layer(ctx, feats, n, set_table, cap_sets, num_sets, set_rowoff, p, out, true, ctx->rowoff_a);

@@ -12,6 +12,8 @@
 #include "dsvt_common.cuh"
 #include "fma_tile.cuh"
 
+#include <limits.h>
+
 namespace {
 using namespace dsvt_fma;
 
@@ -20,6 +22,8 @@ struct FmaGeom {
   int TMn;   // nominal rows per tile: a set belongs to the tile its first row falls in
   int LDQ;   // row stride of the wide buffer (>= 3C, LDQ % 32 == 4)
   int C, hidden, heads, d, tau;
+  // relative position bias: entries per head, strides of the x and y offsets, index of the zero offset
+  int rb_len, rb_sx, rb_sy, rb_centre;
 };
 
 // row[c] = LN(row[c] + add[c]) (gain g == NULL: plain sum).  One warp per row; result left in `row`
@@ -59,6 +63,7 @@ layer_fma_kernel(dsvt_fused_args a, FmaGeom g, int32_t* __restrict__ status) {
   int* rowvox = reinterpret_cast<int*>(pbuf + kWarps * 128);  // [TM]
   int* set_lo = rowvox + TM;                                   // [TM + 1]
   int* misc = set_lo + TM + 1;                                 // [4]
+  int* rowlin = misc + 4;                                      // [TM] bias: x * rb_sx + y * rb_sy + z of each row
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const dsvt_layer_params& p = a.p;
   const WT* Wqkv = reinterpret_cast<const WT*>(p.W_qkv);
@@ -127,6 +132,31 @@ layer_fma_kernel(dsvt_fused_args a, FmaGeom g, int32_t* __restrict__ status) {
     const int rm_used = (rows + 15) >> 4;
     const int rows_pad = rm_used << 4;
     const int C4 = C >> 2;
+    if (p.rpb) {
+      // The bias index is linear in the offset, so one integer per row serves every (query, key) pair.  A set
+      // spread wider than the table's extent is reported.
+      for (int si = warp; si < nsets; si += kWarps) {
+        int lo[3] = {INT_MAX, INT_MAX, INT_MAX}, hi[3] = {INT_MIN, INT_MIN, INT_MIN};
+        for (int r = set_lo[si] + lane; r < set_lo[si + 1]; r += 32) {
+          const int v = rowvox[r];
+          int4 c = make_int4(0, 0, 0, 0);
+          if (v >= 0) {
+            c = __ldg(reinterpret_cast<const int4*>(p.coords) + v);
+            lo[0] = min(lo[0], c.y); hi[0] = max(hi[0], c.y);
+            lo[1] = min(lo[1], c.z); hi[1] = max(hi[1], c.z);
+            lo[2] = min(lo[2], c.w); hi[2] = max(hi[2], c.w);
+          }
+          rowlin[r] = c.y * g.rb_sx + c.z * g.rb_sy + c.w;
+        }
+        bool wide = false;
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+          const int l = -warp_max_int(-lo[q]), h = warp_max_int(hi[q]);
+          wide |= (h >= l) && (h - l > p.rpb_extent[q] - 1);
+        }
+        if (wide && lane == 0) atomicOr(status, DSVT_STATUS_BAD_INDEX);
+      }
+    }
     auto gather = [&](bool with_pe) {
       for (int r = warp; r < rows_pad; r += kWarps) {
         const int v = r < rows ? rowvox[r] : -1;
@@ -166,6 +196,7 @@ layer_fma_kernel(dsvt_fused_args a, FmaGeom g, int32_t* __restrict__ status) {
         const float* Qb = Bs + (size_t)r0 * LDQ + h * d;
         const float* Kb = Qb + C;
         const float* Vb = Qb + 2 * C;
+        const float* bias = p.rpb ? p.rpb + (size_t)h * g.rb_len : nullptr;
         for (int qa = 0; qa < m; ++qa) {
           const float4* q4 = reinterpret_cast<const float4*>(Qb + (size_t)qa * LDQ);
           float lg[4];
@@ -182,6 +213,10 @@ layer_fma_kernel(dsvt_fused_args a, FmaGeom g, int32_t* __restrict__ status) {
                 s = fmaf(qv.x, kv.x, s); s = fmaf(qv.y, kv.y, s); s = fmaf(qv.z, kv.z, s); s = fmaf(qv.w, kv.w, s);
               }
               lg[u] = s * scale;
+              if (bias) {
+                const int idx = rowlin[r0 + qa] - rowlin[r0 + kb] + g.rb_centre;
+                lg[u] += __ldg(bias + min(max(idx, 0), g.rb_len - 1));
+              }
               mx = fmaxf(mx, lg[u]);
             }
           }
@@ -245,7 +280,7 @@ layer_fma_kernel(dsvt_fused_args a, FmaGeom g, int32_t* __restrict__ status) {
 
 size_t fma_smem_bytes(const FmaGeom& g) {
   size_t fl = (size_t)g.TM * g.C + (size_t)g.TM * g.LDQ + kKC * kNC + kWarps * 128;
-  size_t in = (size_t)g.TM + (g.TM + 1) + 4;
+  size_t in = (size_t)g.TM + (g.TM + 1) + 4 + g.TM;
   return fl * 4 + in * 4 + 16;
 }
 
@@ -278,6 +313,14 @@ int dsvt_launch_layer_fma(dsvt_ctx* ctx, const dsvt_fused_args& a) {
   const dsvt_layer_params& p = a.p;
   FmaGeom g;
   g.C = p.C; g.hidden = a.attention_only ? 0 : p.hidden; g.heads = p.heads; g.d = p.C / p.heads; g.tau = p.set_size;
+  g.rb_len = g.rb_sx = g.rb_sy = g.rb_centre = 0;
+  if (p.rpb) {
+    const int L = p.rpb_extent[0], W = p.rpb_extent[1], H = p.rpb_extent[2];
+    g.rb_sy = 2 * H - 1;
+    g.rb_sx = (2 * W - 1) * g.rb_sy;
+    g.rb_len = (2 * L - 1) * g.rb_sx;
+    g.rb_centre = (L - 1) * g.rb_sx + (W - 1) * g.rb_sy + (H - 1);
+  }
   g.LDQ = 3 * p.C + (36 - (3 * p.C) % 32) % 32;  // LDQ % 32 == 4: conflict-free 128-bit row-strided loads
   static const int kTiles[] = {128, 96, 64, 48, 32, 16};
   g.TM = 0;

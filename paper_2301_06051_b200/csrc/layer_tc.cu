@@ -1479,7 +1479,7 @@ bool dsvt_make_weight_map(void* tensor_map, const void* w, int rows, int cols, i
 // Shapes the tensor-core kernel covers; everything else goes to the FMA kernel.
 bool dsvt_layer_tc_supported(const dsvt_fused_args& a) {
   const dsvt_layer_params& p = a.p;
-  if (p.precision != DSVT_BF16_FP32ACC || p.pe) return false;
+  if (p.precision != DSVT_BF16_FP32ACC || p.pe || p.rpb) return false;
   const int d = p.C / p.heads;
   const bool shape = (p.C == 192 && d == 24) || (p.C == 128 && (d == 16 || d == 32)) || (p.C == 64 && d == 16);
   if (!shape || p.set_size > 96) return false;
