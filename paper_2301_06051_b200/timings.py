@@ -1,6 +1,6 @@
 """Per-configuration device timings of the path: partition (both axes), blocks, pooling, whole backbone.
 
-    python -m paper_2301_06051_b200.timings [--configs 1 2 3 4 5] [--steps 20]
+    python -m paper_2301_06051_b200.timings [--configs 1 2 3 4 5] [--steps 20] [--hybrid] [--bev]
 
 One JSON line per configuration.  Times are CUDA-event medians over `steps` passes on synthetic frames that are
 resident in HBM; a 256 MiB write flushes L2 before every pass.  bench.py measures the headline configuration under
@@ -51,6 +51,37 @@ def time_staged(cfg, steps: int, device: int = 0):
            "voxels_out": int(oc.shape[0])}
     out.update({"t_%s_ms" % k: float(np.median(v)) for k, v in spans.items()})
     out["frames_per_s"] = cfg["batch"] / (out["t_backbone_ms"] * 1e-3)
+    return out
+
+
+def time_bev(cid: int, steps: int, device: int = 0):
+    """dsvt_bev_scatter on the configuration's frame (its input features stand in for the backbone's output): the
+    whole call (cell map clear + mark + dense writer), both layouts; bytes = the map written + features and coords read."""
+    cfg = di.make_config(cid)
+    dev = torch.device("cuda", device)
+    ctx = api.Context(cfg["n"], 8, cfg["C"], device=device)
+    coords = torch.from_numpy(cfg["coords"]).to(dev)
+    x = torch.from_numpy(cfg["feats"]).to(dev)
+    flush = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device=dev)
+    out = {"config": cid, "name": cfg["name"], "voxels": cfg["n"], "grid": list(cfg["grid"]), "C": cfg["C"]}
+    for tag, last in (("channels_first", False), ("channels_last", True)):
+        m = ctx.bev_scatter(coords, x, cfg["batch"], cfg["grid"], last)
+        ts = []
+        for it in range(3 + steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ctx.bev_scatter(coords, x, cfg["batch"], cfg["grid"], last, out=m)
+            e1.record()
+            torch.cuda.synchronize(dev)
+            ts.append(e0.elapsed_time(e1))
+        t = float(np.median(ts[3:]))
+        nbytes = 4 * (m.numel() + x.numel() + coords.numel())
+        out.update({"t_%s_ms" % tag: t, "gbs_%s" % tag: nbytes / t * 1e-6})
+        del m
+    out["map_mb"] = 4e-6 * cfg["batch"] * cfg["C"] * int(np.prod(cfg["grid"]))
+    if ctx.status_sync() != 0:
+        raise SystemExit("device status word is not clean")
     return out
 
 
@@ -127,10 +158,14 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--hybrid", action="store_true",
                     help="alternate the configuration's windows with doubled, displaced ones (single-stage configurations)")
+    ap.add_argument("--bev", action="store_true", help="time the BEV projection of each configuration's frame instead")
     args = ap.parse_args()
     api.load()
     for cid in args.configs:
-        print(json.dumps(time_config(cid, args.steps, hybrid=args.hybrid)), flush=True)
+        if args.bev:
+            print(json.dumps(time_bev(cid, args.steps)), flush=True)
+        else:
+            print(json.dumps(time_config(cid, args.steps, hybrid=args.hybrid)), flush=True)
 
 
 if __name__ == "__main__":
