@@ -55,6 +55,9 @@ struct TcGeom {
   int n_f1;     // hidden / NF
   int mode;     // 0: attention only, 1: attention + residual + LN1, 2: full layer
   uint32_t off_a, off_kv, off_stage, off_par;  // byte offsets from the 1024-aligned base
+  // relative position bias (rb_len == 0: none): entries per head, strides of the x and y offsets in the table,
+  // index of the zero offset
+  int rb_len, rb_sx, rb_sy, rb_centre;
 };
 
 struct Misc {  // small shared state beside the big regions
@@ -87,8 +90,16 @@ struct Misc {  // small shared state beside the big regions
   // row lists, double buffered: the loader warps fill buffer (k + 1) & 1 while the compute warps work on tile k;
   // the compute warps gather tile k + 1 as soon as tile k's MMAs no longer read the A operand
   int rowvox[2][kTM];              // tile row -> voxel (-1: none)
-  short set_lo[2][kTM + 1];        // first tile row of each set of the tile
+  unsigned char set_lo[2][kTM + 1];  // first tile row of each set of the tile
   unsigned char row_lo[2][kTM], row_n[2][kTM];  // per tile row: first row and row count of its set
+  // relative position bias.  The table index is linear in the coordinate offset, so one integer per row,
+  // x * rb_sx + y * rb_sy + z, serves every (query, key) pair: index = lin[query] - lin[key] + rb_centre.  Offsets
+  // inside a set are below 2^15 in magnitude, so the low 16 bits are kept and differences are taken modulo 2^16.
+  // Written by the gather of a tile (after the previous tile's attention), read by the tile's attention.
+  const float* rpb;
+  const int4* coords;
+  int rb_len, rb_sx, rb_sy, rb_centre, rb_ext[3];
+  short rowlin[kTM];
 };
 __shared__ Misc s_mi;
 
@@ -272,17 +283,24 @@ struct TcMaps {
   CUtensorMap qkv, o, w1, w2;
 };
 
+// Relative position bias of (query, key) from their rows' linear coordinates; `tab` is the head's table, `root`
+// the square root of the head dimension (the scores are still unscaled dot products when the bias is added).
+__device__ __forceinline__ float rpb_term(const float* __restrict__ tab, int lin_q, int lin_k, float root) {
+  const int idx = (int)(short)(lin_q - lin_k) + s_mi.rb_centre;
+  return __ldg(tab + min((unsigned)idx, (unsigned)(s_mi.rb_len - 1))) * root;  // (a negative index clamps too)
+}
+
 // ---------------------------------------------------------------------------------------------
 // Attention of one tile with mma.sync: one warp per (set, head, 16-query block).
 // D = head dim (16 / 24 / 32), NT = key blocks of 8 a set can have.
 // ---------------------------------------------------------------------------------------------
-template <int C, int D, int NT>
+template <int C, int D, int NT, bool RPB>
 __device__ __noinline__ void attend_tile() {
   constexpr int DC = D / 8;  // 16-byte chunks per head
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t a_base = s_mi.sbase + s_mi.off_a, k_base = s_mi.sbase + s_mi.off_kv;
   const uint32_t v_base = k_base + (C / 64) * (kTM * 128);
-  const short* set_lo = s_mi.set_lo[s_mi.buf];
+  const unsigned char* set_lo = s_mi.set_lo[s_mi.buf];
   const int nsets = s_mi.nsets, heads = s_mi.heads;
   const int g = lane >> 2, t4 = lane & 3;
   const float sc = 1.4426950408889634f * rsqrtf((float)D);  // log2(e) / sqrt(d)
@@ -314,6 +332,22 @@ __device__ __noinline__ void attend_tile() {
           mma_16816(s[j], qa, kf[0], kf[1]);
           if (D == 24) mma_1688(s[j], qb[0], qb[1], kf[2]);
           if (D == 32) mma_16816(s[j], qb, kf[2], kf[3]);
+        }
+      }
+      if (RPB) {
+        const float root = sqrtf((float)D);
+        const float* tab = s_mi.rpb + (size_t)h * s_mi.rb_len;
+        const int linA = s_mi.rowlin[min(q0 + g, kTM - 1)], linB = s_mi.rowlin[min(q0 + g + 8, kTM - 1)];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+          if (j < ntu) {
+            const int kr = r0 + 8 * j + 2 * t4;  // (rows past the tile are masked below: any entry will do)
+            const int lk0 = s_mi.rowlin[min(kr, kTM - 1)], lk1 = s_mi.rowlin[min(kr + 1, kTM - 1)];
+            s[j][0] += rpb_term(tab, linA, lk0, root);
+            s[j][1] += rpb_term(tab, linA, lk1, root);
+            s[j][2] += rpb_term(tab, linB, lk0, root);
+            s[j][3] += rpb_term(tab, linB, lk1, root);
+          }
         }
       }
       // masked softmax over the set's m keys (rows g and g + 8 of the query block)
@@ -392,7 +426,7 @@ __device__ __noinline__ void attend_tile() {
 // many tiny sets cost one item per 16 rows instead of one per set.
 // NTB = key blocks of 8 a row block can need: ceil((2 tau + 14) / 8).
 // ---------------------------------------------------------------------------------------------
-template <int C, int D, int NTB>
+template <int C, int D, int NTB, bool RPB>
 __device__ __noinline__ void attend_blocked() {
   constexpr int DC = D / 8;  // 16-byte chunks per head
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -419,6 +453,9 @@ __device__ __noinline__ void attend_blocked() {
     const unsigned nA = ra < rows ? (unsigned)row_n[ra] : 0u;
     const unsigned loB = rb < rows ? (unsigned)(row_lo[rb] - k_lo) : 0u;
     const unsigned nB = rb < rows ? (unsigned)row_n[rb] : 0u;
+    const float root = sqrtf((float)D);
+    const float* tab = RPB ? s_mi.rpb + (size_t)h * s_mi.rb_len : nullptr;
+    const int linA = RPB ? s_mi.rowlin[min(ra, kTM - 1)] : 0, linB = RPB ? s_mi.rowlin[min(rb, kTM - 1)] : 0;
     uint32_t qa[4], qb[4];
     {
       const int row = q0 + (lane & 15);  // <= 127
@@ -449,6 +486,14 @@ __device__ __noinline__ void attend_blocked() {
           if (D == 24) mma_1688(s[jj], qb[0], qb[1], kf[2]);
           if (D == 32) mma_16816(s[jj], qb, kf[2], kf[3]);
           const unsigned key = (unsigned)(8 * (j0 + jj) + 2 * t4);
+          if (RPB) {
+            const int kr = k_lo + (int)key;  // (rows past the tile are masked below: any entry will do)
+            const int lk0 = s_mi.rowlin[min(kr, kTM - 1)], lk1 = s_mi.rowlin[min(kr + 1, kTM - 1)];
+            s[jj][0] += rpb_term(tab, linA, lk0, root);
+            s[jj][1] += rpb_term(tab, linA, lk1, root);
+            s[jj][2] += rpb_term(tab, linB, lk0, root);
+            s[jj][3] += rpb_term(tab, linB, lk1, root);
+          }
           if (key - loA >= nA) s[jj][0] = -INFINITY;  // unsigned: also true for key < lo
           if (key + 1u - loA >= nA) s[jj][1] = -INFINITY;
           if (key - loB >= nB) s[jj][2] = -INFINITY;
@@ -770,6 +815,7 @@ __device__ __forceinline__ void loader_sync() { asm volatile("bar.sync 6, %0;" :
 
 // Distinct slots of each set -> tile rows (Eq. 4), per-row set ranges, per-set first rows: one thread per
 // set (a tile of a sparse region holds dozens of tiny sets), walking the set's table row.
+template <bool RPB>
 __device__ __forceinline__ void loader_row_list(int b, int lt, int s_lo, int nsets, int base) {
   const int32_t* __restrict__ table = s_mi.table;
   const int32_t* __restrict__ rowoff = s_mi.rowoff;
@@ -782,10 +828,23 @@ __device__ __forceinline__ void loader_row_list(int b, int lt, int s_lo, int nse
     const int cnt_max = inside ? min(cap, kTM - lb) : 0;  // tile rows this set may fill
     int pos = 0, prev = 0;
     bool bad = false;
+    constexpr bool rpb = RPB;
+    int lo3[3] = {INT_MAX, INT_MAX, INT_MAX}, hi3[3] = {INT_MIN, INT_MIN, INT_MIN};
     for (int k0 = 0; k0 < tau; k0 += 8) {
       int v4[8];  // eight independent loads per round trip to L2 (the loader warps run a whole tile ahead)
 #pragma unroll
       for (int u = 0; u < 8; ++u) v4[u] = k0 + u < tau ? __ldg(trow + k0 + u) : 0;
+      if (rpb) {  // a set spread wider than the bias table's extent is reported
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          if (k0 + u < tau && v4[u] >= 0 && v4[u] < n) {
+            const int4 c = __ldg(s_mi.coords + v4[u]);
+            lo3[0] = min(lo3[0], c.y); hi3[0] = max(hi3[0], c.y);
+            lo3[1] = min(lo3[1], c.z); hi3[1] = max(hi3[1], c.z);
+            lo3[2] = min(lo3[2], c.w); hi3[2] = max(hi3[2], c.w);
+          }
+        }
+      }
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         if (k0 + u < tau) {
@@ -804,12 +863,14 @@ __device__ __forceinline__ void loader_row_list(int b, int lt, int s_lo, int nse
         }
       }
     }
-    s_mi.set_lo[b][si] = (short)min(max(lb, 0), kTM);
+    s_mi.set_lo[b][si] = (unsigned char)min(max(lb, 0), kTM);
+    if (rpb)
+      for (int q = 0; q < 3; ++q) bad |= hi3[q] >= lo3[q] && hi3[q] - lo3[q] > s_mi.rb_ext[q] - 1;
     if (bad || pos != cap) atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX);
   }
 }
 
-template <int C>
+template <int C, bool RPB>
 __device__ __noinline__ void loader_role() {
   const int lt = threadIdx.x - 32 * kLoadWarp0, lane = lt & 31;
   volatile int* abort_flag = &s_mi.abort_flag;
@@ -839,8 +900,8 @@ __device__ __noinline__ void loader_role() {
         s_mi.row_n[b][i] = 1;
       }
       loader_sync();
-      loader_row_list(b, lt, s_lo, nsets, base);
-      if (lt == 0) s_mi.set_lo[b][nsets] = (short)rows;
+      loader_row_list<RPB>(b, lt, s_lo, nsets, base);
+      if (lt == 0) s_mi.set_lo[b][nsets] = (unsigned char)rows;
     }
     if (lt == 0) s_mi.next_rows[b] = nsets < 0 ? -1 : rows;
     mbar_arrive(&s_mi.rl_ready[b]);
@@ -854,6 +915,7 @@ __device__ __noinline__ void loader_role() {
 // alive across the calls.
 
 // Row list of a CTA's first tile by the compute warps (one warp per set), into buffer 0.
+template <bool RPB>
 __device__ __noinline__ void phase_row_list() {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int32_t* __restrict__ table = s_mi.table;
@@ -865,11 +927,18 @@ __device__ __noinline__ void phase_row_list() {
     const int lb = rowoff[s] - base, cap = rowoff[s + 1] - rowoff[s];
     const int cnt_max = (lb >= 0 && lb < kTM) ? min(cap, kTM - lb) : 0;
     int cnt = 0;
+    int lo3[3] = {INT_MAX, INT_MAX, INT_MAX}, hi3[3] = {INT_MIN, INT_MIN, INT_MIN};
     for (int k0 = 0; k0 < tau; k0 += 32) {
       const int k = k0 + lane;
       int v = -1;
       bool uniq = false;
       if (k < tau) { v = trow[k]; uniq = (k == 0) || (v != trow[k - 1]); }
+      if (RPB && v >= 0 && v < n) {
+        const int4 c = __ldg(s_mi.coords + v);
+        lo3[0] = min(lo3[0], c.y); hi3[0] = max(hi3[0], c.y);
+        lo3[1] = min(lo3[1], c.z); hi3[1] = max(hi3[1], c.z);
+        lo3[2] = min(lo3[2], c.w); hi3[2] = max(hi3[2], c.w);
+      }
       const unsigned bal = __ballot_sync(0xffffffffu, uniq);
       const int pos = cnt + __popc(bal & ((1u << lane) - 1u));
       if (uniq && pos < cnt_max) {
@@ -882,17 +951,25 @@ __device__ __noinline__ void phase_row_list() {
       s_mi.row_lo[0][lb + i] = (unsigned char)lb;
       s_mi.row_n[0][lb + i] = (unsigned char)cnt_max;
     }
+    bool wide = false;
+    if (RPB) {  // a set spread wider than the bias table's extent is reported
+#pragma unroll
+      for (int q = 0; q < 3; ++q) {
+        const int l = __reduce_min_sync(0xffffffffu, lo3[q]), hmax = __reduce_max_sync(0xffffffffu, hi3[q]);
+        wide |= hmax >= l && hmax - l > s_mi.rb_ext[q] - 1;
+      }
+    }
     if (lane == 0) {
-      s_mi.set_lo[0][si] = (short)min(max(lb, 0), kTM);
-      if (cnt != cap) atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX);
+      s_mi.set_lo[0][si] = (unsigned char)min(max(lb, 0), kTM);
+      if (cnt != cap || wide) atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX);
     }
   }
-  if (tid == 0) s_mi.set_lo[0][nsets] = (short)s_mi.rows;
+  if (tid == 0) s_mi.set_lo[0][nsets] = (unsigned char)s_mi.rows;
 }
 
 // Gather (Eq. 4): the fp32 rows listed in buffer b -> bf16 A operand, four rows in flight per warp; all 128 rows
 // are written (rows past the tile as zeros).
-template <int C>
+template <int C, bool RPB>
 __device__ __noinline__ void phase_gather(int b, int rows) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float* __restrict__ x = s_mi.x;
@@ -909,6 +986,14 @@ __device__ __noinline__ void phase_gather(int b, int rows) {
         const float4* src = reinterpret_cast<const float4*>(x + (size_t)v * C) + 2 * lane;
         f[u][0] = __ldg(src);
         f[u][1] = __ldg(src + 1);
+      }
+      if (RPB && lane == 31) {  // (lane 31 carries no feature columns: C / 8 <= 24)
+        int lin = 0;
+        if (v >= 0) {
+          const int4 c = __ldg(s_mi.coords + v);
+          lin = c.y * s_mi.rb_sx + c.z * s_mi.rb_sy + c.w;
+        }
+        s_mi.rowlin[r] = (short)lin;
       }
     }
     if (lane < (C >> 3)) {
@@ -1150,7 +1235,7 @@ __device__ __noinline__ void phase_epi_f2() {
 // the odd MLP-1 pieces; region 2 = [512 - C, 512): x1 + b_2 parked by the output-projection epilogue, then
 // the MLP-2 accumulator.  Each region has its own full / free barrier pair.  For C = 192 regions 1 and 2
 // overlap, which is why the MMA issuer waits for region 2 before it starts the next tile's V.
-template <int C, int D, int NT, bool BLOCKED>
+template <int C, int D, int NT, bool BLOCKED, bool RPB>
 __device__ __forceinline__ void compute_role() {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
   constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
@@ -1173,7 +1258,7 @@ __device__ __forceinline__ void compute_role() {
     ok = mbar_wait(&s_mi.rl_ready[b], (uint32_t)((k + 1) >> 1) & 1u, abort_flag) && ok;
     const int nr = s_mi.next_rows[b];
     if (ok && nr >= 0) {
-      phase_gather<C>(b, nr);
+      phase_gather<C, RPB>(b, nr);
       fence_proxy_async();
       mbar_arrive(&s_mi.x_ready);
     }
@@ -1205,9 +1290,9 @@ __device__ __forceinline__ void compute_role() {
     if (k == 0) {  // nothing runs ahead of a CTA's first tile: the compute warps list and gather it themselves,
                    // as a rule already during the kernel's set-up
       if (!listed) {
-        phase_row_list();
+        phase_row_list<RPB>();
         compute_sync();
-        phase_gather<C>(0, rows);
+        phase_gather<C, RPB>(0, rows);
         fence_proxy_async();
       }
       mbar_arrive(&s_mi.x_ready);  // X is in place
@@ -1224,9 +1309,9 @@ __device__ __forceinline__ void compute_role() {
     compute_sync();
     // ---- attention inside each set ----
     if (BLOCKED)
-      attend_blocked<C, D, NT>();
+      attend_blocked<C, D, NT, RPB>();
     else
-      attend_tile<C, D, NT>();
+      attend_tile<C, D, NT, RPB>();
     fence_proxy_async();
     mbar_arrive(&s_mi.a_ready);  // attention output is the A operand of the output projection
     compute_sync();              // every warp is done with K and V: their region becomes fp32 staging
@@ -1273,7 +1358,7 @@ __device__ __forceinline__ void compute_role() {
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int C, int D, int NT, bool BLOCKED>
+template <int C, int D, int NT, bool BLOCKED, bool RPB>
 __global__ void __launch_bounds__(kThreads, 1)
 layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant__ TcGeom g,
                 const __grid_constant__ TcMaps maps, int32_t* __restrict__ status) {
@@ -1317,6 +1402,9 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
     mi->n = a.n; mi->tau = g.tau; mi->heads = g.heads; mi->mode = g.mode; mi->NF = g.NF; mi->n_f1 = g.n_f1;
     mi->ln1 = a.p.ln1_g != nullptr; mi->ln2 = a.p.ln2_g != nullptr;
     mi->eps = a.p.ln_eps;
+    mi->rpb = a.p.rpb; mi->coords = reinterpret_cast<const int4*>(a.p.coords);
+    mi->rb_len = g.rb_len; mi->rb_sx = g.rb_sx; mi->rb_sy = g.rb_sy; mi->rb_centre = g.rb_centre;
+    mi->rb_ext[0] = a.p.rpb_extent[0]; mi->rb_ext[1] = a.p.rpb_extent[1]; mi->rb_ext[2] = a.p.rpb_extent[2];
     mi->s_lo = mi->nsets = mi->base = mi->rows = mi->buf = mi->pre0 = 0;
     mi->next_rows[0] = mi->next_rows[1] = -1;
   }
@@ -1364,9 +1452,9 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
         mi->row_n[0][tid] = 1;
       }
       compute_sync();
-      phase_row_list();
+      phase_row_list<RPB>();
       compute_sync();
-      phase_gather<C>(0, rows);
+      phase_gather<C, RPB>(0, rows);
       fence_proxy_async();
     }
   }
@@ -1402,9 +1490,9 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
     if ((tid & 31) == 0) mma_role<C>(a, g, rc);
     __syncwarp();
   } else if (warp >= kLoadWarp0) {
-    loader_role<C>();
+    loader_role<C, RPB>();
   } else {
-    compute_role<C, D, NT, BLOCKED>();
+    compute_role<C, D, NT, BLOCKED, RPB>();
   }
   // ---- teardown: everyone meets here, then the allocating warp returns the TMEM columns ----
   tc_fence_before();
@@ -1449,14 +1537,21 @@ bool make_weight_map(CUtensorMap* m, const void* w, int rows, int cols, int box_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int C, int D, int NT, bool BLOCKED>
-int launch_tc(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
-  cudaError_t e =
-      cudaFuncSetAttribute(layer_tc_kernel<C, D, NT, BLOCKED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+template <int C, int D, int NT, bool BLOCKED, bool RPB>
+int launch_tc_one(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
+  cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<C, D, NT, BLOCKED, RPB>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
-  layer_tc_kernel<C, D, NT, BLOCKED><<<grid, kThreads, smem, ctx->stream>>>(a, g, maps, ctx->status);
+  layer_tc_kernel<C, D, NT, BLOCKED, RPB><<<grid, kThreads, smem, ctx->stream>>>(a, g, maps, ctx->status);
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
+}
+
+// The position bias is a compile-time variant: a layer without one runs a kernel that holds none of its code.
+template <int C, int D, int NT, bool BLOCKED>
+int launch_tc(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
+  if (g.rb_len != 0) return launch_tc_one<C, D, NT, BLOCKED, true>(ctx, a, g, maps, grid, smem);
+  return launch_tc_one<C, D, NT, BLOCKED, false>(ctx, a, g, maps, grid, smem);
 }
 
 template <int C, int D>
@@ -1479,7 +1574,11 @@ bool dsvt_make_weight_map(void* tensor_map, const void* w, int rows, int cols, i
 // Shapes the tensor-core kernel covers; everything else goes to the FMA kernel.
 bool dsvt_layer_tc_supported(const dsvt_fused_args& a) {
   const dsvt_layer_params& p = a.p;
-  if (p.precision != DSVT_BF16_FP32ACC || p.pe || p.rpb) return false;
+  if (p.precision != DSVT_BF16_FP32ACC || p.pe) return false;
+  if (p.rpb) {  // row coordinates are kept as 16-bit linear indices: every table offset must be below 2^15
+    const int64_t len = (int64_t)(2 * p.rpb_extent[0] - 1) * (2 * p.rpb_extent[1] - 1) * (2 * p.rpb_extent[2] - 1);
+    if (len > 32767) return false;
+  }
   const int d = p.C / p.heads;
   const bool shape = (p.C == 192 && d == 24) || (p.C == 128 && (d == 16 || d == 32)) || (p.C == 64 && d == 16);
   if (!shape || p.set_size > 96) return false;
@@ -1499,6 +1598,14 @@ int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a) {
   g.nkb_h = g.hidden / 64;
   g.NF = (g.hidden % 128 == 0 && C >= 128) ? 128 : 64;
   g.n_f1 = g.hidden / g.NF;
+  g.rb_len = g.rb_sx = g.rb_sy = g.rb_centre = 0;
+  if (p.rpb) {
+    const int L = p.rpb_extent[0], W = p.rpb_extent[1], H = p.rpb_extent[2];
+    g.rb_sy = 2 * H - 1;
+    g.rb_sx = (2 * W - 1) * g.rb_sy;
+    g.rb_len = (2 * L - 1) * g.rb_sx;
+    g.rb_centre = (L - 1) * g.rb_sx + (W - 1) * g.rb_sy + (H - 1);
+  }
   const uint32_t a_bytes = kTM * C * 2;
   g.off_a = 0;
   g.off_kv = a_bytes;

@@ -53,7 +53,7 @@ class Stage:
         src = x
         for blk, sp in zip(self.blocks, self.specs):
             t = self.tables_of[sp]
-            self.ctx.block(src, t[0], t[1], blk, y)
+            self.ctx.block(src, t[0], t[1], blk, y, coords=coords)  # (coords: read by layers with a position bias)
             src = y
         return y
 
@@ -137,7 +137,7 @@ class StagedBackbone:
                 on_step("s%d_partition" % i)
             src = feats
             for blk in stage.blocks:
-                self.ctx.block(src, stage.tables[0], stage.tables[1], blk, y)
+                self.ctx.block(src, stage.tables[0], stage.tables[1], blk, y, coords=coords)
                 src = y
             if on_step:
                 on_step("s%d_blocks" % i)

@@ -1,6 +1,6 @@
 """Per-configuration device timings of the path: partition (both axes), blocks, pooling, whole backbone.
 
-    python -m paper_2301_06051_b200.timings [--configs 1 2 3 4 5] [--steps 20] [--hybrid] [--bev]
+    python -m paper_2301_06051_b200.timings [--configs 1 2 3 4 5] [--steps 20] [--hybrid] [--rpb] [--bev]
 
 One JSON line per configuration.  Times are CUDA-event medians over `steps` passes on synthetic frames that are
 resident in HBM; a 256 MiB write flushes L2 before every pass.  bench.py measures the headline configuration under
@@ -85,10 +85,22 @@ def time_bev(cid: int, steps: int, device: int = 0):
     return out
 
 
-def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False):
+def add_position_bias(cfg, seed: int = 0):
+    """Gives every layer of a single-stage configuration a random relative position bias table for its window."""
+    rng = np.random.default_rng(seed)
+    L, W, H = cfg["window"]
+    for blk in cfg["blocks"]:
+        for layer in blk:
+            layer["rpb"] = rng.standard_normal((cfg["heads"], (2 * L - 1) * (2 * W - 1) * (2 * H - 1))).astype(np.float32)
+            layer["rpb_extent"] = (L, W, H)
+
+
+def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False, rpb: bool = False):
     cfg = di.make_config(cid)
     if cfg.get("stages"):
         return time_staged(cfg, steps, device)
+    if rpb:
+        add_position_bias(cfg)
     dev = torch.device("cuda", device)
     if hybrid:
         # hybrid window partition (Sec. 3.2): every second block works on windows twice as large in x and y,
@@ -113,7 +125,7 @@ def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False):
         stage.partition(c)
         mark(tag + "partition")
         for blk in stage.blocks:
-            bb.ctx.block(src, stage.tables[0], stage.tables[1], blk, dst)
+            bb.ctx.block(src, stage.tables[0], stage.tables[1], blk, dst, coords=c)
             src = dst
         mark(tag + "blocks")
 
@@ -139,7 +151,7 @@ def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False):
         spans.setdefault("backbone", []).append(r[0][1].elapsed_time(r[-1][1]))
     med = {k: float(np.median(v)) for k, v in spans.items()}
     nb1 = len(bb.stage1.blocks)
-    out = {"config": cid, "name": cfg["name"] + (" + hybrid windows" if hybrid else ""), "voxels": cfg["n"], "precision": cfg["precision"],
+    out = {"config": cid, "name": cfg["name"] + (" + hybrid windows" if hybrid else "") + (" + position bias" if rpb else ""), "voxels": cfg["n"], "precision": cfg["precision"],
            "sets": int(bb.stage1.tables[0].num_sets.item()),
            "t_partition_ms": med["s1_partition"], "t_block_ms": med["s1_blocks"] / nb1,
            "voxels_per_s_per_block": cfg["n"] / (med["s1_blocks"] / nb1 * 1e-3),
@@ -158,6 +170,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--hybrid", action="store_true",
                     help="alternate the configuration's windows with doubled, displaced ones (single-stage configurations)")
+    ap.add_argument("--rpb", action="store_true",
+                    help="give every layer a relative position bias table for its window (single-stage configurations)")
     ap.add_argument("--bev", action="store_true", help="time the BEV projection of each configuration's frame instead")
     args = ap.parse_args()
     api.load()
@@ -165,7 +179,7 @@ def main():
         if args.bev:
             print(json.dumps(time_bev(cid, args.steps)), flush=True)
         else:
-            print(json.dumps(time_config(cid, args.steps, hybrid=args.hybrid)), flush=True)
+            print(json.dumps(time_config(cid, args.steps, hybrid=args.hybrid, rpb=args.rpb)), flush=True)
 
 
 if __name__ == "__main__":

@@ -35,6 +35,9 @@ def _with_bias(rng, layer, heads, extent, oracle):
     (34, 3000, (96, 96, 1), (30, 30, 1), 90, 128, 8, False),
     (35, 1500, (48, 48, 1), (12, 12, 1), 36, 192, 8, True),
     (36, 1200, (48, 48, 2), (12, 12, 2), 48, 192, 8, True),
+    (37, 3000, (96, 96, 1), (30, 30, 1), 90, 128, 8, True),    # one attention item per set (set size above 48)
+    (38, 2000, (60, 60, 1), (12, 12, 1), 36, 128, 4, True),    # head dimension 32
+    (39, 900, (24, 24, 40), (12, 12, 32), 36, 64, 4, True),    # a table too long for 16-bit row indices
 ])
 def test_set_attention_with_relative_position_bias(gpu, oracle, seed, n, grid, window, tau, C, heads, bf16):
     cfg = di.random_case(seed, n, grid, window, tau, C, heads, bf16=bf16)
@@ -103,6 +106,75 @@ def test_bias_table_narrower_than_a_set_is_flagged(gpu, oracle):
     # a bias without coordinates is refused on the host
     with pytest.raises(gpu.DsvtError):
         ctx.set_attention(x, upload_table(ok), w, out, coords=None)
+
+
+@pytest.mark.parametrize("cid", [2, 6])
+def test_full_size_frame_with_bias_on_sampled_windows(gpu, oracle, cid):
+    """One block of the full-size frame (bf16 weights, tensor-core kernel, several tiles per thread block) with a
+    bias table per layer; whole sampled windows are recomputed by the oracle.  A table cut for a smaller window
+    than the partition's is reported and harms nothing else."""
+    cfg = di.make_config(cid)
+    rng = np.random.default_rng(cid)
+    heads, window, tau = cfg["heads"], cfg["window"], cfg["set_size"]
+    layers = [_with_bias(rng, l, heads, window, oracle) for l in cfg["blocks"][0]]
+    n = cfg["n"]
+    ctx = gpu.Context(n, _nwin(cfg["batch"], cfg["grid"], window), cfg["C"])
+    ws = [gpu.device_weights(l, gpu.BF16_FP32ACC, ctx.device) for l in layers]
+    x, coords = dev(cfg["feats"]), dev(cfg["coords"])
+    t0, t1 = ctx.partition_rotated(coords, cfg["batch"], cfg["grid"], window, tau)
+    y = torch.empty_like(x)
+    ctx.block(x, t0, t1, ws, y, coords=coords)
+    assert ctx.status_sync() == 0
+    got = y.cpu().numpy()
+    assert np.all(np.isfinite(got))
+    # whole windows holding about 2500 voxels
+    p = oracle.partition(cfg["coords"], cfg["batch"], cfg["grid"], window, tau, 0)
+    order = np.concatenate([[np.argmax(p.win_count)], rng.permutation(np.flatnonzero(p.win_count > 0))])
+    sel, total = [], 0
+    for w in order:
+        sel.append(p.perm[p.win_start[w]:p.win_start[w + 1]])
+        total += sel[-1].shape[0]
+        if total >= 2500:
+            break
+    sel = np.sort(np.unique(np.concatenate(sel)))
+    sc, sf = cfg["coords"][sel], cfg["feats"][sel]
+    p0 = oracle.partition(sc, cfg["batch"], cfg["grid"], window, tau, 0).set_table
+    p1 = oracle.partition(sc, cfg["batch"], cfg["grid"], window, tau, 1).set_table
+    want = oracle.block(sf, p0, p1, layers, coords=sc)
+    check_close(got[sel], want, "bf16", "config %d block with bias" % cid)
+    plain = oracle.block(sf, p0, p1, cfg["blocks"][0])
+    assert np.abs(plain - want).max() > 1e-2
+    # too small a table: reported by the status word, results stay finite
+    small = tuple(max(1, v // 2) for v in window)
+    ws_small = [gpu.device_weights(_with_bias(rng, l, heads, small, oracle), gpu.BF16_FP32ACC, ctx.device)
+                for l in cfg["blocks"][0]]
+    ctx.block(x, t0, t1, ws_small, y, coords=coords)
+    assert ctx.status_sync() & gpu.STATUS_BAD_INDEX
+    assert torch.isfinite(y).all()
+
+
+def test_bias_table_narrower_than_a_set_is_flagged_on_the_tensor_core_path(gpu, oracle):
+    rng = np.random.default_rng(4)
+    n, C, heads, tau = 40, 64, 4, 4
+    L = _with_bias(rng, di.make_layer(rng, C, heads, 0, False, True), heads, (3, 3, 1), oracle)
+    coords = np.zeros((n, 4), dtype=np.int32)
+    coords[:, 1] = np.arange(n) % 8
+    coords[:, 2] = np.arange(n) // 8
+    ctx = gpu.Context(n, 8, C)
+    w = gpu.device_weights(L, gpu.BF16_FP32ACC, ctx.device)
+    xh = rng.standard_normal((n, C), dtype=np.float32)
+    x = dev(xh)
+    ok = np.array([[0, 1, 2, 2], [8, 9, 10, 10]], dtype=np.int32)
+    out = torch.zeros((n, C), device="cuda")
+    ctx.set_attention(x, upload_table(ok), w, out, coords=dev(coords))
+    assert ctx.status_sync() == 0
+    want, covered = oracle.set_attention(xh, ok, L["W_qkv"], L["b_qkv"], L["W_o"], L["b_o"], heads, rpb=L["rpb"],
+                                         coords=coords, rpb_extent=(3, 3, 1))
+    check_close(out.cpu().numpy()[covered == 1], want[covered == 1], "bf16", "caller-made table with bias")
+    wide = np.array([[0, 1, 2, 3], [8, 9, 10, 10]], dtype=np.int32)
+    ctx.set_attention(x, upload_table(wide), w, out, coords=dev(coords))
+    assert ctx.status_sync() & gpu.STATUS_BAD_INDEX
+    assert torch.isfinite(out).all()
 
 
 # ------------------------------------------------------------------------------------------------ BEV projection
