@@ -58,6 +58,62 @@ class Stage:
         return y
 
 
+class FrameStream:
+    """Runs frames that live in pinned host memory through a Stage with the copies off the critical path: frame
+    k + 1 is uploaded and frame k - 1 downloaded while frame k's kernels run (one upload stream, the context's
+    stream for the kernels, one download stream; `depth` sets of device buffers).  Every frame is still copied in,
+    computed and copied out in full; only the waiting is overlapped."""
+
+    def __init__(self, stage: Stage, max_voxels: int, C: int, depth: int = 2):
+        self.stage, self.depth = stage, int(depth)
+        ctx = stage.ctx
+        dev = ctx.device
+        self.compute = ctx.stream
+        self.up, self.down = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        cap = max(int(max_voxels), 1)
+        self.coords = [torch.empty((cap, 4), dtype=torch.int32, device=dev) for _ in range(self.depth)]
+        self.x = [torch.empty((cap, C), dtype=torch.float32, device=dev) for _ in range(self.depth)]
+        self.y = [torch.empty((cap, C), dtype=torch.float32, device=dev) for _ in range(self.depth)]
+        self.uploaded = [torch.cuda.Event() for _ in range(self.depth)]
+        self.computed = [torch.cuda.Event() for _ in range(self.depth)]
+        self.downloaded = [torch.cuda.Event() for _ in range(self.depth)]
+        self.count = 0
+
+    def submit(self, coords_h: torch.Tensor, feats_h: torch.Tensor, out_h: torch.Tensor) -> None:
+        """Enqueues one frame: coords_h int32 [n, 4], feats_h float32 [n, C], out_h float32 [n, C], all pinned host
+        tensors that must stay untouched until `wait()` returns (out_h is written by then).  Does not block unless the
+        caller is `depth` frames ahead of the device."""
+        assert coords_h.is_pinned() and feats_h.is_pinned() and out_h.is_pinned(), "pinned host memory only"
+        n = int(feats_h.shape[0])
+        s = self.count % self.depth
+        reuse = self.count >= self.depth
+        with torch.cuda.stream(self.up):
+            if reuse:
+                self.up.wait_event(self.computed[s])   # the frame that last used these inputs has been computed
+            c, x = self.coords[s][:n], self.x[s][:n]
+            c.copy_(coords_h, non_blocking=True)
+            x.copy_(feats_h, non_blocking=True)
+            self.uploaded[s].record(self.up)
+        self.compute.wait_event(self.uploaded[s])
+        if reuse:
+            self.compute.wait_event(self.downloaded[s])  # y[s] of that frame has reached the host
+        y = self.y[s][:n]
+        with torch.cuda.stream(self.compute):
+            self.stage.forward(c, x, y)
+            self.computed[s].record(self.compute)
+        with torch.cuda.stream(self.down):
+            self.down.wait_event(self.computed[s])
+            out_h.copy_(y, non_blocking=True)
+            self.downloaded[s].record(self.down)
+        self.count += 1
+
+    def wait(self) -> None:
+        """Blocks until every submitted frame's output is in its host tensor."""
+        self.down.synchronize()
+        self.compute.synchronize()
+        self.up.synchronize()
+
+
 class Backbone:
     """One or two stages with an optional attention-style pooling step between them."""
 

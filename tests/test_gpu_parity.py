@@ -363,6 +363,34 @@ def test_in_place_and_repeatability(gpu):
     assert np.array_equal(a, b)  # no atomics on the float path: bitwise repeatable
 
 
+def test_frame_stream_overlaps_copies_without_mixing_frames(gpu):
+    """Seven different frames (different sizes and contents) through pipeline.FrameStream with two buffer sets:
+    every host output equals the frame's own device-resident run."""
+    from paper_2301_06051_b200 import pipeline
+
+    base = di.make_config(2, n_override=9000)
+    n_max = 9000
+    ctx = gpu.Context(n_max, _nwin(base["batch"], base["grid"], base["window"]), base["C"])
+    st = pipeline.Stage(ctx, base["blocks"][:2], base["batch"], base["grid"], base["window"], base["set_size"],
+                        precision_of(base), n_max)
+    frames = []
+    for k, n in enumerate([9000, 4000, 7000, 1, 8999, 2500, 6000]):
+        rng = np.random.default_rng(100 + k)
+        coords = di.unique_cells(rng, n, base["grid"], base["batch"])
+        feats = rng.standard_normal((n, base["C"]), dtype=np.float32)
+        frames.append((torch.from_numpy(coords).pin_memory(), torch.from_numpy(feats).pin_memory(),
+                       torch.full((n, base["C"]), 5.0).pin_memory()))
+    fs = pipeline.FrameStream(st, n_max, base["C"], depth=2)
+    for c, f, o in frames:
+        fs.submit(c, f, o)
+    fs.wait()
+    assert ctx.status_sync() == 0
+    for c, f, o in frames:
+        y = torch.empty((f.shape[0], base["C"]), device="cuda")
+        st.forward(c.cuda(), f.cuda(), y)
+        assert torch.equal(y.cpu(), o)
+
+
 # ------------------------------------------------------------------------------------------------
 # pooling
 # ------------------------------------------------------------------------------------------------
