@@ -291,140 +291,14 @@ __device__ __forceinline__ float rpb_term(const float* __restrict__ tab, int lin
 }
 
 // ---------------------------------------------------------------------------------------------
-// Attention of one tile with mma.sync: one warp per (set, head, 16-query block).
-// D = head dim (16 / 24 / 32), NT = key blocks of 8 a set can have.
-// ---------------------------------------------------------------------------------------------
-template <int C, int D, int NT, bool RPB>
-__device__ __noinline__ void attend_tile() {
-  constexpr int DC = D / 8;  // 16-byte chunks per head
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t a_base = s_mi.sbase + s_mi.off_a, k_base = s_mi.sbase + s_mi.off_kv;
-  const uint32_t v_base = k_base + (C / 64) * (kTM * 128);
-  const unsigned char* set_lo = s_mi.set_lo[s_mi.buf];
-  const int nsets = s_mi.nsets, heads = s_mi.heads;
-  const int g = lane >> 2, t4 = lane & 3;
-  const float sc = 1.4426950408889634f * rsqrtf((float)D);  // log2(e) / sqrt(d)
-  int item = 0;
-  for (int si = 0; si < nsets; ++si) {
-    const int r0 = set_lo[si], m = set_lo[si + 1] - r0;
-    const int mtiles = (m + 15) >> 4, ntu = (m + 7) >> 3;
-    for (int hm = 0; hm < heads * mtiles; ++hm, ++item) {
-      if ((item % kComputeWarps) != warp) continue;
-      const int h = hm / mtiles, mt = hm - h * mtiles;
-      const int c0 = h * DC;
-      const int q0 = r0 + 16 * mt;
-      // Q fragments (A operand, 16 x D)
-      uint32_t qa[4], qb[4];
-      {
-        const int row = min(q0 + (lane & 15), kTM - 1);
-        ldsm_x4(a_base + swz(row, c0 + (lane >> 4)), qa);
-        if (D > 16) ldsm_x4(a_base + swz(row, c0 + 2 + ((D == 32) ? (lane >> 4) : 0)), qb);
-      }
-      float s[NT][4];
-#pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
-        if (j < ntu) {
-          uint32_t kf[4];
-          const int row = min(r0 + 8 * j + (lane & 7), kTM - 1);
-          const int ch = min(lane >> 3, DC - 1);
-          ldsm_x4(k_base + swz(row, c0 + ch), kf);
-          mma_16816(s[j], qa, kf[0], kf[1]);
-          if (D == 24) mma_1688(s[j], qb[0], qb[1], kf[2]);
-          if (D == 32) mma_16816(s[j], qb, kf[2], kf[3]);
-        }
-      }
-      if (RPB) {
-        const float root = sqrtf((float)D);
-        const float* tab = s_mi.rpb + (size_t)h * s_mi.rb_len;
-        const int linA = s_mi.rowlin[min(q0 + g, kTM - 1)], linB = s_mi.rowlin[min(q0 + g + 8, kTM - 1)];
-#pragma unroll
-        for (int j = 0; j < NT; ++j) {
-          if (j < ntu) {
-            const int kr = r0 + 8 * j + 2 * t4;  // (rows past the tile are masked below: any entry will do)
-            const int lk0 = s_mi.rowlin[min(kr, kTM - 1)], lk1 = s_mi.rowlin[min(kr + 1, kTM - 1)];
-            s[j][0] += rpb_term(tab, linA, lk0, root);
-            s[j][1] += rpb_term(tab, linA, lk1, root);
-            s[j][2] += rpb_term(tab, linB, lk0, root);
-            s[j][3] += rpb_term(tab, linB, lk1, root);
-          }
-        }
-      }
-      // masked softmax over the set's m keys (rows g and g + 8 of the query block)
-      float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        const int key = 8 * j + 2 * t4;
-        if (key >= m) s[j][0] = s[j][2] = -INFINITY;
-        if (key + 1 >= m) s[j][1] = s[j][3] = -INFINITY;
-        mx0 = fmaxf(mx0, fmaxf(s[j][0], s[j][1]));
-        mx1 = fmaxf(mx1, fmaxf(s[j][2], s[j][3]));
-      }
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-      float l0 = 0.f, l1 = 0.f;
-#pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        s[j][0] = exp2f((s[j][0] - mx0) * sc);
-        s[j][1] = exp2f((s[j][1] - mx0) * sc);
-        s[j][2] = exp2f((s[j][2] - mx1) * sc);
-        s[j][3] = exp2f((s[j][3] - mx1) * sc);
-        l0 += s[j][0] + s[j][1];
-        l1 += s[j][2] + s[j][3];
-      }
-      l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-      l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-      l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-      l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-      // O = P V
-      float o[DC][4];
-#pragma unroll
-      for (int dn = 0; dn < DC; ++dn) o[dn][0] = o[dn][1] = o[dn][2] = o[dn][3] = 0.f;
-#pragma unroll
-      for (int kk = 0; kk < (NT + 1) / 2; ++kk) {
-        if (2 * kk < ntu) {
-          constexpr int kLast = NT - 1;
-          const int j1 = (2 * kk + 1 <= kLast) ? 2 * kk + 1 : kLast;
-          const bool two = (2 * kk + 1 <= kLast);
-          uint32_t pa[4];
-          pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-          pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-          pa[2] = two ? pack_bf16(s[j1][0], s[j1][1]) : 0u;
-          pa[3] = two ? pack_bf16(s[j1][2], s[j1][3]) : 0u;
-          const int row = min(r0 + 16 * kk + (lane & 15), kTM - 1);
-#pragma unroll
-          for (int dn = 0; dn < DC; ++dn) {
-            uint32_t vf[2];
-            ldsm_x2_trans(v_base + swz(row, c0 + dn), vf);
-            mma_16816(o[dn], pa, vf[0], vf[1]);
-          }
-        }
-      }
-      const float i0 = 1.0f / l0, i1 = 1.0f / l1;
-      const int qa_row = 16 * mt + g;
-#pragma unroll
-      for (int dn = 0; dn < DC; ++dn) {
-        // the query rows of this block and head are dead now: their slots take the attention output
-        if (qa_row < m)
-          asm volatile("st.shared.b32 [%0], %1;" ::"r"(a_base + swz(q0 + g, c0 + dn) + 4 * t4),
-                       "r"(pack_bf16(o[dn][0] * i0, o[dn][1] * i0)) : "memory");
-        if (qa_row + 8 < m)
-          asm volatile("st.shared.b32 [%0], %1;" ::"r"(a_base + swz(q0 + g + 8, c0 + dn) + 4 * t4),
-                       "r"(pack_bf16(o[dn][2] * i1, o[dn][3] * i1)) : "memory");
-      }
-    }
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Attention of one tile, blocked by 16 consecutive tile rows instead of by set: one warp per (row
+// Attention of one tile with mma.sync, blocked by 16 consecutive tile rows rather than by set: one warp per (row
 // block, head).  The keys of a block are the rows of every set that the block touches; a score is
 // kept only where query and key belong to the same set (row_lo / row_n give each row's set range).
 // The arithmetic per query row is exactly the per-set softmax attention, but sparse regions with
-// many tiny sets cost one item per 16 rows instead of one per set.
-// NTB = key blocks of 8 a row block can need: ceil((2 tau + 14) / 8).
+// many tiny sets cost one item per 16 rows instead of one per set, and the running softmax over passes of four key
+// blocks keeps the registers low for sets of any size (a version with one item per set and all of a set's scores in
+// registers spilled for set sizes near 96 and was a quarter slower there).
+// NTB = key blocks of 8 a row block can need: ceil((2 tau + 14) / 8), at most the 16 of a whole tile.
 // ---------------------------------------------------------------------------------------------
 template <int C, int D, int NTB, bool RPB>
 __device__ __noinline__ void attend_blocked() {
@@ -1235,7 +1109,7 @@ __device__ __noinline__ void phase_epi_f2() {
 // the odd MLP-1 pieces; region 2 = [512 - C, 512): x1 + b_2 parked by the output-projection epilogue, then
 // the MLP-2 accumulator.  Each region has its own full / free barrier pair.  For C = 192 regions 1 and 2
 // overlap, which is why the MMA issuer waits for region 2 before it starts the next tile's V.
-template <int C, int D, int NT, bool BLOCKED, bool RPB>
+template <int C, int D, int NT, bool RPB>
 __device__ __forceinline__ void compute_role() {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
   constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
@@ -1308,10 +1182,7 @@ __device__ __forceinline__ void compute_role() {
     phase_epi_bf16<QC, false, true>(0u, 0, ParOff<C>::b_q, s_mi.off_a, 0, rows);
     compute_sync();
     // ---- attention inside each set ----
-    if (BLOCKED)
-      attend_blocked<C, D, NT, RPB>();
-    else
-      attend_tile<C, D, NT, RPB>();
+    attend_blocked<C, D, NT, RPB>();
     fence_proxy_async();
     mbar_arrive(&s_mi.a_ready);  // attention output is the A operand of the output projection
     compute_sync();              // every warp is done with K and V: their region becomes fp32 staging
@@ -1358,7 +1229,7 @@ __device__ __forceinline__ void compute_role() {
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int C, int D, int NT, bool BLOCKED, bool RPB>
+template <int C, int D, int NT, bool RPB>
 __global__ void __launch_bounds__(kThreads, 1)
 layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant__ TcGeom g,
                 const __grid_constant__ TcMaps maps, int32_t* __restrict__ status) {
@@ -1492,7 +1363,7 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   } else if (warp >= kLoadWarp0) {
     loader_role<C, RPB>();
   } else {
-    compute_role<C, D, NT, BLOCKED, RPB>();
+    compute_role<C, D, NT, RPB>();
   }
   // ---- teardown: everyone meets here, then the allocating warp returns the TMEM columns ----
   tc_fence_before();
@@ -1537,30 +1408,30 @@ bool make_weight_map(CUtensorMap* m, const void* w, int rows, int cols, int box_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int C, int D, int NT, bool BLOCKED, bool RPB>
+template <int C, int D, int NT, bool RPB>
 int launch_tc_one(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
-  cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<C, D, NT, BLOCKED, RPB>,
+  cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<C, D, NT, RPB>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
-  layer_tc_kernel<C, D, NT, BLOCKED, RPB><<<grid, kThreads, smem, ctx->stream>>>(a, g, maps, ctx->status);
+  layer_tc_kernel<C, D, NT, RPB><<<grid, kThreads, smem, ctx->stream>>>(a, g, maps, ctx->status);
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
 }
 
 // The position bias is a compile-time variant: a layer without one runs a kernel that holds none of its code.
-template <int C, int D, int NT, bool BLOCKED>
+template <int C, int D, int NT>
 int launch_tc(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
-  if (g.rb_len != 0) return launch_tc_one<C, D, NT, BLOCKED, true>(ctx, a, g, maps, grid, smem);
-  return launch_tc_one<C, D, NT, BLOCKED, false>(ctx, a, g, maps, grid, smem);
+  if (g.rb_len != 0) return launch_tc_one<C, D, NT, true>(ctx, a, g, maps, grid, smem);
+  return launch_tc_one<C, D, NT, false>(ctx, a, g, maps, grid, smem);
 }
 
 template <int C, int D>
 int launch_tc_nt(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
-  // up to set size 48 the attention runs per 16-row block (key blocks: ceil((2 tau + 14) / 8)); larger
-  // sets keep one item per set (key blocks: ceil(tau / 8))
-  if (g.tau <= 36) return launch_tc<C, D, 11, true>(ctx, a, g, maps, grid, smem);
-  if (g.tau <= 48) return launch_tc<C, D, 14, true>(ctx, a, g, maps, grid, smem);
-  return launch_tc<C, D, 12, false>(ctx, a, g, maps, grid, smem);
+  // NT = key blocks of 8 a 16-row block can need: the rows of every set it touches, ceil((2 tau + 14) / 8), at most
+  // the 16 blocks of a whole tile
+  if (g.tau <= 36) return launch_tc<C, D, 11>(ctx, a, g, maps, grid, smem);
+  if (g.tau <= 48) return launch_tc<C, D, 14>(ctx, a, g, maps, grid, smem);
+  return launch_tc<C, D, 16>(ctx, a, g, maps, grid, smem);
 }
 
 }  // namespace
