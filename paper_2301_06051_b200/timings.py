@@ -88,7 +88,8 @@ def time_bev(cid: int, steps: int, device: int = 0):
 def add_position_bias(cfg, seed: int = 0):
     """Gives every layer of a single-stage configuration a random relative position bias table for its window."""
     rng = np.random.default_rng(seed)
-    L, W, H = cfg["window"]
+    wins = [cfg["window"]] + [w for w, _ in cfg.get("block_windows") or []]
+    L, W, H = (max(w[a] for w in wins) for a in range(3))  # one table extent that covers every block's windows
     for blk in cfg["blocks"]:
         for layer in blk:
             layer["rpb"] = rng.standard_normal((cfg["heads"], (2 * L - 1) * (2 * W - 1) * (2 * H - 1))).astype(np.float32)
@@ -99,8 +100,6 @@ def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False, rpb
     cfg = di.make_config(cid)
     if cfg.get("stages"):
         return time_staged(cfg, steps, device)
-    if rpb:
-        add_position_bias(cfg)
     dev = torch.device("cuda", device)
     if hybrid:
         # hybrid window partition (Sec. 3.2): every second block works on windows twice as large in x and y,
@@ -108,6 +107,8 @@ def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False, rpb
         w = cfg["window"]
         big = (2 * w[0], 2 * w[1], w[2])
         cfg["block_windows"] = [(w, None) if i % 2 == 0 else (big, (w[0], w[1], 0)) for i in range(len(cfg["blocks"]))]
+    if rpb:
+        add_position_bias(cfg)
     bb = pipeline.Backbone(cfg, device=device)
     coords = torch.from_numpy(cfg["coords"]).to(dev)
     x = torch.from_numpy(cfg["feats"]).to(dev)
@@ -124,8 +125,9 @@ def time_config(cid: int, steps: int, device: int = 0, hybrid: bool = False, rpb
     def run_stage(stage, c, src, dst, tag):
         stage.partition(c)
         mark(tag + "partition")
-        for blk in stage.blocks:
-            bb.ctx.block(src, stage.tables[0], stage.tables[1], blk, dst, coords=c)
+        for blk, sp in zip(stage.blocks, stage.specs):
+            t = stage.tables_of[sp]  # (hybrid windows: every block runs on the tables of its own cut)
+            bb.ctx.block(src, t[0], t[1], blk, dst, coords=c)
             src = dst
         mark(tag + "blocks")
 
