@@ -795,6 +795,8 @@ __device__ __noinline__ void phase_row_list() {
   const int32_t* __restrict__ table = s_mi.table;
   const int32_t* __restrict__ rowoff = s_mi.rowoff;
   const int n = s_mi.n, tau = s_mi.tau, s_lo = s_mi.s_lo, nsets = s_mi.nsets, base = s_mi.base;
+  // (runs once per CTA: loops kept rolled, the kernel's text is better spent elsewhere)
+#pragma unroll 1
   for (int si = warp; si < nsets; si += kComputeWarps) {
     const int s = s_lo + si;
     const int32_t* trow = table + (size_t)s * tau;
@@ -802,6 +804,7 @@ __device__ __noinline__ void phase_row_list() {
     const int cnt_max = (lb >= 0 && lb < kTM) ? min(cap, kTM - lb) : 0;
     int cnt = 0;
     int lo3[3] = {INT_MAX, INT_MAX, INT_MAX}, hi3[3] = {INT_MIN, INT_MIN, INT_MIN};
+#pragma unroll 1
     for (int k0 = 0; k0 < tau; k0 += 32) {
       const int k = k0 + lane;
       int v = -1;
@@ -821,6 +824,7 @@ __device__ __noinline__ void phase_row_list() {
       }
       cnt += __popc(bal);
     }
+#pragma unroll 1
     for (int i = lane; i < cnt_max; i += 32) {
       s_mi.row_lo[0][lb + i] = (unsigned char)lb;
       s_mi.row_n[0][lb + i] = (unsigned char)cnt_max;
