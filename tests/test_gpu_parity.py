@@ -405,6 +405,9 @@ def test_frame_stream_overlaps_copies_without_mixing_frames(gpu):
     ((60, 60, 1), (2, 2, 1), 2, 5000, 128, 8, True, True),     # several tiles per CTA, ragged last tile
     ((30, 30, 4), (3, 3, 2), 1, 2500, 64, 4, False, True),      # 18 slots per region
     ((50, 50, 1), (2, 1, 1), 1, 2000, 128, 4, False, True),     # 2 slots: 64 regions per tile
+    ((36, 36, 2), (2, 2, 2), 1, 1500, 64, 8, True, True),       # head dim 8
+    ((40, 40, 1), (2, 2, 1), 1, 1200, 192, 4, True, True),      # head dim 48
+    ((260, 260, 1), (2, 2, 1), 1, 45000, 64, 4, False, True),   # more tiles than SMs: several tiles per CTA
 ])
 def test_pool_matches_oracle(gpu, oracle, grid, pool, batch, n, C, heads, with_pe, bf16, mask_empty):
     rng = np.random.default_rng(n + C)
