@@ -187,11 +187,17 @@ class Context:
             raise RuntimeError("the DSVT library needs a CUDA device; there is no CPU path")
         self.device = torch.device("cuda", device)
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        self.limits = (int(max_voxels), int(max_windows), int(max_channels))
         self._h = C.c_void_p()
         rc = self.lib.dsvt_create(C.byref(self._h), device, C.c_void_p(self.stream.cuda_stream), int(max_voxels),
                                   int(max_windows), int(max_channels))
         if rc != OK:
             raise DsvtError(rc, "dsvt_create")
+
+    def sibling(self, stream: torch.cuda.Stream) -> "Context":
+        """A second context with the same limits on the same device, bound to `stream` (its own workspace and
+        status word: calls on the two contexts may overlap on the GPU)."""
+        return Context(*self.limits, device=self.device.index, stream=stream)
 
     def close(self):
         if self._h:

@@ -36,40 +36,62 @@ class Stage:
             (tuple(w), None if sh is None else tuple(sh)) for w, sh in block_windows]
         assert len(specs) == len(self.blocks)
         self.specs = specs
-        self.tables_of = {}
-        for sp in specs:
-            if sp not in self.tables_of:
-                self.tables_of[sp] = new_tables()
+        self._new_tables = new_tables
+        self.tables_of = self.new_table_set()
         self.tables = self.tables_of[specs[0]] if specs else new_tables()  # the first block's pair
 
-    def partition(self, coords: torch.Tensor):
-        for (window, shift), tables in self.tables_of.items():
-            self.ctx.partition_rotated(coords, self.batch, self.grid, window, self.set_size, out=tuple(tables),
-                                       shift=shift)
+    def new_table_set(self) -> Dict:
+        """One pair of set tables per distinct (window, shift) of the stage's blocks."""
+        out = {}
+        for sp in self.specs:
+            if sp not in out:
+                out[sp] = self._new_tables()
+        return out
+
+    def partition(self, coords: torch.Tensor, ctx: Optional[api.Context] = None, tables_of: Optional[Dict] = None):
+        """Fills the stage's tables, or those of another table set, through the stage's context or another one."""
+        ctx = self.ctx if ctx is None else ctx
+        for (window, shift), tables in (self.tables_of if tables_of is None else tables_of).items():
+            ctx.partition_rotated(coords, self.batch, self.grid, window, self.set_size, out=tuple(tables), shift=shift)
+
+    def run_blocks(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor,
+                   tables_of: Optional[Dict] = None) -> torch.Tensor:
+        """Every block on tables that are already filled; the result ends up in y."""
+        tables_of = self.tables_of if tables_of is None else tables_of
+        src = x
+        for blk, sp in zip(self.blocks, self.specs):
+            t = tables_of[sp]
+            self.ctx.block(src, t[0], t[1], blk, y, coords=coords)  # (coords: read by layers with a position bias)
+            src = y
+        return y
 
     def forward(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
         """Partition (both axes of every distinct window cut) then every block; the result ends up in y."""
         self.partition(coords)
-        src = x
-        for blk, sp in zip(self.blocks, self.specs):
-            t = self.tables_of[sp]
-            self.ctx.block(src, t[0], t[1], blk, y, coords=coords)  # (coords: read by layers with a position bias)
-            src = y
-        return y
+        return self.run_blocks(coords, x, y)
 
 
 class FrameStream:
     """Runs frames that live in pinned host memory through a Stage with the copies off the critical path: frame
     k + 1 is uploaded and frame k - 1 downloaded while frame k's kernels run (one upload stream, the context's
     stream for the kernels, one download stream; `depth` sets of device buffers).  Every frame is still copied in,
-    computed and copied out in full; only the waiting is overlapped."""
+    computed and copied out in full; only the waiting is overlapped.  With `partition_ahead` the set tables of
+    frame k + 1 (which need its coordinates only) are built on a fourth stream through a second context, into
+    that frame's own table set, while frame k's blocks run: the partition's short kernels fill the SMs a layer
+    launch leaves idle towards its end instead of standing between two frames' layer launches."""
 
-    def __init__(self, stage: Stage, max_voxels: int, C: int, depth: int = 2):
+    def __init__(self, stage: Stage, max_voxels: int, C: int, depth: int = 2, partition_ahead: bool = True):
         self.stage, self.depth = stage, int(depth)
         ctx = stage.ctx
         dev = ctx.device
         self.compute = ctx.stream
         self.up, self.down = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        self.prep = self.prep_ctx = None
+        if partition_ahead:
+            self.prep = torch.cuda.Stream(dev)
+            self.prep_ctx = ctx.sibling(self.prep)
+            self.tables = [stage.new_table_set() for _ in range(self.depth)]
+            self.partitioned = [torch.cuda.Event() for _ in range(self.depth)]
         cap = max(int(max_voxels), 1)
         self.coords = [torch.empty((cap, 4), dtype=torch.int32, device=dev) for _ in range(self.depth)]
         self.x = [torch.empty((cap, C), dtype=torch.float32, device=dev) for _ in range(self.depth)]
@@ -98,8 +120,19 @@ class FrameStream:
         if reuse:
             self.compute.wait_event(self.downloaded[s])  # y[s] of that frame has reached the host
         y = self.y[s][:n]
+        if self.prep is not None:
+            self.prep.wait_event(self.uploaded[s])
+            if reuse:
+                self.prep.wait_event(self.computed[s])  # the blocks that last read this table set are done
+            with torch.cuda.stream(self.prep):
+                self.stage.partition(c, ctx=self.prep_ctx, tables_of=self.tables[s])
+                self.partitioned[s].record(self.prep)
+            self.compute.wait_event(self.partitioned[s])
         with torch.cuda.stream(self.compute):
-            self.stage.forward(c, x, y)
+            if self.prep is not None:
+                self.stage.run_blocks(c, x, y, tables_of=self.tables[s])
+            else:
+                self.stage.forward(c, x, y)
             self.computed[s].record(self.compute)
         with torch.cuda.stream(self.down):
             self.down.wait_event(self.computed[s])
@@ -112,6 +145,15 @@ class FrameStream:
         self.down.synchronize()
         self.compute.synchronize()
         self.up.synchronize()
+        if self.prep is not None:
+            self.prep.synchronize()
+
+    def status_sync(self) -> int:
+        """Synchronises and returns (and clears) the device status bits of every context the stream uses."""
+        bits = self.stage.ctx.status_sync()
+        if self.prep_ctx is not None:
+            bits |= self.prep_ctx.status_sync()
+        return bits
 
 
 class Backbone:

@@ -363,9 +363,11 @@ def test_in_place_and_repeatability(gpu):
     assert np.array_equal(a, b)  # no atomics on the float path: bitwise repeatable
 
 
-def test_frame_stream_overlaps_copies_without_mixing_frames(gpu):
-    """Seven different frames (different sizes and contents) through pipeline.FrameStream with two buffer sets:
-    every host output equals the frame's own device-resident run."""
+@pytest.mark.parametrize("partition_ahead", [False, True])
+def test_frame_stream_overlaps_copies_without_mixing_frames(gpu, partition_ahead):
+    """Seven different frames (different sizes and contents) through pipeline.FrameStream with two buffer sets,
+    with and without the next frame's partition running ahead on its own stream: every host output equals the
+    frame's own device-resident run."""
     from paper_2301_06051_b200 import pipeline
 
     base = di.make_config(2, n_override=9000)
@@ -380,11 +382,11 @@ def test_frame_stream_overlaps_copies_without_mixing_frames(gpu):
         feats = rng.standard_normal((n, base["C"]), dtype=np.float32)
         frames.append((torch.from_numpy(coords).pin_memory(), torch.from_numpy(feats).pin_memory(),
                        torch.full((n, base["C"]), 5.0).pin_memory()))
-    fs = pipeline.FrameStream(st, n_max, base["C"], depth=2)
+    fs = pipeline.FrameStream(st, n_max, base["C"], depth=2, partition_ahead=partition_ahead)
     for c, f, o in frames:
         fs.submit(c, f, o)
     fs.wait()
-    assert ctx.status_sync() == 0
+    assert fs.status_sync() == 0
     for c, f, o in frames:
         y = torch.empty((f.shape[0], base["C"]), device="cuda")
         st.forward(c.cuda(), f.cuda(), y)
