@@ -226,13 +226,14 @@ def run_ours(args):
         stage.forward(coords, x, y)
 
     # end to end: every step uploads its frame from pinned host memory, runs the step and downloads the result;
-    # pipeline.FrameStream overlaps the copies of neighbouring steps with the kernels (two sets of device buffers)
-    frames = pipeline.FrameStream(stage, n, C, depth=2)
-    outs_h = [out_h, torch.empty((n, C), dtype=torch.float32).pin_memory()]
+    # pipeline.FrameStream overlaps the copies and the partition of neighbouring steps with the kernels and alternates
+    # the steps between two compute streams (four sets of device buffers)
+    frames = pipeline.FrameStream(stage, n, C, depth=4, lanes=2)
+    outs_h = [out_h] + [torch.empty((n, C), dtype=torch.float32).pin_memory() for _ in range(3)]
 
     def run_e2e(steps):
         for k in range(steps):
-            frames.submit(coords_h, feats_h, outs_h[k & 1])
+            frames.submit(coords_h, feats_h, outs_h[k & 3])
         frames.wait()
 
     for _ in range(max(args.warmup, 3)):
@@ -242,13 +243,43 @@ def run_ours(args):
     if ctx.status_sync() != 0:
         raise SystemExit("device status word is not clean after warm-up")
 
-    # ---- timed region: K steps, L2 flushed (outside the events) before each ----
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3 + nb)] for _ in range(args.steps)]
+    # ---- timed region: K steps, inputs resident in HBM, through the pipeline a stream of frames runs in: the next
+    # step's partition on its own stream, consecutive steps alternating between two compute streams.  The steps
+    # rotate over four sets of (coords, x, y), 199 MB at configuration 2: larger than L2. ----
+    R = 4
+    cs = [coords] + [coords.clone() for _ in range(R - 1)]
+    xs = [x] + [x.clone() for _ in range(R - 1)]
+    ys = [torch.empty_like(x) for _ in range(R)]
+    resident = pipeline.FrameStream(stage, n, C, depth=R, lanes=2)
+    for k in range(2 * R):
+        resident.submit_resident(cs[k % R], xs[k % R], ys[k % R])
+    barrier()
+    if resident.status_sync() != 0:
+        raise SystemExit("device status word is not clean after the pipeline's warm-up")
+    ev_begin, ev_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local_rank)
     sampler.start()
-    launches0 = ctx.launch_count()
+    launches0 = resident.launch_count()
     barrier()
     t_begin = time.perf_counter()
+    ev_begin.record(stream)
+    resident.fence(ev_begin)
+    for k in range(args.steps):
+        resident.submit_resident(cs[k % R], xs[k % R], ys[k % R])
+    resident.join(stream)
+    ev_end.record(stream)
+    barrier()
+    t_end = time.perf_counter()
+    launches = resident.launch_count() - launches0
+    clocks = sampler.stop(t_begin, t_end)
+    total_ms = float(ev_begin.elapsed_time(ev_end))
+    if resident.status_sync() != 0:
+        raise SystemExit("device status word is not clean after the timed region")
+
+    # ---- one step at a time on one stream, L2 flushed (outside the events) before each: the latency of a step and
+    # its parts (partition, blocks, layer launch), which the roofline figure is taken from ----
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3 + nb)] for _ in range(args.steps)]
+    barrier()
     for k in range(args.steps):
         flush.zero_()
         e = ev[k]
@@ -261,23 +292,21 @@ def run_ours(args):
             src = y
             e[2 + b].record(stream)
     barrier()
-    t_end = time.perf_counter()
-    launches = ctx.launch_count() - launches0
-    clocks = sampler.stop(t_begin, t_end)
     t_step = np.array([e[0].elapsed_time(e[1 + nb]) for e in ev])  # ms
     t_part = np.array([e[0].elapsed_time(e[1]) for e in ev])
     t_blocks = np.array([[e[1 + b].elapsed_time(e[2 + b]) for b in range(nb)] for e in ev])
-    total_ms = float(t_step.sum())
+    if any(not torch.equal(o, y) for o in ys):
+        raise SystemExit("pipelined outputs differ from the one-step-at-a-time run")
 
     # ---- end to end through the public API with pinned host buffers ----
-    run_e2e(3)
+    run_e2e(4)
     barrier()
     e_steps = max(3, min(args.steps, 200))  # (the first upload and the last download are not overlapped)
     t0 = time.perf_counter()
     run_e2e(e_steps)
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e_steps
-    if not torch.equal(outs_h[0], outs_h[1]) or not torch.equal(outs_h[0], y.cpu()):
+    if any(not torch.equal(o, outs_h[0]) for o in outs_h[1:]) or not torch.equal(outs_h[0], y.cpu()):
         raise SystemExit("end-to-end outputs differ from the device-resident run")
     if frames.status_sync() != 0:
         raise SystemExit("device status word is not clean after the end-to-end steps")
@@ -323,22 +352,30 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if cfg["precision"] == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": workload_name(args.config, cfg),
-                   "l2": "L2 flushed by a %d MiB write before every step" % (L2_FLUSH_BYTES >> 20),
+                   "l2": "timed steps rotate over %d sets of inputs and outputs (%d MB, larger than L2); the "
+                         "one-step-at-a-time figures: L2 flushed by a %d MiB write before every step"
+                         % (R, R * (2 * x.numel() + coords.numel()) * 4 // 1000000, L2_FLUSH_BYTES >> 20),
+                   "pipeline": "inputs resident in HBM; the next step's partition on its own stream, consecutive "
+                               "steps alternate between two compute streams; CUDA events around all K steps",
                    "num_sets": S, "pad_ratio": pad, "frames_per_rank": 1},
         "frames_per_sec": world / (ms_per_step * 1e-3),
+        "step_latency_ms": float(t_step.mean()),
         "t_partition_ms": float(t_part.mean()), "t_block_ms": float(t_blocks.mean()),
         "clocks": clocks,
         "e2e": {"value": job_throughput(world, n * nb, e2e_ms), "unit": "voxels/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(coords_h.numel() * 4 + feats_h.numel() * 4),
                 "d2h_bytes_per_step": int(out_h.numel() * 4), "steps": e_steps,
                 "how": "pipeline.FrameStream: per step one upload, one backbone pass, one download; copies of "
-                       "neighbouring steps overlap the kernels and the next step's partition runs on its own stream "
-                       "under the current step's layer launches; wall clock over all steps"},
+                       "neighbouring steps overlap the kernels, the next step's partition runs on its own stream "
+                       "under the current step's layer launches, consecutive steps alternate between two compute "
+                       "streams; wall clock over all steps"},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "fused DSVT layer", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                      "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"], "peak_source": peaks["source"],
                      "flops_per_launch": flops_per_launch, "ms_per_launch": layer_ms,
+                     "timing": "launch duration from the one-step-at-a-time run (a launch alone on the GPU)",
+                     "achieved_in_pipeline": flops_per_launch * 2 * nb / (ms_per_step * 1e-3) / 1e12,
                      "traffic": LAYER_DRAM_BYTES_PER_LAUNCH if args.config == 2 else None},
         "cpu_baseline": cpu,
     }))

@@ -55,13 +55,14 @@ class Stage:
             ctx.partition_rotated(coords, self.batch, self.grid, window, self.set_size, out=tuple(tables), shift=shift)
 
     def run_blocks(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor,
-                   tables_of: Optional[Dict] = None) -> torch.Tensor:
+                   tables_of: Optional[Dict] = None, ctx: Optional[api.Context] = None) -> torch.Tensor:
         """Every block on tables that are already filled; the result ends up in y."""
         tables_of = self.tables_of if tables_of is None else tables_of
+        ctx = self.ctx if ctx is None else ctx
         src = x
         for blk, sp in zip(self.blocks, self.specs):
             t = tables_of[sp]
-            self.ctx.block(src, t[0], t[1], blk, y, coords=coords)  # (coords: read by layers with a position bias)
+            ctx.block(src, t[0], t[1], blk, y, coords=coords)  # (coords: read by layers with a position bias)
             src = y
         return y
 
@@ -76,15 +77,22 @@ class FrameStream:
     k + 1 is uploaded and frame k - 1 downloaded while frame k's kernels run (one upload stream, the context's
     stream for the kernels, one download stream; `depth` sets of device buffers).  Every frame is still copied in,
     computed and copied out in full; only the waiting is overlapped.  With `partition_ahead` the set tables of
-    frame k + 1 (which need its coordinates only) are built on a fourth stream through a second context, into
-    that frame's own table set, while frame k's blocks run: the partition's short kernels fill the SMs a layer
-    launch leaves idle towards its end instead of standing between two frames' layer launches."""
+    frame k + 1 (which need its coordinates only) are built on a stream of their own through a second context,
+    into that frame's own table set, while frame k's blocks run: the partition's short kernels fill the SMs a
+    layer launch leaves idle towards its end instead of standing between two frames' layer launches.  With
+    `lanes` = 2, consecutive frames alternate between two compute streams (each with its own context), so that a
+    layer launch of one frame starts on the SMs the other frame's launch has already left: frames are
+    independent, and a launch of one CTA per SM with an odd number of tiles leaves SMs idle for its second half."""
 
-    def __init__(self, stage: Stage, max_voxels: int, C: int, depth: int = 2, partition_ahead: bool = True):
-        self.stage, self.depth = stage, int(depth)
+    def __init__(self, stage: Stage, max_voxels: int, C: int, depth: int = 2, partition_ahead: bool = True,
+                 lanes: int = 1):
+        self.stage, self.depth, self.lanes = stage, int(depth), int(lanes)
+        assert self.lanes == 1 or (partition_ahead and self.depth >= 2 * self.lanes), \
+            "several lanes need partition_ahead and two buffer sets per lane"
         ctx = stage.ctx
         dev = ctx.device
-        self.compute = ctx.stream
+        self.compute = [ctx.stream] + [torch.cuda.Stream(dev) for _ in range(self.lanes - 1)]
+        self.ctxs = [ctx] + [ctx.sibling(st) for st in self.compute[1:]]
         self.up, self.down = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
         self.prep = self.prep_ctx = None
         if partition_ahead:
@@ -92,14 +100,50 @@ class FrameStream:
             self.prep_ctx = ctx.sibling(self.prep)
             self.tables = [stage.new_table_set() for _ in range(self.depth)]
             self.partitioned = [torch.cuda.Event() for _ in range(self.depth)]
-        cap = max(int(max_voxels), 1)
-        self.coords = [torch.empty((cap, 4), dtype=torch.int32, device=dev) for _ in range(self.depth)]
-        self.x = [torch.empty((cap, C), dtype=torch.float32, device=dev) for _ in range(self.depth)]
-        self.y = [torch.empty((cap, C), dtype=torch.float32, device=dev) for _ in range(self.depth)]
+        self.cap, self.C = max(int(max_voxels), 1), int(C)
+        self.coords = self.x = self.y = None  # device copies of host frames: allocated by the first submit()
         self.uploaded = [torch.cuda.Event() for _ in range(self.depth)]
         self.computed = [torch.cuda.Event() for _ in range(self.depth)]
         self.downloaded = [torch.cuda.Event() for _ in range(self.depth)]
         self.count = 0
+
+    def _streams(self):
+        return self.compute + [self.up, self.down] + ([self.prep] if self.prep is not None else [])
+
+    def fence(self, event: torch.cuda.Event) -> None:
+        """Nothing submitted from now on starts before `event` has happened."""
+        for st in self._streams():
+            st.wait_event(event)
+
+    def join(self, stream: torch.cuda.Stream) -> None:
+        """Makes `stream` wait for everything submitted so far."""
+        for st in self._streams():
+            if st != stream:
+                e = torch.cuda.Event()
+                e.record(st)
+                stream.wait_event(e)
+
+    def submit_resident(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor) -> None:
+        """Enqueues one frame that already lives in device memory (no copies): partition on the look-ahead stream,
+        blocks on the frame's lane, result in y.  The caller rotates over `depth` sets of (coords, x, y): a set may
+        be handed in again once `depth` - 1 other frames have been submitted after it."""
+        assert self.prep is not None and self.depth % self.lanes == 0
+        s = self.count % self.depth
+        lane = self.count % self.lanes
+        compute, ctx = self.compute[lane], self.ctxs[lane]
+        if self.count >= self.depth:
+            self.prep.wait_event(self.computed[s])  # the blocks that last read this table set are done
+        with torch.cuda.stream(self.prep):
+            self.stage.partition(coords, ctx=self.prep_ctx, tables_of=self.tables[s])
+            self.partitioned[s].record(self.prep)
+        compute.wait_event(self.partitioned[s])
+        with torch.cuda.stream(compute):  # (the frame that last wrote y ran on this lane: same stream, in order)
+            self.stage.run_blocks(coords, x, y, tables_of=self.tables[s], ctx=ctx)
+            self.computed[s].record(compute)
+        self.count += 1
+
+    def launch_count(self) -> int:
+        return sum(c.launch_count() for c in self.ctxs + ([self.prep_ctx] if self.prep_ctx is not None else []))
 
     def submit(self, coords_h: torch.Tensor, feats_h: torch.Tensor, out_h: torch.Tensor) -> None:
         """Enqueues one frame: coords_h int32 [n, 4], feats_h float32 [n, C], out_h float32 [n, C], all pinned host
@@ -107,7 +151,14 @@ class FrameStream:
         caller is `depth` frames ahead of the device."""
         assert coords_h.is_pinned() and feats_h.is_pinned() and out_h.is_pinned(), "pinned host memory only"
         n = int(feats_h.shape[0])
+        if self.x is None:
+            dev = self.stage.ctx.device
+            self.coords = [torch.empty((self.cap, 4), dtype=torch.int32, device=dev) for _ in range(self.depth)]
+            self.x = [torch.empty((self.cap, self.C), dtype=torch.float32, device=dev) for _ in range(self.depth)]
+            self.y = [torch.empty((self.cap, self.C), dtype=torch.float32, device=dev) for _ in range(self.depth)]
         s = self.count % self.depth
+        lane = self.count % self.lanes
+        compute, ctx = self.compute[lane], self.ctxs[lane]
         reuse = self.count >= self.depth
         with torch.cuda.stream(self.up):
             if reuse:
@@ -116,9 +167,9 @@ class FrameStream:
             c.copy_(coords_h, non_blocking=True)
             x.copy_(feats_h, non_blocking=True)
             self.uploaded[s].record(self.up)
-        self.compute.wait_event(self.uploaded[s])
+        compute.wait_event(self.uploaded[s])
         if reuse:
-            self.compute.wait_event(self.downloaded[s])  # y[s] of that frame has reached the host
+            compute.wait_event(self.downloaded[s])  # y[s] of that frame has reached the host
         y = self.y[s][:n]
         if self.prep is not None:
             self.prep.wait_event(self.uploaded[s])
@@ -127,13 +178,13 @@ class FrameStream:
             with torch.cuda.stream(self.prep):
                 self.stage.partition(c, ctx=self.prep_ctx, tables_of=self.tables[s])
                 self.partitioned[s].record(self.prep)
-            self.compute.wait_event(self.partitioned[s])
-        with torch.cuda.stream(self.compute):
+            compute.wait_event(self.partitioned[s])
+        with torch.cuda.stream(compute):
             if self.prep is not None:
-                self.stage.run_blocks(c, x, y, tables_of=self.tables[s])
+                self.stage.run_blocks(c, x, y, tables_of=self.tables[s], ctx=ctx)
             else:
                 self.stage.forward(c, x, y)
-            self.computed[s].record(self.compute)
+            self.computed[s].record(compute)
         with torch.cuda.stream(self.down):
             self.down.wait_event(self.computed[s])
             out_h.copy_(y, non_blocking=True)
@@ -143,16 +194,17 @@ class FrameStream:
     def wait(self) -> None:
         """Blocks until every submitted frame's output is in its host tensor."""
         self.down.synchronize()
-        self.compute.synchronize()
+        for st in self.compute:
+            st.synchronize()
         self.up.synchronize()
         if self.prep is not None:
             self.prep.synchronize()
 
     def status_sync(self) -> int:
         """Synchronises and returns (and clears) the device status bits of every context the stream uses."""
-        bits = self.stage.ctx.status_sync()
-        if self.prep_ctx is not None:
-            bits |= self.prep_ctx.status_sync()
+        bits = 0
+        for ctx in self.ctxs + ([self.prep_ctx] if self.prep_ctx is not None else []):
+            bits |= ctx.status_sync()
         return bits
 
 

@@ -363,10 +363,10 @@ def test_in_place_and_repeatability(gpu):
     assert np.array_equal(a, b)  # no atomics on the float path: bitwise repeatable
 
 
-@pytest.mark.parametrize("partition_ahead", [False, True])
-def test_frame_stream_overlaps_copies_without_mixing_frames(gpu, partition_ahead):
-    """Seven different frames (different sizes and contents) through pipeline.FrameStream with two buffer sets,
-    with and without the next frame's partition running ahead on its own stream: every host output equals the
+@pytest.mark.parametrize("partition_ahead,lanes,depth", [(False, 1, 2), (True, 1, 2), (True, 2, 4)])
+def test_frame_stream_overlaps_copies_without_mixing_frames(gpu, partition_ahead, lanes, depth):
+    """Seven different frames (different sizes and contents) through pipeline.FrameStream: plain, with the next
+    frame's partition running ahead on its own stream, and with two compute lanes: every host output equals the
     frame's own device-resident run."""
     from paper_2301_06051_b200 import pipeline
 
@@ -382,7 +382,7 @@ def test_frame_stream_overlaps_copies_without_mixing_frames(gpu, partition_ahead
         feats = rng.standard_normal((n, base["C"]), dtype=np.float32)
         frames.append((torch.from_numpy(coords).pin_memory(), torch.from_numpy(feats).pin_memory(),
                        torch.full((n, base["C"]), 5.0).pin_memory()))
-    fs = pipeline.FrameStream(st, n_max, base["C"], depth=2, partition_ahead=partition_ahead)
+    fs = pipeline.FrameStream(st, n_max, base["C"], depth=depth, partition_ahead=partition_ahead, lanes=lanes)
     for c, f, o in frames:
         fs.submit(c, f, o)
     fs.wait()
@@ -391,6 +391,44 @@ def test_frame_stream_overlaps_copies_without_mixing_frames(gpu, partition_ahead
         y = torch.empty((f.shape[0], base["C"]), device="cuda")
         st.forward(c.cuda(), f.cuda(), y)
         assert torch.equal(y.cpu(), o)
+
+
+def test_frame_stream_resident_frames_on_two_lanes(gpu):
+    """Ten device-resident frames (four rotating buffer sets, different sizes and contents) through the two-lane
+    pipeline with the partition running ahead: every output equals the frame's own single-stream run."""
+    from paper_2301_06051_b200 import pipeline
+
+    base = di.make_config(2, n_override=8000)
+    n_max = 8000
+    ctx = gpu.Context(n_max, _nwin(base["batch"], base["grid"], base["window"]), base["C"])
+    st = pipeline.Stage(ctx, base["blocks"][:2], base["batch"], base["grid"], base["window"], base["set_size"],
+                        precision_of(base), n_max)
+    fs = pipeline.FrameStream(st, n_max, base["C"], depth=4, lanes=2)
+    sizes = [8000, 3000, 1, 7999, 5000, 6500, 2, 4000, 8000, 1000]
+    bufs = [(torch.empty((n_max, 4), dtype=torch.int32, device="cuda"), torch.empty((n_max, base["C"]), device="cuda"),
+             torch.empty((n_max, base["C"]), device="cuda")) for _ in range(4)]
+    want, got = [], []
+    for k, n in enumerate(sizes):
+        rng = np.random.default_rng(500 + k)
+        c = torch.from_numpy(di.unique_cells(rng, n, base["grid"], base["batch"])).cuda()
+        f = torch.from_numpy(rng.standard_normal((n, base["C"]), dtype=np.float32)).cuda()
+        y = torch.empty_like(f)
+        st.forward(c, f, y)
+        want.append(y.cpu())
+        torch.cuda.synchronize()
+        if k >= 4:  # the set is handed in again: its previous frame's result must have been read first
+            fs.join(torch.cuda.current_stream())
+            got.append(bufs[k % 4][2][: sizes[k - 4]].cpu())
+        cb, xb, yb = bufs[k % 4]
+        cb[:n].copy_(c); xb[:n].copy_(f)
+        torch.cuda.synchronize()
+        fs.submit_resident(cb[:n], xb[:n], yb[:n])
+    fs.wait()
+    for k in range(len(sizes) - 4, len(sizes)):
+        got.append(bufs[k % 4][2][: sizes[k]].cpu())
+    assert fs.status_sync() == 0
+    for k, (g, w) in enumerate(zip(got, want)):
+        assert torch.equal(g, w), "frame %d" % k
 
 
 # ------------------------------------------------------------------------------------------------
