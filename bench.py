@@ -226,14 +226,17 @@ def run_ours(args):
         stage.forward(coords, x, y)
 
     # end to end: every step uploads its frame from pinned host memory, runs the step and downloads the result;
-    # pipeline.FrameStream overlaps the copies and the partition of neighbouring steps with the kernels and alternates
-    # the steps between two compute streams (four sets of device buffers)
-    frames = pipeline.FrameStream(stage, n, C, depth=4, lanes=2)
-    outs_h = [out_h] + [torch.empty((n, C), dtype=torch.float32).pin_memory() for _ in range(3)]
+    # pipeline.FrameStream overlaps the copies and the partition of neighbouring steps with the kernels and deals
+    # the steps out to four compute streams (eight sets of device buffers)
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    LANES, R = 4, 8                 # compute streams, rotating sets of buffers
+    lane_ctas = (sms + 2) // 3      # CTAs per layer launch: the four lanes ask for more CTAs than there are SMs
+    frames = pipeline.FrameStream(stage, n, C, depth=R, lanes=LANES, layer_ctas=lane_ctas)
+    outs_h = [out_h] + [torch.empty((n, C), dtype=torch.float32).pin_memory() for _ in range(R - 1)]
 
     def run_e2e(steps):
         for k in range(steps):
-            frames.submit(coords_h, feats_h, outs_h[k & 3])
+            frames.submit(coords_h, feats_h, outs_h[k % R])
         frames.wait()
 
     for _ in range(max(args.warmup, 3)):
@@ -244,13 +247,13 @@ def run_ours(args):
         raise SystemExit("device status word is not clean after warm-up")
 
     # ---- timed region: K steps, inputs resident in HBM, through the pipeline a stream of frames runs in: the next
-    # step's partition on its own stream, consecutive steps alternating between two compute streams.  The steps
-    # rotate over four sets of (coords, x, y), 199 MB at configuration 2: larger than L2. ----
-    R = 4
+    # step's partition on its own stream, consecutive steps dealt out to four compute streams whose layer launches
+    # take a third of the SMs each.  The steps rotate over eight sets of (coords, x, y), 397 MB at configuration 2:
+    # larger than L2. ----
     cs = [coords] + [coords.clone() for _ in range(R - 1)]
     xs = [x] + [x.clone() for _ in range(R - 1)]
     ys = [torch.empty_like(x) for _ in range(R)]
-    resident = pipeline.FrameStream(stage, n, C, depth=R, lanes=2)
+    resident = pipeline.FrameStream(stage, n, C, depth=R, lanes=LANES, layer_ctas=lane_ctas)
     for k in range(2 * R):
         resident.submit_resident(cs[k % R], xs[k % R], ys[k % R])
     barrier()
@@ -299,7 +302,7 @@ def run_ours(args):
         raise SystemExit("pipelined outputs differ from the one-step-at-a-time run")
 
     # ---- end to end through the public API with pinned host buffers ----
-    run_e2e(4)
+    run_e2e(R)
     barrier()
     e_steps = max(3, min(args.steps, 200))  # (the first upload and the last download are not overlapped)
     t0 = time.perf_counter()
@@ -356,7 +359,8 @@ def run_ours(args):
                          "one-step-at-a-time figures: L2 flushed by a %d MiB write before every step"
                          % (R, R * (2 * x.numel() + coords.numel()) * 4 // 1000000, L2_FLUSH_BYTES >> 20),
                    "pipeline": "inputs resident in HBM; the next step's partition on its own stream, consecutive "
-                               "steps alternate between two compute streams; CUDA events around all K steps",
+                               "steps dealt out to %d compute streams, %d CTAs per layer launch; CUDA events around "
+                               "all K steps" % (LANES, lane_ctas),
                    "num_sets": S, "pad_ratio": pad, "frames_per_rank": 1},
         "frames_per_sec": world / (ms_per_step * 1e-3),
         "step_latency_ms": float(t_step.mean()),
@@ -367,7 +371,7 @@ def run_ours(args):
                 "d2h_bytes_per_step": int(out_h.numel() * 4), "steps": e_steps,
                 "how": "pipeline.FrameStream: per step one upload, one backbone pass, one download; copies of "
                        "neighbouring steps overlap the kernels, the next step's partition runs on its own stream "
-                       "under the current step's layer launches, consecutive steps alternate between two compute "
+                       "under the current step's layer launches, consecutive steps dealt out to four compute "
                        "streams; wall clock over all steps"},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "fused DSVT layer", "bound": "tensor", "achieved": achieved,

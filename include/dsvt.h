@@ -78,6 +78,13 @@ int dsvt_last_cuda_error(const dsvt_ctx* ctx);
 const char* dsvt_error_string(int code);
 /* Number of kernels this context has launched since it was created. */
 int64_t dsvt_launch_count(const dsvt_ctx* ctx);
+/* Caps the number of persistent CTAs (one per SM) the tensor-core layer kernel is launched with on this
+ * context: max_ctas >= 1, or 0 for "as many as the device has SMs" (the default).  A context that shares the
+ * GPU with other contexts' launches (several frames in flight on several streams) runs its tiles on fewer
+ * CTAs, each taking more tiles, so that a launch's set-up is spread over more work and launches of different
+ * frames run side by side.  No counterpart in the paper (a launch parameter).  Returns DSVT_ERR_INVALID_ARG
+ * for a NULL context or a negative value. */
+int dsvt_set_layer_ctas(dsvt_ctx* ctx, int32_t max_ctas);
 
 /*
  * Rotated set partition: Sec. 3.2 "Dynamic set partition" (window partition, Eq. 1 inner-window

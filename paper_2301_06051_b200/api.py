@@ -23,7 +23,7 @@ STATUS_BAD_COORD, STATUS_TABLE_OVERFLOW, STATUS_BAD_INDEX, STATUS_DUPLICATE_CELL
 
 EXPORTS = [
     "dsvt_create", "dsvt_destroy", "dsvt_status_sync", "dsvt_last_cuda_error", "dsvt_error_string",
-    "dsvt_launch_count", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_set_attention_rpb", "dsvt_layer", "dsvt_block", "dsvt_pool",
+    "dsvt_launch_count", "dsvt_set_layer_ctas", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_set_attention_rpb", "dsvt_layer", "dsvt_block", "dsvt_pool",
     "dsvt_bev_scatter",
 ]
 
@@ -68,6 +68,7 @@ def load():
     lib.dsvt_error_string.restype = C.c_char_p
     lib.dsvt_launch_count.argtypes = [vp]
     lib.dsvt_launch_count.restype = i64
+    lib.dsvt_set_layer_ctas.argtypes = [vp, i32]
     lib.dsvt_partition.argtypes = [vp, vp, i32, i32, p3, p3, i32, i32, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.dsvt_partition_rotated.argtypes = [vp, vp, i32, i32, p3, p3, i32, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.dsvt_partition_shifted.argtypes = [vp, vp, i32, i32, p3, p3, p3, i32, vp, i32, vp, vp, vp, vp, vp, vp]
@@ -224,6 +225,10 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.dsvt_launch_count(self._h))
+
+    def set_layer_ctas(self, max_ctas: int) -> None:
+        """Caps the tensor-core layer kernel's persistent CTAs on this context (0: one per SM)."""
+        self._check(self.lib.dsvt_set_layer_ctas(self._h, int(max_ctas)), "dsvt_set_layer_ctas")
 
     # ---- dsvt_partition ----
     def partition(self, coords: torch.Tensor, batch: int, grid, window, set_size: int, axis: int,

@@ -127,6 +127,7 @@ extern "C" int dsvt_create(dsvt_ctx** out, int device, void* cuda_stream, int64_
   c->max_windows = max_windows;
   c->max_channels = max_channels;
   c->sm_count = prop.multiProcessorCount;
+  c->layer_ctas = 0;
   c->last_cuda_error = 0;
   c->launches = 0;
   c->cell_map = nullptr;
@@ -173,6 +174,11 @@ extern "C" int dsvt_status_sync(dsvt_ctx* ctx, int32_t* bits) {
 
 extern "C" int dsvt_last_cuda_error(const dsvt_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 extern "C" int64_t dsvt_launch_count(const dsvt_ctx* ctx) { return ctx ? ctx->launches : 0; }
+extern "C" int dsvt_set_layer_ctas(dsvt_ctx* ctx, int32_t max_ctas) {
+  if (!ctx || max_ctas < 0) return DSVT_ERR_INVALID_ARG;
+  ctx->layer_ctas = max_ctas;
+  return DSVT_OK;
+}
 
 extern "C" const char* dsvt_error_string(int code) {
   switch (code) {

@@ -12,6 +12,7 @@ struct dsvt_ctx {
   int64_t max_voxels, max_windows;
   int32_t max_channels;
   int sm_count;
+  int layer_ctas;  // cap on the tensor-core layer kernel's grid (0: sm_count)
   int last_cuda_error;
   int64_t launches;
   // one device allocation carved into the arrays below

@@ -1500,6 +1500,7 @@ int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a) {
   // one CTA per SM, but no more CTAs than there can be sets
   int64_t grid = a.cap_sets < a.n ? a.cap_sets : a.n;
   if (grid > ctx->sm_count) grid = ctx->sm_count;
+  if (ctx->layer_ctas > 0 && grid > ctx->layer_ctas) grid = ctx->layer_ctas;
   if (grid < 1) grid = 1;
   const int d = C / p.heads;
   if (C == 192) return launch_tc_nt<192, 24>(ctx, a, g, maps, (int)grid, smem);

@@ -85,14 +85,19 @@ class FrameStream:
     independent, and a launch of one CTA per SM with an odd number of tiles leaves SMs idle for its second half."""
 
     def __init__(self, stage: Stage, max_voxels: int, C: int, depth: int = 2, partition_ahead: bool = True,
-                 lanes: int = 1):
+                 lanes: int = 1, layer_ctas: int = 0):
         self.stage, self.depth, self.lanes = stage, int(depth), int(lanes)
         assert self.lanes == 1 or (partition_ahead and self.depth >= 2 * self.lanes), \
             "several lanes need partition_ahead and two buffer sets per lane"
         ctx = stage.ctx
         dev = ctx.device
-        self.compute = [ctx.stream] + [torch.cuda.Stream(dev) for _ in range(self.lanes - 1)]
-        self.ctxs = [ctx] + [ctx.sibling(st) for st in self.compute[1:]]
+        if self.lanes == 1:  # the stage's own context and stream
+            self.compute, self.ctxs = [ctx.stream], [ctx]
+        else:  # every lane on a stream and a context of its own; `layer_ctas` caps their layer launches' CTAs
+            self.compute = [torch.cuda.Stream(dev) for _ in range(self.lanes)]
+            self.ctxs = [ctx.sibling(st) for st in self.compute]
+            for c in self.ctxs:
+                c.set_layer_ctas(layer_ctas)
         self.up, self.down = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
         self.prep = self.prep_ctx = None
         if partition_ahead:

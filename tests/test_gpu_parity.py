@@ -363,7 +363,7 @@ def test_in_place_and_repeatability(gpu):
     assert np.array_equal(a, b)  # no atomics on the float path: bitwise repeatable
 
 
-@pytest.mark.parametrize("partition_ahead,lanes,depth", [(False, 1, 2), (True, 1, 2), (True, 2, 4)])
+@pytest.mark.parametrize("partition_ahead,lanes,depth", [(False, 1, 2), (True, 1, 2), (True, 2, 4), (True, 4, 8)])
 def test_frame_stream_overlaps_copies_without_mixing_frames(gpu, partition_ahead, lanes, depth):
     """Seven different frames (different sizes and contents) through pipeline.FrameStream: plain, with the next
     frame's partition running ahead on its own stream, and with two compute lanes: every host output equals the
@@ -403,7 +403,7 @@ def test_frame_stream_resident_frames_on_two_lanes(gpu):
     ctx = gpu.Context(n_max, _nwin(base["batch"], base["grid"], base["window"]), base["C"])
     st = pipeline.Stage(ctx, base["blocks"][:2], base["batch"], base["grid"], base["window"], base["set_size"],
                         precision_of(base), n_max)
-    fs = pipeline.FrameStream(st, n_max, base["C"], depth=4, lanes=2)
+    fs = pipeline.FrameStream(st, n_max, base["C"], depth=4, lanes=2, layer_ctas=20)  # several tiles per CTA
     sizes = [8000, 3000, 1, 7999, 5000, 6500, 2, 4000, 8000, 1000]
     bufs = [(torch.empty((n_max, 4), dtype=torch.int32, device="cuda"), torch.empty((n_max, base["C"]), device="cuda"),
              torch.empty((n_max, base["C"]), device="cuda")) for _ in range(4)]
