@@ -393,6 +393,25 @@ def test_frame_stream_overlaps_copies_without_mixing_frames(gpu, partition_ahead
         assert torch.equal(y.cpu(), o)
 
 
+def test_layer_cta_cap_keeps_results_and_rejects_negative_values(gpu):
+    """dsvt_set_layer_ctas: a block on 7 CTAs (dozens of tiles each) is bitwise the block on one CTA per SM."""
+    cfg = di.make_config(2, n_override=20000)
+    n, C = cfg["n"], cfg["C"]
+    ctx = gpu.Context(n, _nwin(cfg["batch"], cfg["grid"], cfg["window"]), C)
+    coords, x = dev(cfg["coords"]), dev(cfg["feats"])
+    t0, t1 = ctx.partition_rotated(coords, cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"])
+    w = [gpu.device_weights(l, precision_of(cfg), ctx.device) for l in cfg["blocks"][0]]
+    full, capped = torch.empty_like(x), torch.empty_like(x)
+    ctx.block(x, t0, t1, w, full)
+    ctx.set_layer_ctas(7)
+    ctx.block(x, t0, t1, w, capped)
+    ctx.set_layer_ctas(0)
+    assert ctx.status_sync() == 0
+    assert torch.equal(full, capped)
+    with pytest.raises(gpu.DsvtError):
+        ctx.set_layer_ctas(-1)
+
+
 def test_frame_stream_resident_frames_on_two_lanes(gpu):
     """Ten device-resident frames (four rotating buffer sets, different sizes and contents) through the two-lane
     pipeline with the partition running ahead: every output equals the frame's own single-stream run."""
