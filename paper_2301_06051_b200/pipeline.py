@@ -80,9 +80,11 @@ class FrameStream:
     frame k + 1 (which need its coordinates only) are built on a stream of their own through a second context,
     into that frame's own table set, while frame k's blocks run: the partition's short kernels fill the SMs a
     layer launch leaves idle towards its end instead of standing between two frames' layer launches.  With
-    `lanes` = 2, consecutive frames alternate between two compute streams (each with its own context), so that a
-    layer launch of one frame starts on the SMs the other frame's launch has already left: frames are
-    independent, and a launch of one CTA per SM with an odd number of tiles leaves SMs idle for its second half."""
+    several `lanes`, consecutive frames are dealt out to that many compute streams (each with its own context), so
+    that a frame's layer launch starts on SMs as other frames' launches leave them: frames are independent, and a
+    launch of one CTA per SM whose tiles do not divide evenly leaves SMs idle towards its end.  `layer_ctas` caps
+    the CTAs of every lane's layer launches (0: one per SM); with the lanes together asking for somewhat more CTAs
+    than the GPU has SMs, each CTA takes more tiles per start-up and one is always waiting for an SM to come free."""
 
     def __init__(self, stage: Stage, max_voxels: int, C: int, depth: int = 2, partition_ahead: bool = True,
                  lanes: int = 1, layer_ctas: int = 0):
