@@ -258,11 +258,36 @@ int dsvt_layer(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* set_tabl
 /*
  * One DSVT block (Eq. 5): the layer with the X-axis table, then the layer with the Y-axis table.
  * layers: HOST array of two parameter structs.  y may alias x.  Every voxel must be covered by
- * both tables (true for tables made by dsvt_partition).
+ * both tables (true for tables made by dsvt_partition).  Same as dsvt_layers with two layers.
  */
 int dsvt_block(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* table_axis0, int32_t cap_sets0,
                const int32_t* num_sets0, const int32_t* set_rowoff0, const int32_t* table_axis1, int32_t cap_sets1,
                const int32_t* num_sets1, const int32_t* set_rowoff1, const dsvt_layer_params layers[2], float* y);
+
+/*
+ * A chain of DSVT layers, e.g. all blocks of a backbone stage (Sec. 3.2: the blocks are stacked, Eq. 5 gives the
+ * two layers of one): layer 0 reads x and writes y, every later layer runs in place on y; layer i runs on
+ * tables[i] with params[i] (for blocks that share their windows: the X-axis table, the Y-axis table, the X-axis
+ * table, ...; with hybrid windows each block brings its own pair).  The result equals num_layers dsvt_layer
+ * calls.  Consecutive layers of one shape that the tensor-core kernel covers (bfloat16 weights, see dsvt_layer)
+ * run as ONE launch of up to DSVT_MAX_CHAIN_LAYERS layers: thread blocks draw row tiles of layer after layer
+ * from a counter, and a tile of layer i starts once the rows it reads carry layer i - 1's completion stamp, so
+ * the chain pays a launch's start-up and tail once.  Every voxel that a later layer reads must be covered by the
+ * table of the layer before it (true for tables made by dsvt_partition from one set of coordinates; otherwise a
+ * bounded wait expires and DSVT_STATUS_TIMEOUT is raised).  All layers have the same C.
+ *
+ *   tables, params   HOST arrays of num_layers entries; the pointers inside are device pointers.
+ *   set_rowoff       as produced by dsvt_partition, or NULL (derived from the table; such a layer runs alone).
+ */
+#define DSVT_MAX_CHAIN_LAYERS 16
+typedef struct dsvt_table_ref {
+  const int32_t* set_table; /* int32 [cap_sets][set_size] */
+  int32_t cap_sets;
+  const int32_t* num_sets;   /* device int32 */
+  const int32_t* set_rowoff; /* int32 [2 * cap_sets + 3] or NULL */
+} dsvt_table_ref;
+int dsvt_layers(dsvt_ctx* ctx, const float* x, int32_t n, int32_t num_layers, const dsvt_table_ref* tables,
+                const dsvt_layer_params* params, float* y);
 
 /*
  * Attention-style 3D pooling (Eq. 6, Eq. 7).  Region of voxel (b,x,y,z): (b, x/l, y/w, z/h) with

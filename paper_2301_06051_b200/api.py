@@ -23,7 +23,7 @@ STATUS_BAD_COORD, STATUS_TABLE_OVERFLOW, STATUS_BAD_INDEX, STATUS_DUPLICATE_CELL
 
 EXPORTS = [
     "dsvt_create", "dsvt_destroy", "dsvt_status_sync", "dsvt_last_cuda_error", "dsvt_error_string",
-    "dsvt_launch_count", "dsvt_set_layer_ctas", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_set_attention_rpb", "dsvt_layer", "dsvt_block", "dsvt_pool",
+    "dsvt_launch_count", "dsvt_set_layer_ctas", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_set_attention_rpb", "dsvt_layer", "dsvt_layers", "dsvt_block", "dsvt_pool",
     "dsvt_bev_scatter",
 ]
 
@@ -48,6 +48,15 @@ class LayerParams(C.Structure):
         ("pe", C.c_void_p),
         ("rpb", C.c_void_p), ("coords", C.c_void_p), ("rpb_extent", C.c_int32 * 3),
     ]
+
+
+class TableRef(C.Structure):
+    """Mirror of dsvt_table_ref."""
+    _fields_ = [("set_table", C.c_void_p), ("cap_sets", C.c_int32), ("num_sets", C.c_void_p),
+                ("set_rowoff", C.c_void_p)]
+
+
+MAX_CHAIN_LAYERS = 16
 
 
 def load():
@@ -78,6 +87,7 @@ def load():
                                            C.c_int, vp]
     lib.dsvt_bev_scatter.argtypes = [vp, vp, vp, i32, i32, i32, p3, i32, vp]
     lib.dsvt_layer.argtypes = [vp, vp, i32, vp, i32, vp, vp, C.POINTER(LayerParams), vp]
+    lib.dsvt_layers.argtypes = [vp, vp, i32, i32, C.POINTER(TableRef), C.POINTER(LayerParams), vp]
     lib.dsvt_block.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, i32, vp, vp, C.POINTER(LayerParams), vp]
     lib.dsvt_pool.argtypes = [vp, vp, vp, i32, i32, i32, p3, p3, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32,
                               C.c_int, vp, vp, i32, vp, vp, vp]
@@ -309,6 +319,22 @@ class Context:
                                  _ptr(table.num_sets), _ptr(table.set_rowoff) if use_rowoff else None, C.byref(p),
                                  _ptr(y))
         self._check(rc, "dsvt_layer")
+        return y
+
+    # ---- dsvt_layers ----
+    def layers(self, x: torch.Tensor, tables: Sequence["SetTable"], ws: Sequence[Dict], y: torch.Tensor,
+               coords: Optional[torch.Tensor] = None, use_rowoff: bool = True) -> torch.Tensor:
+        """A chain of layers, layer i on tables[i] with weights ws[i]: the first reads x, all write y."""
+        L = len(ws)
+        assert len(tables) == L
+        tr = (TableRef * max(L, 1))()
+        pr = (LayerParams * max(L, 1))()
+        for i, (t, w) in enumerate(zip(tables, ws)):
+            tr[i].set_table, tr[i].cap_sets, tr[i].num_sets = _ptr(t.set_table), t.cap_sets, _ptr(t.num_sets)
+            tr[i].set_rowoff = _ptr(t.set_rowoff) if use_rowoff else None
+            pr[i] = layer_params(w, t.set_size, None, coords)
+        rc = self.lib.dsvt_layers(self._h, _ptr(x), int(x.shape[0]), L, tr, pr, _ptr(y))
+        self._check(rc, "dsvt_layers")
         return y
 
     # ---- dsvt_block ----

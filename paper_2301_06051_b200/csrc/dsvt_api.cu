@@ -44,6 +44,8 @@ void carve(dsvt_ctx* c, unsigned char* base, size_t* total) {
   c->bm_zero = k.take<int32_t>(2 * (nw + 1) + 2 * c->bm_words);
   c->bm_wordrank = k.take<int32_t>(2 * c->bm_words);
   c->bm_dup = k.take<int32_t>(nv);
+  c->tc_counter = k.take<int32_t>(64);
+  c->row_stamp = k.take<int32_t>(nv);
   *total = align_up(k.off, 256);
 }
 
@@ -104,6 +106,43 @@ int check_common(const dsvt_ctx* ctx, const float* x, const float* y, int32_t n,
   return DSVT_OK;
 }
 
+
+// A chain of layers, layer i on tables[i]: layer 0 reads x and writes y, the later ones run in place on y.
+// Consecutive layers of one shape that the tensor-core kernel covers share a launch; the rest run one by one.
+int run_layers(dsvt_ctx* ctx, const float* x, int32_t n, int32_t num_layers, const dsvt_table_ref* tables,
+               const dsvt_layer_params* params, float* y) {
+  dsvt_fused_args chain[DSVT_MAX_CHAIN_LAYERS];
+  int len = 0;
+  auto flush = [&]() -> int {
+    if (len == 0) return DSVT_OK;
+    const int rc = dsvt_launch_layers_tc(ctx, chain, len);
+    len = 0;
+    return rc;
+  };
+  for (int i = 0; i < num_layers; ++i) {
+    const dsvt_table_ref& t = tables[i];
+    if (n == 0 || t.cap_sets == 0) continue;
+    dsvt_fused_args a;
+    a.x = i == 0 ? x : y; a.y = y; a.n = n;
+    a.table = t.set_table; a.num_sets = t.num_sets; a.rowoff = t.set_rowoff; a.cap_sets = t.cap_sets;
+    a.p = params[i];
+    a.attention_only = 0;
+    const bool tc = t.set_rowoff != nullptr && dsvt_layer_tc_supported(a);
+    if (len > 0 && (!tc || len == DSVT_MAX_CHAIN_LAYERS || !dsvt_layer_tc_chainable(chain[0], a))) {
+      const int rc = flush();
+      if (rc != DSVT_OK) return rc;
+    }
+    if (tc) {
+      chain[len++] = a;
+      continue;
+    }
+    const int rc = run_layer(ctx, a.x, n, t.set_table, t.cap_sets, t.num_sets, t.set_rowoff, params[i], y, false,
+                             (i & 1) ? ctx->rowoff_b : ctx->rowoff_a);
+    if (rc != DSVT_OK) return rc;
+  }
+  return flush();
+}
+
 }  // namespace
 
 extern "C" int dsvt_create(dsvt_ctx** out, int device, void* cuda_stream, int64_t max_voxels, int64_t max_windows,
@@ -132,6 +171,8 @@ extern "C" int dsvt_create(dsvt_ctx** out, int device, void* cuda_stream, int64_
   c->launches = 0;
   c->cell_map = nullptr;
   c->cell_map_entries = 0;
+  c->maps = nullptr;
+  c->stamp_serial = 0;
   size_t total = 0;
   carve(c, nullptr, &total);
   cudaError_t e = cudaMalloc(&c->arena, total);
@@ -141,7 +182,9 @@ extern "C" int dsvt_create(dsvt_ctx** out, int device, void* cuda_stream, int64_
   }
   c->arena_bytes = total;
   carve(c, (unsigned char*)c->arena, &total);
-  if (cudaMemsetAsync(c->status, 0, 64 * sizeof(int32_t), c->stream) != cudaSuccess) {
+  if (cudaMemsetAsync(c->status, 0, 64 * sizeof(int32_t), c->stream) != cudaSuccess ||
+      cudaMemsetAsync(c->tc_counter, 0, 64 * sizeof(int32_t), c->stream) != cudaSuccess ||
+      cudaMemsetAsync(c->row_stamp, 0, (size_t)max_voxels * sizeof(int32_t), c->stream) != cudaSuccess) {
     cudaFree(c->arena);
     delete c;
     return DSVT_ERR_CUDA;
@@ -156,6 +199,7 @@ extern "C" int dsvt_destroy(dsvt_ctx* ctx) {
   cudaStreamSynchronize(ctx->stream);
   if (ctx->cell_map) cudaFree(ctx->cell_map);
   cudaFree(ctx->arena);
+  if (ctx->maps) dsvt_map_cache_destroy(ctx->maps);
   delete ctx;
   return DSVT_OK;
 }
@@ -234,23 +278,27 @@ extern "C" int dsvt_layer(dsvt_ctx* ctx, const float* x, int32_t n, const int32_
   return run_layer(ctx, x, n, set_table, cap_sets, num_sets, set_rowoff, *params, y, false, ctx->rowoff_a);
 }
 
+extern "C" int dsvt_layers(dsvt_ctx* ctx, const float* x, int32_t n, int32_t num_layers, const dsvt_table_ref* tables,
+                           const dsvt_layer_params* params, float* y) {
+  if (!ctx || num_layers < 0 || (num_layers > 0 && (!tables || !params))) return DSVT_ERR_INVALID_ARG;
+  for (int i = 0; i < num_layers; ++i) {
+    int rc = check_common(ctx, x, y, n, tables[i].set_table, tables[i].cap_sets, tables[i].num_sets);
+    if (rc != DSVT_OK) return rc;
+    rc = check_layer_shape(ctx, params[i], false);
+    if (rc != DSVT_OK) return rc;
+    if (params[i].C != params[0].C) return DSVT_ERR_INVALID_ARG;
+  }
+  return run_layers(ctx, x, n, num_layers, tables, params, y);
+}
+
 extern "C" int dsvt_block(dsvt_ctx* ctx, const float* x, int32_t n, const int32_t* table_axis0, int32_t cap_sets0,
                           const int32_t* num_sets0, const int32_t* set_rowoff0, const int32_t* table_axis1,
                           int32_t cap_sets1, const int32_t* num_sets1, const int32_t* set_rowoff1,
                           const dsvt_layer_params layers[2], float* y) {
   if (!layers) return DSVT_ERR_INVALID_ARG;
-  int rc = check_common(ctx, x, y, n, table_axis0, cap_sets0, num_sets0);
-  if (rc != DSVT_OK) return rc;
-  rc = check_common(ctx, x, y, n, table_axis1, cap_sets1, num_sets1);
-  if (rc != DSVT_OK) return rc;
-  for (int i = 0; i < 2; ++i) {
-    rc = check_layer_shape(ctx, layers[i], false);
-    if (rc != DSVT_OK) return rc;
-  }
-  if (layers[0].C != layers[1].C) return DSVT_ERR_INVALID_ARG;
   // X-axis layer writes y (every voxel is in one set, so every row of y is produced); the Y-axis
   // layer then runs in place on y.
-  rc = run_layer(ctx, x, n, table_axis0, cap_sets0, num_sets0, set_rowoff0, layers[0], y, false, ctx->rowoff_a);
-  if (rc != DSVT_OK) return rc;
-  return run_layer(ctx, y, n, table_axis1, cap_sets1, num_sets1, set_rowoff1, layers[1], y, false, ctx->rowoff_b);
+  const dsvt_table_ref tables[2] = {{table_axis0, cap_sets0, num_sets0, set_rowoff0},
+                                    {table_axis1, cap_sets1, num_sets1, set_rowoff1}};
+  return dsvt_layers(ctx, x, n, 2, tables, layers, y);
 }

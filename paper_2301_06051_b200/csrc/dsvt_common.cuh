@@ -6,6 +6,9 @@
 
 #include "dsvt.h"
 
+struct dsvt_map_cache;  // tensor maps of the weight matrices seen so far (layer_tc.cu)
+void dsvt_map_cache_destroy(dsvt_map_cache* c);
+
 struct dsvt_ctx {
   int device;
   cudaStream_t stream;
@@ -34,6 +37,12 @@ struct dsvt_ctx {
   int32_t* bm_zero;      // [2 (max_windows + 1) + 2 bm_words] window counts, duplicate counts, bitmaps
   int32_t* bm_wordrank;  // [2 bm_words] popcount prefix of each bitmap word inside its window
   int32_t* bm_dup;       // [max_voxels] -1, or the voxel's ticket among the duplicates of its window
+  // tensor-core layer kernel: tile counter of a launch ([0] next tile, [1] CTAs that have left; zero between
+  // launches), per-voxel completion stamps of a chain of layers, and the serial number the stamps are built from
+  int32_t* tc_counter;   // [2]
+  int32_t* row_stamp;    // [max_voxels]
+  uint32_t stamp_serial;
+  dsvt_map_cache* maps;
   // pooling: dense cell -> voxel map, grown on demand
   int32_t* cell_map;
   size_t cell_map_entries;
@@ -85,6 +94,11 @@ int dsvt_launch_layer_fma(dsvt_ctx* ctx, const dsvt_fused_args& a);
 // tcgen05 path: bfloat16 weights, C in {64, 128, 192}, head dim in {16, 24, 32}, set size <= 96.
 bool dsvt_layer_tc_supported(const dsvt_fused_args& a);
 int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a);
+// A chain of layers in one launch: layers[0] reads its x and writes y; layers[i > 0] run in place on that y.  Every
+// layer passes dsvt_layer_tc_supported and dsvt_layer_tc_chainable(layers[0], layers[i]); at most
+// DSVT_MAX_CHAIN_LAYERS layers; every voxel a later layer reads must be written by the layer before it.
+bool dsvt_layer_tc_chainable(const dsvt_fused_args& a, const dsvt_fused_args& b);
+int dsvt_launch_layers_tc(dsvt_ctx* ctx, const dsvt_fused_args* layers, int n_layers);
 // CUtensorMap (128 bytes, 64-byte aligned) of a row-major bf16 matrix [rows][cols]: boxes of 64 columns x box_rows
-// rows, 128-byte swizzle.  Returns false if the driver cannot encode it.
-bool dsvt_make_weight_map(void* tensor_map, const void* w, int rows, int cols, int box_rows);
+// rows, 128-byte swizzle; encoded once per matrix and context.  Returns false if the driver cannot encode it.
+bool dsvt_cached_weight_map(dsvt_ctx* ctx, void* tensor_map, const void* w, int rows, int cols, int box_rows);

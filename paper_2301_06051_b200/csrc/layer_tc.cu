@@ -1,18 +1,24 @@
-// Fused DSVT layer on the 5th-generation tensor cores (tcgen05 + TMEM), bfloat16 operands, fp32
+// Fused DSVT layers on the 5th-generation tensor cores (tcgen05 + TMEM), bfloat16 operands, fp32
 // accumulation: gather (Eq. 4) -> QKV projection -> per-set multi-head attention (Eq. 5) -> output
 // projection -> residual + LayerNorm -> MLP with GELU -> residual + LayerNorm -> scatter (App. B.1.1).
 //
-// One persistent CTA per SM.  Whole sets are packed greedily into tiles of at most 128 distinct rows (the
-// UMMA M); the tile plan comes from the partition (tile t goes to CTA t mod gridDim.x), or, without a
-// plan, each CTA cuts its own contiguous row segment into tiles.
+// One launch runs a chain of layers (one layer, the two layers of a block, or every block of a stage): layer 0
+// reads x and writes y, the later layers run in place on y.  Whole sets are packed into tiles of at most 128
+// distinct rows (the UMMA M) by the partition's tile plan.  The persistent CTAs (one per SM) draw tiles from a
+// global counter, all tiles of layer 0 first, then layer 1, ...; a tile of layer l may be gathered as soon as
+// each of its rows carries layer l - 1's completion stamp (one int per voxel, written after the row's store), so
+// no CTA ever waits for a whole layer to end, and a launch pays its start-up and its tail once per chain rather
+// than once per layer.  Tiles are taken in counter order and a tile only ever waits for tiles with a smaller
+// number, so the tile with the smallest unfinished number can always run: no CTA has to be resident for another
+// to make progress.
 //
 // Roles (640 threads): warps 0-15 compute (gather, TMEM epilogues, attention); warp 16 is the scheduler
-// and TMA producer: it publishes tiles through a two-entry ring, two ahead, and streams the layer's
+// and TMA producer: it draws tiles, publishes them through a two-entry ring, two ahead, and streams the layer's
 // weight matrices through a three-stage shared-memory ring with plain (single-CTA) TMA loads; warp 17
-// allocates TMEM and issues the tcgen05.mma instructions; warps 18-19 build the next tile's row list
-// while the current tile is computed.  The compute warps gather the next tile's rows as soon as the
-// current tile's MMAs have stopped reading the A operand, so that its first projections overlap the
-// current tile's tail.
+// allocates TMEM and issues the tcgen05.mma instructions; warp 18 builds the next tile's row list
+// while the current tile is computed and waits for its rows' stamps; warp 19 stamps a finished tile's rows.
+// The compute warps gather the next tile's rows as soon as the current tile's MMAs have stopped reading the A
+// operand (if its rows are ready by then), so that its first projections overlap the current tile's tail.
 //
 // The projections of a layer are chunks of at most 192 output columns (K, V, Q, O, MLP-1 in pieces of
 // 128 or 64 hidden columns, MLP-2), accumulated in three TMEM regions (map at compute_role) so the
@@ -26,12 +32,15 @@
 // (mma.sync m16n8k16 with ldmatrix) reads it without bank conflicts and writes its result straight
 // into the A operand of the output projection.
 //
-// Every wait on an mbarrier is bounded; a wait that gives up raises DSVT_STATUS_TIMEOUT and all roles
-// leave their loops.
+// Every wait (on an mbarrier, on a row stamp) is bounded; a wait that gives up raises DSVT_STATUS_TIMEOUT and
+// all roles leave their loops.
 #include <cuda.h>
 #include <limits.h>
 
+#include <mutex>
+#include <new>
 #include <type_traits>
+#include <vector>
 
 #include "dsvt_common.cuh"
 
@@ -41,12 +50,15 @@ constexpr int kTM = 128;               // tile rows = UMMA M
 constexpr int kComputeWarps = 16;
 constexpr int kComputeThreads = 32 * kComputeWarps;
 constexpr int kTmaWarp = kComputeWarps, kMmaWarp = kComputeWarps + 1;
-constexpr int kLoadWarp0 = kComputeWarps + 2, kLoadWarps = 2;  // row-list + gather warps, one tile ahead
+constexpr int kLoadWarp0 = kComputeWarps + 2, kLoadWarps = 1;  // row-list warp, one tile ahead
 constexpr int kLoadThreads = 32 * kLoadWarps;
-constexpr int kThreads = kComputeThreads + 64 + kLoadThreads;
+constexpr int kStampWarp = kLoadWarp0 + kLoadWarps;  // writes the completion stamps of a finished tile's rows
+constexpr int kThreads = kComputeThreads + 64 + kLoadThreads + 32;
 constexpr int kStages = 3;             // weight ring depth
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxPolls = 1 << 20;
+constexpr int kStampPolls = 1 << 18;  // polls of a row's stamp, about a microsecond each
+constexpr int kMaxLayers = DSVT_MAX_CHAIN_LAYERS;  // layers one launch can chain
 
 struct TcGeom {
   int hidden, heads, tau;
@@ -56,8 +68,30 @@ struct TcGeom {
   int mode;     // 0: attention only, 1: attention + residual + LN1, 2: full layer
   uint32_t off_a, off_kv, off_stage, off_par;  // byte offsets from the 1024-aligned base
   // relative position bias (rb_len == 0: none): entries per head, strides of the x and y offsets in the table,
-  // index of the zero offset
-  int rb_len, rb_sx, rb_sy, rb_centre;
+  // index of the zero offset, extent of the table
+  int rb_len, rb_sx, rb_sy, rb_centre, rb_ext[3];
+};
+
+// One layer of a launch's chain: weight tensor maps, per-layer vectors, and the set table the layer runs on.
+struct alignas(64) TcLayer {
+  CUtensorMap qkv, o, w1, w2;
+  const float *b_qkv, *b_o, *b_1, *b_2, *ln1_g, *ln1_b, *ln2_g, *ln2_b, *rpb;
+  const int32_t *table, *num_sets, *rowoff;
+  int32_t cap_sets;
+  float eps;
+};
+
+struct TcArgs {
+  const float* x;        // input of layer 0
+  float* y;              // output of every layer; input of the layers after the first
+  const int4* coords;    // (b, x, y, z) per voxel: read only with a position bias
+  int32_t n, n_layers;
+  int32_t* counter;      // [0] next tile of the launch, [1] CTAs that have left; both zero between launches
+  int32_t* row_stamp;    // [n] completion stamps (n_layers > 1)
+  int32_t stamp_base;    // layer l's stamp is stamp_base + l + 1
+  int32_t* status;
+  TcGeom g;
+  TcLayer layer[kMaxLayers];
 };
 
 struct Misc {  // small shared state beside the big regions
@@ -65,18 +99,23 @@ struct Misc {  // small shared state beside the big regions
   unsigned long long full[kStages], empty[kStages], acc_full[3], acc_free[3];
   unsigned long long a_ready;   // compute warps -> MMA: attention output / x1 / MLP hidden is in place
   unsigned long long x_ready;   // compute warps -> MMA: the gathered rows of a tile are in the A operand
-  unsigned long long rl_ready[2];  // loader warps -> compute: row-list buffer b describes its next tile
-  unsigned long long rl_free[2];   // compute -> loader warps: row-list buffer b is no longer read
+  unsigned long long rl_ready[2];   // loader warp -> compute: row-list buffer b describes its next tile
+  unsigned long long dep_ready[2];  // loader warp -> compute: the rows listed in buffer b carry the previous layer's stamp
+  unsigned long long rl_free[2];    // compute + stamp warp -> loader warp: row-list buffer b is no longer read
+  unsigned long long stored[2];     // compute -> stamp warp: the tile listed in buffer b has been stored
+  unsigned long long drain;         // MMA issuer: every MMA issued before an abort has completed
   unsigned long long sched_full[2], sched_empty[2];
   uint32_t tmem_base;
   int abort_flag;
-  int tile[2][4];  // ring of tiles: first set, number of sets (< 0: no more tiles), first row, rows
+  int exit_at;   // tile iteration at which the compute warps left their loop (-1: still running; read by the stamp warp)
+  int tile[2][6];  // ring of tiles: first set, number of sets (< 0: no more tiles), first row, rows, layer
+  // the scheduler's view of the chain: tiles before the end of each layer, sets per layer, plan or not
+  int tile_end[kMaxLayers], lay_S[kMaxLayers];
+  unsigned char lay_plan[kMaxLayers];
   // launch constants, written once before the roles start: the phase functions read them from here
   // instead of taking them as arguments, so that nothing has to stay in registers across their calls
-  const float* x;
+  const float* x;   // input rows of the tile the compute warps are working on
   float* y;
-  const int32_t* table;
-  const int32_t* rowoff;
   int32_t* status;
   unsigned char* sm;   // 1024-aligned base of the dynamic shared memory (generic address)
   uint32_t sbase;      // the same as a shared-space address
@@ -84,13 +123,13 @@ struct Misc {  // small shared state beside the big regions
   int n, tau, heads, mode, NF, n_f1, ln1, ln2;
   float eps;
   // the tile the compute warps are working on, and which row-list buffer describes it
-  int s_lo, nsets, base, rows, buf;
-  int pre0;  // the CTA's first tile was listed and gathered during the kernel's set-up
-  int next_rows[2];  // rows of the tile listed in buffer b (< 0: there is no such tile), valid after rl_ready[b]
-  // row lists, double buffered: the loader warps fill buffer (k + 1) & 1 while the compute warps work on tile k;
+  int s_lo, nsets, base, rows, buf, layer;
+  int next_rows[2];        // rows of the tile listed in buffer b (< 0: there is no such tile), valid after rl_ready[b]
+  const float* next_x[2];  // where that tile's input rows are read from
+  int st_rows[2], st_stamp[2];  // for the stamp warp: rows of the stored tile in buffer b, the stamp they get (0: none)
+  // row lists, double buffered: the loader warp fills buffer (k + 1) & 1 while the compute warps work on tile k;
   // the compute warps gather tile k + 1 as soon as tile k's MMAs no longer read the A operand
   int rowvox[2][kTM];              // tile row -> voxel (-1: none)
-  unsigned char set_lo[2][kTM + 1];  // first tile row of each set of the tile
   unsigned char row_lo[2][kTM], row_n[2][kTM];  // per tile row: first row and row count of its set
   // relative position bias.  The table index is linear in the coordinate offset, so one integer per row,
   // x * rb_sx + y * rb_sy + z, serves every (query, key) pair: index = lin[query] - lin[key] + rb_centre.  Offsets
@@ -279,10 +318,6 @@ __device__ __forceinline__ float2 gelu_fast2(float2 t) {
   return __ffma2_rn(m, h, make_float2(fmaxf(t.x, 0.f), fmaxf(t.y, 0.f)));
 }
 
-struct TcMaps {
-  CUtensorMap qkv, o, w1, w2;
-};
-
 // Relative position bias of (query, key) from their rows' linear coordinates; `tab` is the head's table, `root`
 // the square root of the head dimension (the scores are still unscaled dot products when the bias is added).
 __device__ __forceinline__ float rpb_term(const float* __restrict__ tab, int lin_q, int lin_k, float root) {
@@ -457,242 +492,227 @@ __device__ __forceinline__ uint32_t stage_off(int r, int c4) {
 // Roles
 // ---------------------------------------------------------------------------------------------
 struct RoleCtx {
-  unsigned char* sm;  // 1024-aligned shared-memory base (generic address) and its shared-space address
-  uint32_t sbase;
+  uint32_t sbase;     // 1024-aligned shared-memory base as a shared-space address
   uint32_t tmem;      // TMEM base address of the CTA's allocation
-  // read by the scheduler thread while the other threads set up shared memory (see prefetch_first_tile)
-  int S;              // number of sets
-  int n_plan;         // tiles in the plan (< 0: no plan)
-  int pre_ok;         // the CTA's first plan tile below is valid
-  int pre_s, pre_ns, pre_base, pre_rows;
   // copies of the kernel parameters the two single-thread roles use (registers instead of parameter-space loads)
-  const int32_t* rowoff;
-  int cap_sets, mode, n_f1, NF, nkb_h;
+  int mode, n_f1, NF, nkb_h, tau, n_layers;
   uint32_t off_a, off_kv, off_stage;
 };
 
-// The scheduler thread's first global reads (set count, plan header, the CTA's first tile and its row range)
-// are issued at kernel entry, so that their two round trips overlap the shared-memory set-up.
-__device__ __forceinline__ void prefetch_first_tile(const dsvt_fused_args& a, RoleCtx& rc) {
-  const int32_t* plan = a.rowoff + a.cap_sets + 1;
-  const int n_plan = plan[0];
-  const int S = min(*a.num_sets, a.cap_sets);
-  // in bounds for every block index: the grid has at most cap_sets CTAs and the plan cap_sets + 2 entries
-  const int f = plan[1 + blockIdx.x], l = plan[2 + blockIdx.x];
-  rc.n_plan = n_plan;
-  rc.S = S;
-  rc.pre_ok = 0;
-  rc.pre_s = rc.pre_ns = rc.pre_base = rc.pre_rows = 0;
-  if (n_plan >= 0 && (int)blockIdx.x < n_plan && f >= 0 && l > f && l <= S && l - f <= kTM) {
-    const int base = a.rowoff[f], rows = a.rowoff[l] - base;
-    if (rows > 0 && rows <= kTM) {
-      rc.pre_ok = 1;
-      rc.pre_s = f; rc.pre_ns = l - f; rc.pre_base = base; rc.pre_rows = rows;
-    }
-  }
+__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
 }
-
+__device__ __forceinline__ void st_relaxed_gpu(int32_t* p, int v) {
+  asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 
 // The scheduler and the MMA issuer are separate (not inlined) functions so that their polling loops get
 // their own, spill-free register allocation; the compute role is inlined into the kernel, where the
 // kernel parameters are constant-bank operands.
 
 // ================= scheduler + TMA producer (one thread) ===============================================
+// Tiles are numbered over the whole chain, layer after layer; a tile's number comes from the launch's counter.
+// Inside a layer, tile t is entry t of the layer's plan (whole sets, at most 128 distinct rows); a layer without
+// a plan is cut by row ranges instead: tile t holds the sets whose first row lies in [t R, (t + 1) R),
+// R = 128 - tau + 1, found by binary search in the row offsets (slower to schedule, same results).
 template <int C>
-__device__ __noinline__ void producer_role(const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps,
-                                           int32_t* __restrict__ status, const RoleCtx rc) {
+__device__ __noinline__ void producer_role(const TcArgs& a, const RoleCtx rc) {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
-  constexpr uint32_t COL_B = C;      // second accumulator buffer
   constexpr uint32_t STAGE_BYTES = C * 128;
-  const uint32_t sbase = rc.sbase, tmem = rc.tmem;
   Misc* mi = &s_mi;
-  const uint32_t a_base = sbase + rc.off_a, kv_base = sbase + rc.off_kv, st_base = sbase + rc.off_stage;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t st_base = rc.sbase + rc.off_stage;
   volatile int* abort_flag = &mi->abort_flag;
-  const int S = rc.S;
+  int32_t* status = a.status;
   const bool mlp = rc.mode == 2;
   const int n_chunks = 4 + (mlp ? rc.n_f1 + 1 : 0);
-  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp;
-  (void)tmem; (void)S; (void)n_chunks; (void)tid;
-    if (lane == 0) {
-      // Tiles come from the plan behind the row offsets (greedy packing of the whole frame, tile t goes to
-      // CTA t mod G); without a plan each CTA packs its own segment, the sets whose first row lies in
-      // [b R / G, (b + 1) R / G).
-      const int32_t* plan = rc.rowoff + rc.cap_sets + 1;
-      const int n_plan = rc.n_plan;
-      int t_next = blockIdx.x;
-      int s = 0, s_end = 0;
-      if (n_plan < 0) {
-        const int R = S > 0 ? rc.rowoff[S] : 0;
-        const int row_lo = (int)(((long long)blockIdx.x * R) / gridDim.x);
-        const int row_hi = (int)(((long long)(blockIdx.x + 1) * R) / gridDim.x);
-        int lo = 0, hi = S;
-        while (lo < hi) { const int m = (lo + hi) >> 1; if (rc.rowoff[m] < row_lo) lo = m + 1; else hi = m; }
-        s = lo;
-        hi = S;
-        while (lo < hi) { const int m = (lo + hi) >> 1; if (rc.rowoff[m] < row_hi) lo = m + 1; else hi = m; }
-        s_end = lo;
-      }
-      // next tile: first set s0, ns sets (< 0: none left), first row, rows
-      auto next_tile = [&](int& s0, int& ns, int& base, int& rows) {
-        ns = -1; base = 0; rows = 0;
-        if (n_plan >= 0) {
-          while (t_next < n_plan) {
-            const int f = plan[1 + t_next], l = plan[2 + t_next];
-            t_next += gridDim.x;
-            if (f < 0 || l <= f || l > S) { atomicOr(status, DSVT_STATUS_BAD_INDEX); continue; }
-            base = rc.rowoff[f];
-            rows = rc.rowoff[l] - base;
-            if (rows <= 0 || rows > kTM || l - f > kTM) { atomicOr(status, DSVT_STATUS_BAD_INDEX); continue; }
-            s0 = f;
-            ns = l - f;
-            return;
-          }
-          return;
-        }
-        while (s0 < s_end) {
-          base = rc.rowoff[s0];
-          const int first = rc.rowoff[s0 + 1] - base;
-          if (first <= 0 || first > kTM) {  // offsets that do not describe a set: skip it
-            atomicOr(status, DSVT_STATUS_BAD_INDEX);
-            ++s0;
-            continue;
-          }
-          int l2 = s0 + 1, h2 = s_end;  // last e in (s0, s_end] with rowoff[e] - base <= 128
-          while (l2 < h2) { const int m = (l2 + h2 + 1) >> 1; if (rc.rowoff[m] - base <= kTM) l2 = m; else h2 = m - 1; }
-          ns = l2 - s0;
-          rows = rc.rowoff[l2] - base;
-          return;
-        }
-      };
-      int stage = 0, slot = 0;
-      uint32_t phase = 0, sphase = 0;
-      int ns, base, rows;
-      if (rc.pre_ok) {  // the first tile was looked up at kernel entry
-        s = rc.pre_s; ns = rc.pre_ns; base = rc.pre_base; rows = rc.pre_rows;
-        t_next += gridDim.x;
+  const int L = rc.n_layers;
+  const int Rv = kTM - rc.tau + 1;
+  // the chain's tile counts
+  int total = 0;
+  for (int l = 0; l < L; ++l) {
+    const TcLayer& ly = a.layer[l];
+    const int S = min(__ldg(ly.num_sets), ly.cap_sets);
+    int T = __ldg(ly.rowoff + ly.cap_sets + 1);
+    mi->lay_S[l] = S;
+    mi->lay_plan[l] = T >= 0;
+    if (T < 0) T = S > 0 ? (__ldg(ly.rowoff + S) + Rv - 1) / Rv : 0;
+    else T = min(T, S);
+    total += max(T, 0);
+    mi->tile_end[l] = total;
+  }
+  // next tile: layer, first set s0, ns sets (< 0: none left), first row, rows
+  auto next_tile = [&](int& lay, int& s0, int& ns, int& base, int& rows) {
+    for (;;) {
+      lay = 0; s0 = 0; ns = -1; base = 0; rows = 0;
+      if (*abort_flag) return;
+      const int g = atomicAdd(a.counter, 1);
+      if (g < 0 || g >= total) return;
+      int l = 0;
+      while (l + 1 < L && g >= mi->tile_end[l]) ++l;
+      const int t = g - (l ? mi->tile_end[l - 1] : 0);
+      const TcLayer& ly = a.layer[l];
+      const int S = mi->lay_S[l];
+      int f, e;
+      if (mi->lay_plan[l]) {
+        const int32_t* plan = ly.rowoff + ly.cap_sets + 1;
+        f = __ldg(plan + 1 + t);
+        e = __ldg(plan + 2 + t);
+        if (f < 0 || e <= f || e > S) { atomicOr(status, DSVT_STATUS_BAD_INDEX); continue; }
       } else {
-        next_tile(s, ns, base, rows);
+        const int r0 = t * Rv, r1 = r0 + Rv;
+        int lo = 0, hi = S;
+        while (lo < hi) { const int m = (lo + hi) >> 1; if (__ldg(ly.rowoff + m) < r0) lo = m + 1; else hi = m; }
+        f = lo;
+        hi = S;
+        while (lo < hi) { const int m = (lo + hi) >> 1; if (__ldg(ly.rowoff + m) < r1) lo = m + 1; else hi = m; }
+        e = lo;
+        if (e <= f) continue;  // no set starts in this row range
       }
-      // Tiles are published two ahead of the weights (the ring has two entries), so that the loader
-      // warps can prepare tile k + 1 while tile k is being computed.
-      int ahead = 0;          // published tiles whose weights have not been streamed yet
-      bool all_out = false;   // the end marker has been published
-      auto publish = [&]() -> bool {
-        if (!mbar_wait(&mi->sched_empty[slot], sphase ^ 1u, abort_flag)) return false;
-        mi->tile[slot][0] = s; mi->tile[slot][1] = ns; mi->tile[slot][2] = base; mi->tile[slot][3] = rows;
-        mbar_arrive(&mi->sched_full[slot]);
-        if (++slot == 2) { slot = 0; sphase ^= 1u; }
-        if (ns < 0) { all_out = true; return true; }
-        ++ahead;
-        s += ns;
-        next_tile(s, ns, base, rows);
-        return true;
-      };
-      if (!publish()) goto producer_done;
-      if (!all_out && !publish()) goto producer_done;
-      while (ahead > 0) {
-        // the layer's weights for one tile, chunk by chunk, K block by K block
-        for (int c = 0; c < n_chunks; ++c) {
-          const CUtensorMap* map;
-          int row0, nkb;
-          uint32_t bytes = STAGE_BYTES;
-          if (c < 3) { map = &maps.qkv; row0 = (c == 0 ? 1 : c == 1 ? 2 : 0) * C; nkb = NKB; }   // K, V, Q
-          else if (c == 3) { map = &maps.o; row0 = 0; nkb = NKB; }
-          else if (c < 4 + rc.n_f1) { map = &maps.w1; row0 = (c - 4) * rc.NF; nkb = NKB; bytes = (uint32_t)rc.NF * 128u; }
-          else { map = &maps.w2; row0 = 0; nkb = rc.nkb_h; }
-          for (int kb = 0; kb < nkb; ++kb) {
-            if (!mbar_wait(&mi->empty[stage], phase ^ 1u, abort_flag)) goto producer_done;
-            mbar_expect_tx(&mi->full[stage], bytes);
-            tma_load_2d(st_base + stage * STAGE_BYTES, map, kb * 64, row0, &mi->full[stage]);
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
-          }
-        }
-        --ahead;
-        if (!all_out && !publish()) goto producer_done;
-      }
-    producer_done:;
+      base = __ldg(ly.rowoff + f);
+      rows = __ldg(ly.rowoff + e) - base;
+      if (rows <= 0 || rows > kTM || e - f > kTM) { atomicOr(status, DSVT_STATUS_BAD_INDEX); continue; }
+      lay = l; s0 = f; ns = e - f;
+      return;
     }
+  };
+  int stage = 0, slot = 0;
+  uint32_t phase = 0, sphase = 0;
+  int issued[kStages];  // loads issued into each stage so far
+#pragma unroll
+  for (int i = 0; i < kStages; ++i) issued[i] = 0;
+  int lay, s, ns, base, rows;
+  int wl[2] = {0, 0}, wcount = 0, wread = 0;  // layers of the published tiles whose weights are still to be streamed
+  bool all_out = false;    // the end marker has been published
+  // Tiles are published two ahead of the weights (the ring has two entries), so that the loader
+  // warp can prepare tile k + 1 while tile k is being computed.
+  auto publish = [&]() -> bool {
+    next_tile(lay, s, ns, base, rows);
+    if (!mbar_wait(&mi->sched_empty[slot], sphase ^ 1u, abort_flag)) return false;
+    mi->tile[slot][0] = s; mi->tile[slot][1] = ns; mi->tile[slot][2] = base; mi->tile[slot][3] = rows;
+    mi->tile[slot][4] = lay;
+    mbar_arrive(&mi->sched_full[slot]);
+    if (++slot == 2) { slot = 0; sphase ^= 1u; }
+    if (ns < 0) { all_out = true; return true; }
+    wl[(wread + wcount) & 1] = lay;
+    ++wcount;
+    return true;
+  };
+  if (!publish()) goto producer_done;
+  if (!all_out && !publish()) goto producer_done;
+  while (wcount > 0) {
+    // the layer's weights for one tile, chunk by chunk, K block by K block
+    const TcLayer& ly = a.layer[wl[wread & 1]];
+    for (int c = 0; c < n_chunks; ++c) {
+      const CUtensorMap* map;
+      int row0, nkb;
+      uint32_t bytes = STAGE_BYTES;
+      if (c < 3) { map = &ly.qkv; row0 = (c == 0 ? 1 : c == 1 ? 2 : 0) * C; nkb = NKB; }   // K, V, Q
+      else if (c == 3) { map = &ly.o; row0 = 0; nkb = NKB; }
+      else if (c < 4 + rc.n_f1) { map = &ly.w1; row0 = (c - 4) * rc.NF; nkb = NKB; bytes = (uint32_t)rc.NF * 128u; }
+      else { map = &ly.w2; row0 = 0; nkb = rc.nkb_h; }
+      for (int kb = 0; kb < nkb; ++kb) {
+        if (!mbar_wait(&mi->empty[stage], phase ^ 1u, abort_flag)) goto producer_done;
+        mbar_expect_tx(&mi->full[stage], bytes);
+        tma_load_2d(st_base + stage * STAGE_BYTES, map, kb * 64, row0, &mi->full[stage]);
+        ++issued[stage];
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+    ++wread;
+    --wcount;
+    if (!all_out && !publish()) goto producer_done;
+  }
+producer_done:
+  if (*abort_flag) {
+    // leaving early: no load may still be writing into this CTA's shared memory when it retires
+#pragma unroll
+    for (int i = 0; i < kStages; ++i)
+      if (issued[i] > 0) {
+        const uint32_t par = (uint32_t)(issued[i] - 1) & 1u;
+        for (int it = 0; it < kMaxPolls && !mbar_try(&mi->full[i], par); ++it) {}
+      }
+  }
 }
 
 // ================= MMA issuer (one thread) =============================================================
 template <int C>
-__device__ __noinline__ void mma_role(const dsvt_fused_args& a, const TcGeom& g, const RoleCtx rc) {
+__device__ __noinline__ void mma_role(const RoleCtx rc) {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
   constexpr uint32_t COL_B = C;      // second accumulator buffer
   constexpr uint32_t STAGE_BYTES = C * 128;
   const uint32_t sbase = rc.sbase, tmem = rc.tmem;
   Misc* mi = &s_mi;
   const uint32_t a_base = sbase + rc.off_a, kv_base = sbase + rc.off_kv, st_base = sbase + rc.off_stage;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile int* abort_flag = &mi->abort_flag;
   const bool mlp = rc.mode == 2;
   const int n_chunks = 4 + (mlp ? rc.n_f1 + 1 : 0);
-  (void)NKB; (void)COL_B; (void)STAGE_BYTES; (void)a_base; (void)kv_base; (void)st_base; (void)lane; (void)warp;
-  (void)tmem; (void)n_chunks; (void)tid;
-    if (lane == 0) {
-      int stage = 0, slot = 0;
-      uint32_t phase = 0, a_phase = 0, x_phase = 0, sphase = 0;
-      uint32_t uses[3] = {0u, 0u, 0u};  // how often each accumulator region has been used
-      for (;;) {
-        if (!mbar_wait(&mi->sched_full[slot], sphase, abort_flag)) break;
-        const int ns = mi->tile[slot][1];
-        mbar_arrive(&mi->sched_empty[slot]);
-        if (++slot == 2) { slot = 0; sphase ^= 1u; }
-        if (ns < 0) break;
-        for (int c = 0; c < n_chunks; ++c) {
-          // a fresh A operand: X (chunks 0-2), attention output (3), x1 (4..), MLP hidden (last)
-          if (c == 0) {
-            if (!mbar_wait(&mi->x_ready, x_phase, abort_flag)) goto mma_done;
-            x_phase ^= 1u;
-          } else if (c == 3 || c == 4 || c == 4 + rc.n_f1) {
-            if (!mbar_wait(&mi->a_ready, a_phase, abort_flag)) goto mma_done;
-            a_phase ^= 1u;
-          }
-          // accumulator placement: K -> region 0, V -> 1, Q -> 0, O -> 0, MLP-1 piece i -> i & 1, MLP-2 -> 2
-          // (on top of the parked x1 + b_2)
-          uint32_t bar, col, n;
-          if (c < 4) { bar = (c == 1) ? 1u : 0u; col = (c == 1) ? COL_B : 0u; n = C; }
-          else if (c < 4 + rc.n_f1) { bar = (uint32_t)(c - 4) & 1u; col = bar * COL_B; n = (uint32_t)rc.NF; }
-          else { bar = 2u; col = kTmemCols - C; n = C; }
-          if (c == 1) {
-            // region 1 may overlap region 2: the previous tile's MLP-2 result must have been read
-            if (!mbar_wait(&mi->acc_free[2], (uses[2] & 1u) ^ 1u, abort_flag)) goto mma_done;
-          }
-          if (bar != 2u && !mbar_wait(&mi->acc_free[bar], (uses[bar] & 1u) ^ 1u, abort_flag)) goto mma_done;
-          ++uses[bar];
-          tc_fence_after();
-          const bool last = mlp && c == 4 + rc.n_f1;
-          const uint32_t abase = last ? kv_base : a_base;
-          const int nkb = last ? rc.nkb_h : NKB;
-          const uint32_t idesc = umma_idesc((int)n);
-          const uint32_t d_tmem = tmem + col;
-          for (int kb = 0; kb < nkb; ++kb) {
-            if (!mbar_wait(&mi->full[stage], phase, abort_flag)) goto mma_done;
-            tc_fence_after();
-            const uint32_t sa = abase + kb * (kTM * 128), sb = st_base + stage * STAGE_BYTES;
-#pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4)
-              umma_bf16(d_tmem, umma_desc(sa + k4 * 32), umma_desc(sb + k4 * 32), idesc, (last || (kb | k4) != 0) ? 1u : 0u);
-            umma_commit(&mi->empty[stage]);  // frees the weight stage once these MMAs have read it
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
-          }
-          umma_commit(&mi->acc_full[bar]);
-        }
+  int stage = 0, slot = 0;
+  uint32_t phase = 0, a_phase = 0, x_phase = 0, sphase = 0;
+  uint32_t uses[3] = {0u, 0u, 0u};  // how often each accumulator region has been used
+  for (;;) {
+    if (!mbar_wait(&mi->sched_full[slot], sphase, abort_flag)) break;
+    const int ns = mi->tile[slot][1];
+    mbar_arrive(&mi->sched_empty[slot]);
+    if (++slot == 2) { slot = 0; sphase ^= 1u; }
+    if (ns < 0) break;
+    for (int c = 0; c < n_chunks; ++c) {
+      // a fresh A operand: X (chunks 0-2), attention output (3), x1 (4..), MLP hidden (last)
+      if (c == 0) {
+        if (!mbar_wait(&mi->x_ready, x_phase, abort_flag)) goto mma_done;
+        x_phase ^= 1u;
+      } else if (c == 3 || c == 4 || c == 4 + rc.n_f1) {
+        if (!mbar_wait(&mi->a_ready, a_phase, abort_flag)) goto mma_done;
+        a_phase ^= 1u;
       }
-    mma_done:;
+      // accumulator placement: K -> region 0, V -> 1, Q -> 0, O -> 0, MLP-1 piece i -> i & 1, MLP-2 -> 2
+      // (on top of the parked x1 + b_2)
+      uint32_t bar, col, n;
+      if (c < 4) { bar = (c == 1) ? 1u : 0u; col = (c == 1) ? COL_B : 0u; n = C; }
+      else if (c < 4 + rc.n_f1) { bar = (uint32_t)(c - 4) & 1u; col = bar * COL_B; n = (uint32_t)rc.NF; }
+      else { bar = 2u; col = kTmemCols - C; n = C; }
+      if (c == 1) {
+        // region 1 may overlap region 2: the previous tile's MLP-2 result must have been read
+        if (!mbar_wait(&mi->acc_free[2], (uses[2] & 1u) ^ 1u, abort_flag)) goto mma_done;
+      }
+      if (bar != 2u && !mbar_wait(&mi->acc_free[bar], (uses[bar] & 1u) ^ 1u, abort_flag)) goto mma_done;
+      ++uses[bar];
+      tc_fence_after();
+      const bool last = mlp && c == 4 + rc.n_f1;
+      const uint32_t abase = last ? kv_base : a_base;
+      const int nkb = last ? rc.nkb_h : NKB;
+      const uint32_t idesc = umma_idesc((int)n);
+      const uint32_t d_tmem = tmem + col;
+      for (int kb = 0; kb < nkb; ++kb) {
+        if (!mbar_wait(&mi->full[stage], phase, abort_flag)) goto mma_done;
+        tc_fence_after();
+        const uint32_t sa = abase + kb * (kTM * 128), sb = st_base + stage * STAGE_BYTES;
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+          umma_bf16(d_tmem, umma_desc(sa + k4 * 32), umma_desc(sb + k4 * 32), idesc, (last || (kb | k4) != 0) ? 1u : 0u);
+        umma_commit(&mi->empty[stage]);  // frees the weight stage once these MMAs have read it
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+      }
+      umma_commit(&mi->acc_full[bar]);
     }
+  }
+mma_done:
+  if (*abort_flag) {
+    // leaving early: the MMAs already issued must have completed before the TMEM columns are returned
+    umma_commit(&mi->drain);
+    for (int it = 0; it < kMaxPolls && !mbar_try(&mi->drain, 0u); ++it) {}
+  }
 }
 
-// ================= loader warps: row list + gather, one tile ahead of the compute warps ==================
+// ================= loader warp: row list, one tile ahead of the compute warps =============================
 __device__ __forceinline__ void loader_sync() { asm volatile("bar.sync 6, %0;" ::"n"(kLoadThreads) : "memory"); }
 
-// Distinct slots of each set -> tile rows (Eq. 4), per-row set ranges, per-set first rows: one thread per
+// Distinct slots of each set -> tile rows (Eq. 4) and per-row set ranges: one thread per
 // set (a tile of a sparse region holds dozens of tiny sets), walking the set's table row.
 template <bool RPB>
-__device__ __forceinline__ void loader_row_list(int b, int lt, int s_lo, int nsets, int base) {
-  const int32_t* __restrict__ table = s_mi.table;
-  const int32_t* __restrict__ rowoff = s_mi.rowoff;
+__device__ __forceinline__ void loader_row_list(const int32_t* __restrict__ table, const int32_t* __restrict__ rowoff,
+                                                int b, int lt, int s_lo, int nsets, int base) {
   const int n = s_mi.n, tau = s_mi.tau;
   for (int si = lt; si < nsets; si += kLoadThreads) {
     const int s = s_lo + si;
@@ -705,7 +725,7 @@ __device__ __forceinline__ void loader_row_list(int b, int lt, int s_lo, int nse
     constexpr bool rpb = RPB;
     int lo3[3] = {INT_MAX, INT_MAX, INT_MAX}, hi3[3] = {INT_MIN, INT_MIN, INT_MIN};
     for (int k0 = 0; k0 < tau; k0 += 8) {
-      int v4[8];  // eight independent loads per round trip to L2 (the loader warps run a whole tile ahead)
+      int v4[8];  // eight independent loads per round trip to L2 (the loader warp runs a whole tile ahead)
 #pragma unroll
       for (int u = 0; u < 8; ++u) v4[u] = k0 + u < tau ? __ldg(trow + k0 + u) : 0;
       if (rpb) {  // a set spread wider than the bias table's extent is reported
@@ -737,7 +757,6 @@ __device__ __forceinline__ void loader_row_list(int b, int lt, int s_lo, int nse
         }
       }
     }
-    s_mi.set_lo[b][si] = (unsigned char)min(max(lb, 0), kTM);
     if (rpb)
       for (int q = 0; q < 3; ++q) bad |= hi3[q] >= lo3[q] && hi3[q] - lo3[q] > s_mi.rb_ext[q] - 1;
     if (bad || pos != cap) atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX);
@@ -745,7 +764,7 @@ __device__ __forceinline__ void loader_row_list(int b, int lt, int s_lo, int nse
 }
 
 template <int C, bool RPB>
-__device__ __noinline__ void loader_role() {
+__device__ __noinline__ void loader_role(const TcArgs& a) {
   const int lt = threadIdx.x - 32 * kLoadWarp0, lane = lt & 31;
   volatile int* abort_flag = &s_mi.abort_flag;
   int slot = 0;
@@ -756,16 +775,12 @@ __device__ __noinline__ void loader_role() {
     // every exit from this loop is taken by all loader threads together
     if (bar_or(6, kLoadThreads, !ok || *abort_flag != 0)) break;
     const int s_lo = s_mi.tile[slot][0], nsets = s_mi.tile[slot][1], base = s_mi.tile[slot][2], rows = s_mi.tile[slot][3];
+    const int lay = s_mi.tile[slot][4];
     __syncwarp();
     if (lane == 0) mbar_arrive(&s_mi.sched_empty[slot]);
     if (++slot == 2) { slot = 0; sphase ^= 1u; }
     const int b = k & 1;
-    if (k == 0) {  // the compute warps list a CTA's first tile themselves (nothing can run ahead of it)
-      mbar_arrive(&s_mi.rl_ready[b]);
-      if (nsets < 0) break;
-      continue;
-    }
-    // buffer b was last used by tile k - 2: the compute warps release it when they are done with that tile
+    // buffer b was last used by tile k - 2: the compute warps and the stamp warp release it when they are done with it
     if (k >= 2) ok = mbar_wait(&s_mi.rl_free[b], (uint32_t)((k >> 1) - 1) & 1u, abort_flag) && ok;
     if (nsets >= 0) {
       for (int i = lt; i < kTM; i += kLoadThreads) {
@@ -774,12 +789,51 @@ __device__ __noinline__ void loader_role() {
         s_mi.row_n[b][i] = 1;
       }
       loader_sync();
-      loader_row_list<RPB>(b, lt, s_lo, nsets, base);
-      if (lt == 0) s_mi.set_lo[b][nsets] = (unsigned char)rows;
+      const TcLayer& ly = a.layer[lay];
+      loader_row_list<RPB>(ly.table, ly.rowoff, b, lt, s_lo, nsets, base);
+      if (lt == 0) s_mi.next_x[b] = lay == 0 ? a.x : a.y;
     }
     if (lt == 0) s_mi.next_rows[b] = nsets < 0 ? -1 : rows;
     mbar_arrive(&s_mi.rl_ready[b]);
     if (nsets < 0) break;
+    // a tile of a later layer reads rows the previous layer wrote, possibly on other SMs: each row must carry that
+    // layer's stamp (written after the row's store) before the tile is gathered
+    if (lay > 0) {
+      loader_sync();  // the row list is complete
+      const int want = a.stamp_base + lay;
+      for (int r = lt; r < rows && ok; r += kLoadThreads) {
+        const int v = s_mi.rowvox[b][r];
+        if (v < 0) continue;
+        int it = 0;
+        while (ld_acquire_gpu(a.row_stamp + v) != want) {
+          if (++it >= kStampPolls || *abort_flag) { *abort_flag = 1; ok = false; break; }
+          __nanosleep(256);
+        }
+      }
+    }
+    mbar_arrive(&s_mi.dep_ready[b]);
+  }
+}
+
+// ================= stamp warp: completion stamps of a stored tile's rows ==================================
+__device__ __noinline__ void stamp_role(int32_t* __restrict__ row_stamp) {
+  const int lane = threadIdx.x & 31;
+  volatile int* abort_flag = &s_mi.abort_flag;
+  for (int k = 0;; ++k) {
+    const int b = k & 1;
+    // (a failed wait has raised the abort flag: the compute warps leave their loop, and so does this warp)
+    if (!mbar_wait(&s_mi.stored[b], (uint32_t)(k >> 1) & 1u, abort_flag)) break;
+    if (s_mi.exit_at == k) break;
+    const int rows = s_mi.st_rows[b], stamp = s_mi.st_stamp[b];
+    if (stamp != 0) {
+      __threadfence();  // the rows' stores (ordered before this warp by the barrier) are visible before the stamps
+      for (int r = lane; r < rows; r += 32) {
+        const int v = s_mi.rowvox[b][r];
+        if (v >= 0) st_relaxed_gpu(row_stamp + v, stamp);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&s_mi.rl_free[b]);
   }
 }
 
@@ -788,69 +842,12 @@ __device__ __noinline__ void loader_role() {
 // rest from s_mi, so that each gets a register allocation of its own and the tile loop keeps almost nothing
 // alive across the calls.
 
-// Row list of a CTA's first tile by the compute warps (one warp per set), into buffer 0.
-template <bool RPB>
-__device__ __noinline__ void phase_row_list() {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int32_t* __restrict__ table = s_mi.table;
-  const int32_t* __restrict__ rowoff = s_mi.rowoff;
-  const int n = s_mi.n, tau = s_mi.tau, s_lo = s_mi.s_lo, nsets = s_mi.nsets, base = s_mi.base;
-  // (runs once per CTA: loops kept rolled, the kernel's text is better spent elsewhere)
-#pragma unroll 1
-  for (int si = warp; si < nsets; si += kComputeWarps) {
-    const int s = s_lo + si;
-    const int32_t* trow = table + (size_t)s * tau;
-    const int lb = rowoff[s] - base, cap = rowoff[s + 1] - rowoff[s];
-    const int cnt_max = (lb >= 0 && lb < kTM) ? min(cap, kTM - lb) : 0;
-    int cnt = 0;
-    int lo3[3] = {INT_MAX, INT_MAX, INT_MAX}, hi3[3] = {INT_MIN, INT_MIN, INT_MIN};
-#pragma unroll 1
-    for (int k0 = 0; k0 < tau; k0 += 32) {
-      const int k = k0 + lane;
-      int v = -1;
-      bool uniq = false;
-      if (k < tau) { v = trow[k]; uniq = (k == 0) || (v != trow[k - 1]); }
-      if (RPB && v >= 0 && v < n) {
-        const int4 c = __ldg(s_mi.coords + v);
-        lo3[0] = min(lo3[0], c.y); hi3[0] = max(hi3[0], c.y);
-        lo3[1] = min(lo3[1], c.z); hi3[1] = max(hi3[1], c.z);
-        lo3[2] = min(lo3[2], c.w); hi3[2] = max(hi3[2], c.w);
-      }
-      const unsigned bal = __ballot_sync(0xffffffffu, uniq);
-      const int pos = cnt + __popc(bal & ((1u << lane) - 1u));
-      if (uniq && pos < cnt_max) {
-        if (v < 0 || v >= n) { atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX); v = -1; }
-        s_mi.rowvox[0][lb + pos] = v;
-      }
-      cnt += __popc(bal);
-    }
-#pragma unroll 1
-    for (int i = lane; i < cnt_max; i += 32) {
-      s_mi.row_lo[0][lb + i] = (unsigned char)lb;
-      s_mi.row_n[0][lb + i] = (unsigned char)cnt_max;
-    }
-    bool wide = false;
-    if (RPB) {  // a set spread wider than the bias table's extent is reported
-#pragma unroll
-      for (int q = 0; q < 3; ++q) {
-        const int l = __reduce_min_sync(0xffffffffu, lo3[q]), hmax = __reduce_max_sync(0xffffffffu, hi3[q]);
-        wide |= hmax >= l && hmax - l > s_mi.rb_ext[q] - 1;
-      }
-    }
-    if (lane == 0) {
-      s_mi.set_lo[0][si] = (unsigned char)min(max(lb, 0), kTM);
-      if (cnt != cap || wide) atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX);
-    }
-  }
-  if (tid == 0) s_mi.set_lo[0][nsets] = (unsigned char)s_mi.rows;
-}
-
 // Gather (Eq. 4): the fp32 rows listed in buffer b -> bf16 A operand, four rows in flight per warp; all 128 rows
 // are written (rows past the tile as zeros).
 template <int C, bool RPB>
 __device__ __noinline__ void phase_gather(int b, int rows) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const float* __restrict__ x = s_mi.x;
+  const float* x = s_mi.next_x[b];
   unsigned char* a_tile = s_mi.sm + s_mi.off_a;
   const int* rowvox = s_mi.rowvox[b];
   for (int r0 = warp; r0 < kTM; r0 += 4 * kComputeWarps) {
@@ -862,8 +859,8 @@ __device__ __noinline__ void phase_gather(int b, int rows) {
       f[u][0] = f[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (v >= 0 && lane < (C >> 3)) {
         const float4* src = reinterpret_cast<const float4*>(x + (size_t)v * C) + 2 * lane;
-        f[u][0] = __ldg(src);
-        f[u][1] = __ldg(src + 1);
+        f[u][0] = __ldcg(src);  // (L2: the rows of a later layer were written during this launch, by any SM)
+        f[u][1] = __ldcg(src + 1);
       }
       if (RPB && lane == 31) {  // (lane 31 carries no feature columns: C / 8 <= 24)
         int lin = 0;
@@ -1109,12 +1106,47 @@ __device__ __noinline__ void phase_epi_f2() {
   *reinterpret_cast<float4*>(stage + stage_off<C>(row, hq * (QC / 4))) = make_float4(t[0], t[1], t[2], t[3]);
 }
 
+// The layer's biases and LayerNorm vectors into the parameter block (absent vectors as zeros), and its scalars.
+// Order of ParOff: b_q, b_v, b_o, b_2, ln1_g, ln1_b, ln2_g, ln2_b, then b_1 (the key bias is not needed).
+template <int C>
+__device__ __forceinline__ void load_layer_params(const TcLayer& ly, int hidden) {
+  float* par = reinterpret_cast<float*>(s_mi.sm + s_mi.off_par);
+  const int n_par = ParOff<C>::vectors * C + hidden;
+  for (int i = threadIdx.x; i < n_par; i += kComputeThreads) {
+    const int which = i / C;
+    const float* v = which == 0 ? ly.b_qkv : which == 1 ? (ly.b_qkv ? ly.b_qkv + 2 * C : nullptr) : which == 2 ? ly.b_o
+                   : which == 3 ? ly.b_2 : which == 4 ? ly.ln1_g : which == 5 ? ly.ln1_b : which == 6 ? ly.ln2_g
+                   : which == 7 ? ly.ln2_b : (ly.b_1 ? ly.b_1 - ParOff<C>::b_1 + which * C : nullptr);
+    par[i] = v ? __ldg(v + i % C) : 0.f;
+  }
+  if (threadIdx.x == 0) {
+    s_mi.ln1 = ly.ln1_g != nullptr;
+    s_mi.ln2 = ly.ln2_g != nullptr;
+    s_mi.eps = ly.eps;
+    s_mi.rpb = ly.rpb;
+  }
+}
+
+// Barrier over the compute threads that also ANDs a predicate.
+__device__ __forceinline__ bool compute_all(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %2, 0;\n\t"
+      "bar.red.and.pred p, 1, %1, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "n"(kComputeThreads), "r"((uint32_t)pred)
+      : "memory");
+  return r != 0;
+}
+
 // TMEM map (512 columns): region 0 = [0, C): K, Q, O and the even MLP-1 pieces; region 1 = [C, 2C): V and
 // the odd MLP-1 pieces; region 2 = [512 - C, 512): x1 + b_2 parked by the output-projection epilogue, then
 // the MLP-2 accumulator.  Each region has its own full / free barrier pair.  For C = 192 regions 1 and 2
 // overlap, which is why the MMA issuer waits for region 2 before it starts the next tile's V.
 template <int C, int D, int NT, bool RPB>
-__device__ __forceinline__ void compute_role() {
+__device__ __forceinline__ void compute_role(const TcArgs& a) {
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
   constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
   constexpr uint32_t COL_B = C;      // accumulator region 1
@@ -1123,6 +1155,8 @@ __device__ __forceinline__ void compute_role() {
   int slot = 0;
   uint32_t sphase = 0;
   bool ok = true;
+  bool gathered = false;  // the tile about to start was gathered under the previous tile's tail
+  int cur_layer = -1;     // layer whose vectors are in the parameter block
   auto acc_wait = [&](uint32_t bar) {
     ok = mbar_wait(&s_mi.acc_full[bar], uses[bar] & 1u, abort_flag) && ok;
     ++uses[bar];
@@ -1130,51 +1164,56 @@ __device__ __forceinline__ void compute_role() {
   };
   // The next tile's rows are gathered as soon as the current tile's MMAs have stopped reading the A operand
   // (the caller has just waited for the accumulator of the last such chunk), so that its first projections
-  // run on the tensor pipe while the compute warps finish the current tile.
+  // run on the tensor pipe while the compute warps finish the current tile; unless its rows are not all stamped
+  // yet: then the gather waits until this tile is done (the row that is missing may be one of this tile's own).
   auto gather_next = [&](int k) {
     const int b = (k + 1) & 1;
-    ok = mbar_wait(&s_mi.rl_ready[b], (uint32_t)((k + 1) >> 1) & 1u, abort_flag) && ok;
+    const uint32_t par = (uint32_t)((k + 1) >> 1) & 1u;
+    ok = mbar_wait(&s_mi.rl_ready[b], par, abort_flag) && ok;
     const int nr = s_mi.next_rows[b];
-    if (ok && nr >= 0) {
+    if (compute_all(ok && nr >= 0 && mbar_try(&s_mi.dep_ready[b], par))) {
       phase_gather<C, RPB>(b, nr);
       fence_proxy_async();
       mbar_arrive(&s_mi.x_ready);
+      gathered = true;
     }
   };
-  for (int k = 0;; ++k) {
+  int k = 0;
+  for (;; ++k) {
     ok = mbar_wait(&s_mi.sched_full[slot], sphase, abort_flag) && ok;
     // also orders the previous tile's last shared-memory reads before this tile's writes; every exit from
     // this loop is taken by all compute threads together
     if (bar_or(1, kComputeThreads, !ok || *abort_flag != 0)) break;
-    const int nsets = s_mi.tile[slot][1], rows = s_mi.tile[slot][3];
+    const int nsets = s_mi.tile[slot][1], rows = s_mi.tile[slot][3], layer = s_mi.tile[slot][4];
     if (threadIdx.x == 0) {
       s_mi.s_lo = s_mi.tile[slot][0];
       s_mi.nsets = nsets;
       s_mi.base = s_mi.tile[slot][2];
       s_mi.rows = rows;
       s_mi.buf = k & 1;
+      s_mi.layer = layer;
+      s_mi.x = layer == 0 ? a.x : a.y;
       if (k >= 1) mbar_arrive(&s_mi.rl_free[(k - 1) & 1]);  // the previous tile's row list is dead
     }
     mbar_arrive(&s_mi.sched_empty[slot]);
     if (++slot == 2) { slot = 0; sphase ^= 1u; }
     if (nsets < 0) break;
-    const bool listed = k != 0 || s_mi.pre0 != 0;  // (pre0 is not written after the kernel's set-up)
-    if (!listed && threadIdx.x < kTM) {
-      s_mi.rowvox[0][threadIdx.x] = -1;
-      s_mi.row_lo[0][threadIdx.x] = (unsigned char)threadIdx.x;
-      s_mi.row_n[0][threadIdx.x] = 1;
+    if (layer != cur_layer) {  // (the previous tile's last use of the block lies before the barrier above)
+      load_layer_params<C>(a.layer[layer], a.g.hidden);
+      cur_layer = layer;
     }
-    compute_sync();  // the tile's fields are visible to the phase functions
-    if (k == 0) {  // nothing runs ahead of a CTA's first tile: the compute warps list and gather it themselves,
-                   // as a rule already during the kernel's set-up
-      if (!listed) {
-        phase_row_list<RPB>();
-        compute_sync();
-        phase_gather<C, RPB>(0, rows);
+    if (!gathered) {  // a CTA's first tile, or a tile whose rows were not ready in time
+      const uint32_t par = (uint32_t)(k >> 1) & 1u;
+      ok = mbar_wait(&s_mi.rl_ready[k & 1], par, abort_flag) && ok;
+      ok = mbar_wait(&s_mi.dep_ready[k & 1], par, abort_flag) && ok;
+      if (compute_all(ok)) {
+        phase_gather<C, RPB>(k & 1, rows);
         fence_proxy_async();
       }
       mbar_arrive(&s_mi.x_ready);  // X is in place
     }
+    gathered = false;
+    compute_sync();  // the tile's fields and the parameter block are visible to the phase functions
 
     // ---- chunks 0..2: K, V, Q epilogues: (+ bias,) to bf16, into the operand layout ----
     // (the attention pads its key blocks up to 15 rows past the tile: those K / V rows must be real bf16)
@@ -1198,33 +1237,40 @@ __device__ __forceinline__ void compute_role() {
     // ---- chunk 3: output projection epilogue: Z + b_o (+ x, LayerNorm) ----
     acc_wait(0u);
     phase_epi_o<C, QC>();
-    if (mode != 2) {  // final result of this call
+    if (mode != 2) {  // final result of this layer
       gather_next(k);  // the output projection was the last chunk to read the A operand
-      compute_sync();
-      phase_store_rows<C>();
-      continue;
+    } else {
+      fence_proxy_async();
+      mbar_arrive(&s_mi.a_ready);  // x1 (bf16) is the A operand of MLP-1
+      // ---- MLP-1 pieces: H = gelu(x1 W_1^T + b_1) as the A operand of MLP-2 ----
+      const int n_f1 = s_mi.n_f1, NF = s_mi.NF;
+      for (int c = 0; c < n_f1; ++c) {
+        const int bar = c & 1;
+        acc_wait((uint32_t)bar);
+        if (NF == 128)
+          phase_epi_bf16<32, true, true>(bar * COL_B, bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
+        else
+          phase_epi_bf16<16, true, true>(bar * COL_B, bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
+      }
+      fence_proxy_async();
+      mbar_arrive(&s_mi.a_ready);  // H is in place
+      gather_next(k);  // the last MLP-1 piece has been drained: nothing reads the A operand any more
+      // ---- MLP-2 epilogue: y = LN2(x1 + M) ----
+      acc_wait(2u);
+      phase_epi_f2<C, QC>();
     }
-    fence_proxy_async();
-    mbar_arrive(&s_mi.a_ready);  // x1 (bf16) is the A operand of MLP-1
-    // ---- MLP-1 pieces: H = gelu(x1 W_1^T + b_1) as the A operand of MLP-2 ----
-    const int n_f1 = s_mi.n_f1, NF = s_mi.NF;
-    for (int c = 0; c < n_f1; ++c) {
-      const int bar = c & 1;
-      acc_wait((uint32_t)bar);
-      if (NF == 128)
-        phase_epi_bf16<32, true, true>(bar * COL_B, bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
-      else
-        phase_epi_bf16<16, true, true>(bar * COL_B, bar, ParOff<C>::b_1 + c * NF, s_mi.off_kv, (c * NF) >> 3, rows);
-    }
-    fence_proxy_async();
-    mbar_arrive(&s_mi.a_ready);  // H is in place
-    gather_next(k);  // the last MLP-1 piece has been drained: nothing reads the A operand any more
-    // ---- MLP-2 epilogue: y = LN2(x1 + M) ----
-    acc_wait(2u);
-    phase_epi_f2<C, QC>();
     compute_sync();
     phase_store_rows<C>();
+    if (threadIdx.x == 0) {
+      s_mi.st_rows[k & 1] = rows;
+      s_mi.st_stamp[k & 1] = a.n_layers > 1 ? a.stamp_base + layer + 1 : 0;
+    }
+    mbar_arrive(&s_mi.stored[k & 1]);  // the stamp warp takes it from here
   }
+  // tell the stamp warp to leave at iteration k, once it is done with tile k - 2 (which signalled on the same barrier)
+  if (k >= 2) mbar_wait(&s_mi.rl_free[k & 1], (uint32_t)((k >> 1) - 1) & 1u, abort_flag);
+  if (threadIdx.x == 0) s_mi.exit_at = k;
+  mbar_arrive(&s_mi.stored[k & 1]);
   if (!ok || *abort_flag) {
     if (threadIdx.x == 0) atomicOr(s_mi.status, DSVT_STATUS_TIMEOUT);
   }
@@ -1234,54 +1280,30 @@ __device__ __forceinline__ void compute_role() {
 // The kernel
 // ---------------------------------------------------------------------------------------------
 template <int C, int D, int NT, bool RPB>
-__global__ void __launch_bounds__(kThreads, 1)
-layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant__ TcGeom g,
-                const __grid_constant__ TcMaps maps, int32_t* __restrict__ status) {
+__global__ void __launch_bounds__(kThreads, 1) layer_tc_kernel(const __grid_constant__ TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   unsigned char* sm = smem_raw + pad;
   Misc* mi = &s_mi;
   const int tid = threadIdx.x, warp = tid >> 5;
-  RoleCtx rc;
-  rc.S = rc.n_plan = rc.pre_ok = rc.pre_s = rc.pre_ns = rc.pre_base = rc.pre_rows = 0;
-  if (tid == 32 * kTmaWarp) prefetch_first_tile(a, rc);
-  // (the scheduler warp takes no part in the set-up loops: its first thread is busy with the plan look-ups)
-  const bool setup = warp != kTmaWarp;
-  const int stid = warp > kTmaWarp ? tid - 32 : tid;  // dense index of the threads that take part
-  constexpr int kSetupThreads = kThreads - 32;
-  // biases and LayerNorm vectors (absent vectors read as zeros): the loads are issued first, the values go to
-  // shared memory at the end of the set-up.  Order of ParOff: b_q, b_v, b_o, b_2, ln1_g, ln1_b, ln2_g, ln2_b,
-  // then b_1 (the key bias is not needed).
-  constexpr int kParSlots = (ParOff<C>::vectors * C + 2 * C + kSetupThreads - 1) / kSetupThreads;
-  const int n_par = ParOff<C>::vectors * C + g.hidden;
-  float pv[kParSlots];
-#pragma unroll
-  for (int j = 0; j < kParSlots; ++j) {
-    const int i = stid + j * kSetupThreads;
-    pv[j] = 0.f;
-    if (setup && i < n_par) {
-      const dsvt_layer_params& p = a.p;
-      const int which = i / C;
-      const float* v = which == 0 ? p.b_qkv : which == 1 ? (p.b_qkv ? p.b_qkv + 2 * C : nullptr) : which == 2 ? p.b_o
-                     : which == 3 ? p.b_2 : which == 4 ? p.ln1_g : which == 5 ? p.ln1_b : which == 6 ? p.ln2_g
-                     : which == 7 ? p.ln2_b : (p.b_1 ? p.b_1 - ParOff<C>::b_1 + which * C : nullptr);
-      if (v) pv[j] = __ldg(v + i % C);
-    }
-  }
+  const TcGeom& g = a.g;
   if (tid == 0) {  // launch constants for the phase functions
     mi->abort_flag = 0;
-    mi->x = a.x; mi->y = a.y; mi->table = a.table; mi->rowoff = a.rowoff; mi->status = status;
+    mi->exit_at = -1;
+    mi->x = a.x; mi->y = a.y; mi->status = a.status;
     mi->sm = sm; mi->sbase = raw + pad;
     mi->off_a = g.off_a; mi->off_kv = g.off_kv; mi->off_par = g.off_par;
     mi->n = a.n; mi->tau = g.tau; mi->heads = g.heads; mi->mode = g.mode; mi->NF = g.NF; mi->n_f1 = g.n_f1;
-    mi->ln1 = a.p.ln1_g != nullptr; mi->ln2 = a.p.ln2_g != nullptr;
-    mi->eps = a.p.ln_eps;
-    mi->rpb = a.p.rpb; mi->coords = reinterpret_cast<const int4*>(a.p.coords);
+    mi->ln1 = mi->ln2 = 0;
+    mi->eps = 0.f;
+    mi->rpb = nullptr; mi->coords = a.coords;
     mi->rb_len = g.rb_len; mi->rb_sx = g.rb_sx; mi->rb_sy = g.rb_sy; mi->rb_centre = g.rb_centre;
-    mi->rb_ext[0] = a.p.rpb_extent[0]; mi->rb_ext[1] = a.p.rpb_extent[1]; mi->rb_ext[2] = a.p.rpb_extent[2];
-    mi->s_lo = mi->nsets = mi->base = mi->rows = mi->buf = mi->pre0 = 0;
+    mi->rb_ext[0] = g.rb_ext[0]; mi->rb_ext[1] = g.rb_ext[1]; mi->rb_ext[2] = g.rb_ext[2];
+    mi->s_lo = mi->nsets = mi->base = mi->rows = mi->buf = mi->layer = 0;
     mi->next_rows[0] = mi->next_rows[1] = -1;
+    mi->next_x[0] = mi->next_x[1] = a.x;
+    mi->st_rows[0] = mi->st_rows[1] = mi->st_stamp[0] = mi->st_stamp[1] = 0;
   }
   if (tid == 32 * kLoadWarp0) {  // barriers
     for (int i = 0; i < kStages; ++i) { mbar_init(&mi->full[i], 1); mbar_init(&mi->empty[i], 1); }
@@ -1291,12 +1313,15 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&mi->sched_full[i], 1);
-      mbar_init(&mi->sched_empty[i], kComputeThreads + 1 + kLoadWarps);  // compute threads, MMA issuer, loader warps
-      mbar_init(&mi->rl_free[i], 1);
+      mbar_init(&mi->sched_empty[i], kComputeThreads + 1 + kLoadWarps);  // compute threads, MMA issuer, loader warp
+      mbar_init(&mi->rl_free[i], 2);  // the compute warps' first thread and the stamp warp
       mbar_init(&mi->rl_ready[i], kLoadThreads);
+      mbar_init(&mi->dep_ready[i], kLoadThreads);
+      mbar_init(&mi->stored[i], kComputeThreads);
     }
     mbar_init(&mi->a_ready, kComputeThreads);
     mbar_init(&mi->x_ready, kComputeThreads);
+    mbar_init(&mi->drain, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kMmaWarp) {
@@ -1304,70 +1329,33 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
                  "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // The compute warps look up the CTA's first tile themselves (the same plan entries the scheduler reads) and
-  // list and gather it right here, under the rest of the set-up; the A operand is not touched by the loops below.
-  if (warp < kComputeWarps) {
-    const int32_t* plan = a.rowoff + a.cap_sets + 1;
-    const int n_plan = plan[0];
-    const int S = min(*a.num_sets, a.cap_sets);
-    const int f = plan[1 + blockIdx.x], l = plan[2 + blockIdx.x];  // in bounds: see prefetch_first_tile
-    bool pre = n_plan >= 0 && (int)blockIdx.x < n_plan && f >= 0 && l > f && l <= S && l - f <= kTM;
-    int base = 0, rows = 0;
-    if (pre) {
-      base = a.rowoff[f];
-      rows = a.rowoff[l] - base;
-      pre = rows > 0 && rows <= kTM;
-    }
-    compute_sync();  // thread 0's constants are in place
-    if (pre) {
-      if (tid == 0) { mi->s_lo = f; mi->nsets = l - f; mi->base = base; mi->rows = rows; mi->buf = 0; mi->pre0 = 1; }
-      if (tid < kTM) {
-        mi->rowvox[0][tid] = -1;
-        mi->row_lo[0][tid] = (unsigned char)tid;
-        mi->row_n[0][tid] = 1;
-      }
-      compute_sync();
-      phase_row_list<RPB>();
-      compute_sync();
-      phase_gather<C, RPB>(0, rows);
-      fence_proxy_async();
-    }
-  }
   // rows of K / V past the end of a tile are read (and masked) by the attention: never let them hold
   // uninitialised bit patterns
   // (the weight ring behind it as well: key blocks that run past row 127 read a little of it)
-  if (setup)
-    for (uint32_t i = stid; i < ((uint32_t)kTM * 2 * C * 2 + kStages * (uint32_t)C * 128u) / 16; i += kSetupThreads)
-      reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
+  for (uint32_t i = tid; i < ((uint32_t)kTM * 2 * C * 2 + kStages * (uint32_t)C * 128u) / 16; i += kThreads)
+    reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_proxy_async();  // the TMA writes that follow must not be overtaken by these generic stores
-  {
-    float* par = reinterpret_cast<float*>(sm + g.off_par);
-#pragma unroll
-    for (int j = 0; j < kParSlots; ++j) {
-      const int i = stid + j * kSetupThreads;
-      if (setup && i < n_par) par[i] = pv[j];
-    }
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  rc.sm = sm;
+  RoleCtx rc;
   rc.sbase = raw + pad;
   rc.tmem = mi->tmem_base;
-  rc.rowoff = a.rowoff; rc.cap_sets = a.cap_sets;
-  rc.mode = g.mode; rc.n_f1 = g.n_f1; rc.NF = g.NF; rc.nkb_h = g.nkb_h;
+  rc.mode = g.mode; rc.n_f1 = g.n_f1; rc.NF = g.NF; rc.nkb_h = g.nkb_h; rc.tau = g.tau; rc.n_layers = a.n_layers;
   rc.off_a = g.off_a; rc.off_kv = g.off_kv; rc.off_stage = g.off_stage;
 
   if (warp == kTmaWarp) {
-    if ((tid & 31) == 0) producer_role<C>(a, g, maps, status, rc);
+    if ((tid & 31) == 0) producer_role<C>(a, rc);
     __syncwarp();
   } else if (warp == kMmaWarp) {
-    if ((tid & 31) == 0) mma_role<C>(a, g, rc);
+    if ((tid & 31) == 0) mma_role<C>(rc);
     __syncwarp();
+  } else if (warp == kStampWarp) {
+    stamp_role(a.row_stamp);
   } else if (warp >= kLoadWarp0) {
-    loader_role<C, RPB>();
+    loader_role<C, RPB>(a);
   } else {
-    compute_role<C, D, NT, RPB>();
+    compute_role<C, D, NT, RPB>(a);
   }
   // ---- teardown: everyone meets here, then the allocating warp returns the TMEM columns ----
   tc_fence_before();
@@ -1375,6 +1363,14 @@ layer_tc_kernel(const __grid_constant__ dsvt_fused_args a, const __grid_constant
   if (warp == kMmaWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(rc.tmem), "r"(kTmemCols) : "memory");
+  }
+  // the last CTA to leave puts the launch's counters back to zero for the next launch on this context
+  if (tid == 0) {
+    const int left = atomicAdd(a.counter + 1, 1);
+    if (left == (int)gridDim.x - 1) {
+      a.counter[0] = 0;
+      a.counter[1] = 0;
+    }
   }
 }
 
@@ -1386,16 +1382,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn encode_fn() {
+  static std::once_flag once;
   static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  std::call_once(once, [] {
     void* ptr = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
         q == cudaDriverEntryPointSuccess)
       fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
+  });
   return fn;
 }
 
@@ -1412,39 +1407,71 @@ bool make_weight_map(CUtensorMap* m, const void* w, int rows, int cols, int box_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+}  // namespace
+
+// Tensor maps are encoded once per (matrix, shape, box) and context and kept: a backbone calls the same layers
+// frame after frame.
+struct dsvt_map_cache {
+  struct Entry {
+    const void* w;
+    int rows, cols, box_rows;
+    CUtensorMap map;
+  };
+  std::vector<Entry> entries;
+  unsigned attr_done = 0;  // kernel instantiations whose shared-memory attribute is set on this context's device
+};
+
+void dsvt_map_cache_destroy(dsvt_map_cache* c) { delete c; }
+
+namespace {
+
+bool cached_weight_map(dsvt_ctx* ctx, CUtensorMap* out, const void* w, int rows, int cols, int box_rows) {
+  if (!ctx->maps) ctx->maps = new (std::nothrow) dsvt_map_cache();
+  if (!ctx->maps) return false;
+  auto& v = ctx->maps->entries;
+  for (const auto& e : v)
+    if (e.w == w && e.rows == rows && e.cols == cols && e.box_rows == box_rows) { *out = e.map; return true; }
+  dsvt_map_cache::Entry e;
+  e.w = w; e.rows = rows; e.cols = cols; e.box_rows = box_rows;
+  if (!make_weight_map(&e.map, w, rows, cols, box_rows)) return false;
+  if (v.size() >= 256) v.erase(v.begin(), v.begin() + 128);  // (a caller that keeps changing its weights)
+  v.push_back(e);
+  *out = e.map;
+  return true;
+}
+
 template <int C, int D, int NT, bool RPB>
-int launch_tc_one(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
-  cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<C, D, NT, RPB>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
-  layer_tc_kernel<C, D, NT, RPB><<<grid, kThreads, smem, ctx->stream>>>(a, g, maps, ctx->status);
+int launch_tc_one(dsvt_ctx* ctx, const TcArgs& a, int grid, size_t smem, int inst) {
+  if (!(ctx->maps->attr_done & (1u << inst))) {  // once per instantiation and context (the attribute is per device)
+    cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<C, D, NT, RPB>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
+    ctx->maps->attr_done |= 1u << inst;
+  }
+  layer_tc_kernel<C, D, NT, RPB><<<grid, kThreads, smem, ctx->stream>>>(a);
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
 }
 
 // The position bias is a compile-time variant: a layer without one runs a kernel that holds none of its code.
 template <int C, int D, int NT>
-int launch_tc(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
-  if (g.rb_len != 0) return launch_tc_one<C, D, NT, true>(ctx, a, g, maps, grid, smem);
-  return launch_tc_one<C, D, NT, false>(ctx, a, g, maps, grid, smem);
+int launch_tc(dsvt_ctx* ctx, const TcArgs& a, int grid, size_t smem, int inst) {
+  if (a.g.rb_len != 0) return launch_tc_one<C, D, NT, true>(ctx, a, grid, smem, 2 * inst + 1);
+  return launch_tc_one<C, D, NT, false>(ctx, a, grid, smem, 2 * inst);
 }
 
 template <int C, int D>
-int launch_tc_nt(dsvt_ctx* ctx, const dsvt_fused_args& a, const TcGeom& g, const TcMaps& maps, int grid, size_t smem) {
+int launch_tc_nt(dsvt_ctx* ctx, const TcArgs& a, int grid, size_t smem, int inst) {
   // NT = key blocks of 8 a 16-row block can need: the rows of every set it touches, ceil((2 tau + 14) / 8), at most
   // the 16 blocks of a whole tile
-  if (g.tau <= 36) return launch_tc<C, D, 11>(ctx, a, g, maps, grid, smem);
-  if (g.tau <= 48) return launch_tc<C, D, 14>(ctx, a, g, maps, grid, smem);
-  return launch_tc<C, D, 16>(ctx, a, g, maps, grid, smem);
+  if (a.g.tau <= 36) return launch_tc<C, D, 11>(ctx, a, grid, smem, 3 * inst);
+  if (a.g.tau <= 48) return launch_tc<C, D, 14>(ctx, a, grid, smem, 3 * inst + 1);
+  return launch_tc<C, D, 16>(ctx, a, grid, smem, 3 * inst + 2);
 }
+
+int tc_hidden(const dsvt_fused_args& a) { return a.attention_only ? 0 : a.p.hidden; }
 
 }  // namespace
-
-// Tensor map of a row-major bf16 matrix [rows][cols] for boxes of 64 columns x box_rows rows with the 128-byte
-// swizzle (the layout every operand tile here uses); false if the driver entry point is missing or refuses.
-bool dsvt_make_weight_map(void* tensor_map, const void* w, int rows, int cols, int box_rows) {
-  return make_weight_map(reinterpret_cast<CUtensorMap*>(tensor_map), w, rows, cols, box_rows);
-}
 
 // Shapes the tensor-core kernel covers; everything else goes to the FMA kernel.
 bool dsvt_layer_tc_supported(const dsvt_fused_args& a) {
@@ -1457,29 +1484,50 @@ bool dsvt_layer_tc_supported(const dsvt_fused_args& a) {
   const int d = p.C / p.heads;
   const bool shape = (p.C == 192 && d == 24) || (p.C == 128 && (d == 16 || d == 32)) || (p.C == 64 && d == 16);
   if (!shape || p.set_size > 96) return false;
-  const int hidden = a.attention_only ? 0 : p.hidden;
+  const int hidden = tc_hidden(a);
   if (hidden != 0 && hidden != p.C && hidden != 2 * p.C) return false;
   return encode_fn() != nullptr;
 }
 
-int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a) {
-  const dsvt_layer_params& p = a.p;
+// Two layers can share a launch if they have the same shape (one kernel instantiation, one geometry).
+bool dsvt_layer_tc_chainable(const dsvt_fused_args& a, const dsvt_fused_args& b) {
+  const dsvt_layer_params &p = a.p, &q = b.p;
+  if (a.attention_only || b.attention_only || a.n != b.n || a.y != b.y) return false;
+  if (p.C != q.C || p.heads != q.heads || tc_hidden(a) != tc_hidden(b) || p.set_size != q.set_size) return false;
+  if ((p.rpb != nullptr) != (q.rpb != nullptr)) return false;
+  if (p.rpb && (p.coords != q.coords || p.rpb_extent[0] != q.rpb_extent[0] || p.rpb_extent[1] != q.rpb_extent[1] ||
+                p.rpb_extent[2] != q.rpb_extent[2]))
+    return false;
+  return true;
+}
+
+// One launch for layers[0 .. n_layers): layers[0] reads its x and writes y, every later layer runs in place on y
+// (its x must be that y).  All layers pass dsvt_layer_tc_supported and are chainable with layers[0].
+int dsvt_launch_layers_tc(dsvt_ctx* ctx, const dsvt_fused_args* layers, int n_layers) {
+  if (n_layers < 1 || n_layers > kMaxLayers) return DSVT_ERR_INVALID_ARG;
+  if (!ctx->maps) ctx->maps = new (std::nothrow) dsvt_map_cache();
+  if (!ctx->maps) return DSVT_ERR_CUDA;
+  const dsvt_fused_args& a0 = layers[0];
+  const dsvt_layer_params& p = a0.p;
   const int C = p.C;
-  TcGeom g;
-  g.hidden = a.attention_only ? 0 : p.hidden;
+  TcArgs ta = {};
+  TcGeom& g = ta.g;
+  g.hidden = tc_hidden(a0);
   g.heads = p.heads;
   g.tau = p.set_size;
-  g.mode = a.attention_only ? 0 : (g.hidden > 0 ? 2 : 1);
+  g.mode = a0.attention_only ? 0 : (g.hidden > 0 ? 2 : 1);
   g.nkb_h = g.hidden / 64;
   g.NF = (g.hidden % 128 == 0 && C >= 128) ? 128 : 64;
   g.n_f1 = g.hidden / g.NF;
   g.rb_len = g.rb_sx = g.rb_sy = g.rb_centre = 0;
+  g.rb_ext[0] = g.rb_ext[1] = g.rb_ext[2] = 0;
   if (p.rpb) {
     const int L = p.rpb_extent[0], W = p.rpb_extent[1], H = p.rpb_extent[2];
     g.rb_sy = 2 * H - 1;
     g.rb_sx = (2 * W - 1) * g.rb_sy;
     g.rb_len = (2 * L - 1) * g.rb_sx;
     g.rb_centre = (L - 1) * g.rb_sx + (W - 1) * g.rb_sy + (H - 1);
+    g.rb_ext[0] = L; g.rb_ext[1] = W; g.rb_ext[2] = H;
   }
   const uint32_t a_bytes = kTM * C * 2;
   g.off_a = 0;
@@ -1488,23 +1536,54 @@ int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a) {
   g.off_par = g.off_stage + kStages * (uint32_t)C * 128u;
   const size_t smem = (size_t)g.off_par + (size_t)(8 * C + g.hidden) * sizeof(float) + 1024;
   if (smem + sizeof(Misc) + 16 > 227 * 1024) return DSVT_ERR_UNSUPPORTED;  // s_mi is static shared memory
-  TcMaps maps;
-  bool okm = make_weight_map(&maps.qkv, p.W_qkv, 3 * C, C, C) && make_weight_map(&maps.o, p.W_o, C, C, C);
-  if (g.hidden > 0)
-    okm = okm && make_weight_map(&maps.w1, p.W_1, g.hidden, C, g.NF) && make_weight_map(&maps.w2, p.W_2, C, g.hidden, C);
-  else {
-    maps.w1 = maps.o;
-    maps.w2 = maps.o;
+  int64_t grid = 1;
+  for (int l = 0; l < n_layers; ++l) {
+    const dsvt_fused_args& a = layers[l];
+    const dsvt_layer_params& q = a.p;
+    TcLayer& ly = ta.layer[l];
+    bool okm = cached_weight_map(ctx, &ly.qkv, q.W_qkv, 3 * C, C, C) && cached_weight_map(ctx, &ly.o, q.W_o, C, C, C);
+    if (g.hidden > 0)
+      okm = okm && cached_weight_map(ctx, &ly.w1, q.W_1, g.hidden, C, g.NF) &&
+            cached_weight_map(ctx, &ly.w2, q.W_2, C, g.hidden, C);
+    else {
+      ly.w1 = ly.o;
+      ly.w2 = ly.o;
+    }
+    if (!okm) return DSVT_ERR_CUDA;
+    ly.b_qkv = q.b_qkv; ly.b_o = q.b_o; ly.rpb = q.rpb;
+    const bool full = !a.attention_only;
+    ly.b_1 = full ? q.b_1 : nullptr; ly.b_2 = full ? q.b_2 : nullptr;
+    ly.ln1_g = full ? q.ln1_g : nullptr; ly.ln1_b = full ? q.ln1_b : nullptr;
+    ly.ln2_g = full ? q.ln2_g : nullptr; ly.ln2_b = full ? q.ln2_b : nullptr;
+    ly.table = a.table; ly.num_sets = a.num_sets; ly.rowoff = a.rowoff; ly.cap_sets = a.cap_sets;
+    ly.eps = q.ln_eps;
+    const int64_t cap = a.cap_sets < a.n ? a.cap_sets : a.n;
+    if (cap > grid) grid = cap;
   }
-  if (!okm) return DSVT_ERR_CUDA;
+  ta.x = a0.x; ta.y = a0.y; ta.n = a0.n; ta.n_layers = n_layers;
+  ta.coords = reinterpret_cast<const int4*>(p.coords);
+  ta.counter = ctx->tc_counter;
+  ta.row_stamp = ctx->row_stamp;
+  ctx->stamp_serial = (ctx->stamp_serial + 1) & 0x3ffffff;  // (stamps of launches 2^26 apart never meet)
+  if (ctx->stamp_serial == 0) ctx->stamp_serial = 1;
+  ta.stamp_base = (int32_t)(ctx->stamp_serial * 32u);
+  ta.status = ctx->status;
   // one CTA per SM, but no more CTAs than there can be sets
-  int64_t grid = a.cap_sets < a.n ? a.cap_sets : a.n;
   if (grid > ctx->sm_count) grid = ctx->sm_count;
   if (ctx->layer_ctas > 0 && grid > ctx->layer_ctas) grid = ctx->layer_ctas;
   if (grid < 1) grid = 1;
   const int d = C / p.heads;
-  if (C == 192) return launch_tc_nt<192, 24>(ctx, a, g, maps, (int)grid, smem);
-  if (C == 128 && d == 16) return launch_tc_nt<128, 16>(ctx, a, g, maps, (int)grid, smem);
-  if (C == 128) return launch_tc_nt<128, 32>(ctx, a, g, maps, (int)grid, smem);
-  return launch_tc_nt<64, 16>(ctx, a, g, maps, (int)grid, smem);
+  if (C == 192) return launch_tc_nt<192, 24>(ctx, ta, (int)grid, smem, 0);
+  if (C == 128 && d == 16) return launch_tc_nt<128, 16>(ctx, ta, (int)grid, smem, 1);
+  if (C == 128) return launch_tc_nt<128, 32>(ctx, ta, (int)grid, smem, 2);
+  return launch_tc_nt<64, 16>(ctx, ta, (int)grid, smem, 3);
+}
+
+int dsvt_launch_layer_tc(dsvt_ctx* ctx, const dsvt_fused_args& a) { return dsvt_launch_layers_tc(ctx, &a, 1); }
+
+// Tensor map of a row-major bf16 matrix [rows][cols] for boxes of 64 columns x box_rows rows with the 128-byte
+// swizzle (the layout every operand tile here uses), from the context's cache; false if the driver entry point is
+// missing or refuses.
+bool dsvt_cached_weight_map(dsvt_ctx* ctx, void* tensor_map, const void* w, int rows, int cols, int box_rows) {
+  return cached_weight_map(ctx, reinterpret_cast<CUtensorMap*>(tensor_map), w, rows, cols, box_rows);
 }

@@ -645,7 +645,7 @@ extern "C" int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feat
     mma_pool::PoolMaps maps;
     const void* wm[4] = {W_q, W_k, W_v, W_o};
     for (int i = 0; i < 4; ++i)
-      if (!dsvt_make_weight_map(&maps.w[i], wm[i], C, C, C)) return DSVT_ERR_CUDA;
+      if (!dsvt_cached_weight_map(ctx, &maps.w[i], wm[i], C, C, C)) return DSVT_ERR_CUDA;
     mma_pool::pool_attn_mma_kernel<<<(unsigned)gridn, mma_pool::kT, smem, st>>>(a, maps, ctx->status);
     DSVT_LAUNCHED(ctx);
     return DSVT_OK;

@@ -59,11 +59,16 @@ class Stage:
         """Every block on tables that are already filled; the result ends up in y."""
         tables_of = self.tables_of if tables_of is None else tables_of
         ctx = self.ctx if ctx is None else ctx
-        src = x
+        # one dsvt_layers call for the whole stage: X-axis table, Y-axis table of every block's window cut
+        tabs, ws = [], []
         for blk, sp in zip(self.blocks, self.specs):
             t = tables_of[sp]
-            ctx.block(src, t[0], t[1], blk, y, coords=coords)  # (coords: read by layers with a position bias)
-            src = y
+            tabs += [t[0], t[1]]
+            ws += [blk[0], blk[1]]
+        src = x
+        for i in range(0, len(ws), api.MAX_CHAIN_LAYERS):
+            ctx.layers(src, tabs[i:i + api.MAX_CHAIN_LAYERS], ws[i:i + api.MAX_CHAIN_LAYERS], y, coords=coords)
+            src = y  # (coords: read by layers with a position bias)
         return y
 
     def forward(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
