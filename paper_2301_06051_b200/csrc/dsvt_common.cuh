@@ -17,6 +17,7 @@ struct dsvt_ctx {
   int sm_count;
   int layer_ctas;  // cap on the tensor-core layer kernel's grid (0: sm_count)
   int last_cuda_error;
+  unsigned attr_flags;  // kernels whose shared-memory attribute has been raised on this context's device
   int64_t launches;
   // one device allocation carved into the arrays below
   void* arena;

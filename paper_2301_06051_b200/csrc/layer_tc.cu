@@ -1335,6 +1335,10 @@ __global__ void __launch_bounds__(kThreads, 1) layer_tc_kernel(const __grid_cons
   for (uint32_t i = tid; i < ((uint32_t)kTM * 2 * C * 2 + kStages * (uint32_t)C * 128u) / 16; i += kThreads)
     reinterpret_cast<uint4*>(sm + g.off_kv)[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_proxy_async();  // the TMA writes that follow must not be overtaken by these generic stores
+  // everything above touched only this CTA's own state; from here on the kernel reads what earlier kernels in the
+  // stream wrote (tables, features, the launch counters): wait for them if this launch was allowed to start early
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -1448,7 +1452,16 @@ int launch_tc_one(dsvt_ctx* ctx, const TcArgs& a, int grid, size_t smem, int ins
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
     ctx->maps->attr_done |= 1u << inst;
   }
-  layer_tc_kernel<C, D, NT, RPB><<<grid, kThreads, smem, ctx->stream>>>(a);
+  // launched so that it may be set up under the tail of the kernel before it in the stream (the partition, an
+  // earlier chain): the kernel waits for that kernel's completion before it reads anything but its parameters
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = ctx->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  cudaError_t le = cudaLaunchKernelEx(&cfg, layer_tc_kernel<C, D, NT, RPB>, a);
+  if (le != cudaSuccess) { ctx->last_cuda_error = (int)le; cudaGetLastError(); return DSVT_ERR_CUDA; }
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
 }

@@ -14,6 +14,14 @@ constexpr int kSortTile = kSortThreads * kSortRounds;  // keys per block per pas
 constexpr int kRadixBits = 8;
 constexpr int kRadix = 1 << kRadixBits;
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start while its
+// predecessor in the stream still runs; it lets its own successor start early and then waits for the predecessor
+// (and everything before it) to have completed and flushed.  Both are no-ops in an ordinary launch.
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ int warp_incl_scan(int v) {
   const int lane = threadIdx.x & 31;
 #pragma unroll
@@ -331,28 +339,28 @@ __global__ void table_unique_count_kernel(const int32_t* __restrict__ table, int
 // row segments).  The greedy chain 0 -> next(0) -> next(next(0)) ... is found by pointer doubling, all
 // sets in parallel: single block, arrays in shared memory.
 constexpr int kPlanMaxSets = 24576;
-__global__ void __launch_bounds__(kScanThreads) tile_plan_kernel(int32_t* rowoff0, int32_t* rowoff1,
-                                                                 const int32_t* __restrict__ num_sets, int32_t cap_sets,
-                                                                 int32_t smax, int32_t max_rows) {
-  extern __shared__ int plan_smem[];
-  int32_t* rowoff = blockIdx.x ? rowoff1 : rowoff0;  // one block per buffer: offsets, then the plan
-  if (!rowoff) return;
+// Dynamic shared memory the plan needs for at most smax sets.
+__host__ __device__ constexpr size_t plan_smem_bytes(int smax) { return (size_t)(smax + 1) * 8 + (size_t)smax + 16; }
+
+// The plan of `rowoff` (its offsets are read, its plan written; a second buffer with the same offsets, e.g. the
+// other sort axis of the same windows, receives a copy).  One block, any size up to 1024 threads.
+__device__ void tile_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int32_t cap_sets, int32_t smax,
+                               int32_t max_rows, int* plan_smem, int* warp_tot) {
   int32_t* plan = rowoff + cap_sets + 1;
-  __shared__ int warp_tot[33];
+  int32_t* plan2 = rowoff_copy ? rowoff_copy + cap_sets + 1 : nullptr;
   int* cur = plan_smem;
   int* nxt = cur + (smax + 1);
   unsigned char* mark = reinterpret_cast<unsigned char*>(nxt + (smax + 1));
-  const int tid = threadIdx.x;
-  const int S = min(*num_sets, cap_sets);
+  const int tid = threadIdx.x, nthr = blockDim.x;
   if (S > smax) {
-    if (tid == 0) plan[0] = -1;
+    if (tid == 0) { plan[0] = -1; if (plan2) plan2[0] = -1; }
     return;
   }
   if (S <= 0) {
-    if (tid == 0) { plan[0] = 0; plan[1] = 0; }
+    if (tid == 0) { plan[0] = 0; plan[1] = 0; if (plan2) { plan2[0] = 0; plan2[1] = 0; } }
     return;
   }
-  for (int s = tid; s < S; s += kScanThreads) {
+  for (int s = tid; s < S; s += nthr) {
     const int base = rowoff[s];
     int e = s + 1;
     const int first = rowoff[s + 1] - base;
@@ -368,22 +376,39 @@ __global__ void __launch_bounds__(kScanThreads) tile_plan_kernel(int32_t* rowoff
   __syncthreads();
   for (int len = 1; len < S; len <<= 1) {
     // marked sets are tile starts; cur = 'next' applied len times
-    for (int s = tid; s < S; s += kScanThreads)
+    for (int s = tid; s < S; s += nthr)
       if (mark[s] && cur[s] < S) mark[cur[s]] = 1;
-    for (int s = tid; s <= S; s += kScanThreads) nxt[s] = cur[cur[s]];
+    for (int s = tid; s <= S; s += nthr) nxt[s] = cur[cur[s]];
     __syncthreads();
     int* t = cur; cur = nxt; nxt = t;
   }
   // ordered compaction of the marks
-  const int chunk = (S + kScanThreads - 1) / kScanThreads;
+  const int chunk = (S + nthr - 1) / nthr;
   const int s0 = min(tid * chunk, S), s1 = min(s0 + chunk, S);
   int cnt = 0;
   for (int s = s0; s < s1; ++s) cnt += mark[s];
   int total;
   int off = block_excl_scan(cnt, warp_tot, &total);
   for (int s = s0; s < s1; ++s)
-    if (mark[s]) plan[1 + off++] = s;
-  if (tid == 0) { plan[0] = total; plan[1 + total] = S; }
+    if (mark[s]) {
+      plan[1 + off] = s;
+      if (plan2) plan2[1 + off] = s;
+      ++off;
+    }
+  if (tid == 0) {
+    plan[0] = total; plan[1 + total] = S;
+    if (plan2) { plan2[0] = total; plan2[1 + total] = S; }
+  }
+}
+
+__global__ void __launch_bounds__(kScanThreads) tile_plan_kernel(int32_t* rowoff0, int32_t* rowoff1,
+                                                                 const int32_t* __restrict__ num_sets, int32_t cap_sets,
+                                                                 int32_t smax, int32_t max_rows) {
+  extern __shared__ int plan_smem[];
+  __shared__ int warp_tot[33];
+  int32_t* rowoff = blockIdx.x ? rowoff1 : rowoff0;  // one block per buffer: offsets, then the plan
+  if (!rowoff) return;
+  tile_plan_body(rowoff, nullptr, min(*num_sets, cap_sets), cap_sets, smax, max_rows, plan_smem, warp_tot);
 }
 
 // ---- bitmap route: ranks by population count instead of sorting --------------------------------
@@ -407,6 +432,7 @@ struct BmJob {
 __global__ void bm_mark_kernel(const int4* __restrict__ coords, int32_t n, PartGeom g, uint32_t Vp, BmJob job,
                                int32_t* __restrict__ win_count, int32_t* __restrict__ dup_count,
                                int32_t* __restrict__ dup, int32_t* __restrict__ status) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // (the scan kernel may be set up meanwhile)
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   int4 c = coords[i];  // (b, x, y, z)
@@ -443,14 +469,44 @@ __global__ void bm_mark_kernel(const int4* __restrict__ coords, int32_t n, PartG
   dup[i] = ticket;
 }
 
-// Block 0: the per-window scans (Eq. 2).  Other blocks: wordrank, one warp per (axis, window).
+// Block 0: the per-window scans (Eq. 2) and the sets' row offsets.  Other blocks: wordrank, one warp per (axis,
+// window).
 __global__ void __launch_bounds__(kScanThreads) bm_scan_kernel(const int32_t* __restrict__ win_count,
                                                                int32_t num_windows, int32_t tau, int32_t* win_start,
                                                                int32_t* win_setoff, int32_t cap_sets,
                                                                int32_t* num_sets0, int32_t* num_sets1, BmJob job,
-                                                               int32_t wpw, int32_t* status) {
+                                                               int32_t wpw, int32_t* rowoff0, int32_t* rowoff1,
+                                                               int32_t* status) {
+  pdl_enter();
   if (blockIdx.x == 0) {
     window_scan_body(win_count, num_windows, tau, win_start, win_setoff, cap_sets, num_sets0, num_sets1, status);
+    if (!rowoff0 && !rowoff1) return;
+    __syncthreads();  // the scans are visible to the whole block
+    // row offsets: set j of a window of N voxels in S sets starts at rank floor(j N / S) (proof of Theorem A.2);
+    // they depend on the windows only, so both axes get the same ones
+    for (int w = threadIdx.x; w < num_windows; w += kScanThreads) {
+      const int N = win_count[w];
+      if (N == 0) continue;
+      const int so = win_setoff[w], S = win_setoff[w + 1] - so, start = win_start[w];
+      for (int j = 0; j < S && so + j < cap_sets; ++j) {
+        const int v = start + (int)(((int64_t)j * N) / S);
+        if (rowoff0) rowoff0[so + j] = v;
+        if (rowoff1) rowoff1[so + j] = v;
+      }
+    }
+    if (threadIdx.x == 0) {
+      const int S_all = min(win_setoff[num_windows], cap_sets);
+      // (with more sets than the caller's capacity the last kept set ends where the first dropped one starts)
+      int end = win_start[num_windows];
+      if (win_setoff[num_windows] > cap_sets) {
+        int lo = 0, hi = num_windows;  // window of set cap_sets
+        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (win_setoff[mid] <= cap_sets) lo = mid; else hi = mid; }
+        const int N = win_count[lo], so = win_setoff[lo], S = win_setoff[lo + 1] - so;
+        end = win_start[lo] + (int)(((int64_t)(cap_sets - so) * N) / S);
+      }
+      if (rowoff0) rowoff0[S_all] = end;
+      if (rowoff1) rowoff1[S_all] = end;
+    }
     return;
   }
   const int lane = threadIdx.x & 31;
@@ -474,8 +530,31 @@ __global__ void __launch_bounds__(kScanThreads) bm_scan_kernel(const int32_t* __
   }
 }
 
-__global__ void bm_place_kernel(int32_t n, BmJob job, int32_t wpw, const int32_t* __restrict__ dup,
-                                const int32_t* __restrict__ win_start) {
+// Rank -> table: a voxel of inner-window rank r in a window of N voxels and S sets fills the slots m = j tau + k of
+// the window's table rows with floor(m N / (S tau)) == r (Eq. 3, exact integers), i.e. m in
+// [ceil(r S tau / N), ceil((r + 1) S tau / N)): one or two slots as a rule, tau of them for a window of one voxel.
+// The last block builds the tile plan meanwhile (the row offsets come from the scan kernel).
+struct FillOut {
+  int32_t* table[2];
+  int32_t* perm[2];   // optional: voxel ids in sorted order
+  int32_t* rowoff[2]; // optional: offsets are read, the plan is written
+};
+__global__ void __launch_bounds__(256) bm_place_fill_kernel(int32_t n, BmJob job, int32_t wpw,
+                                                            const int32_t* __restrict__ dup,
+                                                            const int32_t* __restrict__ win_count,
+                                                            const int32_t* __restrict__ win_start,
+                                                            const int32_t* __restrict__ win_setoff, int32_t tau,
+                                                            int32_t cap_sets, const int32_t* __restrict__ num_sets,
+                                                            FillOut out, int32_t smax) {
+  extern __shared__ int plan_smem[];
+  __shared__ int warp_tot[33];
+  pdl_enter();
+  if (blockIdx.x == gridDim.x - 1) {  // the plan (one for both axes: their row offsets are the same)
+    int32_t* r0 = out.rowoff[0] ? out.rowoff[0] : out.rowoff[1];
+    int32_t* r1 = out.rowoff[0] ? out.rowoff[1] : nullptr;
+    if (r0) tile_plan_body(r0, r1, min(*num_sets, cap_sets), cap_sets, smax, 128, plan_smem, warp_tot);
+    return;
+  }
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const int ticket = dup[i];
@@ -492,7 +571,15 @@ __global__ void bm_place_kernel(int32_t n, BmJob job, int32_t wpw, const int32_t
         const size_t last = (size_t)win * wpw + (wpw - 1);
         r = job.ax[a].wordrank[last] + __popc(job.ax[a].bitmap[last]) + ticket;
       }
-      job.ax[a].sorted[win_start[win] + r] = i;
+      const int start = win_start[win];
+      if (out.perm[a]) out.perm[a][start + r] = i;
+      const uint64_t N = (uint64_t)win_count[win];
+      const int so = win_setoff[win];
+      const uint64_t St = (uint64_t)(win_setoff[win + 1] - so) * (uint64_t)tau;
+      const uint64_t m_lo = ((uint64_t)r * St + N - 1) / N, m_hi = ((uint64_t)(r + 1) * St + N - 1) / N;
+      const int64_t room = ((int64_t)cap_sets - so) * tau;  // slots of this window that fit the caller's table
+      int32_t* dst = out.table[a] + (size_t)so * tau;
+      for (uint64_t m = m_lo; m < m_hi && (int64_t)m < room; ++m) dst[m] = i;
     }
   }
 }
@@ -553,12 +640,11 @@ int dsvt_launch_rowoff_from_table(dsvt_ctx* ctx, const int32_t* table, int32_t c
 static int launch_tile_plans(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap_sets, int32_t* set_rowoff,
                              int32_t* set_rowoff1) {
   const int32_t smax = cap_sets < kPlanMaxSets ? cap_sets : kPlanMaxSets;
-  const size_t smem = (size_t)(smax + 1) * 8 + (size_t)smax + 16;
-  static bool attr_set = false;
-  if (!attr_set) {
+  const size_t smem = plan_smem_bytes(smax);
+  if (smem > 48 * 1024 && !(ctx->attr_flags & 2u)) {  // (once per context: the attribute belongs to its device)
     DSVT_CUDA_TRY(ctx, cudaFuncSetAttribute(tile_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)((size_t)(kPlanMaxSets + 1) * 8 + kPlanMaxSets + 16)));
-    attr_set = true;
+                                            (int)plan_smem_bytes(kPlanMaxSets)));
+    ctx->attr_flags |= 2u;
   }
   tile_plan_kernel<<<set_rowoff1 ? 2 : 1, kScanThreads, smem, ctx->stream>>>(set_rowoff, set_rowoff1, num_sets,
                                                                             cap_sets, smax, 128);
@@ -689,7 +775,19 @@ int32_t bitmap_words_per_window(const dsvt_ctx* ctx, const PartCall& pc) {
   return (int32_t)wpw;
 }
 
-// Bitmap route: one or both axes in six launches.
+// A launch that may overlap its predecessor's tail (see pdl_enter).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+// Bitmap route: one or both axes in three launches and a memset.
 int partition_bitmap(dsvt_ctx* ctx, const PartCall& pc, int32_t wpw, int naxes, const PartOut* o) {
   cudaStream_t st = ctx->stream;
   const int32_t n = pc.n, nw = pc.nw;
@@ -715,31 +813,34 @@ int partition_bitmap(dsvt_ctx* ctx, const PartCall& pc, int32_t wpw, int naxes, 
   DSVT_LAUNCHED(ctx);
   int64_t rank_blocks = dsvt_ceil_div((int64_t)naxes * nw, kScanThreads / 32);
   if (rank_blocks > 2 * (int64_t)ctx->sm_count) rank_blocks = 2 * (int64_t)ctx->sm_count;
-  bm_scan_kernel<<<(unsigned)(1 + rank_blocks), kScanThreads, 0, st>>>(
-      counts, nw, pc.set_size, ctx->win_start, ctx->win_setoff, pc.cap_sets, o[0].num_sets,
-      naxes > 1 ? o[1].num_sets : nullptr, job, wpw, ctx->status);
+  int32_t* r0 = o[0].set_rowoff;
+  int32_t* r1 = naxes > 1 ? o[1].set_rowoff : nullptr;
+  DSVT_CUDA_TRY(ctx, launch_pdl(bm_scan_kernel, dim3((unsigned)(1 + rank_blocks)), dim3(kScanThreads), 0, st,
+                                (const int32_t*)counts, nw, pc.set_size, ctx->win_start, ctx->win_setoff, pc.cap_sets,
+                                o[0].num_sets, naxes > 1 ? o[1].num_sets : (int32_t*)nullptr, job, wpw, r0, r1,
+                                ctx->status));
   DSVT_LAUNCHED(ctx);
-  bm_place_kernel<<<vox_blocks, 256, 0, st>>>(n, job, wpw, ctx->bm_dup, ctx->win_start);
-  DSVT_LAUNCHED(ctx);
+  // plan capacity: no more sets than floor(n / tau) + non-empty windows
   const int64_t s_bound = sets_bound(pc);
-  if (s_bound > 0) {
-    FillAxis f0{ctx->vals[0], o[0].num_sets, o[0].set_table, o[0].set_rowoff};
-    FillAxis f1 = f0;
-    if (naxes > 1) f1 = FillAxis{ctx->vals[1], o[1].num_sets, o[1].set_table, o[1].set_rowoff};
-    table_fill_kernel<<<dim3((unsigned)dsvt_ceil_div(s_bound, 8), (unsigned)naxes), 256, 0, st>>>(
-        f0, f1, counts, ctx->win_start, ctx->win_setoff, nw, pc.set_size);
-    DSVT_LAUNCHED(ctx);
-    int32_t* r0 = o[0].set_rowoff;
-    int32_t* r1 = naxes > 1 ? o[1].set_rowoff : nullptr;
-    if (!r0) { r0 = r1; r1 = nullptr; }
-    if (r0) {
-      int rc = launch_tile_plans(ctx, o[0].num_sets, pc.cap_sets, r0, r1);
-      if (rc != DSVT_OK) return rc;
-    }
+  const int32_t smax = (int32_t)(s_bound < kPlanMaxSets ? s_bound : kPlanMaxSets);
+  const size_t smem = (r0 || r1) ? plan_smem_bytes(smax) : 0;
+  if (smem > 48 * 1024 && !(ctx->attr_flags & 1u)) {  // (once per context: the attribute belongs to its device)
+    DSVT_CUDA_TRY(ctx, cudaFuncSetAttribute(bm_place_fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)plan_smem_bytes(kPlanMaxSets)));
+    ctx->attr_flags |= 1u;
   }
-  for (int a = 0; a < naxes; ++a)
-    if (o[a].perm)
-      DSVT_CUDA_TRY(ctx, cudaMemcpyAsync(o[a].perm, ctx->vals[a], sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToDevice, st));
+  FillOut fo;
+  for (int a = 0; a < 2; ++a) {
+    const bool on = a < naxes;
+    fo.table[a] = on ? o[a].set_table : nullptr;
+    fo.perm[a] = on ? o[a].perm : nullptr;
+    fo.rowoff[a] = on ? o[a].set_rowoff : nullptr;
+  }
+  DSVT_CUDA_TRY(ctx, launch_pdl(bm_place_fill_kernel, dim3(vox_blocks + 1), dim3(256), smem, st, n, job, wpw,
+                                (const int32_t*)ctx->bm_dup, (const int32_t*)counts, (const int32_t*)ctx->win_start,
+                                (const int32_t*)ctx->win_setoff, pc.set_size, pc.cap_sets,
+                                (const int32_t*)o[0].num_sets, fo, smax));
+  DSVT_LAUNCHED(ctx);
   return copy_window_arrays(ctx, pc, counts);
 }
 
