@@ -360,13 +360,18 @@ __device__ void tile_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int
     if (tid == 0) { plan[0] = 0; plan[1] = 0; if (plan2) { plan2[0] = 0; plan2[1] = 0; } }
     return;
   }
+  // the offsets once into shared memory (the second pointer array is free until the doubling rounds): every set
+  // then finds the end of the tile that would start with it by a binary search there
+  int* ro = nxt;
+  for (int s = tid; s <= S; s += nthr) ro[s] = rowoff[s];
+  __syncthreads();
   for (int s = tid; s < S; s += nthr) {
-    const int base = rowoff[s];
+    const int base = ro[s];
     int e = s + 1;
-    const int first = rowoff[s + 1] - base;
+    const int first = ro[s + 1] - base;
     if (first > 0 && first <= max_rows) {  // last e in (s, S] with rowoff[e] - base <= max_rows
       int lo = s + 1, hi = min(S, s + max_rows);
-      while (lo < hi) { const int m = (lo + hi + 1) >> 1; if (rowoff[m] - base <= max_rows) lo = m; else hi = m - 1; }
+      while (lo < hi) { const int m = (lo + hi + 1) >> 1; if (ro[m] - base <= max_rows) lo = m; else hi = m - 1; }
       e = lo;
     }
     cur[s] = e;
@@ -533,13 +538,13 @@ __global__ void __launch_bounds__(kScanThreads) bm_scan_kernel(const int32_t* __
 // Rank -> table: a voxel of inner-window rank r in a window of N voxels and S sets fills the slots m = j tau + k of
 // the window's table rows with floor(m N / (S tau)) == r (Eq. 3, exact integers), i.e. m in
 // [ceil(r S tau / N), ceil((r + 1) S tau / N)): one or two slots as a rule, tau of them for a window of one voxel.
-// The last block builds the tile plan meanwhile (the row offsets come from the scan kernel).
+// Block 0 builds the tile plan meanwhile (the row offsets come from the scan kernel).
 struct FillOut {
   int32_t* table[2];
   int32_t* perm[2];   // optional: voxel ids in sorted order
   int32_t* rowoff[2]; // optional: offsets are read, the plan is written
 };
-__global__ void __launch_bounds__(256) bm_place_fill_kernel(int32_t n, BmJob job, int32_t wpw,
+__global__ void __launch_bounds__(kScanThreads) bm_place_fill_kernel(int32_t n, BmJob job, int32_t wpw,
                                                             const int32_t* __restrict__ dup,
                                                             const int32_t* __restrict__ win_count,
                                                             const int32_t* __restrict__ win_start,
@@ -549,13 +554,13 @@ __global__ void __launch_bounds__(256) bm_place_fill_kernel(int32_t n, BmJob job
   extern __shared__ int plan_smem[];
   __shared__ int warp_tot[33];
   pdl_enter();
-  if (blockIdx.x == gridDim.x - 1) {  // the plan (one for both axes: their row offsets are the same)
+  if (blockIdx.x == 0) {  // the plan (one for both axes: their row offsets are the same)
     int32_t* r0 = out.rowoff[0] ? out.rowoff[0] : out.rowoff[1];
     int32_t* r1 = out.rowoff[0] ? out.rowoff[1] : nullptr;
     if (r0) tile_plan_body(r0, r1, min(*num_sets, cap_sets), cap_sets, smax, 128, plan_smem, warp_tot);
     return;
   }
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const int i = (blockIdx.x - 1) * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const int ticket = dup[i];
 #pragma unroll
@@ -836,7 +841,8 @@ int partition_bitmap(dsvt_ctx* ctx, const PartCall& pc, int32_t wpw, int naxes, 
     fo.perm[a] = on ? o[a].perm : nullptr;
     fo.rowoff[a] = on ? o[a].set_rowoff : nullptr;
   }
-  DSVT_CUDA_TRY(ctx, launch_pdl(bm_place_fill_kernel, dim3(vox_blocks + 1), dim3(256), smem, st, n, job, wpw,
+  const unsigned fill_blocks = (unsigned)dsvt_ceil_div(n, kScanThreads);
+  DSVT_CUDA_TRY(ctx, launch_pdl(bm_place_fill_kernel, dim3(fill_blocks + 1), dim3(kScanThreads), smem, st, n, job, wpw,
                                 (const int32_t*)ctx->bm_dup, (const int32_t*)counts, (const int32_t*)ctx->win_start,
                                 (const int32_t*)ctx->win_setoff, pc.set_size, pc.cap_sets,
                                 (const int32_t*)o[0].num_sets, fo, smax));
