@@ -5,10 +5,12 @@ A step is one pass of the whole path over one frame: rotated set partition (both
 every DSVT block of the backbone (configuration 2: 32,000 pillars on 468 x 468, C = 192, 8 heads,
 set size 36, four blocks of two layers with MLP and LayerNorm, bfloat16 weights, fp32 accumulate).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2] [--per-config 1 3 ...]
 
 Prints one JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own frame: the path shards
-by frame with no collective, so scaling is weak.
+by frame with no collective, so scaling is weak.  Besides the headline configuration's figures the line carries
+`per_config` (latency of the path's parts at the other configurations, one frame at a time) and `rooflines` (one
+entry per kind of kernel: fused layers, pooling, partition, BEV projection, the fp32 layer path).
 """
 from __future__ import annotations
 
@@ -37,9 +39,31 @@ def _peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one fused-layer launch at configuration 2, from the ncu capture
-# summarised in profiles/layer_tc_kernel_config2.md (25.63 MB read + 0.06 MB written: the output stays in L2).
-LAYER_DRAM_BYTES_PER_LAUNCH = 25.69e6
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "layer_tc_kernel_dram.json")
+KERNEL_SOURCES = ("layer_tc.cu", "dsvt_common.cuh")
+
+
+def kernel_revision() -> str:
+    """Hash of the layer kernel's source files: ties a stored counter reading to the kernel that was measured."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2301_06051_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic(cid: int):
+    """DRAM bytes of one layer-chain launch from the stored ncu reading, or None if there is none for this
+    configuration or the kernel's source has changed since it was taken."""
+    try:
+        rec = json.load(open(TRAFFIC_FILE))
+    except (OSError, ValueError):
+        return None
+    if rec.get("kernel_revision") != kernel_revision() or rec.get("config") != cid:
+        return None
+    return rec.get("dram_bytes_per_launch")
 
 
 class ClockSampler:
@@ -187,6 +211,163 @@ def run_reference(args):
     }))
 
 
+def _frame_buffers(cfg, dev):
+    import torch
+
+    coords = torch.from_numpy(cfg["coords"]).to(dev)
+    x = torch.from_numpy(cfg["feats"]).to(dev)
+    return coords, x
+
+
+def _median_ms(pairs):
+    return float(np.median([a.elapsed_time(b) for a, b in pairs]))
+
+
+def table_stats(table, set_size, C, hidden):
+    """(#sets, pad ratio, algorithmic FLOP of one layer) of a filled set table."""
+    S = int(table.num_sets.item())
+    ro = table.set_rowoff[: S + 1].cpu().numpy()
+    n = int(ro[-1]) if S else 0
+    pad = 1.0 - n / (S * set_size) if S else 0.0
+    return S, pad, algorithmic_flops_per_layer(ro, C, hidden)
+
+
+def partition_bytes(n: int, S: int, set_size: int) -> float:
+    """Algorithmic bytes of the rotated partition (both axes): coordinates read once; per axis a key and a sorted
+    id per voxel, the set table and the row offsets written."""
+    return 16.0 * n + 2.0 * (8.0 * n + 4.0 * set_size * S + 4.0 * (S + 1))
+
+
+def time_config(cid: int, dev, reps: int, flush):
+    """One frame at a time, L2 flushed before each pass: CUDA-event medians of the path's parts at a configuration."""
+    import torch
+
+    import dsvt_inputs as di
+    from paper_2301_06051_b200 import pipeline
+
+    cfg = di.make_config(cid)
+    stream = torch.cuda.current_stream(dev)
+    coords, x = _frame_buffers(cfg, dev)
+    n, C = cfg["n"], cfg["C"]
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    out = {"config": cid, "name": cfg["name"], "voxels": n, "C": C, "precision": cfg["precision"],
+           "window": list(cfg["window"]), "set_size": cfg["set_size"]}
+    if cfg.get("stages"):  # the voxel variant's layout: stages of one block with pooling along z between them
+        bb = pipeline.StagedBackbone(cfg, device=dev.index)
+        recs = []
+        for it in range(2 + reps):
+            flush.zero_()
+            marks = [("start", ev())]
+            oc, of = bb.forward(coords, x, lambda tag: marks.append((tag, ev())))
+            recs.append(marks)
+        torch.cuda.synchronize(dev)
+        if bb.ctx.status_sync() != 0:
+            raise SystemExit("device status word is not clean (config %d)" % cid)
+        spans = {}
+        for r in recs[2:]:
+            for (_, e0), (t1, e1) in zip(r[:-1], r[1:]):
+                spans.setdefault(t1, []).append(e0.elapsed_time(e1))
+            spans.setdefault("backbone", []).append(r[0][1].elapsed_time(r[-1][1]))
+        med = {k: float(np.median(v)) for k, v in spans.items()}
+        out.update({"voxels_out": int(oc.shape[0]), "stages": len(cfg["stages"]),
+                    "t_partition_ms": [med["s%d_partition" % i] for i in range(len(cfg["stages"]))],
+                    "t_block_ms": [med["s%d_blocks" % i] / len(st["blocks"]) for i, st in enumerate(cfg["stages"])],
+                    "t_pool_ms": [med["s%d_pool" % i] for i in range(len(cfg["pools"]))],
+                    "t_backbone_ms": med["backbone"], "frames_per_s": cfg["batch"] / (med["backbone"] * 1e-3),
+                    "note": "the pooled voxel count is read back on the host between stages (inside t_backbone_ms)"})
+        return out, None
+    bb = pipeline.Backbone(cfg, device=dev.index)
+    y = torch.empty_like(x)
+    st1, nb1 = bb.stage1, len(cfg["blocks"])
+    recs = []
+    m = n
+    for it in range(2 + reps):
+        flush.zero_()
+        r = {"t0": ev()}
+        st1.partition(coords)
+        r["t1"] = ev()
+        st1.run_blocks(coords, x, y)
+        r["t2"] = ev()
+        if bb.stage2:
+            oc, of, num, _, _ = bb.ctx.pool(coords, y, cfg["batch"], cfg["grid"], bb.pool_shape, bb.pool_w)
+            r["t3"] = ev()
+            m = int(num.item())  # the pooled voxel count sizes the second stage's tensors (a host read-back)
+            r["t4"] = ev()
+            bb.stage2.partition(oc[:m])
+            r["t5"] = ev()
+            bb.stage2.run_blocks(oc[:m], of[:m], of[:m])
+            r["t6"] = ev()
+        recs.append(r)
+    torch.cuda.synchronize(dev)
+    if bb.ctx.status_sync() != 0:
+        raise SystemExit("device status word is not clean (config %d)" % cid)
+    recs = recs[2:]
+    span = lambda a, b: _median_ms([(r[a], r[b]) for r in recs])
+    hidden = int(cfg["blocks"][0][0].get("hidden", 0))
+    S, pad, fl0 = table_stats(st1.tables[0], cfg["set_size"], C, hidden)
+    _, _, fl1 = table_stats(st1.tables[1], cfg["set_size"], C, hidden)
+    t_part, t_blocks = span("t0", "t1"), span("t1", "t2")
+    last = "t6" if bb.stage2 else "t2"
+    t_bb = span("t0", last)
+    out.update({"sets": S, "pad_ratio": pad, "t_partition_ms": t_part, "t_block_ms": t_blocks / nb1,
+                "voxel_blocks_per_s": n * nb1 / (t_blocks * 1e-3), "t_backbone_ms": t_bb,
+                "frames_per_s": cfg["batch"] / (t_bb * 1e-3),
+                "layer_tflops": nb1 * (fl0 + fl1) / (t_blocks * 1e-3) / 1e12,
+                "partition_gbs": partition_bytes(n, S, cfg["set_size"]) / (t_part * 1e-3) / 1e9})
+    extra = {"flops_stage1": nb1 * (fl0 + fl1), "t_stage1_blocks_ms": t_blocks, "n": n, "S": S}
+    if bb.stage2:
+        nb2 = len(cfg["blocks_after_pool"])
+        ns = int(np.prod(bb.pool_shape))
+        out.update({"t_pool_ms": span("t2", "t3"), "pooled_voxels": m, "t_partition2_ms": span("t4", "t5"),
+                    "t_block2_ms": span("t5", "t6") / nb2,
+                    "note": "the pooled voxel count is read back on the host between the stages (inside t_backbone_ms)"})
+        extra.update({"pool": {"t_ms": out["t_pool_ms"], "bytes": 4.0 * C * (n + m) + 16.0 * (n + m), "n": n, "m": m,
+                               "slots": ns}})
+    return out, extra
+
+
+def fma_peak_tflops(ctx, dev):
+    """FP32 FMA rate of this device, measured with the library's probe kernel (8 independent chains per thread,
+    two blocks of 1024 threads per SM)."""
+    import torch
+
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    sink = torch.zeros(4, dtype=torch.float32, device=dev)
+    ctx.fma_probe(2 * sms, 1024, 1 << 12, sink)  # warm-up
+    best = 0.0
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        flops = ctx.fma_probe(2 * sms, 1024, 1 << 16, sink)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        best = max(best, flops / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+    return best
+
+
+def time_bev(cfg, ctx, dev, reps, flush):
+    import torch
+
+    coords, x = _frame_buffers(cfg, dev)
+    m = ctx.bev_scatter(coords, x, cfg["batch"], cfg["grid"], False)
+    pairs = []
+    for it in range(2 + reps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.bev_scatter(coords, x, cfg["batch"], cfg["grid"], False, out=m)
+        e1.record()
+        pairs.append((e0, e1))
+    torch.cuda.synchronize(dev)
+    t = _median_ms(pairs[2:])
+    return t, 4.0 * (m.numel() + x.numel() + coords.numel())
+
+
 def run_ours(args):
     import torch
 
@@ -203,8 +384,8 @@ def run_ours(args):
     api.load()  # no fallback: a missing library is an error
 
     cfg = di.make_config(args.config)
-    if cfg.get("pool_shape"):
-        raise SystemExit("bench.py times single-stage configurations (1-4)")
+    if cfg.get("pool_shape") or cfg.get("stages"):
+        raise SystemExit("the headline run takes a single-stage configuration (1-4, 6); 5 and 7 are per_config entries")
     n, C, nb = cfg["n"], cfg["C"], len(cfg["blocks"])
     bb = pipeline.Backbone(cfg, device=local_rank)
     ctx, stage = bb.ctx, bb.stage1
@@ -222,15 +403,11 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    def step_device():
-        stage.forward(coords, x, y)
-
-    # end to end: every step uploads its frame from pinned host memory, runs the step and downloads the result;
-    # pipeline.FrameStream overlaps the copies and the partition of neighbouring steps with the kernels and deals
-    # the steps out to four compute streams (eight sets of device buffers)
+    # a stream of frames: pipeline.FrameStream builds the next step's set tables on a stream of its own and deals
+    # consecutive steps out to LANES compute streams (R rotating sets of device buffers)
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    LANES, R = 4, 8                 # compute streams, rotating sets of buffers
-    lane_ctas = (sms + 2) // 3      # CTAs per layer launch: the four lanes ask for more CTAs than there are SMs
+    LANES, R = args.lanes, 8    # compute streams, rotating sets of buffers
+    lane_ctas = args.lane_ctas if args.lane_ctas > 0 else (sms if LANES == 1 else (sms * 2) // (LANES + 1))
     frames = pipeline.FrameStream(stage, n, C, depth=R, lanes=LANES, layer_ctas=lane_ctas)
     outs_h = [out_h] + [torch.empty((n, C), dtype=torch.float32).pin_memory() for _ in range(R - 1)]
 
@@ -241,15 +418,14 @@ def run_ours(args):
 
     for _ in range(max(args.warmup, 3)):
         flush.zero_()
-        step_device()
+        stage.forward(coords, x, y)
     barrier()
     if ctx.status_sync() != 0:
         raise SystemExit("device status word is not clean after warm-up")
 
-    # ---- timed region: K steps, inputs resident in HBM, through the pipeline a stream of frames runs in: the next
-    # step's partition on its own stream, consecutive steps dealt out to four compute streams whose layer launches
-    # take a third of the SMs each.  The steps rotate over eight sets of (coords, x, y), 397 MB at configuration 2:
-    # larger than L2. ----
+    # ---- timed region: K steps, inputs resident in HBM, through the frame pipeline.  The steps rotate over R sets
+    # of (coords, x, y), larger than L2 together.  The K-step region is repeated until at least half a second of
+    # GPU time has passed (so that the clock sampler has samples inside it); the median repeat is reported. ----
     cs = [coords] + [coords.clone() for _ in range(R - 1)]
     xs = [x] + [x.clone() for _ in range(R - 1)]
     ys = [torch.empty_like(x) for _ in range(R)]
@@ -259,31 +435,38 @@ def run_ours(args):
     barrier()
     if resident.status_sync() != 0:
         raise SystemExit("device status word is not clean after the pipeline's warm-up")
-    ev_begin, ev_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local_rank)
     sampler.start()
     launches0 = resident.launch_count()
     barrier()
     t_begin = time.perf_counter()
-    ev_begin.record(stream)
-    resident.fence(ev_begin)
-    for k in range(args.steps):
-        resident.submit_resident(cs[k % R], xs[k % R], ys[k % R])
-    resident.join(stream)
-    ev_end.record(stream)
-    barrier()
+    repeats, host_us, gpu_ms = [], [], 0.0
+    while gpu_ms < 500.0 and len(repeats) < 2000:
+        ev_begin, ev_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev_begin.record(stream)
+        resident.fence(ev_begin)
+        h0 = time.perf_counter()
+        for k in range(args.steps):
+            resident.submit_resident(cs[k % R], xs[k % R], ys[k % R])
+        host_us.append((time.perf_counter() - h0) * 1e6 / args.steps)
+        resident.join(stream)
+        ev_end.record(stream)
+        barrier()
+        repeats.append(float(ev_begin.elapsed_time(ev_end)))
+        gpu_ms += repeats[-1]
     t_end = time.perf_counter()
-    launches = resident.launch_count() - launches0
+    launches = (resident.launch_count() - launches0) // len(repeats)
     clocks = sampler.stop(t_begin, t_end)
-    total_ms = float(ev_begin.elapsed_time(ev_end))
+    total_ms = float(np.median(repeats))
     if resident.status_sync() != 0:
         raise SystemExit("device status word is not clean after the timed region")
 
     # ---- one step at a time on one stream, L2 flushed (outside the events) before each: the latency of a step and
     # its parts (partition; all blocks as one chained launch, which the roofline figure is taken from) ----
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    lat_steps = max(10, min(args.steps, 100))
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(lat_steps)]
     barrier()
-    for k in range(args.steps):
+    for k in range(lat_steps):
         flush.zero_()
         e = ev[k]
         e[0].record(stream)
@@ -296,9 +479,9 @@ def run_ours(args):
     t_part = np.array([e[0].elapsed_time(e[1]) for e in ev])
     t_chain = np.array([e[1].elapsed_time(e[2]) for e in ev])
     # the same blocks as one launch per block (dsvt_block), for comparison
-    evb = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+    evb = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(lat_steps)]
     yb = torch.empty_like(y)
-    for k in range(args.steps):
+    for k in range(lat_steps):
         flush.zero_()
         evb[k][0].record(stream)
         src = x
@@ -337,14 +520,76 @@ def run_ours(args):
     ms_per_step = total_ms / args.steps
     value = job_throughput(world, n * nb, ms_per_step)
     peaks = _peaks()
-    # dominant kernel: the fused layer kernel, two launches per block
-    S = int(stage.tables[0].num_sets.item())
-    fl = [algorithmic_flops_per_layer(stage.tables[a].set_rowoff[: S + 1].cpu().numpy(), C, cfg["hidden"])
-          for a in (0, 1)]
-    flops_per_launch = nb * (fl[0] + fl[1])  # one launch runs every layer of the stage
-    launch_ms = float(t_chain.mean())
+    # dominant kernel: the fused layer kernel, one launch for all layers of the stage
+    hidden = int(cfg["blocks"][0][0].get("hidden", 0))
+    S, pad, fl0 = table_stats(stage.tables[0], cfg["set_size"], C, hidden)
+    _, _, fl1 = table_stats(stage.tables[1], cfg["set_size"], C, hidden)
+    flops_per_launch = nb * (fl0 + fl1)
+    launch_ms = float(np.median(t_chain))
     achieved = flops_per_launch / (launch_ms * 1e-3) / 1e12
-    pad = 1.0 - n / (S * cfg["set_size"])
+    bf16 = cfg["precision"] == "bf16"
+
+    # ---- the other configurations and the other kinds of kernel (rank 0, one GPU) ----
+    per_config, rooflines = [], []
+    fma_peak = fma_peak_tflops(ctx, dev)
+    if bf16:
+        layer_roof = {"kernel": "fused DSVT layers (one launch per stage)", "config": args.config, "bound": "tensor",
+                      "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                      "frac": achieved / peaks["bf16_tflops"], "flops": flops_per_launch, "ms": launch_ms}
+    else:
+        layer_roof = {"kernel": "fused DSVT layers, fp32 FMA path (one launch per layer)", "config": args.config,
+                      "bound": "alu", "achieved": achieved, "peak": fma_peak, "unit": "TFLOP/s",
+                      "frac": achieved / fma_peak, "flops": flops_per_launch, "ms": launch_ms,
+                      "peak_source": "measured in this run with the library's FMA probe kernel"}
+    rooflines.append(layer_roof)
+    t_p = float(np.median(t_part))
+    pb = partition_bytes(n, S, cfg["set_size"])
+    rooflines.append({"kernel": "rotated partition (both axes; memset + 3 launches)", "config": args.config,
+                      "bound": "hbm", "bytes": pb, "ms": t_p, "achieved": pb / (t_p * 1e-3) / 1e9,
+                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": pb / (t_p * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                      "note": "a few MB of traffic: bound by the latency of three dependent launches, not by HBM"})
+    if world == 1 and args.per_config:
+        t_b, bev_bytes = time_bev(cfg, ctx, dev, 10, flush)
+        rooflines.append({"kernel": "BEV projection (cell-map clear + mark + dense writer)", "config": args.config,
+                          "bound": "hbm", "bytes": bev_bytes, "ms": t_b, "achieved": bev_bytes / (t_b * 1e-3) / 1e9,
+                          "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                          "frac": bev_bytes / (t_b * 1e-3) / 1e9 / peaks["hbm_gbs"]})
+        for cid in args.per_config:
+            if cid == args.config:
+                continue
+            pc, extra = time_config(cid, dev, 10, flush)
+            per_config.append(pc)
+            if extra is None:
+                continue
+            if pc["precision"] == "bf16":
+                a_t = extra["flops_stage1"] / (extra["t_stage1_blocks_ms"] * 1e-3) / 1e12
+                pc["roofline_frac"] = a_t / peaks["bf16_tflops"]
+                rooflines.append({"kernel": "fused DSVT layers (one launch per stage)", "config": cid,
+                                  "bound": "tensor", "achieved": a_t, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                  "frac": a_t / peaks["bf16_tflops"], "flops": extra["flops_stage1"],
+                                  "ms": extra["t_stage1_blocks_ms"]})
+            else:
+                a_t = extra["flops_stage1"] / (extra["t_stage1_blocks_ms"] * 1e-3) / 1e12
+                pc["roofline_frac"] = a_t / fma_peak
+                rooflines.append({"kernel": "fused DSVT layers, fp32 FMA path (one launch per layer)", "config": cid,
+                                  "bound": "alu", "achieved": a_t, "peak": fma_peak, "unit": "TFLOP/s",
+                                  "frac": a_t / fma_peak, "flops": extra["flops_stage1"],
+                                  "ms": extra["t_stage1_blocks_ms"],
+                                  "peak_source": "measured in this run with the library's FMA probe kernel",
+                                  "note": "2,000 voxels: 56 thread blocks of work, bound by launch and memory "
+                                          "latency rather than by the FMA pipes"})
+            if "pool" in extra:
+                pl = extra["pool"]
+                # Eq. 7: key and value maps on every padded slot, query and output maps per region
+                pflops = 2.0 * C * C * (2.0 * pl["m"] * pl["slots"] + 2.0 * pl["m"])
+                t_hbm = pl["bytes"] / (peaks["hbm_gbs"] * 1e9) * 1e3
+                t_tc = pflops / (peaks["bf16_tflops"] * 1e12) * 1e3
+                rooflines.append({"kernel": "attention-style pooling (mark, scan, finish, fused attention kernel)",
+                                  "config": cid, "bound": "hbm" if t_hbm >= t_tc else "tensor", "bytes": pl["bytes"],
+                                  "flops": pflops, "ms": pl["t_ms"], "ms_at_hbm_peak": t_hbm,
+                                  "ms_at_tensor_peak": t_tc, "frac": max(t_hbm, t_tc) / pl["t_ms"],
+                                  "achieved": pl["bytes"] / (pl["t_ms"] * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                                  "unit": "GB/s"})
 
     # ---- CPU oracle on a bounded sample (reported baseline, not a target) ----
     from oracle import ref
@@ -365,36 +610,41 @@ def run_ours(args):
     print(json.dumps({
         "metric": METRIC, "value": value, "unit": "voxels/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16" if cfg["precision"] == "bf16" else "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
         "config": {"workload": workload_name(args.config, cfg),
                    "l2": "timed steps rotate over %d sets of inputs and outputs (%d MB, larger than L2); the "
                          "one-step-at-a-time figures: L2 flushed by a %d MiB write before every step"
                          % (R, R * (2 * x.numel() + coords.numel()) * 4 // 1000000, L2_FLUSH_BYTES >> 20),
                    "pipeline": "inputs resident in HBM; the next step's partition on its own stream, consecutive "
-                               "steps dealt out to %d compute streams, %d CTAs per layer launch; CUDA events around "
-                               "all K steps" % (LANES, lane_ctas),
+                               "steps dealt out to %d compute stream(s), %d CTAs per layer launch; the K-step region "
+                               "repeated %d times (%.0f ms of GPU time), median repeat reported; CUDA events around "
+                               "each repeat" % (LANES, lane_ctas, len(repeats), gpu_ms),
                    "num_sets": S, "pad_ratio": pad, "frames_per_rank": 1},
         "frames_per_sec": world / (ms_per_step * 1e-3),
-        "step_latency_ms": float(t_step.mean()),
-        "t_partition_ms": float(t_part.mean()), "t_block_ms": launch_ms / nb,
-        "t_block_ms_one_launch_per_block": float(t_blockwise.mean()) / nb,
+        "step_latency_ms": float(np.median(t_step)),
+        "t_partition_ms": t_p, "t_block_ms": launch_ms / nb,
+        "t_block_ms_one_launch_per_block": float(np.median(t_blockwise)) / nb,
+        "host_us_per_step": float(np.median(host_us)),
         "clocks": clocks,
         "e2e": {"value": job_throughput(world, n * nb, e2e_ms), "unit": "voxels/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(coords_h.numel() * 4 + feats_h.numel() * 4),
                 "d2h_bytes_per_step": int(out_h.numel() * 4), "steps": e_steps,
                 "how": "pipeline.FrameStream: per step one upload, one backbone pass, one download; copies of "
                        "neighbouring steps overlap the kernels, the next step's partition runs on its own stream "
-                       "under the current step's layer launches, consecutive steps dealt out to four compute "
-                       "streams; wall clock over all steps"},
+                       "under the current step's layer launch; wall clock over all steps"},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "fused DSVT layer", "bound": "tensor", "achieved": achieved,
-                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                     "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"], "peak_source": peaks["source"],
+        "roofline": {"kernel": layer_roof["kernel"], "bound": layer_roof["bound"], "achieved": achieved,
+                     "peak": layer_roof["peak"], "unit": "TFLOP/s", "frac": layer_roof["frac"],
+                     "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if bf16 else None,
+                     "peak_source": peaks["source"] if bf16 else layer_roof["peak_source"],
                      "flops_per_launch": flops_per_launch, "ms_per_launch": launch_ms,
-                     "layers_per_launch": 2 * nb,
+                     "layers_per_launch": 2 * nb if bf16 else 1,
                      "timing": "launch duration from the one-step-at-a-time run (a launch alone on the GPU)",
                      "achieved_in_pipeline": flops_per_launch / (ms_per_step * 1e-3) / 1e12,
-                     "traffic": LAYER_DRAM_BYTES_PER_LAUNCH if args.config == 2 else None},
+                     "traffic": measured_traffic(args.config), "kernel_revision": kernel_revision()},
+        "fp32_fma_peak_tflops": fma_peak,
+        "rooflines": rooflines,
+        "per_config": per_config,
         "cpu_baseline": cpu,
     }))
     if world > 1:
@@ -408,6 +658,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--per-config", type=int, nargs="*", default=[1, 3, 4, 5, 6, 7],
+                    help="configurations timed one frame at a time for the per_config list (none: skip)")
+    ap.add_argument("--lanes", type=int, default=2, help="compute streams of the frame pipeline")
+    ap.add_argument("--lane-ctas", type=int, default=0, help="CTAs per layer launch in the pipeline (0: automatic)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

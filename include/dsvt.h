@@ -329,6 +329,16 @@ int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feats, int32_t 
 int dsvt_bev_scatter(dsvt_ctx* ctx, const int32_t* coords, const float* feats, int32_t n, int32_t C, int32_t batch,
                      const int32_t grid[3], int32_t channels_last, float* out);
 
+/*
+ * A measurement aid (the paper has no counterpart): launches a kernel of `blocks` x `threads` threads that
+ * each run `iters` rounds of eight independent fp32 fused multiply-adds and nothing else, on the context's stream.
+ * A benchmark times it to learn the FP32 FMA rate of the device, which bounds the fp32 layer path (that path's
+ * arithmetic runs on the FMA pipes, not on the tensor cores).  *flops (HOST, optional) receives the number of
+ * floating-point operations of the launch (2 per multiply-add); sink is a device float the kernel may write.
+ * threads: a multiple of 32, at most 1024.
+ */
+int dsvt_fma_probe(dsvt_ctx* ctx, int32_t blocks, int32_t threads, int32_t iters, float* sink, int64_t* flops);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,7 @@ STATUS_BAD_COORD, STATUS_TABLE_OVERFLOW, STATUS_BAD_INDEX, STATUS_DUPLICATE_CELL
 EXPORTS = [
     "dsvt_create", "dsvt_destroy", "dsvt_status_sync", "dsvt_last_cuda_error", "dsvt_error_string",
     "dsvt_launch_count", "dsvt_set_layer_ctas", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_set_attention_rpb", "dsvt_layer", "dsvt_layers", "dsvt_block", "dsvt_pool",
-    "dsvt_bev_scatter",
+    "dsvt_bev_scatter", "dsvt_fma_probe",
 ]
 
 _lib = None
@@ -87,6 +87,7 @@ def load():
                                            C.c_int, vp]
     lib.dsvt_bev_scatter.argtypes = [vp, vp, vp, i32, i32, i32, p3, i32, vp]
     lib.dsvt_layer.argtypes = [vp, vp, i32, vp, i32, vp, vp, C.POINTER(LayerParams), vp]
+    lib.dsvt_fma_probe.argtypes = [vp, i32, i32, i32, vp, C.POINTER(i64)]
     lib.dsvt_layers.argtypes = [vp, vp, i32, i32, C.POINTER(TableRef), C.POINTER(LayerParams), vp]
     lib.dsvt_block.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, i32, vp, vp, C.POINTER(LayerParams), vp]
     lib.dsvt_pool.argtypes = [vp, vp, vp, i32, i32, i32, p3, p3, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32,
@@ -347,6 +348,14 @@ class Context:
                                  _ptr(t1.num_sets), _ptr(t1.set_rowoff), arr, _ptr(y))
         self._check(rc, "dsvt_block")
         return y
+
+    # ---- dsvt_fma_probe ----
+    def fma_probe(self, blocks: int, threads: int, iters: int, sink: torch.Tensor) -> int:
+        """Enqueues the FP32 FMA probe kernel; returns the floating-point operations of the launch."""
+        flops = C.c_int64(0)
+        rc = self.lib.dsvt_fma_probe(self._h, int(blocks), int(threads), int(iters), _ptr(sink), C.byref(flops))
+        self._check(rc, "dsvt_fma_probe")
+        return int(flops.value)
 
     # ---- dsvt_bev_scatter ----
     def bev_scatter(self, coords: torch.Tensor, feats: torch.Tensor, batch: int, grid, channels_last: bool = False,
