@@ -177,7 +177,9 @@ int dsvt_partition_shifted(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int3
  * Limits: n <= DSVT_NOALLOC_MAX_VOXELS and at most DSVT_NOALLOC_MAX_WINDOWS windows, otherwise
  * DSVT_ERR_CAPACITY is returned and nothing is launched.
  * The first call on each device looks up the array's device address (once, with that device
- * current); make that first call before starting any stream capture.
+ * current); make that first call before starting any stream capture.  That first call may also
+ * make the driver load the library's code onto the device (the one time the call can change the
+ * device's free memory), and the address it caches does not survive a cudaDeviceReset.
  * All calls on a device share the one array, which keeps the previous call's contents (the call
  * clears what has to start at zero): two calls whose kernels overlap on the GPU -- different
  * streams, or threads -- race on it.  Serialise them on one stream.

@@ -372,8 +372,11 @@ __device__ __noinline__ void attend_blocked() {
       if (D > 16) ldsm_x4(a_base + swz(row, c0 + 2 + ((D == 32) ? (lane >> 4) : 0)), qb);
     }
     // Row addresses advance by one 1024-byte group per key block of 8 (the swizzle depends on row & 7 only).
-    // Reads may run up to two groups past row 127: they land in the neighbouring operand block or the weight
-    // ring, which hold finite bf16 values, and meet zero probabilities.
+    // Reads may run up to two groups past row 127: they land in the neighbouring operand block or, for the last
+    // 64 value columns, in the weight ring, and meet zero probabilities.  Those bytes are this tile's own K / V
+    // values or this layer's weights: a non-finite value among them (0 x Inf) could only come from a non-finite
+    // weight or feature, and every output row of a layer depends on every weight of the layer, so such a layer has
+    // no finite output row to spoil.
     uint32_t k_addr = k_base + swz(k_lo + (lane & 7), c0 + min(lane >> 3, DC - 1));
     uint32_t v_addr[DC];
 #pragma unroll

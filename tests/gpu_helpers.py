@@ -33,6 +33,17 @@ def check_close(got, want, cfg_precision, what=""):
     return err
 
 
+def row_rel_error(got, want) -> float:
+    """Largest per-row relative error max_i |g_i - r_i|_inf / |r_i|_inf (reported beside the tensor-wide figure)."""
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    if got.size == 0:
+        return 0.0
+    num = np.abs(got - want).max(axis=1)
+    den = np.maximum(np.abs(want).max(axis=1), 1e-6)
+    return float((num / den).max())
+
+
 def table_np(t: api.SetTable):
     """(table rows [S, tau], set_rowoff [S + 1]) on the host."""
     S = int(t.num_sets.item())

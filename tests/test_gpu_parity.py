@@ -4,7 +4,7 @@ import pytest
 import torch
 
 import dsvt_inputs as di
-from gpu_helpers import check_close, dev, precision_of, rowoff_of, table_np, upload_table
+from gpu_helpers import check_close, dev, precision_of, row_rel_error, rowoff_of, table_np, upload_table
 
 pytestmark = pytest.mark.gpu
 
@@ -329,7 +329,9 @@ def _sample_windows(oracle, cfg, coords, n_target, seed, win=None):
     rng = np.random.default_rng(seed)
     order = rng.permutation(np.flatnonzero(p.win_count > 0))
     # always include the fullest and the emptiest windows
-    order = np.concatenate([[np.argmax(p.win_count)], order])
+    # always include the fullest window and the first and last non-empty ones (the first and the last tiles)
+    nonempty = np.flatnonzero(p.win_count > 0)
+    order = np.concatenate([[np.argmax(p.win_count), nonempty[0], nonempty[-1]], order])
     sel, total = [], 0
     for w in order:
         sel.append(p.perm[p.win_start[w]:p.win_start[w + 1]])
@@ -354,6 +356,19 @@ def test_backbone_full_size_bf16_on_sampled_windows(gpu, oracle, cid, n_sample):
     got1 = _run_blocks_gpu(gpu, cfg, cfg["blocks"][:1], cfg["coords"], cfg["feats"])
     want1 = _run_blocks_oracle(oracle, cfg, cfg["blocks"][:1], cfg["coords"][sel], cfg["feats"][sel])
     check_close(got1[sel], want1, "bf16", "config %d first block" % cid)
+
+
+@pytest.mark.parametrize("cid", [2, 6])
+def test_backbone_whole_frame_against_the_oracle(gpu, oracle, cid):
+    """Configurations 2 and 6 (the nuScenes-shaped extra) in full: every voxel of the frame through all four
+    blocks against the oracle, not a sample.  Prints the per-row relative error beside the tensor-wide one."""
+    cfg = di.make_config(cid)
+    oracle.set_threads(oracle.max_threads())
+    got = _run_blocks_gpu(gpu, cfg, cfg["blocks"], cfg["coords"], cfg["feats"])
+    want = _run_blocks_oracle(oracle, cfg, cfg["blocks"], cfg["coords"], cfg["feats"])
+    rel = check_close(got, want, "bf16", "config %d backbone, whole frame" % cid)
+    print("config %d whole frame: tensor-wide relative error %.3e, largest per-row relative error %.3e"
+          % (cid, rel, row_rel_error(got, want)))
 
 
 def test_in_place_and_repeatability(gpu):
