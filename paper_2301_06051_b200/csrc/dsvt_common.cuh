@@ -103,3 +103,20 @@ int dsvt_launch_layers_tc(dsvt_ctx* ctx, const dsvt_fused_args* layers, int n_la
 // CUtensorMap (128 bytes, 64-byte aligned) of a row-major bf16 matrix [rows][cols]: boxes of 64 columns x box_rows
 // rows, 128-byte swizzle; encoded once per matrix and context.  Returns false if the driver cannot encode it.
 bool dsvt_cached_weight_map(dsvt_ctx* ctx, void* tensor_map, const void* w, int rows, int cols, int box_rows);
+
+// Attention-style pooling with the projections on tcgen05 (pool_tc.cu): bfloat16 weights, C / head dim as for the
+// layer kernel, a power-of-two number of slots per region (at most 32).  The region bookkeeping (cell map, region
+// keys, output count) has been done by the caller.
+struct dsvt_pool_tc_call {
+  const float* feats;
+  const int32_t* cell_map;
+  const int32_t* region_key;
+  const int32_t* num_out;
+  int32_t cap_m, n;
+  const void* W[4];  // W_q, W_k, W_v, W_o
+  const float *b_q, *b_k, *b_v, *b_o, *slot_pe;
+  float* out_feats;
+  int32_t C, heads, nslots, mask_empty;
+};
+bool dsvt_pool_tc_supported(int C, int heads, int nslots);
+int dsvt_launch_pool_tc(dsvt_ctx* ctx, const dsvt_pool_tc_call& c);

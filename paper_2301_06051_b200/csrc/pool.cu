@@ -630,7 +630,17 @@ extern "C" int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feat
   a.W_q = W_q; a.W_k = W_k; a.W_v = W_v; a.W_o = W_o;
   a.b_q = b_q; a.b_k = b_k; a.b_v = b_v; a.b_o = b_o; a.slot_pe = slot_pe;
   a.out_feats = out_feats; a.C = C; a.heads = heads; a.nslots = (int32_t)nslots; a.mask_empty = mask_empty ? 1 : 0;
-  // bfloat16 weights, C in {64, 128, 192}, head dim <= 32: the tensor-core kernel
+  // bfloat16 weights, a power-of-two number of slots: the projections on tcgen05
+  if (precision == DSVT_BF16_FP32ACC && dsvt_pool_tc_supported(C, heads, (int)nslots)) {
+    dsvt_pool_tc_call c;
+    c.feats = feats; c.cell_map = ctx->cell_map; c.region_key = ctx->region_key; c.num_out = num_out;
+    c.cap_m = cap_m; c.n = n;
+    c.W[0] = W_q; c.W[1] = W_k; c.W[2] = W_v; c.W[3] = W_o;
+    c.b_q = b_q; c.b_k = b_k; c.b_v = b_v; c.b_o = b_o; c.slot_pe = slot_pe;
+    c.out_feats = out_feats; c.C = C; c.heads = heads; c.nslots = (int32_t)nslots; c.mask_empty = mask_empty ? 1 : 0;
+    return dsvt_launch_pool_tc(ctx, c);
+  }
+  // bfloat16 weights, C in {64, 128, 192}, head dim <= 32: other slot counts: the mma.sync kernel
   if (precision == DSVT_BF16_FP32ACC && (C == 64 || C == 128 || C == 192) && heads <= mma_pool::kMaxHeads) {
     a.TM = mma_pool::kRows;
     a.LDQ = 0;

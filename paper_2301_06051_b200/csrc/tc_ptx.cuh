@@ -106,11 +106,19 @@ __device__ __forceinline__ void tmem_st16_at(uint32_t taddr, const float (&v)[N]
         "f"(v[OFF + 12]), "f"(v[OFF + 13]), "f"(v[OFF + 14]), "f"(v[OFF + 15])
       : "memory");
 }
+template <int OFF, int N>
+__device__ __forceinline__ void tmem_ld8_at(uint32_t taddr, float (&r)[N]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=f"(r[OFF + 0]), "=f"(r[OFF + 1]), "=f"(r[OFF + 2]), "=f"(r[OFF + 3]), "=f"(r[OFF + 4]), "=f"(r[OFF + 5]),
+                 "=f"(r[OFF + 6]), "=f"(r[OFF + 7])
+               : "r"(taddr));
+}
 template <int N>
 __device__ __forceinline__ void tmem_ld_row(uint32_t taddr, float (&r)[N]) {
-  static_assert(N == 16 || N == 32 || N == 48, "column count per thread");
+  static_assert(N == 16 || N == 24 || N == 32 || N == 48, "column count per thread");
   tmem_ld16_at<0>(taddr, r);
-  if constexpr (N > 16) tmem_ld16_at<16>(taddr + 16, r);
+  if constexpr (N == 24) tmem_ld8_at<16>(taddr + 16, r);
+  if constexpr (N > 24) tmem_ld16_at<16>(taddr + 16, r);
   if constexpr (N > 32) tmem_ld16_at<32>(taddr + 32, r);
 }
 template <int N>
