@@ -40,7 +40,7 @@ def _peaks():
 
 
 TRAFFIC_FILE = os.path.join(ROOT, "profiles", "layer_tc_kernel_dram.json")
-KERNEL_SOURCES = ("layer_tc.cu", "dsvt_common.cuh")
+KERNEL_SOURCES = ("layer_tc.cu", "tc_ptx.cuh")
 
 
 def kernel_revision() -> str:

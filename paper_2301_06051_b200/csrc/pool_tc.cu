@@ -141,46 +141,72 @@ struct PoolTcArgs {
 };
 
 // ================= compute warps: gather + Eq. 6 ========================================================
-// One warp per region: its slot rows (four in flight), the channel-wise maximum, X~ rows and P rows as bf16.
+// Work item = (region, 16-byte channel chunk): the chunk of every slot row of the region (all loads of a thread's
+// items in flight together), the channel-wise maximum, X~ rows and P rows as bf16.
+template <int C, int NS>
+__device__ __forceinline__ void pool_gather_ns(const PoolTcArgs& a, unsigned char* xs, unsigned char* ps, int nr) {
+  constexpr int C4 = C / 4, TR = kTM / NS, ITEMS = TR * C4;
+  constexpr int PER = (ITEMS + kComputeThreads - 1) / kComputeThreads;  // items per thread
+  constexpr int GROUP = NS <= 4 ? NS : 4;                               // slot rows loaded together
+  static_assert(PER * GROUP <= 16, "loads in flight per thread");
+  const int tid = threadIdx.x;
+  float4 mx[PER];
+#pragma unroll
+  for (int j = 0; j < PER; ++j) mx[j] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+  for (int s0 = 0; s0 < NS; s0 += GROUP) {
+    float4 f[PER][GROUP];
+    int vv[PER][GROUP];
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const int i = tid + j * kComputeThreads, ri = i / C4, c4 = i - ri * C4;
+#pragma unroll
+      for (int u = 0; u < GROUP; ++u) {
+        vv[j][u] = (i < ITEMS && ri < nr) ? s_pm.rowvox[ri * NS + s0 + u] : -1;
+        f[j][u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (vv[j][u] >= 0) f[j][u] = __ldg(reinterpret_cast<const float4*>(a.feats + (size_t)vv[j][u] * C) + c4);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const int i = tid + j * kComputeThreads, ri = i / C4, c4 = i - ri * C4;
+      if (i >= ITEMS) continue;
+      const bool live = ri < nr;
+#pragma unroll
+      for (int u = 0; u < GROUP; ++u) {
+        const int s = s0 + u, r = ri * NS + s;
+        float4 g = f[j][u];
+        if (live && (!a.mask_empty || vv[j][u] >= 0)) {
+          mx[j].x = fmaxf(mx[j].x, g.x); mx[j].y = fmaxf(mx[j].y, g.y); mx[j].z = fmaxf(mx[j].z, g.z); mx[j].w = fmaxf(mx[j].w, g.w);
+        }
+        if (live && a.slot_pe) {
+          const float4 e = __ldg(reinterpret_cast<const float4*>(a.slot_pe + (size_t)s * C) + c4);
+          g.x += e.x; g.y += e.y; g.z += e.z; g.w += e.w;
+        }
+        *reinterpret_cast<uint2*>(xs + swz(r, c4 >> 1) + (c4 & 1) * 8) = make_uint2(pack_bf16(g.x, g.y), pack_bf16(g.z, g.w));
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int i = tid + j * kComputeThreads, ri = i / C4, c4 = i - ri * C4;
+    if (i >= ITEMS) continue;
+    const float4 m4 = ri < nr ? mx[j] : make_float4(0.f, 0.f, 0.f, 0.f);
+    const uint2 p2 = make_uint2(pack_bf16(m4.x, m4.y), pack_bf16(m4.z, m4.w));
+#pragma unroll
+    for (int s = 0; s < NS; ++s)  // the region's maximum, once per slot row
+      *reinterpret_cast<uint2*>(ps + swz(ri * NS + s, c4 >> 1) + (c4 & 1) * 8) = p2;
+  }
+}
+
 template <int C>
 __device__ __forceinline__ void pool_gather(const PoolTcArgs& a, unsigned char* xs, unsigned char* ps, int nr, int ns) {
-  constexpr int C4 = C / 4;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int TR = kTM / ns;
-  for (int ri = warp; ri < TR; ri += kComputeWarps) {
-    for (int c4 = lane; c4 < C4; c4 += 32) {
-      float4 mx = make_float4(0.f, 0.f, 0.f, 0.f);
-      const bool live = ri < nr;
-      if (live) mx = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-      for (int s0 = 0; s0 < ns; s0 += 4) {
-        float4 f[4];
-        int vv[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          vv[u] = (live && s0 + u < ns) ? s_pm.rowvox[ri * ns + s0 + u] : -1;
-          f[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (vv[u] >= 0) f[u] = __ldg(reinterpret_cast<const float4*>(a.feats + (size_t)vv[u] * C) + c4);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (s0 + u < ns) {
-            const int s = s0 + u, r = ri * ns + s;
-            if (live && (!a.mask_empty || vv[u] >= 0)) {
-              mx.x = fmaxf(mx.x, f[u].x); mx.y = fmaxf(mx.y, f[u].y); mx.z = fmaxf(mx.z, f[u].z); mx.w = fmaxf(mx.w, f[u].w);
-            }
-            if (live && a.slot_pe) {
-              const float4 e = __ldg(reinterpret_cast<const float4*>(a.slot_pe + (size_t)s * C) + c4);
-              f[u].x += e.x; f[u].y += e.y; f[u].z += e.z; f[u].w += e.w;
-            }
-            *reinterpret_cast<uint2*>(xs + swz(r, c4 >> 1) + (c4 & 1) * 8) =
-                make_uint2(pack_bf16(f[u].x, f[u].y), pack_bf16(f[u].z, f[u].w));
-          }
-        }
-      }
-      const uint2 p2 = make_uint2(pack_bf16(mx.x, mx.y), pack_bf16(mx.z, mx.w));
-      for (int s = 0; s < ns; ++s)  // the region's maximum, once per slot row
-        *reinterpret_cast<uint2*>(ps + swz(ri * ns + s, c4 >> 1) + (c4 & 1) * 8) = p2;
-    }
+  switch (ns) {
+    case 1: pool_gather_ns<C, 1>(a, xs, ps, nr); break;
+    case 2: pool_gather_ns<C, 2>(a, xs, ps, nr); break;
+    case 4: pool_gather_ns<C, 4>(a, xs, ps, nr); break;
+    case 8: pool_gather_ns<C, 8>(a, xs, ps, nr); break;
+    case 16: pool_gather_ns<C, 16>(a, xs, ps, nr); break;
+    default: pool_gather_ns<C, 32>(a, xs, ps, nr); break;
   }
 }
 
@@ -249,16 +275,22 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const __grid_const
       ++uses[bar];
       tc_fence_after();
     };
+    // tile row -> voxel through the region list and the dense cell map (looked up one tile ahead)
+    auto row_voxel = [&](int tl) {
+      const int t = blockIdx.x + tl * gridDim.x, r_lo = t * TR, nr = min(TR, m - r_lo);
+      int v = -1;
+      if (tl < my_tiles && tid < kTM && tid / ns < nr)
+        v = __ldg(a.cell_map + (size_t)__ldg(a.region_key + r_lo + tid / ns) * ns + (tid & (ns - 1)));
+      return v;
+    };
+    int v_next = row_voxel(0);
     for (int tl = 0; tl < my_tiles; ++tl) {
       const int t = blockIdx.x + tl * gridDim.x;
       const int r_lo = t * TR, nr = min(TR, m - r_lo);
       compute_sync();  // the previous tile's staging rows have been stored; its operands are dead
-      if (tid < kTM) {
-        int v = -1;
-        if (tid / ns < nr) v = a.cell_map[(size_t)a.region_key[r_lo + tid / ns] * ns + (tid & (ns - 1))];
-        s_pm.rowvox[tid] = v;
-      }
+      if (tid < kTM) s_pm.rowvox[tid] = v_next;
       compute_sync();
+      v_next = row_voxel(tl + 1);
       pool_gather<C>(a, xs, ps, nr, ns);
       fence_proxy_async();
       mbar_arrive(&s_pm.ab_ready);
@@ -276,9 +308,13 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const __grid_const
         tmem_wait_ld();
         float acc = 0.f;
 #pragma unroll
-        for (int c = 0; c < D; ++c) {
+        for (int c = 0; c < D; c += 4) {
           const int cc = hq * QC + j * D + c;
-          acc = fmaf(q[c] + par[cc], k[c] + par[C + cc], acc);
+          const float4 bq = *reinterpret_cast<const float4*>(par + cc), bk = *reinterpret_cast<const float4*>(par + C + cc);
+          acc = fmaf(q[c] + bq.x, k[c] + bk.x, acc);
+          acc = fmaf(q[c + 1] + bq.y, k[c + 1] + bk.y, acc);
+          acc = fmaf(q[c + 2] + bq.z, k[c + 2] + bk.z, acc);
+          acc = fmaf(q[c + 3] + bq.w, k[c + 3] + bk.w, acc);
         }
         const float lg = key_ok ? acc * scale : -INFINITY;
         float mx = lg;
@@ -300,10 +336,16 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const __grid_const
         tc_fence_before();
         mbar_arrive(&s_pm.acc_free[0]);
 #pragma unroll
-        for (int cc = 0; cc < QC; ++cc) {
-          float t2 = p[cc / D] * v[cc];
-          for (int o = ns >> 1; o > 0; o >>= 1) t2 += __shfl_xor_sync(0xffffffffu, t2, o);
-          v[cc] = live ? t2 + par[2 * C + hq * QC + cc] : 0.f;  // the probabilities sum to one: + b_v once
+        for (int c4 = 0; c4 < QC; c4 += 4) {
+          const float4 bv = *reinterpret_cast<const float4*>(par + 2 * C + hq * QC + c4);
+          const float b4[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int cc = c4 + e;
+            float t2 = p[cc / D] * v[cc];
+            for (int o = ns >> 1; o > 0; o >>= 1) t2 += __shfl_xor_sync(0xffffffffu, t2, o);
+            v[cc] = live ? t2 + b4[e] : 0.f;  // the probabilities sum to one: + b_v once
+          }
         }
 #pragma unroll
         for (int q8 = 0; q8 < QC / 8; ++q8)
@@ -323,10 +365,11 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const __grid_const
         mbar_arrive(&s_pm.acc_free[1]);
         if (live && s_of == 0) {  // (X~ is dead: the value projection has been read)
 #pragma unroll
-          for (int q4 = 0; q4 < QC / 4; ++q4)
+          for (int q4 = 0; q4 < QC / 4; ++q4) {
+            const float4 bo = *reinterpret_cast<const float4*>(par + 3 * C + hq * QC + 4 * q4);
             *reinterpret_cast<float4*>(xs + out_off<C>(ri, hq * (QC / 4) + q4)) =
-                make_float4(o[4 * q4] + par[3 * C + hq * QC + 4 * q4], o[4 * q4 + 1] + par[3 * C + hq * QC + 4 * q4 + 1],
-                            o[4 * q4 + 2] + par[3 * C + hq * QC + 4 * q4 + 2], o[4 * q4 + 3] + par[3 * C + hq * QC + 4 * q4 + 3]);
+                make_float4(o[4 * q4] + bo.x, o[4 * q4 + 1] + bo.y, o[4 * q4 + 2] + bo.z, o[4 * q4 + 3] + bo.w);
+          }
         }
       }
       compute_sync();
