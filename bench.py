@@ -279,7 +279,7 @@ def time_config(cid: int, dev, reps: int, flush):
                     "t_block_ms": [med["s%d_blocks" % i] / len(st["blocks"]) for i, st in enumerate(cfg["stages"])],
                     "t_pool_ms": [med["s%d_pool" % i] for i in range(len(cfg["pools"]))],
                     "t_backbone_ms": med["backbone"], "frames_per_s": cfg["batch"] / (med["backbone"] * 1e-3),
-                    "note": "the pooled voxel count is read back on the host between stages (inside t_backbone_ms)"})
+                    "note": "no host read-back between the stages: the pooled voxel counts stay on the device"})
         return out, None
     bb = pipeline.Backbone(cfg, device=dev.index)
     y = torch.empty_like(x)
@@ -296,17 +296,18 @@ def time_config(cid: int, dev, reps: int, flush):
         if bb.stage2:
             oc, of, num, _, _ = bb.ctx.pool(coords, y, cfg["batch"], cfg["grid"], bb.pool_shape, bb.pool_w)
             r["t3"] = ev()
-            m = int(num.item())  # the pooled voxel count sizes the second stage's tensors (a host read-back)
-            r["t4"] = ev()
-            bb.stage2.partition(oc[:m])
+            r["t4"] = r["t3"]  # (no read-back: the second stage reads the pooled voxel count on the device)
+            bb.stage2.partition(oc, n_dev=num)
             r["t5"] = ev()
-            bb.stage2.run_blocks(oc[:m], of[:m], of[:m])
+            bb.stage2.run_blocks(oc, of, of)
             r["t6"] = ev()
         recs.append(r)
     torch.cuda.synchronize(dev)
     if bb.ctx.status_sync() != 0:
         raise SystemExit("device status word is not clean (config %d)" % cid)
     recs = recs[2:]
+    if bb.stage2:
+        m = int(num.item())
     span = lambda a, b: _median_ms([(r[a], r[b]) for r in recs])
     hidden = int(cfg["blocks"][0][0].get("hidden", 0))
     S, pad, fl0 = table_stats(st1.tables[0], cfg["set_size"], C, hidden)
@@ -325,7 +326,7 @@ def time_config(cid: int, dev, reps: int, flush):
         ns = int(np.prod(bb.pool_shape))
         out.update({"t_pool_ms": span("t2", "t3"), "pooled_voxels": m, "t_partition2_ms": span("t4", "t5"),
                     "t_block2_ms": span("t5", "t6") / nb2,
-                    "note": "the pooled voxel count is read back on the host between the stages (inside t_backbone_ms)"})
+                    "note": "no host read-back between the stages: the pooled voxel count stays on the device"})
         extra.update({"pool": {"t_ms": out["t_pool_ms"], "bytes": 4.0 * C * (n + m) + 16.0 * (n + m), "n": n, "m": m,
                                "slots": ns}})
     return out, extra

@@ -157,6 +157,21 @@ int dsvt_partition_shifted(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int3
                            int32_t* win_count, int32_t* win_setoff);
 
 /*
+ * dsvt_partition_shifted for a frame whose voxel count lives on the device (Sec. 3.2 and Sec. 3.3: the stage after
+ * an attention-style pooling partitions the pooled voxels, whose number the pooling has just written to device
+ * memory).  The call takes the first min(n, *n_dev) voxels of coords; n is the capacity the launches are sized by.
+ * n_dev NULL gives dsvt_partition_shifted exactly.  Everything downstream (num_sets, the tables, the row offsets
+ * whose last entry is the voxel count) follows the device count, so dsvt_layers / dsvt_block can run on the tables
+ * with n = the capacity and no host read-back in between.  Needs the bitmap route (key space within 64 Mi keys);
+ * otherwise DSVT_ERR_UNSUPPORTED.
+ */
+int dsvt_partition_counted(dsvt_ctx* ctx, const int32_t* coords, int32_t n, const int32_t* n_dev, int32_t batch,
+                           const int32_t grid[3], const int32_t window[3], const int32_t shift[3], int32_t set_size,
+                           int32_t* const set_table[2], int32_t cap_sets, int32_t* const num_sets[2],
+                           int32_t* const set_rowoff[2], int32_t* const perm[2], int32_t* win_start,
+                           int32_t* win_count, int32_t* win_setoff);
+
+/*
  * dsvt_partition without any allocation.  (The paper has no counterpart: this is a deployment
  * variant of dsvt_partition, computing exactly the same table.)
  *
@@ -312,6 +327,18 @@ int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feats, int32_t 
               const void* W_o, const float* b_q, const float* b_k, const float* b_v, const float* b_o,
               const float* slot_pe, int32_t heads, int32_t mask_empty, int precision, int32_t* out_coords,
               float* out_feats, int32_t cap_m, int32_t* num_out, int32_t* region_of, int32_t* slot_of);
+
+/*
+ * dsvt_pool for an input whose voxel count lives on the device (the second and later poolings of a backbone with
+ * several pooled stages, Appendix B.1.1): the first min(n, *n_dev) voxels are pooled; n is the capacity.  n_dev
+ * NULL gives dsvt_pool exactly.
+ */
+int dsvt_pool_counted(dsvt_ctx* ctx, const int32_t* coords, const float* feats, int32_t n, const int32_t* n_dev,
+                      int32_t C, int32_t batch, const int32_t grid[3], const int32_t pool[3], const void* W_q,
+                      const void* W_k, const void* W_v, const void* W_o, const float* b_q, const float* b_k,
+                      const float* b_v, const float* b_o, const float* slot_pe, int32_t heads, int32_t mask_empty,
+                      int precision, int32_t* out_coords, float* out_feats, int32_t cap_m, int32_t* num_out,
+                      int32_t* region_of, int32_t* slot_of);
 
 /*
  * Projection of the backbone's voxel features to a dense bird's-eye-view map (Sec. 3.1).  The z

@@ -23,7 +23,7 @@ STATUS_BAD_COORD, STATUS_TABLE_OVERFLOW, STATUS_BAD_INDEX, STATUS_DUPLICATE_CELL
 
 EXPORTS = [
     "dsvt_create", "dsvt_destroy", "dsvt_status_sync", "dsvt_last_cuda_error", "dsvt_error_string",
-    "dsvt_launch_count", "dsvt_set_layer_ctas", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_set_attention_rpb", "dsvt_layer", "dsvt_layers", "dsvt_block", "dsvt_pool",
+    "dsvt_launch_count", "dsvt_set_layer_ctas", "dsvt_partition", "dsvt_partition_rotated", "dsvt_partition_shifted", "dsvt_partition_counted", "dsvt_pool_counted", "dsvt_partition_noalloc", "dsvt_set_attention", "dsvt_set_attention_rpb", "dsvt_layer", "dsvt_layers", "dsvt_block", "dsvt_pool",
     "dsvt_bev_scatter", "dsvt_fma_probe",
 ]
 
@@ -81,6 +81,9 @@ def load():
     lib.dsvt_partition.argtypes = [vp, vp, i32, i32, p3, p3, i32, i32, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.dsvt_partition_rotated.argtypes = [vp, vp, i32, i32, p3, p3, i32, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.dsvt_partition_shifted.argtypes = [vp, vp, i32, i32, p3, p3, p3, i32, vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.dsvt_partition_counted.argtypes = [vp, vp, i32, vp, i32, p3, p3, p3, i32, vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.dsvt_pool_counted.argtypes = [vp, vp, vp, i32, vp, i32, i32, p3, p3, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32,
+                                      i32, C.c_int, vp, vp, i32, vp, vp, vp]
     lib.dsvt_partition_noalloc.argtypes = [vp, vp, i32, i32, p3, p3, i32, i32, vp, i32, vp, vp, vp, C.POINTER(i32)]
     lib.dsvt_set_attention.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, i32, vp, vp, vp, vp, i32, vp, C.c_int, vp]
     lib.dsvt_set_attention_rpb.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, p3,
@@ -266,9 +269,10 @@ class Context:
 
     # ---- dsvt_partition_rotated ----
     def partition_rotated(self, coords: torch.Tensor, batch: int, grid, window, set_size: int,
-                          cap_sets: Optional[int] = None, out=None, shift=None):
+                          cap_sets: Optional[int] = None, out=None, shift=None, n_dev: Optional[torch.Tensor] = None):
         """Both sort axes in one call; returns (X-axis SetTable, Y-axis SetTable).  `shift` displaces the window
-        cut (dsvt_partition_shifted); None calls dsvt_partition_rotated."""
+        cut (dsvt_partition_shifted); None calls dsvt_partition_rotated.  `n_dev` (device int32) gives the voxel
+        count where it lives on the device (dsvt_partition_counted); coords' length is then the capacity."""
         n = int(coords.shape[0])
         if out is None:
             cap = int(cap_sets) if cap_sets is not None else max(n, 1)
@@ -283,7 +287,11 @@ class Context:
         tail = (int(set_size), pair(t0.set_table, t1.set_table), t0.cap_sets, pair(t0.num_sets, t1.num_sets),
                 pair(t0.set_rowoff, t1.set_rowoff), pair(t0.perm, t1.perm), _ptr(t0.win_start), _ptr(t0.win_count),
                 _ptr(t0.win_setoff))
-        if shift is None:
+        if n_dev is not None:
+            rc = self.lib.dsvt_partition_counted(self._h, _ptr(coords), n, _ptr(n_dev), int(batch), _i3(grid),
+                                                 _i3(window), None if shift is None else _i3(shift), *tail)
+            self._check(rc, "dsvt_partition_counted")
+        elif shift is None:
             rc = self.lib.dsvt_partition_rotated(self._h, _ptr(coords), n, int(batch), _i3(grid), _i3(window), *tail)
             self._check(rc, "dsvt_partition_rotated")
         else:
@@ -374,8 +382,10 @@ class Context:
 
     # ---- dsvt_pool ----
     def pool(self, coords: torch.Tensor, feats: torch.Tensor, batch: int, grid, pool_shape, w: Dict,
-             mask_empty: int = 0, cap_m: Optional[int] = None, extras: bool = False):
-        """Returns (out_coords [cap_m,4], out_feats [cap_m,C], num_out [1], region_of, slot_of)."""
+             mask_empty: int = 0, cap_m: Optional[int] = None, extras: bool = False,
+             n_dev: Optional[torch.Tensor] = None):
+        """Returns (out_coords [cap_m,4], out_feats [cap_m,C], num_out [1], region_of, slot_of).  `n_dev` (device
+        int32): the input's voxel count where it lives on the device (dsvt_pool_counted)."""
         n, Cc = int(feats.shape[0]), int(feats.shape[1])
         cap = int(cap_m) if cap_m is not None else max(n, 1)
         dev = self.device
@@ -384,10 +394,14 @@ class Context:
         num = torch.zeros(1, dtype=torch.int32, device=dev)
         reg = torch.empty(max(n, 1), dtype=torch.int32, device=dev) if extras else None
         slot = torch.empty(max(n, 1), dtype=torch.int32, device=dev) if extras else None
-        rc = self.lib.dsvt_pool(self._h, _ptr(coords), _ptr(feats), n, Cc, int(batch), _i3(grid), _i3(pool_shape),
-                                _ptr(w["W_q"]), _ptr(w["W_k"]), _ptr(w["W_v"]), _ptr(w["W_o"]), _ptr(w.get("b_q")),
-                                _ptr(w.get("b_k")), _ptr(w.get("b_v")), _ptr(w.get("b_o")), _ptr(w.get("slot_pe")),
-                                int(w["heads"]), int(mask_empty), int(w["precision"]), _ptr(oc), _ptr(of), cap,
-                                _ptr(num), _ptr(reg), _ptr(slot))
-        self._check(rc, "dsvt_pool")
+        tail = (Cc, int(batch), _i3(grid), _i3(pool_shape), _ptr(w["W_q"]), _ptr(w["W_k"]), _ptr(w["W_v"]),
+                _ptr(w["W_o"]), _ptr(w.get("b_q")), _ptr(w.get("b_k")), _ptr(w.get("b_v")), _ptr(w.get("b_o")),
+                _ptr(w.get("slot_pe")), int(w["heads"]), int(mask_empty), int(w["precision"]), _ptr(oc), _ptr(of), cap,
+                _ptr(num), _ptr(reg), _ptr(slot))
+        if n_dev is not None:
+            rc = self.lib.dsvt_pool_counted(self._h, _ptr(coords), _ptr(feats), n, _ptr(n_dev), *tail)
+            self._check(rc, "dsvt_pool_counted")
+        else:
+            rc = self.lib.dsvt_pool(self._h, _ptr(coords), _ptr(feats), n, *tail)
+            self._check(rc, "dsvt_pool")
         return oc, of, num, reg, slot

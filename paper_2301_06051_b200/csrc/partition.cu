@@ -434,11 +434,13 @@ struct BmJob {
   int32_t naxes;
 };
 
-__global__ void bm_mark_kernel(const int4* __restrict__ coords, int32_t n, PartGeom g, uint32_t Vp, BmJob job,
+__global__ void bm_mark_kernel(const int4* __restrict__ coords, int32_t n_max, const int32_t* __restrict__ n_dev,
+                               PartGeom g, uint32_t Vp, BmJob job,
                                int32_t* __restrict__ win_count, int32_t* __restrict__ dup_count,
                                int32_t* __restrict__ dup, int32_t* __restrict__ status) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // (the scan kernel may be set up meanwhile)
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n = n_dev ? min(max(*n_dev, 0), n_max) : n_max;  // (a count that lives on the device)
   if (i >= n) return;
   int4 c = coords[i];  // (b, x, y, z)
   const bool bad =
@@ -544,7 +546,8 @@ struct FillOut {
   int32_t* perm[2];   // optional: voxel ids in sorted order
   int32_t* rowoff[2]; // optional: offsets are read, the plan is written
 };
-__global__ void __launch_bounds__(kScanThreads) bm_place_fill_kernel(int32_t n, BmJob job, int32_t wpw,
+__global__ void __launch_bounds__(kScanThreads) bm_place_fill_kernel(int32_t n_max, const int32_t* __restrict__ n_dev,
+                                                                     BmJob job, int32_t wpw,
                                                             const int32_t* __restrict__ dup,
                                                             const int32_t* __restrict__ win_count,
                                                             const int32_t* __restrict__ win_start,
@@ -561,6 +564,7 @@ __global__ void __launch_bounds__(kScanThreads) bm_place_fill_kernel(int32_t n, 
     return;
   }
   const int i = (blockIdx.x - 1) * blockDim.x + threadIdx.x;
+  const int n = n_dev ? min(max(*n_dev, 0), n_max) : n_max;
   if (i >= n) return;
   const int ticket = dup[i];
 #pragma unroll
@@ -679,6 +683,7 @@ struct PartOut {  // device outputs of one sort axis
 
 struct PartCall {
   const int32_t* coords;
+  const int32_t* n_dev;  // optional device count: the call takes min(n, *n_dev) voxels
   int32_t n, set_size, cap_sets, nw;
   PartGeom g;
   uint64_t V;
@@ -708,7 +713,7 @@ int validate(dsvt_ctx* ctx, const int32_t* coords, int32_t n, int32_t batch, con
   if (V >= (1ull << 31) || num_windows >= (1ull << 31) || num_windows * V > 0xFFFFFFFFull) return DSVT_ERR_UNSUPPORTED;
   g.V = (uint32_t)V;
   if (n > ctx->max_voxels || (int64_t)num_windows > ctx->max_windows) return DSVT_ERR_CAPACITY;
-  pc->coords = coords; pc->n = n; pc->set_size = set_size; pc->cap_sets = cap_sets;
+  pc->coords = coords; pc->n_dev = nullptr; pc->n = n; pc->set_size = set_size; pc->cap_sets = cap_sets;
   pc->nw = (int32_t)num_windows;
   pc->V = V;
   return DSVT_OK;
@@ -813,7 +818,7 @@ int partition_bitmap(dsvt_ctx* ctx, const PartCall& pc, int32_t wpw, int naxes, 
     job.ax[a].axis = o[b].axis;
   }
   const unsigned vox_blocks = (unsigned)dsvt_ceil_div(n, 256);
-  bm_mark_kernel<<<vox_blocks, 256, 0, st>>>((const int4*)pc.coords, n, pc.g, (uint32_t)wpw * 32u, job, counts,
+  bm_mark_kernel<<<vox_blocks, 256, 0, st>>>((const int4*)pc.coords, n, pc.n_dev, pc.g, (uint32_t)wpw * 32u, job, counts,
                                              dup_count, ctx->bm_dup, ctx->status);
   DSVT_LAUNCHED(ctx);
   int64_t rank_blocks = dsvt_ceil_div((int64_t)naxes * nw, kScanThreads / 32);
@@ -842,7 +847,7 @@ int partition_bitmap(dsvt_ctx* ctx, const PartCall& pc, int32_t wpw, int naxes, 
     fo.rowoff[a] = on ? o[a].set_rowoff : nullptr;
   }
   const unsigned fill_blocks = (unsigned)dsvt_ceil_div(n, kScanThreads);
-  DSVT_CUDA_TRY(ctx, launch_pdl(bm_place_fill_kernel, dim3(fill_blocks + 1), dim3(kScanThreads), smem, st, n, job, wpw,
+  DSVT_CUDA_TRY(ctx, launch_pdl(bm_place_fill_kernel, dim3(fill_blocks + 1), dim3(kScanThreads), smem, st, n, pc.n_dev, job, wpw,
                                 (const int32_t*)ctx->bm_dup, (const int32_t*)counts, (const int32_t*)ctx->win_start,
                                 (const int32_t*)ctx->win_setoff, pc.set_size, pc.cap_sets,
                                 (const int32_t*)o[0].num_sets, fo, smax));
@@ -883,10 +888,21 @@ extern "C" int dsvt_partition_shifted(dsvt_ctx* ctx, const int32_t* coords, int3
                                       int32_t* const num_sets[2], int32_t* const set_rowoff[2],
                                       int32_t* const perm[2], int32_t* win_start, int32_t* win_count,
                                       int32_t* win_setoff) {
+  return dsvt_partition_counted(ctx, coords, n, nullptr, batch, grid, window, shift, set_size, set_table, cap_sets,
+                                num_sets, set_rowoff, perm, win_start, win_count, win_setoff);
+}
+
+extern "C" int dsvt_partition_counted(dsvt_ctx* ctx, const int32_t* coords, int32_t n, const int32_t* n_dev,
+                                      int32_t batch, const int32_t grid[3], const int32_t window[3],
+                                      const int32_t shift[3], int32_t set_size, int32_t* const set_table[2],
+                                      int32_t cap_sets, int32_t* const num_sets[2], int32_t* const set_rowoff[2],
+                                      int32_t* const perm[2], int32_t* win_start, int32_t* win_count,
+                                      int32_t* win_setoff) {
   if (!set_table || !num_sets || !num_sets[0] || !num_sets[1]) return DSVT_ERR_INVALID_ARG;
   PartCall pc;
   int rc = validate(ctx, coords, n, batch, grid, window, shift, set_size, cap_sets, &pc);
   if (rc != DSVT_OK) return rc;
+  pc.n_dev = n_dev;
   if (n > 0 && (!set_table[0] || !set_table[1])) return DSVT_ERR_INVALID_ARG;
   pc.win_start = win_start; pc.win_count = win_count; pc.win_setoff = win_setoff;
   PartOut o[2];
@@ -894,6 +910,7 @@ extern "C" int dsvt_partition_shifted(dsvt_ctx* ctx, const int32_t* coords, int3
     o[a] = PartOut{a, set_table[a], num_sets[a], set_rowoff ? set_rowoff[a] : nullptr, perm ? perm[a] : nullptr};
   const int32_t wpw = bitmap_words_per_window(ctx, pc);
   if (wpw > 0) return partition_bitmap(ctx, pc, wpw, 2, o);
+  if (n_dev && n > 0 && cap_sets > 0) return DSVT_ERR_UNSUPPORTED;  // (the sorting route wants the count on the host)
   rc = partition_sorted(ctx, pc, o[0]);
   if (rc != DSVT_OK) return rc;
   return partition_sorted(ctx, pc, o[1]);

@@ -27,10 +27,12 @@ __device__ __forceinline__ int4 clamp_coord(int4 c, const PoolGeom& g, int32_t* 
 }
 
 // Each voxel claims its cell of the dense (region, slot) map and marks its region as non-empty.
-__global__ void pool_mark_kernel(const int4* __restrict__ coords, int32_t n, PoolGeom g, int32_t* __restrict__ cell_map,
+__global__ void pool_mark_kernel(const int4* __restrict__ coords, int32_t n_max, const int32_t* __restrict__ n_dev,
+                                 PoolGeom g, int32_t* __restrict__ cell_map,
                                  int32_t* __restrict__ region_flag, uint32_t* __restrict__ vox_region,
                                  int32_t* __restrict__ slot_of, int32_t* __restrict__ status) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n = n_dev ? min(max(*n_dev, 0), n_max) : n_max;  // (a count that lives on the device)
   if (i >= n) return;
   const int4 c = clamp_coord(coords[i], g, status);
   const int X = c.y / g.l, Y = c.z / g.w, Z = c.w / g.h;
@@ -44,7 +46,8 @@ __global__ void pool_mark_kernel(const int4* __restrict__ coords, int32_t n, Poo
 }
 
 // region rank -> output row: coordinates, region id per output row, region_of per voxel.
-__global__ void pool_finish_kernel(int32_t n, PoolGeom g, const uint32_t* __restrict__ vox_region,
+__global__ void pool_finish_kernel(int32_t n_max, const int32_t* __restrict__ n_dev, PoolGeom g,
+                                   const uint32_t* __restrict__ vox_region,
                                    const int32_t* __restrict__ region_rank, int32_t num_regions, int32_t cap_m,
                                    int32_t* __restrict__ out_coords, int32_t* __restrict__ region_key,
                                    int32_t* __restrict__ region_of, int32_t* __restrict__ num_out,
@@ -55,6 +58,7 @@ __global__ void pool_finish_kernel(int32_t n, PoolGeom g, const uint32_t* __rest
     if (m > cap_m) atomicOr(status, DSVT_STATUS_TABLE_OVERFLOW);
     *num_out = min(m, cap_m);
   }
+  const int n = n_dev ? min(max(*n_dev, 0), n_max) : n_max;
   if (i >= n) return;
   const uint32_t region = vox_region[i];
   const int r = region_rank[region];
@@ -575,6 +579,18 @@ extern "C" int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feat
                          const float* b_o, const float* slot_pe, int32_t heads, int32_t mask_empty, int precision,
                          int32_t* out_coords, float* out_feats, int32_t cap_m, int32_t* num_out, int32_t* region_of,
                          int32_t* slot_of) {
+  return dsvt_pool_counted(ctx, coords, feats, n, nullptr, C, batch, grid, pool, W_q, W_k, W_v, W_o, b_q, b_k, b_v, b_o,
+                           slot_pe, heads, mask_empty, precision, out_coords, out_feats, cap_m, num_out, region_of,
+                           slot_of);
+}
+
+extern "C" int dsvt_pool_counted(dsvt_ctx* ctx, const int32_t* coords, const float* feats, int32_t n,
+                                 const int32_t* n_dev, int32_t C, int32_t batch, const int32_t grid[3],
+                                 const int32_t pool[3], const void* W_q, const void* W_k, const void* W_v,
+                                 const void* W_o, const float* b_q, const float* b_k, const float* b_v,
+                                 const float* b_o, const float* slot_pe, int32_t heads, int32_t mask_empty,
+                                 int precision, int32_t* out_coords, float* out_feats, int32_t cap_m,
+                                 int32_t* num_out, int32_t* region_of, int32_t* slot_of) {
   if (!ctx || !grid || !pool || !num_out || n < 0 || batch < 1 || cap_m < 0 || C < 1 || heads < 1)
     return DSVT_ERR_INVALID_ARG;
   if (precision != DSVT_FP32 && precision != DSVT_BF16_FP32ACC) return DSVT_ERR_INVALID_ARG;
@@ -614,12 +630,12 @@ extern "C" int dsvt_pool(dsvt_ctx* ctx, const int32_t* coords, const float* feat
   DSVT_CUDA_TRY(ctx, cudaMemsetAsync(ctx->cell_map, 0xFF, cells * sizeof(int32_t), st));
   DSVT_CUDA_TRY(ctx, cudaMemsetAsync(ctx->win_count, 0, sizeof(int32_t) * (size_t)(num_regions + 1), st));
   const unsigned vb = (unsigned)dsvt_ceil_div(n, 256);
-  pool_mark_kernel<<<vb, 256, 0, st>>>((const int4*)coords, n, g, ctx->cell_map, ctx->win_count, ctx->keys[0], slot_of,
+  pool_mark_kernel<<<vb, 256, 0, st>>>((const int4*)coords, n, n_dev, g, ctx->cell_map, ctx->win_count, ctx->keys[0], slot_of,
                                        ctx->status);
   DSVT_LAUNCHED(ctx);
   int rc = dsvt_launch_scan_i32(ctx, ctx->win_count, ctx->win_start, num_regions, nullptr);
   if (rc != DSVT_OK) return rc;
-  pool_finish_kernel<<<vb, 256, 0, st>>>(n, g, ctx->keys[0], ctx->win_start, (int32_t)num_regions, cap_m, out_coords,
+  pool_finish_kernel<<<vb, 256, 0, st>>>(n, n_dev, g, ctx->keys[0], ctx->win_start, (int32_t)num_regions, cap_m, out_coords,
                                          ctx->region_key, region_of, num_out, ctx->status);
   DSVT_LAUNCHED(ctx);
   if (cap_m == 0) return DSVT_OK;

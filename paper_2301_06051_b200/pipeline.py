@@ -48,11 +48,14 @@ class Stage:
                 out[sp] = self._new_tables()
         return out
 
-    def partition(self, coords: torch.Tensor, ctx: Optional[api.Context] = None, tables_of: Optional[Dict] = None):
-        """Fills the stage's tables, or those of another table set, through the stage's context or another one."""
+    def partition(self, coords: torch.Tensor, ctx: Optional[api.Context] = None, tables_of: Optional[Dict] = None,
+                  n_dev: Optional[torch.Tensor] = None):
+        """Fills the stage's tables, or those of another table set, through the stage's context or another one.
+        `n_dev`: the voxel count as a device int32 (coords then has the stage's capacity)."""
         ctx = self.ctx if ctx is None else ctx
         for (window, shift), tables in (self.tables_of if tables_of is None else tables_of).items():
-            ctx.partition_rotated(coords, self.batch, self.grid, window, self.set_size, out=tuple(tables), shift=shift)
+            ctx.partition_rotated(coords, self.batch, self.grid, window, self.set_size, out=tuple(tables), shift=shift,
+                                  n_dev=n_dev)
 
     def run_blocks(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor,
                    tables_of: Optional[Dict] = None, ctx: Optional[api.Context] = None) -> torch.Tensor:
@@ -252,17 +255,26 @@ class Backbone:
             self.stage2 = Stage(self.ctx, cfg["blocks_after_pool"], cfg["batch"], self.pooled_grid, window,
                                 cfg["set_size"], self.precision, n)
 
-    def forward(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor):
-        """Returns (coords_out, feats_out, num_out); for a single stage these are (coords, y, None)."""
+    def forward_async(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor):
+        """Enqueues the whole pass without a host read-back: the pooled voxel count stays on the device, the second
+        stage's calls are sized by the capacity and read the count there.  Returns (coords_out, feats_out, num_out)
+        at full capacity (rows past *num_out are not written); for a single stage (coords, y, None)."""
         self.stage1.forward(coords, x, y)
         if not self.stage2:
             return coords, y, None
         oc, of, num, _, _ = self.ctx.pool(coords, y, self.cfg["batch"], self.cfg["grid"], self.pool_shape, self.pool_w)
-        # the pooled voxel count lives on the device; the second stage needs it as a tensor extent
-        m = int(num.item())
-        oc, of = oc[:m], of[:m]
-        self.stage2.forward(oc, of, of)
+        self.stage2.partition(oc, n_dev=num)
+        self.stage2.run_blocks(oc, of, of)
         return oc, of, num
+
+    def forward(self, coords: torch.Tensor, x: torch.Tensor, y: torch.Tensor):
+        """Returns (coords_out, feats_out, num_out) cut to the pooled voxel count (one read-back, after everything
+        has been enqueued); for a single stage these are (coords, y, None)."""
+        oc, of, num = self.forward_async(coords, x, y)
+        if num is None:
+            return oc, of, None
+        m = int(num.item())
+        return oc[:m], of[:m], num
 
 
 class StagedBackbone:
@@ -291,24 +303,23 @@ class StagedBackbone:
 
     def forward(self, coords: torch.Tensor, x: torch.Tensor, on_step=None):
         """Returns (coords, feats) of the last stage.  on_step(tag), if given, is called after every call group."""
-        feats = x
+        feats, num = x, None  # num: the current stage's voxel count on the device (None: all of coords)
         for i, stage in enumerate(self.stages):
             y = torch.empty_like(feats)
-            stage.partition(coords)
+            stage.partition(coords, n_dev=num)
             if on_step:
                 on_step("s%d_partition" % i)
-            src = feats
-            for blk in stage.blocks:
-                self.ctx.block(src, stage.tables[0], stage.tables[1], blk, y, coords=coords)
-                src = y
+            stage.run_blocks(coords, feats, y)
             if on_step:
                 on_step("s%d_blocks" % i)
             feats = y
             if i < len(self.pool_w):
-                oc, of, num, _, _ = self.ctx.pool(coords, feats, self.cfg["batch"], self.grids[i],
-                                                  self.cfg["pools"][i]["shape"], self.pool_w[i])
-                m = int(num.item())  # the pooled voxel count sizes the next stage's tensors
-                coords, feats = oc[:m], of[:m]
+                # (no read-back: the next stage is sized by the capacity and reads the pooled count on the device)
+                coords, feats, num, _, _ = self.ctx.pool(coords, feats, self.cfg["batch"], self.grids[i],
+                                                         self.cfg["pools"][i]["shape"], self.pool_w[i], n_dev=num)
                 if on_step:
                     on_step("s%d_pool" % i)
+        if num is not None:  # one read-back at the end, to cut the results to size
+            m = int(num.item())
+            coords, feats = coords[:m], feats[:m]
         return coords, feats

@@ -581,3 +581,36 @@ def test_dsvt_v_stage_layout_on_sampled_windows(gpu, oracle):
     pos = {k: i for i, k in enumerate(key(oc).tolist())}
     rows = np.array([pos[k] for k in key(cs).tolist()])
     check_close(of[rows], fs, "bf16", "DSVT-V stage layout, %d output voxels" % rows.shape[0])
+
+
+def test_counts_that_live_on_the_device(gpu, oracle):
+    """dsvt_partition_counted and dsvt_pool_counted: the voxel count is read on the device, the arrays have the
+    capacity's length and garbage past the count.  The tables are bit-exact those of the oracle for the counted
+    voxels; the pooling equals dsvt_pool on the truncated arrays; a count of zero gives empty results."""
+    rng = np.random.default_rng(5)
+    grid, window, tau, n, k = (60, 60, 2), (12, 12, 2), 36, 3000, 1777
+    coords = di.unique_cells(rng, n, grid, 1)
+    junk = coords.copy()
+    junk[k:] = 10 ** 6  # (would raise the bad-coordinate bit if it were read)
+    ctx = gpu.Context(n, _nwin(1, grid, window), 64)
+    cnt = dev(np.array([k], dtype=np.int32))
+    both = ctx.partition_rotated(dev(junk), 1, grid, window, tau, n_dev=cnt)
+    assert ctx.status_sync() == 0
+    for axis in (0, 1):
+        _compare_table(both[axis], oracle.partition(coords[:k], 1, grid, window, tau, axis), k, axis, extras=False)
+    zero = dev(np.array([0], dtype=np.int32))
+    both = ctx.partition_rotated(dev(junk), 1, grid, window, tau, n_dev=zero)
+    assert ctx.status_sync() == 0 and int(both[0].num_sets.item()) == 0 and int(both[1].num_sets.item()) == 0
+    assert int(both[0].set_rowoff[0].item()) == 0 and int(both[0].set_rowoff[both[0].cap_sets + 1].item()) == 0
+    # pooling
+    C, heads = 64, 4
+    feats = rng.standard_normal((n, C), dtype=np.float32)
+    w = gpu.device_weights(di.make_pool_weights(rng, C, heads, True), gpu.BF16_FP32ACC, ctx.device)
+    ctx2 = gpu.Context(n, 30 * 30 * 2, C)
+    oc, of, num, _, _ = ctx2.pool(dev(junk), dev(feats), 1, grid, (2, 2, 1), w, n_dev=cnt)
+    rc, rf, rnum, _, _ = ctx2.pool(dev(coords[:k]), dev(feats[:k]), 1, grid, (2, 2, 1), w)
+    assert ctx2.status_sync() == 0
+    m = int(rnum.item())
+    assert int(num.item()) == m and torch.equal(oc[:m], rc[:m]) and torch.equal(of[:m], rf[:m])
+    oc, of, num, _, _ = ctx2.pool(dev(junk), dev(feats), 1, grid, (2, 2, 1), w, n_dev=zero)
+    assert ctx2.status_sync() == 0 and int(num.item()) == 0
