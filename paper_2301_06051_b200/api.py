@@ -332,7 +332,8 @@ class Context:
 
     # ---- dsvt_layers ----
     def layers(self, x: torch.Tensor, tables: Sequence["SetTable"], ws: Sequence[Dict], y: torch.Tensor,
-               coords: Optional[torch.Tensor] = None, use_rowoff: bool = True) -> torch.Tensor:
+               coords: Optional[torch.Tensor] = None, use_rowoff: bool = True,
+               pe: Optional[torch.Tensor] = None) -> torch.Tensor:
         """A chain of layers, layer i on tables[i] with weights ws[i]: the first reads x, all write y."""
         L = len(ws)
         assert len(tables) == L
@@ -341,7 +342,7 @@ class Context:
         for i, (t, w) in enumerate(zip(tables, ws)):
             tr[i].set_table, tr[i].cap_sets, tr[i].num_sets = _ptr(t.set_table), t.cap_sets, _ptr(t.num_sets)
             tr[i].set_rowoff = _ptr(t.set_rowoff) if use_rowoff else None
-            pr[i] = layer_params(w, t.set_size, None, coords)
+            pr[i] = layer_params(w, t.set_size, pe, coords)
         rc = self.lib.dsvt_layers(self._h, _ptr(x), int(x.shape[0]), L, tr, pr, _ptr(y))
         self._check(rc, "dsvt_layers")
         return y

@@ -75,6 +75,7 @@ struct TcGeom {
 struct alignas(64) TcLayer {
   CUtensorMap qkv, o, w1, w2;
   const float *b_qkv, *b_o, *b_1, *b_2, *ln1_g, *ln1_b, *ln2_g, *ln2_b, *rpb;
+  const float* pe;  // positional term added to the input of the query and key maps, [n][C], or NULL
   const int32_t *table, *num_sets, *rowoff;
   int32_t cap_sets;
   float eps;
@@ -114,6 +115,7 @@ struct Misc {  // small shared state beside the big regions
   // launch constants, written once before the roles start: the phase functions read them from here
   // instead of taking them as arguments, so that nothing has to stay in registers across their calls
   const float* x;   // input rows of the tile the compute warps are working on
+  const float* pe;  // the layer's positional term (kernels with one)
   float* y;
   int32_t* status;
   unsigned char* sm;   // 1024-aligned base of the dynamic shared memory (generic address)
@@ -342,6 +344,7 @@ struct RoleCtx {
   uint32_t tmem;      // TMEM base address of the CTA's allocation
   // copies of the kernel parameters the two single-thread roles use (registers instead of parameter-space loads)
   int mode, n_f1, NF, nkb_h, tau, n_layers;
+  int pe;  // the value projection comes first and the A operand is rewritten (x + pe) before the key and query ones
   uint32_t off_a, off_kv, off_stage;
 };
 
@@ -454,7 +457,10 @@ __device__ __noinline__ void producer_role(const TcArgs& a, const RoleCtx rc) {
       const CUtensorMap* map;
       int row0, nkb;
       uint32_t bytes = STAGE_BYTES;
-      if (c < 3) { map = &ly.qkv; row0 = (c == 0 ? 1 : c == 1 ? 2 : 0) * C; nkb = NKB; }   // K, V, Q
+      if (c < 3) {  // K, V, Q; with a positional term V, K, Q
+        map = &ly.qkv; nkb = NKB;
+        row0 = (rc.pe ? (c == 0 ? 2 : c == 1 ? 1 : 0) : (c == 0 ? 1 : c == 1 ? 2 : 0)) * C;
+      }
       else if (c == 3) { map = &ly.o; row0 = 0; nkb = NKB; }
       else if (c < 4 + rc.n_f1) { map = &ly.w1; row0 = (c - 4) * rc.NF; nkb = NKB; bytes = (uint32_t)rc.NF * 128u; }
       else { map = &ly.w2; row0 = 0; nkb = rc.nkb_h; }
@@ -505,7 +511,7 @@ __device__ __noinline__ void mma_role(const RoleCtx rc) {
     if (ns < 0) break;
     for (int c = 0; c < n_chunks; ++c) {
       // a fresh A operand: X (chunks 0-2), attention output (3), x1 (4..), MLP hidden (last)
-      if (c == 0) {
+      if (c == 0 || (c == 1 && rc.pe)) {  // (with a positional term the operand is rewritten after the V chunk)
         if (!mbar_wait(&mi->x_ready, x_phase, abort_flag)) goto mma_done;
         x_phase ^= 1u;
       } else if (c == 3 || c == 4 || c == 4 + rc.n_f1) {
@@ -515,10 +521,11 @@ __device__ __noinline__ void mma_role(const RoleCtx rc) {
       // accumulator placement: K -> region 0, V -> 1, Q -> 0, O -> 0, MLP-1 piece i -> i & 1, MLP-2 -> 2
       // (on top of the parked x1 + b_2)
       uint32_t bar, col, n;
-      if (c < 4) { bar = (c == 1) ? 1u : 0u; col = (c == 1) ? COL_B : 0u; n = C; }
+      const int c_v = rc.pe ? 0 : 1;  // the V chunk
+      if (c < 4) { bar = (c == c_v) ? 1u : 0u; col = (c == c_v) ? COL_B : 0u; n = C; }
       else if (c < 4 + rc.n_f1) { bar = (uint32_t)(c - 4) & 1u; col = bar * COL_B; n = (uint32_t)rc.NF; }
       else { bar = 2u; col = kTmemCols - C; n = C; }
-      if (c == 1) {
+      if (c == c_v) {
         // region 1 may overlap region 2: the previous tile's MLP-2 result must have been read
         if (!mbar_wait(&mi->acc_free[2], (uses[2] & 1u) ^ 1u, abort_flag)) goto mma_done;
       }
@@ -689,11 +696,12 @@ __device__ __noinline__ void stamp_role(int32_t* __restrict__ row_stamp) {
 // alive across the calls.
 
 // Gather (Eq. 4): the fp32 rows listed in buffer b -> bf16 A operand, four rows in flight per warp; all 128 rows
-// are written (rows past the tile as zeros).
-template <int C, bool RPB>
+// are written (rows past the tile as zeros).  ADD_PE: the current tile's rows once more, with the positional
+// term added (the operand of the key and query projections).
+template <int C, bool RPB, bool ADD_PE>
 __device__ __noinline__ void phase_gather(int b, int rows) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const float* x = s_mi.next_x[b];
+  const float* x = ADD_PE ? s_mi.x : s_mi.next_x[b];
   unsigned char* a_tile = s_mi.sm + s_mi.off_a;
   const int* rowvox = s_mi.rowvox[b];
   for (int r0 = warp; r0 < kTM; r0 += 4 * kComputeWarps) {
@@ -707,8 +715,14 @@ __device__ __noinline__ void phase_gather(int b, int rows) {
         const float4* src = reinterpret_cast<const float4*>(x + (size_t)v * C) + 2 * lane;
         f[u][0] = __ldcg(src);  // (L2: the rows of a later layer were written during this launch, by any SM)
         f[u][1] = __ldcg(src + 1);
+        if (ADD_PE) {
+          const float4* pp = reinterpret_cast<const float4*>(s_mi.pe + (size_t)v * C) + 2 * lane;
+          const float4 p0 = __ldg(pp), p1 = __ldg(pp + 1);
+          f[u][0].x += p0.x; f[u][0].y += p0.y; f[u][0].z += p0.z; f[u][0].w += p0.w;
+          f[u][1].x += p1.x; f[u][1].y += p1.y; f[u][1].z += p1.z; f[u][1].w += p1.w;
+        }
       }
-      if (RPB && lane == 31) {  // (lane 31 carries no feature columns: C / 8 <= 24)
+      if (RPB && !ADD_PE && lane == 31) {  // (lane 31 carries no feature columns: C / 8 <= 24)
         int lin = 0;
         if (v >= 0) {
           const int4 c = __ldg(s_mi.coords + v);
@@ -970,6 +984,7 @@ __device__ __forceinline__ void load_layer_params(const TcLayer& ly, int hidden)
     s_mi.ln2 = ly.ln2_g != nullptr;
     s_mi.eps = ly.eps;
     s_mi.rpb = ly.rpb;
+    s_mi.pe = ly.pe;
   }
 }
 
@@ -991,8 +1006,9 @@ __device__ __forceinline__ bool compute_all(bool pred) {
 // the odd MLP-1 pieces; region 2 = [512 - C, 512): x1 + b_2 parked by the output-projection epilogue, then
 // the MLP-2 accumulator.  Each region has its own full / free barrier pair.  For C = 192 regions 1 and 2
 // overlap, which is why the MMA issuer waits for region 2 before it starts the next tile's V.
-template <int C, int D, int NT, bool RPB>
+template <int C, int D, int NT, int VAR>
 __device__ __forceinline__ void compute_role(const TcArgs& a) {
+  constexpr bool RPB = VAR == 1, PE = VAR == 2;
   constexpr int NKB = C / 64;        // K blocks of a C-deep contraction
   constexpr int QC = C / 4;          // epilogue columns per thread for a C-wide chunk (four threads per row)
   constexpr uint32_t COL_B = C;      // accumulator region 1
@@ -1018,7 +1034,7 @@ __device__ __forceinline__ void compute_role(const TcArgs& a) {
     ok = mbar_wait(&s_mi.rl_ready[b], par, abort_flag) && ok;
     const int nr = s_mi.next_rows[b];
     if (compute_all(ok && nr >= 0 && mbar_try(&s_mi.dep_ready[b], par))) {
-      phase_gather<C, RPB>(b, nr);
+      phase_gather<C, RPB, false>(b, nr);
       fence_proxy_async();
       mbar_arrive(&s_mi.x_ready);
       gathered = true;
@@ -1053,7 +1069,7 @@ __device__ __forceinline__ void compute_role(const TcArgs& a) {
       ok = mbar_wait(&s_mi.rl_ready[k & 1], par, abort_flag) && ok;
       ok = mbar_wait(&s_mi.dep_ready[k & 1], par, abort_flag) && ok;
       if (compute_all(ok)) {
-        phase_gather<C, RPB>(k & 1, rows);
+        phase_gather<C, RPB, false>(k & 1, rows);
         fence_proxy_async();
       }
       mbar_arrive(&s_mi.x_ready);  // X is in place
@@ -1063,10 +1079,22 @@ __device__ __forceinline__ void compute_role(const TcArgs& a) {
 
     // ---- chunks 0..2: K, V, Q epilogues: (+ bias,) to bf16, into the operand layout ----
     // (the attention pads its key blocks up to 15 rows past the tile: those K / V rows must be real bf16)
-    acc_wait(0u);
-    phase_epi_bf16<QC, false, false>(0u, 0, 0, s_mi.off_kv, 0, rows + 16);
-    acc_wait(1u);
-    phase_epi_bf16<QC, false, true>(COL_B, 1, ParOff<C>::b_v, s_mi.off_kv + NKB * kTM * 128, 0, rows + 16);
+    if (PE) {
+      // the values come from the bare rows; the operand is then rewritten with the positional term added, for
+      // the keys and the queries (the V chunk's accumulator being complete, nothing reads the operand any more)
+      acc_wait(1u);
+      phase_epi_bf16<QC, false, true>(COL_B, 1, ParOff<C>::b_v, s_mi.off_kv + NKB * kTM * 128, 0, rows + 16);
+      phase_gather<C, false, true>(k & 1, rows);
+      fence_proxy_async();
+      mbar_arrive(&s_mi.x_ready);
+      acc_wait(0u);
+      phase_epi_bf16<QC, false, false>(0u, 0, 0, s_mi.off_kv, 0, rows + 16);
+    } else {
+      acc_wait(0u);
+      phase_epi_bf16<QC, false, false>(0u, 0, 0, s_mi.off_kv, 0, rows + 16);
+      acc_wait(1u);
+      phase_epi_bf16<QC, false, true>(COL_B, 1, ParOff<C>::b_v, s_mi.off_kv + NKB * kTM * 128, 0, rows + 16);
+    }
     acc_wait(0u);
     phase_epi_bf16<QC, false, true>(0u, 0, ParOff<C>::b_q, s_mi.off_a, 0, rows);
     compute_sync();
@@ -1125,8 +1153,10 @@ __device__ __forceinline__ void compute_role(const TcArgs& a) {
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int C, int D, int NT, bool RPB>
+// VAR: 0 plain, 1 relative position bias on the logits, 2 additive positional term on the query / key inputs
+template <int C, int D, int NT, int VAR>
 __global__ void __launch_bounds__(kThreads, 1) layer_tc_kernel(const __grid_constant__ TcArgs a) {
+  constexpr bool RPB = VAR == 1;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -1143,7 +1173,7 @@ __global__ void __launch_bounds__(kThreads, 1) layer_tc_kernel(const __grid_cons
     mi->n = a.n; mi->tau = g.tau; mi->heads = g.heads; mi->mode = g.mode; mi->NF = g.NF; mi->n_f1 = g.n_f1;
     mi->ln1 = mi->ln2 = 0;
     mi->eps = 0.f;
-    mi->rpb = nullptr; mi->coords = a.coords;
+    mi->rpb = nullptr; mi->pe = nullptr; mi->coords = a.coords;
     mi->rb_len = g.rb_len; mi->rb_sx = g.rb_sx; mi->rb_sy = g.rb_sy; mi->rb_centre = g.rb_centre;
     mi->rb_ext[0] = g.rb_ext[0]; mi->rb_ext[1] = g.rb_ext[1]; mi->rb_ext[2] = g.rb_ext[2];
     mi->s_lo = mi->nsets = mi->base = mi->rows = mi->buf = mi->layer = 0;
@@ -1193,6 +1223,7 @@ __global__ void __launch_bounds__(kThreads, 1) layer_tc_kernel(const __grid_cons
   rc.tmem = mi->tmem_base;
   rc.mode = g.mode; rc.n_f1 = g.n_f1; rc.NF = g.NF; rc.nkb_h = g.nkb_h; rc.tau = g.tau; rc.n_layers = a.n_layers;
   rc.off_a = g.off_a; rc.off_kv = g.off_kv; rc.off_stage = g.off_stage;
+  rc.pe = VAR == 2;
 
   if (warp == kTmaWarp) {
     if ((tid & 31) == 0) producer_role<C>(a, rc);
@@ -1205,7 +1236,7 @@ __global__ void __launch_bounds__(kThreads, 1) layer_tc_kernel(const __grid_cons
   } else if (warp >= kLoadWarp0) {
     loader_role<C, RPB>(a);
   } else {
-    compute_role<C, D, NT, RPB>(a);
+    compute_role<C, D, NT, VAR>(a);
   }
   // ---- teardown: everyone meets here, then the allocating warp returns the TMEM columns ----
   tc_fence_before();
@@ -1290,10 +1321,10 @@ bool cached_weight_map(dsvt_ctx* ctx, CUtensorMap* out, const void* w, int rows,
   return true;
 }
 
-template <int C, int D, int NT, bool RPB>
+template <int C, int D, int NT, int VAR>
 int launch_tc_one(dsvt_ctx* ctx, const TcArgs& a, int grid, size_t smem, int inst) {
   if (!(ctx->maps->attr_done & (1u << inst))) {  // once per instantiation and context (the attribute is per device)
-    cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<C, D, NT, RPB>,
+    cudaError_t e = cudaFuncSetAttribute(layer_tc_kernel<C, D, NT, VAR>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return DSVT_ERR_CUDA; }
     ctx->maps->attr_done |= 1u << inst;
@@ -1306,17 +1337,23 @@ int launch_tc_one(dsvt_ctx* ctx, const TcArgs& a, int grid, size_t smem, int ins
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, layer_tc_kernel<C, D, NT, RPB>, a);
+  cudaError_t le = cudaLaunchKernelEx(&cfg, layer_tc_kernel<C, D, NT, VAR>, a);
   if (le != cudaSuccess) { ctx->last_cuda_error = (int)le; cudaGetLastError(); return DSVT_ERR_CUDA; }
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
 }
 
-// The position bias is a compile-time variant: a layer without one runs a kernel that holds none of its code.
+// The position bias and the positional term are compile-time variants: a layer without them runs a kernel that
+// holds none of their code.
 template <int C, int D, int NT>
 int launch_tc(dsvt_ctx* ctx, const TcArgs& a, int grid, size_t smem, int inst) {
-  if (a.g.rb_len != 0) return launch_tc_one<C, D, NT, true>(ctx, a, grid, smem, 2 * inst + 1);
-  return launch_tc_one<C, D, NT, false>(ctx, a, grid, smem, 2 * inst);
+  if (a.g.rb_len != 0) return launch_tc_one<C, D, NT, 1>(ctx, a, grid, smem, 2 * inst + 1);
+  if (a.layer[0].pe) {
+    // (the variant with a positional term is built for the paper's shape only: C = 192, set size up to 48)
+    if constexpr (C == 192 && NT <= 14) return launch_tc_one<C, D, NT, 2>(ctx, a, grid, smem, 24 + inst);
+    return DSVT_ERR_UNSUPPORTED;
+  }
+  return launch_tc_one<C, D, NT, 0>(ctx, a, grid, smem, 2 * inst);
 }
 
 template <int C, int D>
@@ -1335,7 +1372,8 @@ int tc_hidden(const dsvt_fused_args& a) { return a.attention_only ? 0 : a.p.hidd
 // Shapes the tensor-core kernel covers; everything else goes to the FMA kernel.
 bool dsvt_layer_tc_supported(const dsvt_fused_args& a) {
   const dsvt_layer_params& p = a.p;
-  if (p.precision != DSVT_BF16_FP32ACC || p.pe) return false;
+  if (p.precision != DSVT_BF16_FP32ACC) return false;
+  if (p.pe && (p.rpb || p.C != 192 || p.set_size > 48)) return false;  // (see launch_tc)
   if (p.rpb) {  // row coordinates are kept as 16-bit linear indices: every table offset must be below 2^15
     const int64_t len = (int64_t)(2 * p.rpb_extent[0] - 1) * (2 * p.rpb_extent[1] - 1) * (2 * p.rpb_extent[2] - 1);
     if (len > 32767) return false;
@@ -1353,7 +1391,7 @@ bool dsvt_layer_tc_chainable(const dsvt_fused_args& a, const dsvt_fused_args& b)
   const dsvt_layer_params &p = a.p, &q = b.p;
   if (a.attention_only || b.attention_only || a.n != b.n || a.y != b.y) return false;
   if (p.C != q.C || p.heads != q.heads || tc_hidden(a) != tc_hidden(b) || p.set_size != q.set_size) return false;
-  if ((p.rpb != nullptr) != (q.rpb != nullptr)) return false;
+  if ((p.rpb != nullptr) != (q.rpb != nullptr) || (p.pe != nullptr) != (q.pe != nullptr)) return false;
   if (p.rpb && (p.coords != q.coords || p.rpb_extent[0] != q.rpb_extent[0] || p.rpb_extent[1] != q.rpb_extent[1] ||
                 p.rpb_extent[2] != q.rpb_extent[2]))
     return false;
@@ -1409,7 +1447,7 @@ int dsvt_launch_layers_tc(dsvt_ctx* ctx, const dsvt_fused_args* layers, int n_la
       ly.w2 = ly.o;
     }
     if (!okm) return DSVT_ERR_CUDA;
-    ly.b_qkv = q.b_qkv; ly.b_o = q.b_o; ly.rpb = q.rpb;
+    ly.b_qkv = q.b_qkv; ly.b_o = q.b_o; ly.rpb = q.rpb; ly.pe = q.pe;
     const bool full = !a.attention_only;
     ly.b_1 = full ? q.b_1 : nullptr; ly.b_2 = full ? q.b_2 : nullptr;
     ly.ln1_g = full ? q.ln1_g : nullptr; ly.ln1_b = full ? q.ln1_b : nullptr;

@@ -133,3 +133,36 @@ def test_a_row_no_earlier_layer_wrote_ends_a_bounded_wait(gpu):
     ctx.layers(x, tabs, ws, z)
     assert ctx.status_sync() == 0
     assert torch.equal(z, y)
+
+
+def test_positional_term_on_the_tensor_core_path(gpu, oracle):
+    """An additive positional term (added to the input of the query and key maps only, not to the values) with
+    bfloat16 weights: one layer alone, attention alone, and a chain of four layers, each against the oracle."""
+    cfg = di.make_config(2, n_override=5000)
+    blocks = cfg["blocks"][:2]
+    ctx, tabs, ws = _setup(gpu, cfg, blocks)
+    rng = np.random.default_rng(11)
+    pe = (0.5 * rng.standard_normal((cfg["n"], cfg["C"]))).astype(np.float32)
+    x, dpe = dev(cfg["feats"]), dev(pe)
+    p0 = oracle.partition(cfg["coords"], 1, cfg["grid"], cfg["window"], cfg["set_size"], 0).set_table
+    p1 = oracle.partition(cfg["coords"], 1, cfg["grid"], cfg["window"], cfg["set_size"], 1).set_table
+    y = torch.empty_like(x)
+    ctx.layer(x, tabs[0], ws[0], y, pe=dpe)
+    assert ctx.status_sync() == 0
+    check_close(y.cpu().numpy(), oracle.layer(cfg["feats"], p0, blocks[0][0], pe=pe), "bf16", "layer with a term")
+    ctx.set_attention(x, tabs[0], ws[0], y, pe=dpe)
+    assert ctx.status_sync() == 0
+    l0 = blocks[0][0]
+    want, _ = oracle.set_attention(cfg["feats"], p0, l0["W_qkv"], l0["b_qkv"], l0["W_o"], l0["b_o"], l0["heads"], pe=pe)
+    rows = np.unique(p0)
+    check_close(y.cpu().numpy()[rows], want[rows], "bf16", "attention with a term")
+    ctx.layers(x, tabs, ws, y, pe=dpe)
+    assert ctx.status_sync() == 0
+    w = cfg["feats"].astype(np.float64)
+    for blk in blocks:
+        w = oracle.block(w, p0, p1, blk, pe=pe)
+    check_close(y.cpu().numpy(), w, "bf16", "chain with a term")
+    # and the term matters: without it the result is another one
+    z = torch.empty_like(x)
+    ctx.layers(x, tabs, ws, z)
+    assert float((y - z).abs().max()) > 1e-2
