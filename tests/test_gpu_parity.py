@@ -614,3 +614,18 @@ def test_counts_that_live_on_the_device(gpu, oracle):
     assert int(num.item()) == m and torch.equal(oc[:m], rc[:m]) and torch.equal(of[:m], rf[:m])
     oc, of, num, _, _ = ctx2.pool(dev(junk), dev(feats), 1, grid, (2, 2, 1), w, n_dev=zero)
     assert ctx2.status_sync() == 0 and int(num.item()) == 0
+
+
+def test_layers_beyond_the_tile_plan_capacity(gpu, oracle):
+    """More sets than the partition's tile plan covers (set size 4: 30,000 sets): the plan entry says "no plan" and the
+    layer kernel cuts its tiles by row ranges.  One block at full size against the oracle on sampled windows."""
+    cfg = di.random_case(21, 110000, (400, 400, 1), (12, 12, 1), 4, 64, 4, hidden=128, layernorm=True, bf16=True)
+    ctx = gpu.Context(cfg["n"], _nwin(1, cfg["grid"], cfg["window"]), 64)
+    t0, t1 = ctx.partition_rotated(dev(cfg["coords"]), 1, cfg["grid"], cfg["window"], 4)
+    S = int(t0.num_sets.item())
+    assert S > 24576 and int(t0.set_rowoff[t0.cap_sets + 1].item()) == -1
+    got = _run_blocks_gpu(gpu, cfg, cfg["blocks"], cfg["coords"], cfg["feats"], ctx=ctx)
+    assert np.all(np.isfinite(got))
+    sel = _sample_windows(oracle, cfg, cfg["coords"], 2500, 3)
+    want = _run_blocks_oracle(oracle, cfg, cfg["blocks"], cfg["coords"][sel], cfg["feats"][sel])
+    check_close(got[sel], want, "bf16", "one block, %d sets without a plan" % S)
