@@ -134,7 +134,8 @@ struct Misc {  // small shared state beside the big regions
   unsigned char row_lo[2][kTM], row_n[2][kTM];  // per tile row: first row and row count of its set
   // relative position bias.  The table index is linear in the coordinate offset, so one integer per row,
   // x * rb_sx + y * rb_sy + z, serves every (query, key) pair: index = lin[query] - lin[key] + rb_centre.  Offsets
-  // inside a set are below 2^15 in magnitude, so the low 16 bits are kept and differences are taken modulo 2^16.
+  // inside a covered set are at most (table length - 1) / 2 < 2^15 in magnitude (tables of up to 65,535 entries
+  // per head), so the low 16 bits are kept and differences are taken modulo 2^16.
   // Written by the gather of a tile (after the previous tile's attention), read by the tile's attention.
   const float* rpb;
   const int4* coords;
@@ -1374,9 +1375,11 @@ bool dsvt_layer_tc_supported(const dsvt_fused_args& a) {
   const dsvt_layer_params& p = a.p;
   if (p.precision != DSVT_BF16_FP32ACC) return false;
   if (p.pe && (p.rpb || p.C != 192 || p.set_size > 48)) return false;  // (see launch_tc)
-  if (p.rpb) {  // row coordinates are kept as 16-bit linear indices: every table offset must be below 2^15
+  if (p.rpb) {
+    // row coordinates are kept as linear indices modulo 2^16 and differences are taken modulo 2^16: exact while every
+    // offset inside a covered set, at most (len - 1) / 2 in magnitude, is below 2^15
     const int64_t len = (int64_t)(2 * p.rpb_extent[0] - 1) * (2 * p.rpb_extent[1] - 1) * (2 * p.rpb_extent[2] - 1);
-    if (len > 32767) return false;
+    if (len > 65535) return false;
   }
   const int d = p.C / p.heads;
   const bool shape = (p.C == 192 && d == 24) || (p.C == 128 && (d == 16 || d == 32)) || (p.C == 64 && d == 16);

@@ -37,7 +37,9 @@ def _with_bias(rng, layer, heads, extent, oracle):
     (36, 1200, (48, 48, 2), (12, 12, 2), 48, 192, 8, True),
     (37, 3000, (96, 96, 1), (30, 30, 1), 90, 128, 8, True),    # one attention item per set (set size above 48)
     (38, 2000, (60, 60, 1), (12, 12, 1), 36, 128, 4, True),    # head dimension 32
-    (39, 900, (24, 24, 40), (12, 12, 32), 36, 64, 4, True),    # a table too long for 16-bit row indices
+    (39, 900, (24, 24, 40), (12, 12, 32), 36, 64, 4, True),    # 33,327 entries: offsets use 16 of the 16 index bits
+    (40, 900, (24, 24, 40), (12, 12, 40), 36, 64, 4, True),    # 41,791 entries per head
+    (43, 900, (32, 32, 40), (16, 16, 36), 36, 64, 4, True),    # 68,231 entries: beyond 16-bit differences (FMA kernel)
 ])
 def test_set_attention_with_relative_position_bias(gpu, oracle, seed, n, grid, window, tau, C, heads, bf16):
     cfg = di.random_case(seed, n, grid, window, tau, C, heads, bf16=bf16)
@@ -83,6 +85,31 @@ def test_block_with_relative_position_bias_and_a_larger_table(gpu, oracle, bf16)
     ctx.layer(x, t0, ws[0], y1, coords=coords)
     check_close(y1.cpu().numpy(), oracle.layer(cfg["feats"], p0, layers[0], coords=cfg["coords"]), cfg["precision"],
                 "biased layer")
+
+
+def test_long_bias_table_runs_on_the_tensor_core_kernel(gpu, oracle):
+    """A table of 33,327 entries per head (window 12 x 12 x 32): row indices are kept modulo 2^16, every offset of a
+    covered set still fits.  Two bf16 layers with such tables go out as one launch (the chained tensor-core kernel;
+    the FMA kernel would take one launch per layer) and match the oracle."""
+    seed, n, grid, window, tau, C, heads = 42, 2500, (36, 36, 40), (12, 12, 32), 36, 192, 8
+    cfg = di.random_case(seed, n, grid, window, tau, C, heads, hidden=384, layernorm=True, bf16=True)
+    rng = np.random.default_rng(seed)
+    layers = [_with_bias(rng, l, heads, window, oracle) for l in cfg["blocks"][0]]
+    ctx = gpu.Context(n, _nwin(1, grid, window), C)
+    ws = [gpu.device_weights(l, precision_of(cfg), ctx.device) for l in layers]
+    x, coords = dev(cfg["feats"]), dev(cfg["coords"])
+    t0, t1 = ctx.partition_rotated(coords, 1, grid, window, tau)
+    y = torch.empty_like(x)
+    before = ctx.launch_count()
+    ctx.block(x, t0, t1, ws, y, coords=coords)
+    assert ctx.launch_count() - before == 1
+    assert ctx.status_sync() == 0
+    p0 = oracle.partition(cfg["coords"], 1, grid, window, tau, 0).set_table
+    p1 = oracle.partition(cfg["coords"], 1, grid, window, tau, 1).set_table
+    want = oracle.block(cfg["feats"], p0, p1, layers, coords=cfg["coords"])
+    check_close(y.cpu().numpy(), want, cfg["precision"], "block with long bias tables")
+    plain = oracle.block(cfg["feats"], p0, p1, cfg["blocks"][0])
+    assert np.abs(plain - want).max() > 1e-2
 
 
 def test_bias_table_narrower_than_a_set_is_flagged(gpu, oracle):
