@@ -972,13 +972,17 @@ __device__ __noinline__ void phase_epi_f2() {
 template <int C>
 __device__ __forceinline__ void load_layer_params(const TcLayer& ly, int hidden) {
   float* par = reinterpret_cast<float*>(s_mi.sm + s_mi.off_par);
+  const uint32_t par_saddr = s_mi.sbase + s_mi.off_par;
   const int n_par = ParOff<C>::vectors * C + hidden;
+  // asynchronous 4-byte copies, all in flight at once: the first reader is the V epilogue, which waits for them
+  // (wait_layer_params) after the K epilogue
   for (int i = threadIdx.x; i < n_par; i += kComputeThreads) {
     const int which = i / C;
     const float* v = which == 0 ? ly.b_qkv : which == 1 ? (ly.b_qkv ? ly.b_qkv + 2 * C : nullptr) : which == 2 ? ly.b_o
                    : which == 3 ? ly.b_2 : which == 4 ? ly.ln1_g : which == 5 ? ly.ln1_b : which == 6 ? ly.ln2_g
                    : which == 7 ? ly.ln2_b : (ly.b_1 ? ly.b_1 - ParOff<C>::b_1 + which * C : nullptr);
-    par[i] = v ? __ldg(v + i % C) : 0.f;
+    if (v) asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(par_saddr + 4u * (uint32_t)i), "l"(v + i % C) : "memory");
+    else par[i] = 0.f;
   }
   if (threadIdx.x == 0) {
     s_mi.ln1 = ly.ln1_g != nullptr;
@@ -987,6 +991,11 @@ __device__ __forceinline__ void load_layer_params(const TcLayer& ly, int hidden)
     s_mi.rpb = ly.rpb;
     s_mi.pe = ly.pe;
   }
+}
+
+__device__ __forceinline__ void wait_layer_params() {
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  compute_sync();
 }
 
 // Barrier over the compute threads that also ANDs a predicate.
@@ -1061,7 +1070,8 @@ __device__ __forceinline__ void compute_role(const TcArgs& a) {
     mbar_arrive(&s_mi.sched_empty[slot]);
     if (++slot == 2) { slot = 0; sphase ^= 1u; }
     if (nsets < 0) break;
-    if (layer != cur_layer) {  // (the previous tile's last use of the block lies before the barrier above)
+    const bool new_params = layer != cur_layer;
+    if (new_params) {  // (the previous tile's last use of the block lies before the barrier above)
       load_layer_params<C>(a.layer[layer], a.g.hidden);
       cur_layer = layer;
     }
@@ -1076,7 +1086,7 @@ __device__ __forceinline__ void compute_role(const TcArgs& a) {
       mbar_arrive(&s_mi.x_ready);  // X is in place
     }
     gathered = false;
-    compute_sync();  // the tile's fields and the parameter block are visible to the phase functions
+    compute_sync();  // the tile's fields are visible to the phase functions
 
     // ---- chunks 0..2: K, V, Q epilogues: (+ bias,) to bf16, into the operand layout ----
     // (the attention pads its key blocks up to 15 rows past the tile: those K / V rows must be real bf16)
@@ -1084,6 +1094,7 @@ __device__ __forceinline__ void compute_role(const TcArgs& a) {
       // the values come from the bare rows; the operand is then rewritten with the positional term added, for
       // the keys and the queries (the V chunk's accumulator being complete, nothing reads the operand any more)
       acc_wait(1u);
+      if (new_params) wait_layer_params();
       phase_epi_bf16<QC, false, true>(COL_B, 1, ParOff<C>::b_v, s_mi.off_kv + NKB * kTM * 128, 0, rows + 16);
       phase_gather<C, false, true>(k & 1, rows);
       fence_proxy_async();
@@ -1094,6 +1105,7 @@ __device__ __forceinline__ void compute_role(const TcArgs& a) {
       acc_wait(0u);
       phase_epi_bf16<QC, false, false>(0u, 0, 0, s_mi.off_kv, 0, rows + 16);
       acc_wait(1u);
+      if (new_params) wait_layer_params();  // (the key epilogue adds no bias: it needs none of the vectors)
       phase_epi_bf16<QC, false, true>(COL_B, 1, ParOff<C>::b_v, s_mi.off_kv + NKB * kTM * 128, 0, rows + 16);
     }
     acc_wait(0u);
