@@ -45,6 +45,9 @@ extern "C" {
 #define DSVT_ERR_TIMEOUT (-5)     /* a bounded device-side wait expired (reported by dsvt_status_sync) */
 #define DSVT_ERR_BAD_INPUT (-6)   /* device-detected bad data (reported by dsvt_status_sync) */
 
+/* Flag on the tile count of a set_rowoff buffer's tile plan (see dsvt_partition). */
+#define DSVT_PLAN_PACKED 0x40000000
+
 #define DSVT_FP32 0
 #define DSVT_BF16_FP32ACC 1
 
@@ -105,13 +108,21 @@ int dsvt_set_layer_ctas(dsvt_ctx* ctx, int32_t max_ctas);
  *               integer floor), j = the set's number inside its window.  Rows are ordered by
  *               ascending window id, then j.  Rows [0, *num_sets) are written.
  *   num_sets    out, device int32: total number of sets.
- *   set_rowoff  out, optional (NULL to skip), int32 [2 * cap_sets + 3].  Entries [0, cap_sets]:
+ *   set_rowoff  out, optional (NULL to skip), int32 [4 * cap_sets + 4].  Entries [0, cap_sets]:
  *               set_rowoff[s] = number of distinct voxels in the sets before s; entry [*num_sets] = n.
- *               Entries from [cap_sets + 1] on: a tile plan for the tensor-core layer kernel (number of
- *               tiles, then the first set of each tile of at most 128 distinct rows; -1 = no plan).
- *               Passing the buffer on to dsvt_set_attention / dsvt_layer / dsvt_block saves them two
- *               passes over the table.  A caller that fills the row offsets by hand sets entry
- *               [cap_sets + 1] to -1.
+ *               Entries from [cap_sets + 1] on: a tile plan for the tensor-core layer kernel, which
+ *               works on tiles of whole sets with at most 128 distinct rows (the sets of Eq. 3 are
+ *               independent of one another, so any of them may share a tile).  Entry [cap_sets + 1]:
+ *               -1 = no plan; T = T tiles in table order, tile t holding the sets
+ *               [e[t], e[t + 1]) with e = entries [cap_sets + 2, cap_sets + 2 + T];
+ *               T | DSVT_PLAN_PACKED = T tiles over a reordering of the sets that fills the tiles
+ *               better: tile t holds the sets order[p] for p in [e[t], e[t + 1]), with
+ *               order = entries [2 cap_sets + 3, 3 cap_sets + 3) a permutation of the sets and
+ *               entries [3 cap_sets + 3, 4 cap_sets + 4) the number of distinct voxels in the sets
+ *               before position p of that order.  Passing the buffer on to dsvt_set_attention /
+ *               dsvt_layer / dsvt_block / dsvt_layers saves them two passes over the table.  A caller
+ *               that fills the row offsets by hand sets entry [cap_sets + 1] to -1 (and may then
+ *               pass 2 * cap_sets + 3 entries only).
  *   perm        out, optional, int32 [n]: voxel indices in (window, inner-window) sorted order.
  *   win_start, win_setoff   out, optional, int32 [num_windows + 1]: exclusive prefix sums of the
  *               per-window voxel counts / set counts over ALL windows (empty ones included).
@@ -301,7 +312,7 @@ typedef struct dsvt_table_ref {
   const int32_t* set_table; /* int32 [cap_sets][set_size] */
   int32_t cap_sets;
   const int32_t* num_sets;   /* device int32 */
-  const int32_t* set_rowoff; /* int32 [2 * cap_sets + 3] or NULL */
+  const int32_t* set_rowoff; /* int32 [4 * cap_sets + 4] or NULL */
 } dsvt_table_ref;
 int dsvt_layers(dsvt_ctx* ctx, const float* x, int32_t n, int32_t num_layers, const dsvt_table_ref* tables,
                 const dsvt_layer_params* params, float* y);

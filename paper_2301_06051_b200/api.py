@@ -158,7 +158,7 @@ class SetTable:
     """Device-side result of dsvt_partition."""
     set_table: torch.Tensor  # int32 [cap_sets, set_size]
     num_sets: torch.Tensor  # int32 [1] (device)
-    set_rowoff: torch.Tensor  # int32 [2 * cap_sets + 3]: row offsets, then the tile plan
+    set_rowoff: torch.Tensor  # int32 [4 * cap_sets + 4]: row offsets, then the tile plan
     cap_sets: int
     set_size: int
     perm: Optional[torch.Tensor] = None
@@ -253,7 +253,7 @@ class Context:
             dev = self.device
             out = SetTable(torch.empty((cap, set_size), dtype=torch.int32, device=dev),
                            torch.zeros(1, dtype=torch.int32, device=dev),
-                           torch.empty(2 * cap + 3, dtype=torch.int32, device=dev), cap, set_size)
+                           torch.empty(4 * cap + 4, dtype=torch.int32, device=dev), cap, set_size)
             if extras:
                 nw = int(batch) * (-(-grid[0] // window[0])) * (-(-grid[1] // window[1])) * (-(-grid[2] // window[2]))
                 out.perm = torch.empty(max(n, 1), dtype=torch.int32, device=dev)
@@ -279,7 +279,7 @@ class Context:
             dev = self.device
             out = tuple(SetTable(torch.empty((cap, set_size), dtype=torch.int32, device=dev),
                                  torch.zeros(1, dtype=torch.int32, device=dev),
-                                 torch.empty(2 * cap + 3, dtype=torch.int32, device=dev), cap, set_size)
+                                 torch.empty(4 * cap + 4, dtype=torch.int32, device=dev), cap, set_size)
                         for _ in range(2))
         t0, t1 = out
         assert t0.cap_sets == t1.cap_sets and t0.set_size == t1.set_size == set_size

@@ -37,8 +37,8 @@ void carve(dsvt_ctx* c, unsigned char* base, size_t* total) {
   c->win_count = k.take<int32_t>(nw + 1);
   c->win_start = k.take<int32_t>(nw + 1);
   c->win_setoff = k.take<int32_t>(nw + 1);
-  c->rowoff_a = k.take<int32_t>(2 * nv + 3);
-  c->rowoff_b = k.take<int32_t>(2 * nv + 3);
+  c->rowoff_a = k.take<int32_t>(4 * nv + 4);
+  c->rowoff_b = k.take<int32_t>(4 * nv + 4);
   c->region_key = k.take<int32_t>(nv);
   c->bm_words = (size_t)1 << 21;  // 64 Mi keys per sort axis
   c->bm_zero = k.take<int32_t>(2 * (nw + 1) + 2 * c->bm_words);

@@ -30,8 +30,8 @@ struct dsvt_ctx {
   int32_t* win_count;   // [max_windows + 1]  (pooling: region occupancy flags)
   int32_t* win_start;   // [max_windows + 1]  (pooling: region rank)
   int32_t* win_setoff;  // [max_windows + 1]
-  int32_t* rowoff_a;    // [2 max_voxels + 3] row offsets + tile plan derived from a caller table
-  int32_t* rowoff_b;    // [2 max_voxels + 3]
+  int32_t* rowoff_a;    // [4 max_voxels + 4] row offsets + tile plan derived from a caller table
+  int32_t* rowoff_b;    // [4 max_voxels + 4]
   int32_t* region_key;  // [max_voxels] pooling: dense region id of each output row
   // partition, bitmap route (bm_words == 0: route not available)
   size_t bm_words;       // bitmap capacity per sort axis, in 32-bit words

@@ -386,9 +386,9 @@ __device__ __noinline__ void producer_role(const TcArgs& a, const RoleCtx rc) {
     const int S = min(__ldg(ly.num_sets), ly.cap_sets);
     int T = __ldg(ly.rowoff + ly.cap_sets + 1);
     mi->lay_S[l] = S;
-    mi->lay_plan[l] = T >= 0;
+    mi->lay_plan[l] = T < 0 ? 0 : (T & DSVT_PLAN_PACKED) ? 2 : 1;  // none / in table order / over a reordering
     if (T < 0) T = S > 0 ? (__ldg(ly.rowoff + S) + Rv - 1) / Rv : 0;
-    else T = min(T, S);
+    else T = min(T & ~DSVT_PLAN_PACKED, S);
     total += max(T, 0);
     mi->tile_end[l] = total;
   }
@@ -420,8 +420,10 @@ __device__ __noinline__ void producer_role(const TcArgs& a, const RoleCtx rc) {
         e = lo;
         if (e <= f) continue;  // no set starts in this row range
       }
-      base = __ldg(ly.rowoff + f);
-      rows = __ldg(ly.rowoff + e) - base;
+      // rows before a position: of the table's own order, or of the packed plan's
+      const int32_t* ro = mi->lay_plan[l] == 2 ? ly.rowoff + 3 * (size_t)ly.cap_sets + 3 : ly.rowoff;
+      base = __ldg(ro + f);
+      rows = __ldg(ro + e) - base;
       if (rows <= 0 || rows > kTM || e - f > kTM) { atomicOr(status, DSVT_STATUS_BAD_INDEX); continue; }
       lay = l; s0 = f; ns = e - f;
       return;
@@ -564,14 +566,22 @@ __device__ __forceinline__ void loader_sync() { asm volatile("bar.sync 6, %0;" :
 
 // Distinct slots of each set -> tile rows (Eq. 4) and per-row set ranges: one thread per
 // set (a tile of a sparse region holds dozens of tiny sets), walking the set's table row.
+// `order` (or NULL: the identity) maps the positions [s_lo, s_lo + nsets) of the tile to sets, `rowoff` holds the
+// rows before each position.
 template <bool RPB>
 __device__ __forceinline__ void loader_row_list(const int32_t* __restrict__ table, const int32_t* __restrict__ rowoff,
-                                                int b, int lt, int s_lo, int nsets, int base) {
+                                                const int32_t* __restrict__ order, int cap_sets, int b, int lt,
+                                                int s_lo, int nsets, int base) {
   const int n = s_mi.n, tau = s_mi.tau;
   for (int si = lt; si < nsets; si += kLoadThreads) {
-    const int s = s_lo + si;
+    const int p = s_lo + si;
+    const int s = order ? __ldg(order + p) : p;
+    if ((unsigned)s >= (unsigned)cap_sets) {  // (only a plan that this library did not write can do that)
+      atomicOr(s_mi.status, DSVT_STATUS_BAD_INDEX);
+      continue;
+    }
     const int32_t* trow = table + (size_t)s * tau;
-    const int lb = __ldg(rowoff + s) - base, cap = __ldg(rowoff + s + 1) - __ldg(rowoff + s);
+    const int lb = __ldg(rowoff + p) - base, cap = __ldg(rowoff + p + 1) - __ldg(rowoff + p);
     const bool inside = lb >= 0 && lb < kTM;
     const int cnt_max = inside ? min(cap, kTM - lb) : 0;  // tile rows this set may fill
     int pos = 0, prev = 0;
@@ -644,7 +654,9 @@ __device__ __noinline__ void loader_role(const TcArgs& a) {
       }
       loader_sync();
       const TcLayer& ly = a.layer[lay];
-      loader_row_list<RPB>(ly.table, ly.rowoff, b, lt, s_lo, nsets, base);
+      const bool packed = s_mi.lay_plan[lay] == 2;
+      loader_row_list<RPB>(ly.table, packed ? ly.rowoff + 3 * (size_t)ly.cap_sets + 3 : ly.rowoff,
+                           packed ? ly.rowoff + 2 * (size_t)ly.cap_sets + 3 : nullptr, ly.cap_sets, b, lt, s_lo, nsets, base);
       if (lt == 0) s_mi.next_x[b] = lay == 0 ? a.x : a.y;
     }
     if (lt == 0) s_mi.next_rows[b] = nsets < 0 ? -1 : rows;

@@ -339,13 +339,164 @@ __global__ void table_unique_count_kernel(const int32_t* __restrict__ table, int
 // row segments).  The greedy chain 0 -> next(0) -> next(next(0)) ... is found by pointer doubling, all
 // sets in parallel: single block, arrays in shared memory.
 constexpr int kPlanMaxSets = 24576;
+// Scratch of the packed plan behind the three per-set arrays: per-warp bin counts of one sorting round, bin
+// starts, bin cursors, the cursors before the round, the histogram.
+constexpr int kPackBins = 132;  // set sizes 1 .. 128, rounded up
+struct PackScratch {
+  unsigned short whist[32][kPackBins];
+  int bin_start[kPackBins], bin_cur[kPackBins], round_base[kPackBins], hist[kPackBins];
+};
 // Dynamic shared memory the plan needs for at most smax sets.
-__host__ __device__ constexpr size_t plan_smem_bytes(int smax) { return (size_t)(smax + 1) * 8 + (size_t)smax + 16; }
+__host__ __device__ constexpr size_t plan_smem_bytes(int smax) {
+  return (size_t)(smax + 1) * 8 + (((size_t)smax + 15) & ~(size_t)15) + 16 + sizeof(PackScratch);
+}
+
+// Packed plan.  Sets are independent of one another, so a tile may hold any of them: the greedy plan in table
+// order leaves a tenth of every tile empty (the next set did not fit), this one deals the sets, sorted by their
+// number of rows (descending, ties in table order), out to T tiles in boustrophedon rounds, largest to tile 0 ..
+// T - 1, the next T to tile T - 1 .. 0, and so on, which levels the tiles' row counts to within a few rows; T is
+// the smallest of a ladder of candidates from ceil(rows / max_rows) upwards for which no tile exceeds max_rows.
+// Written behind the plan header: the sets in tile order (order[p]) and the rows before each position (prow[p]);
+// tile t covers positions [plan[1 + t], plan[2 + t]).  Returns false (nothing written) if some set has no row or
+// more than max_rows, or no candidate below `limit` tiles (the plan in table order, which the caller has written) fits.
+struct PlanWindows {  // optional: the windows behind the sets (sets of a window are consecutive), or win_setoff = NULL
+  const int32_t* win_setoff;
+  const int32_t* win_count;
+  int32_t num_windows;
+};
+__device__ bool packed_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int32_t cap_sets, int32_t smax,
+                                 int32_t max_rows, int limit, PlanWindows pw, int* plan_smem, int* warp_tot) {
+  const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+  if (max_rows >= kPackBins || nthr <= max_rows || (nthr & 31) != 0) return false;
+  int* srt = plan_smem;                // set ids, sorted by rows descending
+  int* ro = srt + (smax + 1);          // row offsets in table order
+  unsigned char* ssz = reinterpret_cast<unsigned char*>(ro + (smax + 1));  // rows of srt[i]
+  PackScratch* ps = reinterpret_cast<PackScratch*>(ssz + (((size_t)smax + 15) & ~(size_t)15));
+  constexpr int kRowMask = 0xffffff;  // (at most smax * max_rows rows: 24 bits hold them)
+  for (int s = tid; s <= S; s += nthr) ro[s] = rowoff[s];
+  for (int b = tid; b < kPackBins; b += nthr) { ps->hist[b] = 0; ps->bin_cur[b] = 0; }
+  __syncthreads();
+  // Sort key of a set: the rows of its window's largest set, so that the sets of a window (whose sizes differ by
+  // at most one) stay neighbours in the sorted order and land in neighbouring tiles.  The same plan serves every
+  // layer on these windows, so the voxels a tile reads were written by tiles a few numbers away in the layer
+  // before, not by tiles anywhere in it.  Kept in the top byte of the set's row offset; 0 = the set's own rows.
+  if (pw.win_setoff && ro[S] <= kRowMask) {
+    for (int w = tid; w < pw.num_windows; w += nthr) {
+      const int so = pw.win_setoff[w], cnt = pw.win_setoff[w + 1] - so;
+      if (cnt <= 0 || so < 0) continue;
+      const int key = (pw.win_count[w] + cnt - 1) / cnt;
+      if (key < 1 || key > max_rows) continue;
+      for (int j = 0; j < cnt && so + j < S; ++j) ro[so + j] |= key << 24;
+    }
+    __syncthreads();
+  }
+  auto rows_of = [&](int q) { return (ro[q + 1] & kRowMask) - (ro[q] & kRowMask); };
+  auto key_of = [&](int q) { const int k = (int)((unsigned)ro[q] >> 24), c = rows_of(q); return k >= c ? k : c; };
+  bool bad = false;
+  for (int s = tid; s < S; s += nthr) {
+    const int c = rows_of(s);
+    if (c < 1 || c > max_rows || ro[S] > kRowMask) bad = true;
+    else atomicAdd(&ps->hist[key_of(s)], 1);
+  }
+  if (__syncthreads_or(bad)) return false;
+  if (tid == 0) {
+    int acc = 0;
+    for (int c = max_rows; c >= 1; --c) { ps->bin_start[c] = acc; acc += ps->hist[c]; }
+  }
+  // stable counting sort, one set per thread and round
+  for (int base = 0; base < S; base += nthr) {
+    for (int i = tid; i < 32 * kPackBins; i += nthr) (&ps->whist[0][0])[i] = 0;
+    __syncthreads();
+    const int s = base + tid;
+    const int c = s < S ? key_of(s) : 0;  // the bin
+    const unsigned same = __match_any_sync(0xffffffffu, c);
+    const int rank = __popc(same & ((1u << lane) - 1u));
+    if (c && rank == 0) ps->whist[warp][c] = (unsigned short)__popc(same);
+    __syncthreads();
+    if (tid >= 1 && tid <= max_rows) {  // bin tid: the warps' counts -> exclusive prefixes
+      int run = 0;
+      for (int w = 0; w < nwarp; ++w) { const int t = ps->whist[w][tid]; ps->whist[w][tid] = (unsigned short)run; run += t; }
+      ps->round_base[tid] = ps->bin_cur[tid];
+      ps->bin_cur[tid] += run;
+    }
+    __syncthreads();
+    if (c) {
+      const int pos = ps->bin_start[c] + ps->round_base[c] + ps->whist[warp][c] + rank;
+      srt[pos] = s;
+      ssz[pos] = (unsigned char)rows_of(s);
+    }
+    __syncthreads();
+  }
+  // rows of tile t when the sorted sets are dealt out to T tiles
+  auto tile_rows = [&](int t, int T) {
+    int sum = 0, r = 0;
+    for (int i0 = 0; i0 < S; i0 += T, ++r) {
+      const int i = i0 + ((r & 1) ? T - 1 - t : t);
+      if (i < S) sum += ssz[i];
+    }
+    return sum;
+  };
+  const int total = ro[S] & kRowMask;
+  const int T0 = (total + max_rows - 1) / max_rows;
+  auto fits = [&](int Tc) {  // (the same answer in every thread)
+    bool over = false;
+    for (int t = tid; t < Tc; t += nthr) over |= tile_rows(t, Tc) > max_rows;
+    return !__syncthreads_or(over);
+  };
+  int T = -1, last = T0 - 1;  // last = the largest count known not to fit
+  const int ladder[14] = {0, 1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64, 96};  // 128ths of T0 on top of T0
+  for (int j = 0; j < 14; ++j) {
+    const int Tj = min(min(S, limit - 1), T0 + (int)(((int64_t)T0 * ladder[j] + 127) / 128));
+    if (Tj <= last) continue;
+    if (fits(Tj)) { T = Tj; break; }
+    last = Tj;
+    if (Tj >= min(S, limit - 1)) break;  // nothing below the plan in table order fits
+  }
+  if (T < 0) return false;
+  while (T - last > 1) {  // between the rungs: bisection (fitting is not monotonic in T; any count that fits will do)
+    const int mid = last + (T - last) / 2;
+    if (fits(mid)) T = mid; else last = mid;
+  }
+  // positions: tile t holds the sets of rounds 0 .. full - 1 and, for rem tiles, one of the last round
+  const int full = S / T, rem = S % T;
+  auto tile_start = [&](int t) { return t * full + ((full & 1) ? max(0, t - (T - rem)) : min(t, rem)); };
+  const int chunk = (T + nthr - 1) / nthr;
+  const int t0 = min(tid * chunk, T), t1 = min(t0 + chunk, T);
+  int local = 0;
+  for (int t = t0; t < t1; ++t) local += tile_rows(t, T);
+  int tot;
+  int rows = block_excl_scan(local, warp_tot, &tot);
+  int32_t* out[2] = {rowoff, rowoff_copy};
+  for (int t = t0; t < t1; ++t) {
+    int p = tile_start(t), r = 0;
+    for (int q = 0; q < 2; ++q)
+      if (out[q]) out[q][cap_sets + 2 + t] = p;
+    for (int i0 = 0; i0 < S; i0 += T, ++r) {
+      const int i = i0 + ((r & 1) ? T - 1 - t : t);
+      if (i >= S) continue;
+      for (int q = 0; q < 2; ++q)
+        if (out[q]) {
+          out[q][2 * (size_t)cap_sets + 3 + p] = srt[i];
+          out[q][3 * (size_t)cap_sets + 3 + p] = rows;
+        }
+      rows += ssz[i];
+      ++p;
+    }
+  }
+  if (tid == 0)
+    for (int q = 0; q < 2; ++q)
+      if (out[q]) {
+        out[q][cap_sets + 1] = T | DSVT_PLAN_PACKED;
+        out[q][cap_sets + 2 + T] = S;
+        out[q][3 * (size_t)cap_sets + 3 + S] = tot;
+      }
+  return true;
+}
 
 // The plan of `rowoff` (its offsets are read, its plan written; a second buffer with the same offsets, e.g. the
 // other sort axis of the same windows, receives a copy).  One block, any size up to 1024 threads.
 __device__ void tile_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int32_t cap_sets, int32_t smax,
-                               int32_t max_rows, int* plan_smem, int* warp_tot) {
+                               int32_t max_rows, PlanWindows pw, int* plan_smem, int* warp_tot) {
   int32_t* plan = rowoff + cap_sets + 1;
   int32_t* plan2 = rowoff_copy ? rowoff_copy + cap_sets + 1 : nullptr;
   int* cur = plan_smem;
@@ -404,16 +555,18 @@ __device__ void tile_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int
     plan[0] = total; plan[1 + total] = S;
     if (plan2) { plan2[0] = total; plan2[1 + total] = S; }
   }
+  __syncthreads();  // the plan in table order stands; a packed one with fewer tiles replaces it (same shared arrays)
+  packed_plan_body(rowoff, rowoff_copy, S, cap_sets, smax, max_rows, total, pw, plan_smem, warp_tot);
 }
 
 __global__ void __launch_bounds__(kScanThreads) tile_plan_kernel(int32_t* rowoff0, int32_t* rowoff1,
                                                                  const int32_t* __restrict__ num_sets, int32_t cap_sets,
-                                                                 int32_t smax, int32_t max_rows) {
+                                                                 int32_t smax, int32_t max_rows, PlanWindows pw) {
   extern __shared__ int plan_smem[];
   __shared__ int warp_tot[33];
   int32_t* rowoff = blockIdx.x ? rowoff1 : rowoff0;  // one block per buffer: offsets, then the plan
   if (!rowoff) return;
-  tile_plan_body(rowoff, nullptr, min(*num_sets, cap_sets), cap_sets, smax, max_rows, plan_smem, warp_tot);
+  tile_plan_body(rowoff, nullptr, min(*num_sets, cap_sets), cap_sets, smax, max_rows, pw, plan_smem, warp_tot);
 }
 
 // ---- bitmap route: ranks by population count instead of sorting --------------------------------
@@ -553,14 +706,15 @@ __global__ void __launch_bounds__(kScanThreads) bm_place_fill_kernel(int32_t n_m
                                                             const int32_t* __restrict__ win_start,
                                                             const int32_t* __restrict__ win_setoff, int32_t tau,
                                                             int32_t cap_sets, const int32_t* __restrict__ num_sets,
-                                                            FillOut out, int32_t smax) {
+                                                            FillOut out, int32_t smax, int32_t num_windows) {
   extern __shared__ int plan_smem[];
   __shared__ int warp_tot[33];
   pdl_enter();
   if (blockIdx.x == 0) {  // the plan (one for both axes: their row offsets are the same)
     int32_t* r0 = out.rowoff[0] ? out.rowoff[0] : out.rowoff[1];
     int32_t* r1 = out.rowoff[0] ? out.rowoff[1] : nullptr;
-    if (r0) tile_plan_body(r0, r1, min(*num_sets, cap_sets), cap_sets, smax, 128, plan_smem, warp_tot);
+    const PlanWindows pw{win_setoff, win_count, num_windows};
+    if (r0) tile_plan_body(r0, r1, min(*num_sets, cap_sets), cap_sets, smax, 128, pw, plan_smem, warp_tot);
     return;
   }
   const int i = (blockIdx.x - 1) * blockDim.x + threadIdx.x;
@@ -647,7 +801,7 @@ int dsvt_launch_rowoff_from_table(dsvt_ctx* ctx, const int32_t* table, int32_t c
 
 // Tile plans behind the row offsets of one or two buffers: set_rowoff + cap_sets + 1 (see include/dsvt.h).
 static int launch_tile_plans(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap_sets, int32_t* set_rowoff,
-                             int32_t* set_rowoff1) {
+                             int32_t* set_rowoff1, PlanWindows pw) {
   const int32_t smax = cap_sets < kPlanMaxSets ? cap_sets : kPlanMaxSets;
   const size_t smem = plan_smem_bytes(smax);
   if (smem > 48 * 1024 && !(ctx->attr_flags & 2u)) {  // (once per context: the attribute belongs to its device)
@@ -656,13 +810,13 @@ static int launch_tile_plans(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap
     ctx->attr_flags |= 2u;
   }
   tile_plan_kernel<<<set_rowoff1 ? 2 : 1, kScanThreads, smem, ctx->stream>>>(set_rowoff, set_rowoff1, num_sets,
-                                                                            cap_sets, smax, 128);
+                                                                            cap_sets, smax, 128, pw);
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
 }
 
 int dsvt_launch_tile_plan(dsvt_ctx* ctx, const int32_t* num_sets, int32_t cap_sets, int32_t* set_rowoff) {
-  return launch_tile_plans(ctx, num_sets, cap_sets, set_rowoff, nullptr);
+  return launch_tile_plans(ctx, num_sets, cap_sets, set_rowoff, nullptr, PlanWindows{nullptr, nullptr, 0});
 }
 
 static int key_bits_for(uint64_t max_key) {
@@ -766,7 +920,8 @@ int partition_sorted(dsvt_ctx* ctx, const PartCall& pc, const PartOut& o) {
       DSVT_LAUNCHED(ctx);
     }
     if (o.set_rowoff && s_bound > 0) {
-      int rc = dsvt_launch_tile_plan(ctx, o.num_sets, cap_sets, o.set_rowoff);
+      int rc = launch_tile_plans(ctx, o.num_sets, cap_sets, o.set_rowoff, nullptr,
+                                 PlanWindows{ctx->win_setoff, ctx->win_count, nw});
       if (rc != DSVT_OK) return rc;
     }
     if (o.perm)
@@ -850,7 +1005,7 @@ int partition_bitmap(dsvt_ctx* ctx, const PartCall& pc, int32_t wpw, int naxes, 
   DSVT_CUDA_TRY(ctx, launch_pdl(bm_place_fill_kernel, dim3(fill_blocks + 1), dim3(kScanThreads), smem, st, n, pc.n_dev, job, wpw,
                                 (const int32_t*)ctx->bm_dup, (const int32_t*)counts, (const int32_t*)ctx->win_start,
                                 (const int32_t*)ctx->win_setoff, pc.set_size, pc.cap_sets,
-                                (const int32_t*)o[0].num_sets, fo, smax));
+                                (const int32_t*)o[0].num_sets, fo, smax, nw));
   DSVT_LAUNCHED(ctx);
   return copy_window_arrays(ctx, pc, counts);
 }

@@ -29,7 +29,7 @@ class Stage:
         def new_tables():
             return [api.SetTable(torch.empty((cap, set_size), dtype=torch.int32, device=dev),
                                  torch.zeros(1, dtype=torch.int32, device=dev),
-                                 torch.empty(2 * cap + 3, dtype=torch.int32, device=dev), cap, set_size)
+                                 torch.empty(4 * cap + 4, dtype=torch.int32, device=dev), cap, set_size)
                     for _ in range(2)]
 
         specs = [(self.window, None)] * len(self.blocks) if block_windows is None else [

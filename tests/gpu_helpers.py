@@ -65,7 +65,7 @@ def upload_table(table: np.ndarray, with_rowoff=True, cap_extra=0) -> api.SetTab
     cap = S + cap_extra
     full = np.full((max(cap, 1), tau), -7, dtype=np.int32)
     full[:S] = table
-    ro = np.zeros(2 * max(cap, 1) + 3, dtype=np.int32)  # row offsets, then "no tile plan"
+    ro = np.zeros(4 * max(cap, 1) + 4, dtype=np.int32)  # row offsets, then "no tile plan"
     ro[: S + 1] = rowoff_of(table)
     ro[(max(cap, 1) if S else 0) + 1] = -1
     return api.SetTable(dev(full), dev(np.array([S], dtype=np.int32)), dev(ro) if with_rowoff else None,

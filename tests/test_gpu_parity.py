@@ -18,6 +18,9 @@ def gpu():
     return api
 
 
+PLAN_PACKED = 0x40000000  # flag on the tile count of a plan over a reordering of the sets
+
+
 def _nwin(batch, grid, window):
     return batch * int(np.prod([-(-g // w) for g, w in zip(grid, window)]))
 
@@ -30,26 +33,42 @@ def _compare_table(t, ref, n, axis, extras=True):
     assert tbl.shape == ref.set_table.shape, (axis, tbl.shape, ref.set_table.shape)
     assert np.array_equal(tbl, ref.set_table), axis
     assert np.array_equal(ro, rowoff_of(ref.set_table)), axis
-    # tile plan behind the row offsets: greedy packing of whole sets into tiles of at most 128 rows
-    plan = t.set_rowoff[t.cap_sets + 1:].cpu().numpy()
+    # tile plan behind the row offsets: whole sets in tiles of at most 128 rows, over a reordering of the sets that
+    # needs fewer tiles than the greedy packing in table order (or in table order, where no reordering was found)
+    tiles = None
+    cap = t.cap_sets
+    full = t.set_rowoff.cpu().numpy()
+    plan = full[cap + 1:]
     S = tbl.shape[0]
-    starts, s = [], 0
+    sizes = np.diff(ro)
+    greedy, s = 0, 0
     while s < S:
-        starts.append(s)
         e = s + 1
         while e < S and ro[e + 1] - ro[s] <= 128:
             e += 1
         s = e
-    if S <= 24576:
-        assert plan[0] == len(starts), axis
-        assert np.array_equal(plan[1:1 + len(starts)], np.array(starts, dtype=np.int32)) and plan[1 + len(starts)] == S
-    else:
+        greedy += 1
+    if S > 24576:
         assert plan[0] == -1
+    elif S > 0:
+        T = int(plan[0]) & ~PLAN_PACKED
+        e = plan[1:2 + T]
+        assert T <= greedy and e[0] == 0 and e[T] == S and np.all(np.diff(e) > 0), axis
+        if int(plan[0]) & PLAN_PACKED:
+            order = full[2 * cap + 3: 2 * cap + 3 + S]
+            prow = full[3 * cap + 3: 3 * cap + 4 + S]
+            assert np.array_equal(np.sort(order), np.arange(S)), axis
+            assert np.array_equal(prow, np.concatenate([[0], np.cumsum(sizes[order])])), axis
+        else:
+            prow = ro
+        assert np.all(prow[e[1:]] - prow[e[:-1]] <= 128), axis
+        tiles = (T, greedy)
     if extras:
         assert np.array_equal(t.perm[:n].cpu().numpy(), ref.perm)
         assert np.array_equal(t.win_count.cpu().numpy(), ref.win_count)
         assert np.array_equal(t.win_start.cpu().numpy(), ref.win_start)
         assert np.array_equal(t.win_setoff.cpu().numpy(), ref.win_setoff)
+    return tiles
 
 
 def _check_partition(gpu, oracle, coords, batch, grid, window, tau, ctx=None):
@@ -65,14 +84,17 @@ def _check_partition(gpu, oracle, coords, batch, grid, window, tau, ctx=None):
     both = ctx.partition_rotated(dc, batch, grid, window, tau)
     assert ctx.status_sync() == 0
     for axis in (0, 1):
-        _compare_table(both[axis], refs[axis], n, axis, extras=False)
-    return ctx
+        tiles = _compare_table(both[axis], refs[axis], n, axis, extras=False)
+    return ctx, tiles
 
 
 @pytest.mark.parametrize("cid", [1, 2, 3, 4, 5, 6])
 def test_partition_bit_exact_on_every_config(gpu, oracle, cid):
     cfg = di.make_config(cid, with_feats=False)
-    _check_partition(gpu, oracle, cfg["coords"], cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"])
+    _, tiles = _check_partition(gpu, oracle, cfg["coords"], cfg["batch"], cfg["grid"], cfg["window"], cfg["set_size"])
+    if cid >= 2:  # LiDAR-shaped frames: the reordered plan saves tiles over the packing in table order
+        print("config %d: %d tiles (%d in table order)" % (cid, tiles[0], tiles[1]))
+        assert tiles[0] < tiles[1] and (cid == 5 or tiles[0] <= 0.95 * tiles[1])
 
 
 @pytest.mark.parametrize("grid,window,batch,n,tau", [
@@ -225,7 +247,12 @@ def test_set_attention_matches_oracle(gpu, oracle, seed, n, grid, window, tau, C
         want, covered = oracle.set_attention(cfg["feats"], ref_t, L["W_qkv"], L["b_qkv"], L["W_o"], L["b_o"], heads)
         assert covered.all()
         check_close(out.cpu().numpy(), want, cfg["precision"], "set_attention axis %d" % axis)
-        assert torch.equal(out, out2)
+        if bf16:  # the tensor-core kernel: a tile plan made without the windows puts the sets into other tiles, and
+            # a set's place in its tile decides how its attention is blocked: same result up to rounding
+            check_close(out2.cpu().numpy(), want, cfg["precision"], "set_attention axis %d, derived offsets" % axis)
+            assert float((out - out2).abs().max()) <= 1e-2 * float(np.abs(want).max())
+        else:
+            assert torch.equal(out, out2)
 
 
 def test_set_attention_arbitrary_table_positional_term_and_untouched_rows(gpu, oracle):

@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 def _blank_table(api, cap, tau):
     return api.SetTable(torch.full((cap, tau), -1, dtype=torch.int32, device="cuda"),
                         torch.full((1,), -1, dtype=torch.int32, device="cuda"),
-                        torch.full((2 * cap + 3,), -1, dtype=torch.int32, device="cuda"), cap, tau)
+                        torch.full((4 * cap + 4,), -1, dtype=torch.int32, device="cuda"), cap, tau)
 
 
 def _same(api, ctx, coords, batch, grid, window, tau, axis, check_memory=True, oracle=None):
@@ -45,8 +45,12 @@ def _same(api, ctx, coords, batch, grid, window, tau, axis, check_memory=True, o
     assert torch.equal(got.set_table[:S], want.set_table[:S])  # integer outputs: bit-exact
     assert torch.equal(got.set_rowoff[: S + 1], want.set_rowoff[: S + 1])
     cap = want.cap_sets  # the tile plan behind the row offsets: tile count, tile starts, terminator
-    tiles = int(want.set_rowoff[cap + 1].item())
+    head = int(want.set_rowoff[cap + 1].item())
+    tiles = head & ~0x40000000 if head >= 0 else 0
     assert torch.equal(got.set_rowoff[cap + 1: cap + 3 + tiles], want.set_rowoff[cap + 1: cap + 3 + tiles])
+    if head >= 0 and head & 0x40000000:  # a plan over reordered sets: the order and the rows before each position
+        assert torch.equal(got.set_rowoff[2 * cap + 3: 2 * cap + 3 + S], want.set_rowoff[2 * cap + 3: 2 * cap + 3 + S])
+        assert torch.equal(got.set_rowoff[3 * cap + 3: 3 * cap + 4 + S], want.set_rowoff[3 * cap + 3: 3 * cap + 4 + S])
     assert torch.all(got.set_table[S:] == -1)  # nothing written past the last set
     if oracle is not None:  # and against the CPU oracle directly, not only through dsvt_partition
         ref = oracle.partition(coords, batch, grid, window, tau, axis)
