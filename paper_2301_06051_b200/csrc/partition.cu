@@ -1,6 +1,8 @@
 // Integer side of the path: window keys, stable LSD radix sort of (key, voxel id) pairs,
 // per-window scans, set table fill (Sec. 3.2, Eq. 1-3).  Everything here is exact int32/uint32/uint64
 // arithmetic, so results are bit-reproducible.
+#include <limits.h>
+
 #include "dsvt_common.cuh"
 
 namespace {
@@ -339,12 +341,12 @@ __global__ void table_unique_count_kernel(const int32_t* __restrict__ table, int
 // row segments).  The greedy chain 0 -> next(0) -> next(next(0)) ... is found by pointer doubling, all
 // sets in parallel: single block, arrays in shared memory.
 constexpr int kPlanMaxSets = 24576;
-// Scratch of the packed plan behind the three per-set arrays: per-warp bin counts of one sorting round, bin
-// starts, bin cursors, the cursors before the round, the histogram.
+// Scratch of the packed plan behind the three per-set arrays: per-warp bin counts / cursors of the counting sort,
+// bin starts, the histogram (later the flags of the tile counts on trial).
 constexpr int kPackBins = 132;  // set sizes 1 .. 128, rounded up
 struct PackScratch {
   unsigned short whist[32][kPackBins];
-  int bin_start[kPackBins], bin_cur[kPackBins], round_base[kPackBins], hist[kPackBins];
+  int bin_start[kPackBins], hist[kPackBins];
 };
 // Dynamic shared memory the plan needs for at most smax sets.
 __host__ __device__ constexpr size_t plan_smem_bytes(int smax) {
@@ -357,24 +359,24 @@ __host__ __device__ constexpr size_t plan_smem_bytes(int smax) {
 // T - 1, the next T to tile T - 1 .. 0, and so on, which levels the tiles' row counts to within a few rows; T is
 // the smallest of a ladder of candidates from ceil(rows / max_rows) upwards for which no tile exceeds max_rows.
 // Written behind the plan header: the sets in tile order (order[p]) and the rows before each position (prow[p]);
-// tile t covers positions [plan[1 + t], plan[2 + t]).  Returns false (nothing written) if some set has no row or
-// more than max_rows, or no candidate below `limit` tiles (the plan in table order, which the caller has written) fits.
+// tile t covers positions [plan[1 + t], plan[2 + t]).  Returns the number of tiles, or 0 (nothing written) if some set
+// has no row or more than max_rows, or no candidate below `limit` tiles fits.
 struct PlanWindows {  // optional: the windows behind the sets (sets of a window are consecutive), or win_setoff = NULL
   const int32_t* win_setoff;
   const int32_t* win_count;
   int32_t num_windows;
 };
-__device__ bool packed_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int32_t cap_sets, int32_t smax,
+__device__ int packed_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int32_t cap_sets, int32_t smax,
                                  int32_t max_rows, int limit, PlanWindows pw, int* plan_smem, int* warp_tot) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
-  if (max_rows >= kPackBins || nthr <= max_rows || (nthr & 31) != 0) return false;
+  if (max_rows >= kPackBins || nthr <= max_rows || (nthr & 31) != 0) return 0;
   int* srt = plan_smem;                // set ids, sorted by rows descending
   int* ro = srt + (smax + 1);          // row offsets in table order
   unsigned char* ssz = reinterpret_cast<unsigned char*>(ro + (smax + 1));  // rows of srt[i]
   PackScratch* ps = reinterpret_cast<PackScratch*>(ssz + (((size_t)smax + 15) & ~(size_t)15));
   constexpr int kRowMask = 0xffffff;  // (at most smax * max_rows rows: 24 bits hold them)
   for (int s = tid; s <= S; s += nthr) ro[s] = rowoff[s];
-  for (int b = tid; b < kPackBins; b += nthr) { ps->hist[b] = 0; ps->bin_cur[b] = 0; }
+  for (int b = tid; b < kPackBins; b += nthr) ps->hist[b] = 0;
   __syncthreads();
   // Sort key of a set: the rows of its window's largest set, so that the sets of a window (whose sizes differ by
   // at most one) stay neighbours in the sorted order and land in neighbouring tiles.  The same plan serves every
@@ -392,41 +394,61 @@ __device__ bool packed_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, i
   }
   auto rows_of = [&](int q) { return (ro[q + 1] & kRowMask) - (ro[q] & kRowMask); };
   auto key_of = [&](int q) { const int k = (int)((unsigned)ro[q] >> 24), c = rows_of(q); return k >= c ? k : c; };
-  bool bad = false;
+  bool bad = ro[S] > kRowMask;
   for (int s = tid; s < S; s += nthr) {
     const int c = rows_of(s);
-    if (c < 1 || c > max_rows || ro[S] > kRowMask) bad = true;
-    else atomicAdd(&ps->hist[key_of(s)], 1);
+    bad |= c < 1 || c > max_rows;
   }
-  if (__syncthreads_or(bad)) return false;
-  if (tid == 0) {
-    int acc = 0;
-    for (int c = max_rows; c >= 1; --c) { ps->bin_start[c] = acc; acc += ps->hist[c]; }
-  }
-  // stable counting sort, one set per thread and round
-  for (int base = 0; base < S; base += nthr) {
-    for (int i = tid; i < 32 * kPackBins; i += nthr) (&ps->whist[0][0])[i] = 0;
-    __syncthreads();
-    const int s = base + tid;
-    const int c = s < S ? key_of(s) : 0;  // the bin
+  if (__syncthreads_or(bad)) return 0;
+  // stable counting sort: every warp takes a contiguous range of the sets; counts per (warp, bin), their prefixes
+  // over the warps, then each warp walks its range again and places its sets
+  for (int i = tid; i < 32 * kPackBins; i += nthr) (&ps->whist[0][0])[i] = 0;
+  __syncthreads();
+  const int per_warp = (S + nwarp - 1) / nwarp;
+  const int w0 = min(warp * per_warp, S), w1 = min(w0 + per_warp, S);
+  for (int b0 = w0; b0 < w1; b0 += 32) {
+    const int s = b0 + lane;
+    const int c = s < w1 ? key_of(s) : 0;  // the bin
     const unsigned same = __match_any_sync(0xffffffffu, c);
-    const int rank = __popc(same & ((1u << lane) - 1u));
-    if (c && rank == 0) ps->whist[warp][c] = (unsigned short)__popc(same);
-    __syncthreads();
-    if (tid >= 1 && tid <= max_rows) {  // bin tid: the warps' counts -> exclusive prefixes
-      int run = 0;
-      for (int w = 0; w < nwarp; ++w) { const int t = ps->whist[w][tid]; ps->whist[w][tid] = (unsigned short)run; run += t; }
-      ps->round_base[tid] = ps->bin_cur[tid];
-      ps->bin_cur[tid] += run;
+    if (c && lane == __ffs(same) - 1) ps->whist[warp][c] = (unsigned short)(ps->whist[warp][c] + __popc(same));
+    __syncwarp();
+  }
+  __syncthreads();
+  if (tid >= 1 && tid <= max_rows) {  // bin tid: the warps' counts -> exclusive prefixes, and the bin's size
+    int run = 0;
+    for (int w = 0; w < nwarp; ++w) { const int t = ps->whist[w][tid]; ps->whist[w][tid] = (unsigned short)run; run += t; }
+    ps->hist[tid] = run;
+  }
+  __syncthreads();
+  if (warp == 0) {  // the bins in descending order of their key: suffix sums, four bins per lane
+    int h[4], mine = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { const int b = 4 * lane + 1 + k; h[k] = b <= max_rows ? ps->hist[b] : 0; mine += h[k]; }
+    int suf = mine;  // this lane's bins and all higher ones
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_down_sync(0xffffffffu, suf, off);
+      if (lane + off < 32) suf += v;
     }
-    __syncthreads();
+    int acc = suf - mine;  // sets in bins above this lane's
+#pragma unroll
+    for (int k = 3; k >= 0; --k) { const int b = 4 * lane + 1 + k; if (b <= max_rows) ps->bin_start[b] = acc; acc += h[k]; }
+  }
+  __syncthreads();
+  for (int b0 = w0; b0 < w1; b0 += 32) {
+    const int s = b0 + lane;
+    const int c = s < w1 ? key_of(s) : 0;
+    const unsigned same = __match_any_sync(0xffffffffu, c);
+    const int before = c ? ps->whist[warp][c] : 0;
     if (c) {
-      const int pos = ps->bin_start[c] + ps->round_base[c] + ps->whist[warp][c] + rank;
+      const int pos = ps->bin_start[c] + before + __popc(same & ((1u << lane) - 1u));
       srt[pos] = s;
       ssz[pos] = (unsigned char)rows_of(s);
     }
-    __syncthreads();
+    __syncwarp();
+    if (c && lane == __ffs(same) - 1) ps->whist[warp][c] = (unsigned short)(before + __popc(same));
+    __syncwarp();
   }
+  __syncthreads();
   // rows of tile t when the sorted sets are dealt out to T tiles
   auto tile_rows = [&](int t, int T) {
     int sum = 0, r = 0;
@@ -438,59 +460,98 @@ __device__ bool packed_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, i
   };
   const int total = ro[S] & kRowMask;
   const int T0 = (total + max_rows - 1) / max_rows;
-  auto fits = [&](int Tc) {  // (the same answer in every thread)
-    bool over = false;
-    for (int t = tid; t < Tc; t += nthr) over |= tile_rows(t, Tc) > max_rows;
-    return !__syncthreads_or(over);
+  // Tile counts are tried a batch at a time (one barrier per batch): over[j] = some tile of candidate j is too full.
+  constexpr int kBatch = 8;
+  int* over = ps->hist;  // (the histogram has served)
+  int cand[kBatch];
+  auto try_batch = [&](int ncand) {
+    if (tid < kBatch) over[tid] = 0;
+    __syncthreads();
+    for (int j = 0; j < ncand; ++j)
+      for (int t = tid; t < cand[j]; t += nthr)
+        if (tile_rows(t, cand[j]) > max_rows) over[j] = 1;
+    __syncthreads();
   };
-  int T = -1, last = T0 - 1;  // last = the largest count known not to fit
-  const int ladder[14] = {0, 1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64, 96};  // 128ths of T0 on top of T0
-  for (int j = 0; j < 14; ++j) {
-    const int Tj = min(min(S, limit - 1), T0 + (int)(((int64_t)T0 * ladder[j] + 127) / 128));
-    if (Tj <= last) continue;
-    if (fits(Tj)) { T = Tj; break; }
-    last = Tj;
-    if (Tj >= min(S, limit - 1)) break;  // nothing below the plan in table order fits
+  const int top = min(S, limit - 1);  // (a plan with as many tiles as `limit` is no gain)
+  int T = -1, last = T0 - 1;          // last = the largest count known not to fit
+  {
+    const int ladder[15] = {0, 1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64, 96, 128};  // 128ths of T0 on top of T0
+    for (int j0 = 0; j0 < 15 && T < 0 && last < top; j0 += 5) {
+      int nc = 0, prev = last;
+      for (int j = j0; j < j0 + 5; ++j) {
+        const int Tj = min(top, T0 + (int)(((int64_t)T0 * ladder[j] + 127) / 128));
+        if (Tj > prev) { cand[nc++] = Tj; prev = Tj; }
+      }
+      if (nc == 0) break;
+      try_batch(nc);
+      for (int j = 0; j < nc && T < 0; ++j) {
+        if (!over[j]) T = cand[j];
+        else last = cand[j];
+      }
+      __syncthreads();  // (everyone has read the flags)
+    }
   }
-  if (T < 0) return false;
-  while (T - last > 1) {  // between the rungs: bisection (fitting is not monotonic in T; any count that fits will do)
-    const int mid = last + (T - last) / 2;
-    if (fits(mid)) T = mid; else last = mid;
+  if (T < 0) return 0;
+  if (T - last - 1 > T0 / 128) {  // between two rungs, if they are more than a percent apart: evenly spaced counts
+    // (fitting is not monotonic in T: any count that fits will do, the smallest found is taken)
+    const int gap = T - last - 1, nc = min(gap, kBatch);
+    for (int j = 0; j < nc; ++j) cand[j] = last + 1 + (int)(((int64_t)j * gap) / nc);
+    try_batch(nc);
+    for (int j = 0; j < nc; ++j)
+      if (!over[j]) { T = cand[j]; break; }
+    __syncthreads();
   }
   // positions: tile t holds the sets of rounds 0 .. full - 1 and, for rem tiles, one of the last round
   const int full = S / T, rem = S % T;
-  auto tile_start = [&](int t) { return t * full + ((full & 1) ? max(0, t - (T - rem)) : min(t, rem)); };
+  const bool extra_first = (full & 1) == 0;  // the last, partial round runs forwards: tiles 0 .. rem - 1 get its sets
+  auto tile_start = [&](int t) { return t * full + (extra_first ? min(t, rem) : max(0, t - (T - rem))); };
+  // rows before each tile: the tiles' row counts (one thread per tile), then a scan over contiguous chunks of them
+  int* tbase = ro;  // (the offsets in table order have served: the sorted sizes are in ssz)
+  __syncthreads();
+  for (int t = tid; t < T; t += nthr) tbase[t] = tile_rows(t, T);
+  __syncthreads();
   const int chunk = (T + nthr - 1) / nthr;
   const int t0 = min(tid * chunk, T), t1 = min(t0 + chunk, T);
   int local = 0;
-  for (int t = t0; t < t1; ++t) local += tile_rows(t, T);
+  for (int t = t0; t < t1; ++t) local += tbase[t];
   int tot;
   int rows = block_excl_scan(local, warp_tot, &tot);
+  for (int t = t0; t < t1; ++t) { const int c = tbase[t]; tbase[t] = rows; rows += c; }
+  __syncthreads();
   int32_t* out[2] = {rowoff, rowoff_copy};
-  for (int t = t0; t < t1; ++t) {
-    int p = tile_start(t), r = 0;
+  for (int t = tid; t <= T; t += nthr) {
+    const int v = t < T ? tile_start(t) : S;
     for (int q = 0; q < 2; ++q)
-      if (out[q]) out[q][cap_sets + 2 + t] = p;
-    for (int i0 = 0; i0 < S; i0 += T, ++r) {
-      const int i = i0 + ((r & 1) ? T - 1 - t : t);
-      if (i >= S) continue;
-      for (int q = 0; q < 2; ++q)
-        if (out[q]) {
-          out[q][2 * (size_t)cap_sets + 3 + p] = srt[i];
-          out[q][3 * (size_t)cap_sets + 3 + p] = rows;
-        }
-      rows += ssz[i];
-      ++p;
+      if (out[q]) out[q][cap_sets + 2 + t] = v;
+  }
+  // one thread per position (neighbouring threads write neighbouring entries): its tile, its round, the rows before it
+  for (int p = tid; p < S; p += nthr) {
+    int t, r;
+    if (extra_first) {
+      const int cut = rem * (full + 1);
+      if (p < cut) { t = p / (full + 1); r = p - t * (full + 1); }
+      else { t = rem + (p - cut) / full; r = (p - cut) - (t - rem) * full; }
+    } else {
+      const int cut = (T - rem) * full;
+      if (p < cut) { t = p / full; r = p - t * full; }
+      else { t = (T - rem) + (p - cut) / (full + 1); r = (p - cut) - (t - (T - rem)) * (full + 1); }
     }
+    int before = tbase[t];
+    for (int k = 0; k < r; ++k) before += ssz[k * T + ((k & 1) ? T - 1 - t : t)];
+    const int set = srt[r * T + ((r & 1) ? T - 1 - t : t)];
+    for (int q = 0; q < 2; ++q)
+      if (out[q]) {
+        out[q][2 * (size_t)cap_sets + 3 + p] = set;
+        out[q][3 * (size_t)cap_sets + 3 + p] = before;
+      }
   }
   if (tid == 0)
     for (int q = 0; q < 2; ++q)
       if (out[q]) {
         out[q][cap_sets + 1] = T | DSVT_PLAN_PACKED;
-        out[q][cap_sets + 2 + T] = S;
         out[q][3 * (size_t)cap_sets + 3 + S] = tot;
       }
-  return true;
+  return T;
 }
 
 // The plan of `rowoff` (its offsets are read, its plan written; a second buffer with the same offsets, e.g. the
@@ -511,6 +572,12 @@ __device__ void tile_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int
     if (tid == 0) { plan[0] = 0; plan[1] = 0; if (plan2) { plan2[0] = 0; plan2[1] = 0; } }
     return;
   }
+  // The packed plan first.  If it comes within an eighth of the fewest tiles there can be, it stands; else the plan
+  // in table order is worked out as well and the one with fewer tiles is kept.
+  const int packed = packed_plan_body(rowoff, rowoff_copy, S, cap_sets, smax, max_rows, INT_MAX, pw, plan_smem, warp_tot);
+  const int fewest = (rowoff[S] + max_rows - 1) / max_rows;
+  if (packed > 0 && packed <= fewest + fewest / 8) return;
+  __syncthreads();  // (the shared arrays are reused)
   // the offsets once into shared memory (the second pointer array is free until the doubling rounds): every set
   // then finds the end of the tile that would start with it by a binary search there
   int* ro = nxt;
@@ -545,6 +612,7 @@ __device__ void tile_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int
   for (int s = s0; s < s1; ++s) cnt += mark[s];
   int total;
   int off = block_excl_scan(cnt, warp_tot, &total);
+  if (packed > 0 && packed < total) return;  // the packed plan has fewer tiles: it stays
   for (int s = s0; s < s1; ++s)
     if (mark[s]) {
       plan[1 + off] = s;
@@ -555,8 +623,6 @@ __device__ void tile_plan_body(int32_t* rowoff, int32_t* rowoff_copy, int S, int
     plan[0] = total; plan[1 + total] = S;
     if (plan2) { plan2[0] = total; plan2[1 + total] = S; }
   }
-  __syncthreads();  // the plan in table order stands; a packed one with fewer tiles replaces it (same shared arrays)
-  packed_plan_body(rowoff, rowoff_copy, S, cap_sets, smax, max_rows, total, pw, plan_smem, warp_tot);
 }
 
 __global__ void __launch_bounds__(kScanThreads) tile_plan_kernel(int32_t* rowoff0, int32_t* rowoff1,

@@ -53,7 +53,8 @@ def _compare_table(t, ref, n, axis, extras=True):
     elif S > 0:
         T = int(plan[0]) & ~PLAN_PACKED
         e = plan[1:2 + T]
-        assert T <= greedy and e[0] == 0 and e[T] == S and np.all(np.diff(e) > 0), axis
+        fewest = -(-int(ro[S]) // 128)  # (a reordered plan within an eighth of this is taken without looking further)
+        assert T <= max(greedy, fewest + fewest // 8) and e[0] == 0 and e[T] == S and np.all(np.diff(e) > 0), axis
         if int(plan[0]) & PLAN_PACKED:
             order = full[2 * cap + 3: 2 * cap + 3 + S]
             prow = full[3 * cap + 3: 3 * cap + 4 + S]
