@@ -89,6 +89,19 @@ def test_chain_without_a_tile_plan(gpu, oracle):
     assert float((y - z).abs().max()) <= 2e-2 * float(np.abs(want).max())
 
 
+@pytest.mark.parametrize("window,tau,n", [((1, 1, 1), 36, 1500), ((2, 1, 1), 36, 2500), ((8, 8, 1), 64, 4096)])
+def test_chain_on_extreme_tile_plans(gpu, oracle, window, tau, n):
+    """Tiles at the limits of the plan: every voxel a window (and a set) of its own, 128 one-row sets per tile;
+    sets of one or two rows; and full windows whose 64-row sets fill a tile in pairs."""
+    cfg = di.random_case(5, n, (64, 64, 1), window, tau, 192, 8, hidden=384, layernorm=True, bf16=True, n_blocks=2)
+    ctx, tabs, ws = _setup(gpu, cfg, cfg["blocks"])
+    x = dev(cfg["feats"])
+    y = torch.empty_like(x)
+    ctx.layers(x, tabs, ws, y)
+    assert ctx.status_sync() == 0
+    check_close(y.cpu().numpy(), _oracle_chain(oracle, cfg, cfg["blocks"]), "bf16", "chain, window %s" % (window,))
+
+
 def test_chain_with_other_tables_per_block(gpu, oracle):
     """Hybrid windows: the second block runs on the tables of another window cut, so a tile of its first layer
     reads rows that tiles anywhere in the previous layer wrote (the stamps are per voxel, not per window)."""

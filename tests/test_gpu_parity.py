@@ -106,6 +106,9 @@ def test_partition_bit_exact_on_every_config(gpu, oracle, cid):
     ((12, 12, 1), (12, 12, 1), 1, 1, 36),      # a single voxel
     ((300, 300, 1), (7, 9, 1), 1, 5000, 90),   # spans several sort tiles and a ragged tail
     ((64, 64, 8), (64, 64, 8), 1, 20000, 48),  # one huge window (20000 voxels -> 417 sets)
+    ((64, 64, 1), (1, 1, 1), 1, 3000, 36),     # every voxel a window of its own: 128 one-row sets per tile
+    ((64, 64, 1), (8, 8, 1), 1, 4096, 64),     # full windows of 64 voxels: every set has 64 rows, two fill a tile
+    ((96, 96, 1), (6, 7, 1), 1, 9216, 42),     # full windows of 42 (36 at the edges): three sets per tile at most
 ])
 def test_partition_bit_exact_small_and_edge_cases(gpu, oracle, grid, window, batch, n, tau):
     rng = np.random.default_rng(n + tau)
