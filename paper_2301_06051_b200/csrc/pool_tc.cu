@@ -275,22 +275,25 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const __grid_const
       ++uses[bar];
       tc_fence_after();
     };
-    // tile row -> voxel through the region list and the dense cell map (looked up one tile ahead)
-    auto row_voxel = [&](int tl) {
+    // tile row -> voxel through the region list and the dense cell map: the region's key is looked up two tiles
+    // ahead and its cell one tile ahead, so that neither load waits for the other inside a tile
+    auto row_key = [&](int tl) {
       const int t = blockIdx.x + tl * gridDim.x, r_lo = t * TR, nr = min(TR, m - r_lo);
-      int v = -1;
-      if (tl < my_tiles && tid < kTM && tid / ns < nr)
-        v = __ldg(a.cell_map + (size_t)__ldg(a.region_key + r_lo + tid / ns) * ns + (tid & (ns - 1)));
-      return v;
+      return (tl < my_tiles && tid < kTM && tid / ns < nr) ? __ldg(a.region_key + r_lo + tid / ns) : -1;
     };
-    int v_next = row_voxel(0);
+    auto row_voxel = [&](int key) {
+      return key >= 0 ? __ldg(a.cell_map + (size_t)key * ns + (tid & (ns - 1))) : -1;
+    };
+    int v_next = row_voxel(row_key(0));
+    int key_next = row_key(1);
     for (int tl = 0; tl < my_tiles; ++tl) {
       const int t = blockIdx.x + tl * gridDim.x;
       const int r_lo = t * TR, nr = min(TR, m - r_lo);
       compute_sync();  // the previous tile's staging rows have been stored; its operands are dead
       if (tid < kTM) s_pm.rowvox[tid] = v_next;
       compute_sync();
-      v_next = row_voxel(tl + 1);
+      v_next = row_voxel(key_next);
+      key_next = row_key(tl + 2);
       pool_gather<C>(a, xs, ps, nr, ns);
       fence_proxy_async();
       mbar_arrive(&s_pm.ab_ready);
@@ -298,12 +301,16 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const __grid_const
       const bool live = ri < nr;
       const bool key_ok = live && (!a.mask_empty || s_pm.rowvox[row] >= 0);
       float p[HQ];
+      float qr[QC];  // this thread's query columns: read at once, so that the value projection can take their region
       acc_wait(0);
+      tmem_ld_row(taddr, qr);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(&s_pm.acc_free[0]);
       acc_wait(1);
 #pragma unroll
       for (int j = 0; j < HQ; ++j) {  // one head at a time: D query and D key columns of this thread's row
-        float q[D], k[D];
-        tmem_ld_row(taddr + j * D, q);
+        float k[D];
         tmem_ld_row(taddr + C + j * D, k);
         tmem_wait_ld();
         float acc = 0.f;
@@ -311,10 +318,10 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const __grid_const
         for (int c = 0; c < D; c += 4) {
           const int cc = hq * QC + j * D + c;
           const float4 bq = *reinterpret_cast<const float4*>(par + cc), bk = *reinterpret_cast<const float4*>(par + C + cc);
-          acc = fmaf(q[c] + bq.x, k[c] + bk.x, acc);
-          acc = fmaf(q[c + 1] + bq.y, k[c + 1] + bk.y, acc);
-          acc = fmaf(q[c + 2] + bq.z, k[c + 2] + bk.z, acc);
-          acc = fmaf(q[c + 3] + bq.w, k[c + 3] + bk.w, acc);
+          acc = fmaf(qr[j * D + c] + bq.x, k[c] + bk.x, acc);
+          acc = fmaf(qr[j * D + c + 1] + bq.y, k[c + 1] + bk.y, acc);
+          acc = fmaf(qr[j * D + c + 2] + bq.z, k[c + 2] + bk.z, acc);
+          acc = fmaf(qr[j * D + c + 3] + bq.w, k[c + 3] + bk.w, acc);
         }
         const float lg = key_ok ? acc * scale : -INFINITY;
         float mx = lg;
@@ -325,7 +332,6 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const __grid_const
         p[j] = sum > 0.f ? e / sum : 0.f;
       }
       tc_fence_before();
-      mbar_arrive(&s_pm.acc_free[0]);
       mbar_arrive(&s_pm.acc_free[1]);
       // ---- weighted sum of the values over the region's slots -> attention output (bf16 operand, P's place) ----
       {
