@@ -69,6 +69,28 @@ struct dsvt_ctx {
     }                                     \
   } while (0)
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start while its
+// predecessor in the stream still runs; it lets its own successor start early and then waits for the predecessor
+// (and everything before it) to have completed and flushed.  Both are no-ops in an ordinary launch.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+
+// A launch that may overlap its predecessor's tail (see pdl_enter).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 static inline int64_t dsvt_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 // ---- launchers implemented in the .cu files (all enqueue on ctx->stream) ----

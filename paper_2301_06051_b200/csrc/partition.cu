@@ -16,13 +16,6 @@ constexpr int kSortTile = kSortThreads * kSortRounds;  // keys per block per pas
 constexpr int kRadixBits = 8;
 constexpr int kRadix = 1 << kRadixBits;
 
-// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start while its
-// predecessor in the stream still runs; it lets its own successor start early and then waits for the predecessor
-// (and everything before it) to have completed and flushed.  Both are no-ops in an ordinary launch.
-__device__ __forceinline__ void pdl_enter() {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-}
 
 __device__ __forceinline__ int warp_incl_scan(int v) {
   const int lane = threadIdx.x & 31;
@@ -59,6 +52,7 @@ __device__ __forceinline__ int block_excl_scan(int v, int* warp_tot, int* total)
 __global__ void __launch_bounds__(kScanThreads) scan_loop_kernel(const int32_t* in, int32_t* out, int64_t count,
                                                                  int32_t* total_out) {
   __shared__ int warp_tot[33];
+  pdl_enter();
   int carry = 0;
   for (int64_t base = 0; base < count; base += kScanTile) {
     int v[kScanItems];
@@ -88,6 +82,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_loop_kernel(const int32_t* 
 __global__ void __launch_bounds__(kScanThreads) scan_local_kernel(const int32_t* in, int32_t* out, int64_t count,
                                                                   int32_t* block_sums) {
   __shared__ int warp_tot[33];
+  pdl_enter();
   int v[kScanItems];
   int s = 0;
   const int64_t i0 = (int64_t)blockIdx.x * kScanTile + (int64_t)threadIdx.x * kScanItems;
@@ -109,6 +104,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_local_kernel(const int32_t*
 __global__ void __launch_bounds__(kScanThreads) scan_add_kernel(int32_t* out, int64_t count,
                                                                 const int32_t* __restrict__ block_offs,
                                                                 int64_t nblocks, int32_t* total_out) {
+  pdl_enter();
   const int add = block_offs[blockIdx.x];
   const int64_t i0 = (int64_t)blockIdx.x * kScanTile + (int64_t)threadIdx.x * kScanItems;
 #pragma unroll
@@ -817,17 +813,22 @@ __global__ void __launch_bounds__(kScanThreads) bm_place_fill_kernel(int32_t n_m
 
 // ---------------------------------------------------------------------------------------------------
 int dsvt_launch_scan_i32(dsvt_ctx* ctx, const int32_t* in, int32_t* out, int64_t count, int32_t* total_out) {
+  // (the scan kernels wait for their predecessor themselves: their launches may overlap its tail)
+  cudaStream_t st = ctx->stream;
   if (count <= 8 * (int64_t)kScanTile) {
-    scan_loop_kernel<<<1, kScanThreads, 0, ctx->stream>>>(in, out, count, total_out);
+    DSVT_CUDA_TRY(ctx, launch_pdl(scan_loop_kernel, dim3(1), dim3(kScanThreads), 0, st, in, out, count, total_out));
     DSVT_LAUNCHED(ctx);
     return DSVT_OK;
   }
   const int64_t nblocks = dsvt_ceil_div(count, kScanTile);
-  scan_local_kernel<<<(unsigned)nblocks, kScanThreads, 0, ctx->stream>>>(in, out, count, ctx->scan_tmp);
+  DSVT_CUDA_TRY(ctx, launch_pdl(scan_local_kernel, dim3((unsigned)nblocks), dim3(kScanThreads), 0, st, in, out, count,
+                                ctx->scan_tmp));
   DSVT_LAUNCHED(ctx);
-  scan_loop_kernel<<<1, kScanThreads, 0, ctx->stream>>>(ctx->scan_tmp, ctx->scan_tmp, nblocks, nullptr);
+  DSVT_CUDA_TRY(ctx, launch_pdl(scan_loop_kernel, dim3(1), dim3(kScanThreads), 0, st, (const int32_t*)ctx->scan_tmp,
+                                ctx->scan_tmp, nblocks, (int32_t*)nullptr));
   DSVT_LAUNCHED(ctx);
-  scan_add_kernel<<<(unsigned)nblocks, kScanThreads, 0, ctx->stream>>>(out, count, ctx->scan_tmp, nblocks, total_out);
+  DSVT_CUDA_TRY(ctx, launch_pdl(scan_add_kernel, dim3((unsigned)nblocks), dim3(kScanThreads), 0, st, out, count,
+                                (const int32_t*)ctx->scan_tmp, nblocks, total_out));
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
 }
@@ -1004,18 +1005,6 @@ int32_t bitmap_words_per_window(const dsvt_ctx* ctx, const PartCall& pc) {
   const uint64_t wpw = (pc.V + 31) / 32;
   if ((uint64_t)pc.nw * wpw > ctx->bm_words || (uint64_t)pc.nw * wpw * 32 > 0xFFFFFFFFull) return 0;
   return (int32_t)wpw;
-}
-
-// A launch that may overlap its predecessor's tail (see pdl_enter).
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 // Bitmap route: one or both axes in three launches and a memset.

@@ -31,6 +31,7 @@ __global__ void pool_mark_kernel(const int4* __restrict__ coords, int32_t n_max,
                                  PoolGeom g, int32_t* __restrict__ cell_map,
                                  int32_t* __restrict__ region_flag, uint32_t* __restrict__ vox_region,
                                  int32_t* __restrict__ slot_of, int32_t* __restrict__ status) {
+  pdl_enter();  // (lets the scan's first kernel start under this one's tail)
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   const int n = n_dev ? min(max(*n_dev, 0), n_max) : n_max;  // (a count that lives on the device)
   if (i >= n) return;
@@ -52,6 +53,7 @@ __global__ void pool_finish_kernel(int32_t n_max, const int32_t* __restrict__ n_
                                    int32_t* __restrict__ out_coords, int32_t* __restrict__ region_key,
                                    int32_t* __restrict__ region_of, int32_t* __restrict__ num_out,
                                    int32_t* __restrict__ status) {
+  pdl_enter();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i == 0) {
     const int m = region_rank[num_regions];
@@ -635,8 +637,9 @@ extern "C" int dsvt_pool_counted(dsvt_ctx* ctx, const int32_t* coords, const flo
   DSVT_LAUNCHED(ctx);
   int rc = dsvt_launch_scan_i32(ctx, ctx->win_count, ctx->win_start, num_regions, nullptr);
   if (rc != DSVT_OK) return rc;
-  pool_finish_kernel<<<vb, 256, 0, st>>>(n, n_dev, g, ctx->keys[0], ctx->win_start, (int32_t)num_regions, cap_m, out_coords,
-                                         ctx->region_key, region_of, num_out, ctx->status);
+  DSVT_CUDA_TRY(ctx, launch_pdl(pool_finish_kernel, dim3(vb), dim3(256), 0, st, n, n_dev, g, (const uint32_t*)ctx->keys[0],
+                                (const int32_t*)ctx->win_start, (int32_t)num_regions, cap_m, out_coords, ctx->region_key,
+                                region_of, num_out, ctx->status));
   DSVT_LAUNCHED(ctx);
   if (cap_m == 0) return DSVT_OK;
 

@@ -249,6 +249,10 @@ __global__ void __launch_bounds__(kThreads, 1) pool_tc_kernel(const __grid_const
     const float* v = which == 0 ? a.b_q : which == 1 ? a.b_k : which == 2 ? a.b_v : a.b_o;
     par[i] = v ? __ldg(v + i % C) : 0.f;
   }
+  // everything above touched this CTA's own state and the call's weights; what follows reads what the kernels before
+  // it in the stream wrote (the region list, the cell map, the number of regions): wait for them if this launch was
+  // allowed to start early
+  pdl_enter();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -413,7 +417,7 @@ int launch_pool_tc(dsvt_ctx* ctx, const PoolTcArgs& a, const PoolTcMaps& maps, i
     DSVT_CUDA_TRY(ctx, cudaFuncSetAttribute(pool_tc_kernel<C, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     ctx->attr_flags |= flag;
   }
-  pool_tc_kernel<C, D><<<grid, kThreads, smem, ctx->stream>>>(a, maps);
+  DSVT_CUDA_TRY(ctx, launch_pdl(pool_tc_kernel<C, D>, dim3(grid), dim3(kThreads), smem, ctx->stream, a, maps));
   DSVT_LAUNCHED(ctx);
   return DSVT_OK;
 }
